@@ -1,0 +1,227 @@
+"""ctypes front end of the CPU oracle (``pipe_oracle.c``).  TEST INFRASTRUCTURE.
+
+Only the test-suite, the smoke check and the benchmark's CPU-baseline leg use this module;
+the CUDA library never does.  ``build()`` compiles the C file with gcc into
+``libpipe_oracle.so`` next to it; everything else marshals NumPy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pipe_oracle.c")
+_LIB = os.path.join(_HERE, "libpipe_oracle.so")
+
+OK, ERR_ARG, ERR_NONFINITE, ERR_ACC_OVERFLOW = 0, 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (plain C, -O2, OpenMP over rows, no contraction of a*b+c)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-Wall", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        _lib = C.CDLL(_LIB)
+        i32, i64, p = C.c_int32, C.c_int64, C.c_void_p
+        _lib.pipe_oracle_threads.restype = C.c_int
+        _lib.pipe_oracle_row_absmax.argtypes = [p, i64, i64, i64, p]
+        _lib.pipe_oracle_select_groups.argtypes = [p, i32, i32, i32, p]
+        _lib.pipe_oracle_expand.argtypes = [p, i64, i64, i64, C.c_int, C.c_int, i32, i32, p, p, p, p, p, p]
+        _lib.pipe_oracle_pack.argtypes = [p, i64, i64, C.c_int, p]
+        _lib.pipe_oracle_quantize_act.argtypes = [p, i64, i64, i64, p, p, i64, p]
+        _lib.pipe_oracle_forward.argtypes = [p, i64, i64, i64, i64, C.c_int, i32, p, p, p, p, C.c_int, C.c_int,
+                                             C.c_float, p, p, i64, p, p, p]
+        _lib.pipe_oracle_ensemble.argtypes = [p, i64, i64, i64, C.c_int, i32, p, p, p, p, C.c_int, p, p, p,
+                                              C.c_int, p, p]
+        _lib.pipe_oracle_balanced_split.argtypes = [C.c_int, C.c_int, p]
+        _lib.pipe_oracle_keep_groups.argtypes = [i32, C.c_double]
+        _lib.pipe_oracle_keep_groups.restype = i32
+    return _lib
+
+
+def threads() -> int:
+    return int(lib().pipe_oracle_threads())
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int):
+        super().__init__(f"oracle returned status {code}")
+        self.code = code
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise OracleError(rc)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+@dataclass
+class Expansion:
+    """Output of the expansion: compacted per-order codes/scales and kept-group lists."""
+    O: int
+    I: int
+    bits: int
+    K: int
+    g: int
+    n_keep: int
+    codes: np.ndarray        # int8 [R_total, I]
+    scales: np.ndarray       # float32 [R_total]
+    kept: np.ndarray         # int32 [K, G]
+    kept_count: np.ndarray   # int32 [K]
+    residual: np.ndarray     # float32 [O, I]
+    absmax: np.ndarray       # float32 [K, O]
+
+    @property
+    def G(self) -> int:
+        return self.O // self.g
+
+    def rows(self, k: int) -> int:
+        return int(self.kept_count[k]) * self.g
+
+    def row_off(self, k: int) -> int:
+        return int(sum(self.rows(j) for j in range(k)))
+
+    @property
+    def R_total(self) -> int:
+        return self.row_off(self.K)
+
+    def order_codes(self, k: int) -> np.ndarray:
+        return self.codes[self.row_off(k):self.row_off(k) + self.rows(k)]
+
+    def order_scales(self, k: int) -> np.ndarray:
+        return self.scales[self.row_off(k):self.row_off(k) + self.rows(k)]
+
+    def order_kept(self, k: int) -> np.ndarray:
+        return self.kept[k, :int(self.kept_count[k])]
+
+    def order_channels(self, k: int) -> np.ndarray:
+        """Output channel of every compacted row of order k."""
+        kg = self.order_kept(k).astype(np.int64)
+        return (kg[:, None] * self.g + np.arange(self.g)[None, :]).reshape(-1)
+
+    def packed(self, k: int) -> np.ndarray:
+        return pack(self.order_codes(k), self.bits)
+
+
+def row_absmax(r: np.ndarray) -> np.ndarray:
+    r = _c(r, np.float32)
+    a = np.empty(r.shape[0], np.float32)
+    _check(lib().pipe_oracle_row_absmax(_ptr(r), r.shape[0], r.shape[1], r.shape[1], _ptr(a)))
+    return a
+
+
+def select_groups(a: np.ndarray, g: int, n_keep: int) -> np.ndarray:
+    a = _c(a, np.float32)
+    G = a.shape[0] // g
+    out = np.empty(n_keep, np.int32)
+    _check(lib().pipe_oracle_select_groups(_ptr(a), G, g, n_keep, _ptr(out)))
+    return out
+
+
+def expand(W: np.ndarray, bits: int, K: int, g: int, n_keep: int) -> Expansion:
+    W = _c(W, np.float32)
+    O, I = W.shape
+    G = O // g
+    R_max = O + (K - 1) * n_keep * g
+    codes = np.zeros((R_max, I), np.int8)
+    scales = np.zeros(R_max, np.float32)
+    kept = np.full((K, G), -1, np.int32)
+    kept_count = np.zeros(K, np.int32)
+    residual = np.empty((O, I), np.float32)
+    absmax = np.empty((K, O), np.float32)
+    _check(lib().pipe_oracle_expand(_ptr(W), O, I, I, bits, K, g, n_keep, _ptr(codes), _ptr(scales), _ptr(kept),
+                                    _ptr(kept_count), _ptr(residual), _ptr(absmax)))
+    R = int(kept_count.astype(np.int64).sum()) * g
+    return Expansion(O, I, bits, K, g, n_keep, codes[:R], scales[:R], kept, kept_count, residual, absmax)
+
+
+def pack(codes: np.ndarray, bits: int) -> np.ndarray:
+    codes = _c(codes, np.int8)
+    rows, I = codes.shape
+    per = 8 // bits
+    out = np.empty((rows, (I + per - 1) // per), np.uint8)
+    _check(lib().pipe_oracle_pack(_ptr(codes), rows, I, bits, _ptr(out)))
+    return out
+
+
+def quantize_act(x: np.ndarray, static_scale: float | None = None):
+    x = _c(x, np.float32)
+    T, I = x.shape
+    xq = np.empty((T, I), np.int8)
+    sx = np.zeros(1, np.float32)
+    ss = None if static_scale is None else np.array([static_scale], np.float32)
+    _check(lib().pipe_oracle_quantize_act(_ptr(x), T, I, I, _ptr(ss), _ptr(xq), I, _ptr(sx)))
+    return xq, np.float32(sx[0])
+
+
+@dataclass
+class Forward:
+    y: np.ndarray          # float32 [T, O]
+    y64: np.ndarray        # float64 [T, O]  same sum in binary64
+    yabs: np.ndarray       # float64 [T, O]  sum of |terms|
+    partials: np.ndarray   # int32 [T, R_total] (only the cluster's columns written)
+
+
+def forward(e: Expansion, xq: np.ndarray, sx, k_begin: int = 0, k_end: int | None = None,
+            bias: np.ndarray | None = None) -> Forward:
+    xq = _c(xq, np.int8)
+    T, I = xq.shape
+    assert I == e.I
+    k_end = e.K if k_end is None else k_end
+    y = np.empty((T, e.O), np.float32)
+    y64 = np.empty((T, e.O), np.float64)
+    yabs = np.empty((T, e.O), np.float64)
+    partials = np.zeros((T, e.R_total), np.int32)
+    b = None if bias is None else _c(bias, np.float32)
+    _check(lib().pipe_oracle_forward(_ptr(xq), T, I, I, e.O, e.K, e.g, _ptr(e.codes), _ptr(e.scales), _ptr(e.kept),
+                                     _ptr(e.kept_count), k_begin, k_end, C.c_float(float(sx)), _ptr(b), _ptr(y),
+                                     e.O, _ptr(y64), _ptr(yabs), _ptr(partials)))
+    return Forward(y, y64, yabs, partials)
+
+
+def ensemble(e: Expansion, xq_m: np.ndarray, sx_m, branch_orders, bias=None, sum_branches=False):
+    """xq_m: [M, T, I] int8; returns (y [M,T,O] or [T,O], partials [T, R_total])."""
+    xq_m = _c(xq_m, np.int8)
+    M, T, I = xq_m.shape
+    bo = _c(branch_orders, np.int32)
+    sx = _c(sx_m, np.float32)
+    y = np.empty((T, e.O) if sum_branches else (M, T, e.O), np.float32)
+    partials = np.zeros((T, e.R_total), np.int32)
+    b = None if bias is None else _c(bias, np.float32)
+    _check(lib().pipe_oracle_ensemble(_ptr(xq_m), T, I, e.O, e.K, e.g, _ptr(e.codes), _ptr(e.scales), _ptr(e.kept),
+                                      _ptr(e.kept_count), M, _ptr(bo), _ptr(sx), _ptr(b), int(bool(sum_branches)),
+                                      _ptr(y), _ptr(partials)))
+    return y, partials
+
+
+def balanced_split(K: int, M: int) -> np.ndarray:
+    out = np.zeros(M, np.int32)
+    _check(lib().pipe_oracle_balanced_split(K, M, _ptr(out)))
+    return out
+
+
+def keep_groups(G: int, gamma: float) -> int:
+    return int(lib().pipe_oracle_keep_groups(G, float(gamma)))
