@@ -1,0 +1,194 @@
+/*
+ * pipe.h -- C ABI of libpipe: the residual-expanded quantized layer of PIPE
+ * (arXiv 2311.15806) on one NVIDIA B200 (sm_100a).
+ *
+ * Conventions that hold for every call unless its comment says otherwise
+ *   - pointers named d_* are DEVICE pointers, h_* are HOST pointers; both are owned by the
+ *     caller.  The library never allocates, frees or keeps device memory; it only queues
+ *     stream-ordered work on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and returns.  Buffers must stay valid until that work has run.
+ *   - matrices are row-major with the last dimension contiguous; ld* are row pitches in
+ *     ELEMENTS.
+ *   - every function returns a pipe_status.  Problems the host can see (null pointers, bad
+ *     shapes, undersized buffers, unsupported combinations) are reported immediately and no
+ *     work is queued.  Problems only the device can see (a NaN/Inf among the weights or
+ *     activations, a bounded wait inside a kernel running out) set a device status word that
+ *     pipe_poll_status reads; the outputs of that call are then unspecified but every access
+ *     stayed in bounds.  Nothing throws, aborts, traps or prints.
+ *   - there is no CPU fallback: without a CUDA device every compute call returns
+ *     PIPE_ERR_CUDA.
+ */
+#ifndef PIPE_H_
+#define PIPE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PIPE_MAX_ORDERS 16
+#define PIPE_BLOB_ALIGN 1024 /* d_blob must be aligned to this many bytes */
+
+typedef enum {
+  PIPE_OK = 0,
+  PIPE_ERR_INVALID_ARG = 1,  /* null pointer, negative size, value out of range */
+  PIPE_ERR_SHAPE = 2,        /* group size does not divide out_features, K/M inconsistent, ... */
+  PIPE_ERR_ALIGNMENT = 3,    /* pointer or pitch not aligned as documented */
+  PIPE_ERR_UNSUPPORTED = 4,  /* valid request this build has no kernel for */
+  PIPE_ERR_WORKSPACE = 5,    /* blob / workspace smaller than pipe_layout says */
+  PIPE_ERR_NONFINITE = 6,    /* device saw NaN or Inf in weights or activations */
+  PIPE_ERR_ACC_OVERFLOW = 7, /* in_features so large that an int32 partial sum could overflow */
+  PIPE_ERR_TIMEOUT = 8,      /* a bounded wait inside a kernel ran out */
+  PIPE_ERR_CUDA = 9          /* a CUDA runtime/driver call failed (no device, launch error) */
+} pipe_status;
+
+/*
+ * One expanded layer.  Sec. 3 "Methodology overview" fixes the quantizer Q (Eq. 1: scale,
+ * round to nearest) and the target bit-width b; Sec. 3.1 the expansion order K (Eq. 3) and
+ * the structured mask with kept fraction gamma; Sec. 3.2 the grouping [K_1..K_M] of
+ * successive orders into M predictors.
+ */
+typedef struct pipe_layer_desc {
+  int32_t out_features;  /* O: rows of W = output channels */
+  int32_t in_features;   /* I: reduction length; a multiple of the codes per byte (1, 2, 4) */
+  int32_t weight_bits;   /* b: 8, 4, or 2 (2 = ternary {-1,0,+1}); activations are int8 */
+  int32_t num_orders;    /* K, 1..PIPE_MAX_ORDERS */
+  int32_t group_size;    /* g: consecutive output channels per sparsity group; divides O */
+  int32_t keep_groups;   /* groups kept by every order >= 2, 1..O/g (order 1 is dense) */
+  int32_t num_branches;  /* M, 1..K */
+  int32_t branch_orders[PIPE_MAX_ORDERS]; /* K_m, sum = K; all zero = balanced default */
+} pipe_layer_desc;
+
+/*
+ * Byte layout of the expanded-layer blob and the workspace sizes, as computed by
+ * pipe_layout.  All offsets are from the start of the blob, so the blob is relocatable:
+ * saving or moving an expanded layer is a plain byte copy.
+ *
+ * For order k (0-based; rows[k] = kept_groups[k] * g rows, compacted in ascending channel
+ * order of the kept groups):
+ *   codes_off[k]  canonical packed codes, [rows[k], canon_row_bytes] bytes.  Two's complement
+ *                 fields, element e of a row at bit offset e*b of the row's little-endian bit
+ *                 stream: int4 -> element 2j in bits 0-3 of byte j, 2j+1 in bits 4-7;
+ *                 ternary -> element 4j+e in bits 2e..2e+1 of byte j (00 = 0, 01 = +1, 11 = -1).
+ *   scales_off[k] float [rows[k]]: lambda_{R^(k)} of each compacted row.
+ *   kept_off[k]   int32 [kept_groups[k]]: ascending indices of the kept groups.
+ *   cum_off[k]    int32 [G + 1]: cum[j] = number of kept groups with index < j (so group j is
+ *                 kept iff cum[j+1] > cum[j], and its first compacted row is cum[j] * g).
+ *   kcodes_off[k] the same codes in the layout the GEMM kernels stream:
+ *                 [rows[k], kernel_row_bytes], rows zero-padded to a multiple of 128 codes,
+ *                 and inside every aligned 32-bit word the fields are interleaved so that
+ *                 masking alone yields int8 lanes in reduction order: int4 -> code 4h+j of
+ *                 the word's 8 codes sits in nibble 2j+h; ternary -> code 4h+j of the word's
+ *                 16 codes sits in bits 8j+2h..8j+2h+1; int8 -> unchanged.
+ */
+typedef struct pipe_layer_layout {
+  int32_t num_groups;        /* G = O / g */
+  int32_t total_rows;        /* R_total = sum_k rows[k] = O + (K-1) * keep_groups * g */
+  int32_t canon_row_bytes;   /* I * b / 8 */
+  int32_t kernel_row_bytes;  /* roundup(I, 128) * b / 8 */
+  int32_t rows[PIPE_MAX_ORDERS];
+  int32_t kept_groups[PIPE_MAX_ORDERS];
+  int32_t branch_orders[PIPE_MAX_ORDERS]; /* the resolved [K_1..K_M] */
+  uint64_t codes_off[PIPE_MAX_ORDERS];
+  uint64_t kcodes_off[PIPE_MAX_ORDERS];
+  uint64_t scales_off[PIPE_MAX_ORDERS];
+  uint64_t kept_off[PIPE_MAX_ORDERS];
+  uint64_t cum_off[PIPE_MAX_ORDERS];
+  uint64_t blob_bytes;        /* size d_blob must have */
+  uint64_t expand_ws_bytes;   /* size d_ws must have for pipe_expand_weights */
+  uint64_t quantize_ws_bytes; /* size d_ws must have for pipe_quantize_act */
+} pipe_layer_layout;
+
+/* Sec. 3.1: gamma is the kept fraction of an order's channel groups ("150 %" = K 2, gamma
+ * 0.5 in Sec. 4.3).  Returns clamp(ceil(gamma * G - 1e-9), 1, G), evaluated in double. */
+int32_t pipe_keep_groups_from_gamma(int32_t num_groups, double gamma);
+
+/* Sec. 3.2 / Appendix A: balanced grouping with the remainder going to the earliest
+ * predictors (K_1 largest): K_m = floor(K/M) + (m <= K mod M).  Reproduces the paper's
+ * [4,4], [3,3,2], [2,2,2,2] and [2,2].  h_out: M ints. */
+pipe_status pipe_default_branches(int32_t num_orders, int32_t num_branches, int32_t* h_out);
+
+/* Validates `desc` and fills `h_out`.  Pure host function, no CUDA call. */
+pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out);
+
+/*
+ * Sec. 3.1 "Residual Expansion" (Eq. 2, Eq. 3 and the masked form that follows them), with
+ * Q of Eq. 1 per output channel (Sec. 4.1: symmetric, per-channel):
+ * for k = 1..K on the running residual r (r = W for k = 1)
+ *     a[o] = max_i |r[o,i]|
+ *     kept_k = all groups (k = 1, or keep_groups = G), else the keep_groups groups with the
+ *              largest max_{o in group} a[o], ties to the lower index, stored ascending
+ *     for rows o of kept groups:  s = a[o] / qmax (qmax = 2^(b-1) - 1, IEEE division),
+ *              q[o,i] = clamp(rne(r[o,i] / s), -qmax, qmax),  r[o,i] = fma(-s, q[o,i], r[o,i]);
+ *              a zero scale gives zero codes and an unchanged residual
+ *     rows of pruned groups keep their residual (R^k has a zero row there).
+ * d_W: float [O, I], pitch ldw, 4-byte aligned (16-byte aligned rows take the fast path).
+ * d_blob: blob_bytes bytes aligned to PIPE_BLOB_ALIGN; fully overwritten.
+ * d_ws: expand_ws_bytes bytes, 256-byte aligned; contents undefined afterwards.
+ * Non-finite weights set PIPE_ERR_NONFINITE in the device status word.
+ */
+pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const float* d_W, int64_t ldw, void* d_blob,
+                                size_t blob_bytes, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * Appendix B, Eq. 9: the layer consumes Q(x) and one scale lambda_x for the whole tensor.
+ * d_static_scale == NULL: lambda_x = max|x| / 127 (IEEE division); otherwise the given
+ * scale is used and values are clamped.  xq = clamp(rne(x / lambda_x), -127, 127);
+ * lambda_x = 0 gives all-zero codes.
+ * d_x: float [T, I] pitch ldx.  d_xq: int8 [T, I] pitch ldxq.  d_sx: 1 float (written).
+ * d_ws: quantize_ws_bytes bytes, 256-byte aligned.  T = 0 is allowed (lambda_x = 0).
+ */
+pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I, int64_t ldx, const float* d_static_scale,
+                              int8_t* d_xq, int64_t ldxq, float* d_sx, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * Appendix B, Eq. 9 without the activation function: all K orders on one input,
+ *     acc_k[t,o] = sum_i xq[t,i] * q_k[o,i]                    (exact int32)
+ *     y[t,o]     = sum_{k ascending, o kept at k} fma(float(acc_k[t,o]), s_k[o] * lambda_x, .) (+ b[o])
+ * i.e. the scale product is formed first, terms are added in ascending order starting from
+ * zero, the bias last.  d_blob: output of pipe_expand_weights for the same desc.
+ * d_xq: int8 [T, I] pitch ldxq; d_sx: 1 float; d_bias: float [O] or NULL;
+ * d_y: float [T, O] pitch ldy.  d_partials (NULL, or int32 [T, total_rows]): when given,
+ * receives acc_k[t, row] at column (sum_{j<k} rows[j]) + compacted row.  T = 0 is a no-op.
+ * PIPE_ERR_ACC_OVERFLOW if 127 * qmax * I >= 2^31.
+ */
+pipe_status pipe_expanded_linear(const pipe_layer_desc* desc, const void* d_blob, const int8_t* d_xq, int64_t T,
+                                 int64_t ldxq, const float* d_sx, const float* d_bias, float* d_y, int64_t ldy,
+                                 int32_t* d_partials, void* stream);
+
+/*
+ * Sec. 3.2 "Ensembling from Expansion", Fig. 2 and Appendix B: predictor m evaluates only the
+ * orders of its cluster (orders sum_{l<m} K_l + 1 .. sum_{l<=m} K_l) on its own input x_m
+ * with its own lambda_{x_m}; the bias belongs to predictor 1; predictor outputs are added
+ * only after the last layer.  One layer of all M predictors as ONE grouped launch.
+ * h_xq_m, h_sx_m, h_y_m: HOST arrays of M device pointers (int8 [T,I] pitch ldxq; 1 float;
+ * float [T,O] pitch ldy); inputs may alias (shared input, the first layer of a network).
+ * sum_branches != 0: only h_y_m[0] is written, with ((y_1 + y_2) + ...) + y_M.
+ * d_partials as in pipe_expanded_linear.
+ */
+pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                  int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
+                                  float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials,
+                                  void* stream);
+
+/* Which GEMM kernel the two forward calls use (process-wide, for tests and measurements):
+ * 0 = automatic, 1 = CUDA-core reference kernel, 2 = tcgen05 tensor-core kernel,
+ * 3 = small-token weight-streaming kernel.  A forced kernel that cannot run the request
+ * makes the forward call return PIPE_ERR_UNSUPPORTED. */
+pipe_status pipe_select_kernel(int32_t which);
+
+/* Number of kernels the library has launched in this process (all calls, all streams). */
+uint64_t pipe_launch_count(void);
+
+/* Synchronises `stream`, returns the device status word of the current device in
+ * *h_status (a pipe_status value; PIPE_OK if nothing went wrong) and clears it. */
+pipe_status pipe_poll_status(void* stream, int32_t* h_status);
+
+const char* pipe_status_string(pipe_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIPE_H_ */
