@@ -1,0 +1,176 @@
+// Host-side logic of libpipe: descriptor validation, blob layout, status word, small utilities.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+
+#include "pipe_common.cuh"
+
+namespace pipe {
+
+__device__ int g_status_word = 0;
+
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_kernel_choice{0};
+
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+int kernel_choice() { return g_kernel_choice.load(); }
+
+int* device_status_word() {
+  // The symbol is per device; look the address up for whichever device is current.
+  int* p = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
+  return p;
+}
+
+static uint64_t align_up64(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
+  if (!d || !out) return PIPE_ERR_INVALID_ARG;
+  if (d->out_features <= 0 || d->in_features <= 0) return PIPE_ERR_INVALID_ARG;
+  if (!(d->weight_bits == 8 || d->weight_bits == 4 || d->weight_bits == 2)) return PIPE_ERR_INVALID_ARG;
+  if (d->num_orders < 1 || d->num_orders > PIPE_MAX_ORDERS) return PIPE_ERR_INVALID_ARG;
+  if (d->group_size < 1) return PIPE_ERR_INVALID_ARG;
+  if (d->out_features % d->group_size != 0) return PIPE_ERR_SHAPE;
+  const int per_byte = 8 / d->weight_bits;
+  if (d->in_features % per_byte != 0) return PIPE_ERR_SHAPE;
+  LayerInfo L;
+  std::memset(&L, 0, sizeof(L));
+  L.O = d->out_features;
+  L.I = d->in_features;
+  L.bits = d->weight_bits;
+  L.K = d->num_orders;
+  L.g = d->group_size;
+  L.G = L.O / L.g;
+  L.n_keep = d->keep_groups;
+  L.M = d->num_branches;
+  L.qmax = (1 << (L.bits - 1)) - 1;
+  if (L.n_keep < 1 || L.n_keep > L.G) return PIPE_ERR_INVALID_ARG;
+  if (L.M < 1 || L.M > L.K) return PIPE_ERR_SHAPE;
+  // int32 partial sums: |acc| <= 127 * qmax * I must stay below 2^31 (Eq. 9 is exact integer work).
+  if (static_cast<int64_t>(127) * L.qmax * L.I >= (static_cast<int64_t>(1) << 31)) return PIPE_ERR_ACC_OVERFLOW;
+
+  int32_t bo[PIPE_MAX_ORDERS] = {0};
+  bool all_zero = true;
+  for (int m = 0; m < PIPE_MAX_ORDERS; ++m) all_zero = all_zero && d->branch_orders[m] == 0;
+  if (all_zero) {
+    for (int m = 0; m < L.M; ++m) bo[m] = L.K / L.M + (m < L.K % L.M ? 1 : 0);
+  } else {
+    int sum = 0;
+    for (int m = 0; m < PIPE_MAX_ORDERS; ++m) {
+      if (m < L.M) {
+        if (d->branch_orders[m] < 1) return PIPE_ERR_SHAPE;
+        bo[m] = d->branch_orders[m];
+        sum += bo[m];
+      } else if (d->branch_orders[m] != 0) {
+        return PIPE_ERR_SHAPE;
+      }
+    }
+    if (sum != L.K) return PIPE_ERR_SHAPE;
+  }
+  L.branch_begin[0] = 0;
+  for (int m = 0; m < L.M; ++m) L.branch_begin[m + 1] = L.branch_begin[m] + bo[m];
+
+  pipe_layer_layout& y = L.lay;
+  y.num_groups = L.G;
+  y.canon_row_bytes = static_cast<int32_t>(static_cast<int64_t>(L.I) * L.bits / 8);
+  y.kernel_row_bytes = static_cast<int32_t>(static_cast<int64_t>(round_up(L.I, kKernelKAlign)) * L.bits / 8);
+  for (int m = 0; m < L.M; ++m) y.branch_orders[m] = bo[m];
+  uint64_t off = kHeaderBytes;
+  int64_t total = 0;
+  for (int k = 0; k < L.K; ++k) {
+    const int kept = (k == 0) ? L.G : L.n_keep;
+    y.kept_groups[k] = kept;
+    y.rows[k] = kept * L.g;
+    total += y.rows[k];
+    y.codes_off[k] = off;
+    off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * y.canon_row_bytes, 256);
+    y.scales_off[k] = off;
+    off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * 4, 256);
+    y.kept_off[k] = off;
+    off = align_up64(off + static_cast<uint64_t>(kept) * 4, 256);
+    y.cum_off[k] = off;
+    off = align_up64(off + static_cast<uint64_t>(L.G + 1) * 4, 1024);
+    y.kcodes_off[k] = off;
+    off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * y.kernel_row_bytes, 1024);
+  }
+  if (total > INT32_MAX) return PIPE_ERR_SHAPE;
+  y.total_rows = static_cast<int32_t>(total);
+  y.blob_bytes = off;
+  // expansion workspace: residual [O, I4] float + absmax [O] + group score [G] + keep flag [G]
+  const uint64_t I4 = round_up(L.I, 4);
+  y.expand_ws_bytes = align_up64(static_cast<uint64_t>(L.O) * I4 * 4, 256) + align_up64(static_cast<uint64_t>(L.O) * 4, 256) +
+                      2 * align_up64(static_cast<uint64_t>(L.G) * 4, 256);
+  y.quantize_ws_bytes = 256;
+  *out = L;
+  return PIPE_OK;
+}
+
+}  // namespace pipe
+
+using namespace pipe;
+
+extern "C" {
+
+int32_t pipe_keep_groups_from_gamma(int32_t num_groups, double gamma) {
+  if (num_groups < 1) return 0;
+  double v = std::ceil(gamma * static_cast<double>(num_groups) - 1e-9);
+  if (!(v >= 1.0)) v = 1.0;
+  if (v > static_cast<double>(num_groups)) v = static_cast<double>(num_groups);
+  return static_cast<int32_t>(v);
+}
+
+pipe_status pipe_default_branches(int32_t K, int32_t M, int32_t* h_out) {
+  if (!h_out || K < 1 || K > PIPE_MAX_ORDERS) return PIPE_ERR_INVALID_ARG;
+  if (M < 1 || M > K) return PIPE_ERR_SHAPE;
+  for (int m = 0; m < M; ++m) h_out[m] = K / M + (m < K % M ? 1 : 0);
+  return PIPE_OK;
+}
+
+pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
+  if (!h_out) return PIPE_ERR_INVALID_ARG;
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  *h_out = L.lay;
+  return PIPE_OK;
+}
+
+pipe_status pipe_select_kernel(int32_t which) {
+  if (which < 0 || which > 3) return PIPE_ERR_INVALID_ARG;
+  g_kernel_choice.store(which);
+  return PIPE_OK;
+}
+
+uint64_t pipe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+pipe_status pipe_poll_status(void* stream, int32_t* h_status) {
+  if (!h_status) return PIPE_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int* word = device_status_word();
+  if (!word) return PIPE_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpyAsync(&v, word, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (v != 0 && cudaMemsetAsync(word, 0, sizeof(int), s) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (v != 0 && cudaStreamSynchronize(s) != cudaSuccess) return PIPE_ERR_CUDA;
+  *h_status = v;
+  return PIPE_OK;
+}
+
+const char* pipe_status_string(pipe_status s) {
+  switch (s) {
+    case PIPE_OK: return "ok";
+    case PIPE_ERR_INVALID_ARG: return "invalid argument";
+    case PIPE_ERR_SHAPE: return "inconsistent shape";
+    case PIPE_ERR_ALIGNMENT: return "misaligned pointer or pitch";
+    case PIPE_ERR_UNSUPPORTED: return "unsupported request";
+    case PIPE_ERR_WORKSPACE: return "blob or workspace too small";
+    case PIPE_ERR_NONFINITE: return "non-finite value in weights or activations";
+    case PIPE_ERR_ACC_OVERFLOW: return "int32 partial sum could overflow";
+    case PIPE_ERR_TIMEOUT: return "bounded device wait expired";
+    case PIPE_ERR_CUDA: return "CUDA call failed";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"
