@@ -1,0 +1,335 @@
+// pipe_expand_weights: residual expansion of a weight matrix (Sec. 3.1, Eq. 2-3 and the masked
+// form), with the per-channel symmetric quantizer of Eq. 1.
+//
+// Per order: [row absmax, only for order 1] -> [group select, orders >= 2] -> one fused pass
+// over the kept rows that divides, rounds, packs both code layouts, updates the residual with
+// one FMA per element and leaves the next order's row absmax behind.  All kernels are
+// HBM-bound streaming passes: 128-bit loads, warp-shuffle reductions, one block per row.
+#include "pipe_common.cuh"
+
+namespace pipe {
+
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, d));
+  return v;
+}
+
+// Max over the block of an unsigned value; result valid in every thread.
+__device__ __forceinline__ uint32_t block_max_u32(uint32_t v) {
+  __shared__ uint32_t part[32];
+  __shared__ uint32_t total;
+  v = warp_max_u32(v);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) part[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < (blockDim.x + 31) / 32 ? part[lane] : 0u;
+    w = warp_max_u32(w);
+    if (lane == 0) total = w;
+  }
+  __syncthreads();
+  const uint32_t r = total;
+  __syncthreads();
+  return r;
+}
+
+// |v| as an ordered unsigned key: for finite floats the order of the keys is the order of the
+// magnitudes, and every Inf/NaN maps to a key >= 0x7f800000.
+__device__ __forceinline__ uint32_t abs_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+// a[o] = max_i |src[o,i]|   (one block per row)
+__global__ void __launch_bounds__(kRowThreads) row_absmax_kernel(const float* __restrict__ src, int64_t ld, int I,
+                                                                 float* __restrict__ a, int* status) {
+  const int o = blockIdx.x;
+  const float* row = src + static_cast<int64_t>(o) * ld;
+  uint32_t m = 0;
+  const bool vec = ((reinterpret_cast<uintptr_t>(row) & 15) == 0);
+  int i0 = 0;
+  if (vec) {
+    const int n4 = I >> 2;
+    const float4* r4 = reinterpret_cast<const float4*>(row);
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+      const float4 v = __ldg(r4 + i);
+      m = max(max(m, abs_key(v.x)), max(abs_key(v.y), max(abs_key(v.z), abs_key(v.w))));
+    }
+    i0 = n4 << 2;
+  }
+  for (int i = i0 + threadIdx.x; i < I; i += blockDim.x) m = max(m, abs_key(row[i]));
+  m = block_max_u32(m);
+  if (threadIdx.x == 0) {
+    a[o] = __uint_as_float(m);
+    if (m >= 0x7f800000u) raise_status(status, PIPE_ERR_NONFINITE);
+  }
+}
+
+// score[j] = max over the g rows of group j of a[] ; one thread per group.
+__global__ void group_score_kernel(const float* __restrict__ a, int G, int g, float* __restrict__ score) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= G) return;
+  float m = 0.f;
+  for (int u = 0; u < g; ++u) m = fmaxf(m, a[static_cast<int64_t>(j) * g + u]);
+  score[j] = m;
+}
+
+// keep[j] = 1 iff fewer than n_keep groups precede j in the order (score descending, index
+// ascending).  Scores are non-negative finite floats, so the comparison is exact and the
+// result does not depend on any reduction order.
+__global__ void group_rank_kernel(const float* __restrict__ score, int G, int n_keep, int32_t* __restrict__ keep) {
+  __shared__ float tile[1024];
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const float sj = j < G ? score[j] : 0.f;
+  int rank = 0;
+  for (int base = 0; base < G; base += 1024) {
+    const int n = min(1024, G - base);
+    __syncthreads();
+    for (int t = threadIdx.x; t < n; t += blockDim.x) tile[t] = score[base + t];
+    __syncthreads();
+    if (j < G) {
+      for (int t = 0; t < n; ++t) {
+        const float si = tile[t];
+        rank += (si > sj) || (si == sj && base + t < j);
+      }
+    }
+  }
+  if (j < G) keep[j] = rank < n_keep ? 1 : 0;
+}
+
+// Exclusive prefix sum of keep[] -> cum[0..G], and the ascending list of kept groups.
+// keep == nullptr means "all groups kept".  Single block of 1024 threads.
+__global__ void __launch_bounds__(1024) group_compact_kernel(const int32_t* __restrict__ keep, int G,
+                                                             int32_t* __restrict__ cum, int32_t* __restrict__ kept) {
+  __shared__ int32_t chunk_sum[1024];
+  const int per = (G + blockDim.x - 1) / blockDim.x;
+  const int b = threadIdx.x * per, e = min(G, b + per);
+  int32_t s = 0;
+  for (int j = b; j < e; ++j) s += keep ? keep[j] : 1;
+  chunk_sum[threadIdx.x] = s;
+  __syncthreads();
+  // inclusive Hillis-Steele scan over the chunk sums
+  for (int d = 1; d < blockDim.x; d <<= 1) {
+    int32_t v = threadIdx.x >= d ? chunk_sum[threadIdx.x - d] : 0;
+    __syncthreads();
+    chunk_sum[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int32_t run = threadIdx.x == 0 ? 0 : chunk_sum[threadIdx.x - 1];
+  for (int j = b; j < e; ++j) {
+    cum[j] = run;
+    if (!keep || keep[j]) kept[run++] = j;
+  }
+  if (threadIdx.x == blockDim.x - 1) cum[G] = chunk_sum[blockDim.x - 1];
+}
+
+// Pack 16 codes (each already in [-qmax, qmax]) into the canonical and the kernel layout.
+// canonical: field e at bit e*b of the stream; kernel: see include/pipe.h.
+template <int BITS>
+__device__ __forceinline__ void pack16(const int (&q)[16], uint32_t (&canon)[4], uint32_t (&kern)[4]) {
+  if (BITS == 8) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v |= (static_cast<uint32_t>(q[4 * w + e]) & 0xffu) << (8 * e);
+      canon[w] = v;
+      kern[w] = v;
+    }
+  } else if (BITS == 4) {
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+      uint32_t c = 0, k = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t f = static_cast<uint32_t>(q[8 * w + e]) & 0xfu;
+        c |= f << (4 * e);
+        const int h = e >> 2, j = e & 3;  // code 4h+j -> nibble 2j+h
+        k |= f << (4 * (2 * j + h));
+      }
+      canon[w] = c;
+      kern[w] = k;
+    }
+  } else {
+    uint32_t c = 0, k = 0;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const uint32_t f = static_cast<uint32_t>(q[e]) & 0x3u;
+      c |= f << (2 * e);
+      const int h = e >> 2, j = e & 3;  // code 4h+j -> bits 8j+2h
+      k |= f << (8 * j + 2 * h);
+    }
+    canon[0] = c;
+    kern[0] = k;
+  }
+}
+
+struct QuantizeRowsArgs {
+  const float* src;      // residual entering this order ([O, ld_src])
+  int64_t ld_src;
+  float* dst;            // residual leaving this order ([O, ld_dst]) or nullptr (last order)
+  int64_t ld_dst;
+  float* a;              // [O] row absmax: read (this order's), overwritten (next order's) if dst
+  const int32_t* kept;   // [rows/g] ascending kept groups
+  uint8_t* codes;        // canonical [rows, canon_row_bytes]
+  uint8_t* kcodes;       // kernel layout [rows, kernel_row_bytes]
+  float* scales;         // [rows]
+  int I, g, qmax;
+  int canon_row_bytes, kernel_row_bytes;
+};
+
+// One block per compacted row: Eq. 1 on the residual, then the residual update of Eq. 3.
+template <int BITS>
+__global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const QuantizeRowsArgs p) {
+  const int n = blockIdx.x;
+  const int o = p.kept[n / p.g] * p.g + n % p.g;
+  const float* src = p.src + static_cast<int64_t>(o) * p.ld_src;
+  float* dst = p.dst ? p.dst + static_cast<int64_t>(o) * p.ld_dst : nullptr;
+  const float fq = static_cast<float>(p.qmax);
+  const float s = __fdiv_rn(p.a[o], fq);
+  __syncthreads();  // every thread has read a[o] before thread 0 overwrites it at the end
+  if (threadIdx.x == 0) p.scales[n] = s;
+  uint8_t* crow = p.codes + static_cast<int64_t>(n) * p.canon_row_bytes;
+  uint8_t* krow = p.kcodes + static_cast<int64_t>(n) * p.kernel_row_bytes;
+  constexpr int kChunkBytes = 16 * BITS / 8;  // bytes of 16 packed codes
+  constexpr int kWords = kChunkBytes / 4;
+  const int I = p.I;
+  const int I_pad = p.kernel_row_bytes * 8 / BITS;
+  const bool src_vec = (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+  const bool dst_vec = dst && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
+  const bool canon_vec = (reinterpret_cast<uintptr_t>(crow) & 3) == 0;
+  uint32_t m = 0;
+  for (int i0 = threadIdx.x * 16; i0 < I_pad; i0 += blockDim.x * 16) {
+    float v[16];
+    const bool full = i0 + 16 <= I;
+    if (full && src_vec) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float4 t = reinterpret_cast<const float4*>(src + i0)[w];  // plain load: src may alias dst
+        v[4 * w] = t.x; v[4 * w + 1] = t.y; v[4 * w + 2] = t.z; v[4 * w + 3] = t.w;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) v[e] = (i0 + e < I) ? src[i0 + e] : 0.f;
+    }
+    int q[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      float c = 0.f;
+      if (s != 0.f) {
+        c = rintf(__fdiv_rn(v[e], s));           // round half to even
+        c = fminf(fmaxf(c, -fq), fq);
+        v[e] = __fmaf_rn(-s, c, v[e]);           // exact new residual, rounded once
+      }
+      q[e] = static_cast<int>(c);
+      m = max(m, abs_key(v[e]));
+    }
+    if (dst) {
+      if (full && dst_vec) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w)
+          reinterpret_cast<float4*>(dst + i0)[w] = make_float4(v[4 * w], v[4 * w + 1], v[4 * w + 2], v[4 * w + 3]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+          if (i0 + e < I) dst[i0 + e] = v[e];
+      }
+    }
+    uint32_t canon[4], kern[4];
+    pack16<BITS>(q, canon, kern);
+    const int byte0 = i0 * BITS / 8;
+    // kernel layout: rows are padded and 16-byte aligned, always whole words
+#pragma unroll
+    for (int w = 0; w < kWords; ++w) reinterpret_cast<uint32_t*>(krow + byte0)[w] = kern[w];
+    if (i0 < I) {
+      if (full && canon_vec) {
+#pragma unroll
+        for (int w = 0; w < kWords; ++w) reinterpret_cast<uint32_t*>(crow + byte0)[w] = canon[w];
+      } else {
+        const int nbytes = min(kChunkBytes, p.canon_row_bytes - byte0);
+        for (int bb = 0; bb < nbytes; ++bb) crow[byte0 + bb] = static_cast<uint8_t>(canon[bb >> 2] >> (8 * (bb & 3)));
+      }
+    }
+  }
+  if (dst) {
+    m = block_max_u32(m);
+    if (threadIdx.x == 0) p.a[o] = __uint_as_float(m);
+  }
+}
+
+__global__ void write_header_kernel(uint32_t* hdr, pipe_layer_desc d) {
+  if (threadIdx.x == 0) {
+    hdr[0] = kBlobMagic;
+    hdr[1] = 1;  // format version
+    int32_t* o = reinterpret_cast<int32_t*>(hdr + 2);
+    o[0] = d.out_features; o[1] = d.in_features; o[2] = d.weight_bits; o[3] = d.num_orders;
+    o[4] = d.group_size; o[5] = d.keep_groups; o[6] = d.num_branches;
+    for (int m = 0; m < PIPE_MAX_ORDERS; ++m) o[7 + m] = d.branch_orders[m];
+  }
+}
+
+}  // namespace pipe
+
+using namespace pipe;
+
+extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const float* d_W, int64_t ldw, void* d_blob,
+                                           size_t blob_bytes, void* d_ws, size_t ws_bytes, void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  if (!d_W || !d_blob || !d_ws) return PIPE_ERR_INVALID_ARG;
+  if (ldw < L.I) return PIPE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_W) & 3) || (reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) ||
+      (reinterpret_cast<uintptr_t>(d_ws) & 255))
+    return PIPE_ERR_ALIGNMENT;
+  if (blob_bytes < L.lay.blob_bytes || ws_bytes < L.lay.expand_ws_bytes) return PIPE_ERR_WORKSPACE;
+  int* status = device_status_word();
+  if (!status) return PIPE_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  uint8_t* ws = static_cast<uint8_t*>(d_ws);
+  const int64_t I4 = round_up(L.I, 4);
+  float* resid = reinterpret_cast<float*>(ws);
+  uint64_t off = round_up<uint64_t>(static_cast<uint64_t>(L.O) * I4 * 4, 256);
+  float* a = reinterpret_cast<float*>(ws + off);
+  off += round_up<uint64_t>(static_cast<uint64_t>(L.O) * 4, 256);
+  float* score = reinterpret_cast<float*>(ws + off);
+  off += round_up<uint64_t>(static_cast<uint64_t>(L.G) * 4, 256);
+  int32_t* keep = reinterpret_cast<int32_t*>(ws + off);
+  uint8_t* blob = static_cast<uint8_t*>(d_blob);
+
+  write_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<uint32_t*>(blob), *desc);
+  row_absmax_kernel<<<L.O, kRowThreads, 0, s>>>(d_W, ldw, L.I, a, status);
+  count_launch(2);
+  for (int k = 0; k < L.K; ++k) {
+    int32_t* kept = reinterpret_cast<int32_t*>(blob + L.lay.kept_off[k]);
+    int32_t* cum = reinterpret_cast<int32_t*>(blob + L.lay.cum_off[k]);
+    const bool dense = (k == 0) || (L.n_keep == L.G);
+    if (!dense) {
+      group_score_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(a, L.G, L.g, score);
+      group_rank_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
+      count_launch(2);
+    }
+    group_compact_kernel<<<1, 1024, 0, s>>>(dense ? nullptr : keep, L.G, cum, kept);
+    count_launch(1);
+    QuantizeRowsArgs q;
+    q.src = (k == 0) ? d_W : resid;
+    q.ld_src = (k == 0) ? ldw : I4;
+    q.dst = (k + 1 < L.K) ? resid : nullptr;
+    q.ld_dst = I4;
+    q.a = a;
+    q.kept = kept;
+    q.codes = blob + L.lay.codes_off[k];
+    q.kcodes = blob + L.lay.kcodes_off[k];
+    q.scales = reinterpret_cast<float*>(blob + L.lay.scales_off[k]);
+    q.I = L.I; q.g = L.g; q.qmax = L.qmax;
+    q.canon_row_bytes = L.lay.canon_row_bytes;
+    q.kernel_row_bytes = L.lay.kernel_row_bytes;
+    const int rows = L.lay.rows[k];
+    if (L.bits == 8) quantize_rows_kernel<8><<<rows, kRowThreads, 0, s>>>(q);
+    else if (L.bits == 4) quantize_rows_kernel<4><<<rows, kRowThreads, 0, s>>>(q);
+    else quantize_rows_kernel<2><<<rows, kRowThreads, 0, s>>>(q);
+    count_launch(1);
+  }
+  return launch_status();
+}

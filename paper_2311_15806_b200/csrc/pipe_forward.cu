@@ -1,0 +1,87 @@
+// pipe_expanded_linear / pipe_ensemble_forward: argument checks and kernel selection.
+#include "pipe_common.cuh"
+
+namespace pipe {
+
+static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, const int8_t* const* xq,
+                               const float* const* sx, float* const* y, const int* k_begin, const int* k_end,
+                               int64_t T, int64_t ldxq, int64_t ldy, const float* d_bias, int sum_branches,
+                               int32_t* d_partials, cudaStream_t stream) {
+  if (!d_blob) return PIPE_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) return PIPE_ERR_ALIGNMENT;
+  if (T < 0 || ldxq < L.I || ldy < L.O) return PIPE_ERR_INVALID_ARG;
+  for (int m = 0; m < M; ++m) {
+    if (!sx[m]) return PIPE_ERR_INVALID_ARG;
+    if (T > 0 && !xq[m]) return PIPE_ERR_INVALID_ARG;
+    if (T > 0 && (m == 0 || !sum_branches) && !y[m]) return PIPE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(sx[m]) & 3) return PIPE_ERR_ALIGNMENT;
+    if ((m == 0 || !sum_branches) && (reinterpret_cast<uintptr_t>(y[m]) & 3)) return PIPE_ERR_ALIGNMENT;
+  }
+  if ((reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3)) return PIPE_ERR_ALIGNMENT;
+  if (T == 0) return PIPE_OK;
+
+  ForwardArgs a;
+  for (int k = 0; k < L.K; ++k) a.order[k] = order_view(L, d_blob, k);
+  a.num_branches = M;
+  for (int m = 0; m < M; ++m) {
+    BranchArgs& b = a.branch[m];
+    b.xq = xq[m];
+    b.sx = sx[m];
+    b.y = sum_branches ? y[0] : y[m];
+    b.k_begin = k_begin[m];
+    b.k_end = k_end[m];
+    b.add_bias = (m == 0);
+    b.accumulate = (sum_branches && m > 0);
+  }
+  a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
+  a.T = T; a.ldxq = ldxq; a.ldy = ldy;
+  a.bias = d_bias;
+  a.partials = d_partials;
+  a.total_rows = L.lay.total_rows;
+  a.kernel_row_bytes = L.lay.kernel_row_bytes;
+  a.canon_row_bytes = L.lay.canon_row_bytes;
+  a.status = device_status_word();
+  if (!a.status) return PIPE_ERR_CUDA;
+
+  const int choice = kernel_choice();
+  if (choice == 1) return forward_reference(a, stream);
+  if (choice == 2) return forward_tcgen05(a, stream);
+  if (choice == 3) return forward_stream(a, stream);
+  pipe_status st = PIPE_ERR_UNSUPPORTED;
+  if (T <= 16) st = forward_stream(a, stream);
+  if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05(a, stream);
+  if (st == PIPE_ERR_UNSUPPORTED) st = forward_reference(a, stream);
+  return st;
+}
+
+}  // namespace pipe
+
+using namespace pipe;
+
+extern "C" pipe_status pipe_expanded_linear(const pipe_layer_desc* desc, const void* d_blob, const int8_t* d_xq, int64_t T,
+                                            int64_t ldxq, const float* d_sx, const float* d_bias, float* d_y, int64_t ldy,
+                                            int32_t* d_partials, void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  const int kb = 0, ke = L.K;
+  return run_forward(L, d_blob, 1, &d_xq, &d_sx, &d_y, &kb, &ke, T, ldxq, ldy, d_bias, 0, d_partials,
+                     static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                             int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
+                                             float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials,
+                                             void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  if (!h_xq_m || !h_sx_m || !h_y_m) return PIPE_ERR_INVALID_ARG;
+  int kb[PIPE_MAX_ORDERS], ke[PIPE_MAX_ORDERS];
+  for (int m = 0; m < L.M; ++m) {
+    kb[m] = L.branch_begin[m];
+    ke[m] = L.branch_begin[m + 1];
+  }
+  return run_forward(L, d_blob, L.M, h_xq_m, h_sx_m, h_y_m, kb, ke, T, ldxq, ldy, d_bias, sum_branches ? 1 : 0,
+                     d_partials, static_cast<cudaStream_t>(stream));
+}
