@@ -1,0 +1,234 @@
+"""Thin ctypes binding of ``libpipe.so`` (the C ABI of ``include/pipe.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch supplies device memory and streams; tensors are passed as raw device pointers.
+There is no fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+MAX_ORDERS = 16
+BLOB_ALIGN = 1024
+
+STATUS_NAMES = ["PIPE_OK", "PIPE_ERR_INVALID_ARG", "PIPE_ERR_SHAPE", "PIPE_ERR_ALIGNMENT", "PIPE_ERR_UNSUPPORTED",
+                "PIPE_ERR_WORKSPACE", "PIPE_ERR_NONFINITE", "PIPE_ERR_ACC_OVERFLOW", "PIPE_ERR_TIMEOUT",
+                "PIPE_ERR_CUDA"]
+(PIPE_OK, PIPE_ERR_INVALID_ARG, PIPE_ERR_SHAPE, PIPE_ERR_ALIGNMENT, PIPE_ERR_UNSUPPORTED, PIPE_ERR_WORKSPACE,
+ PIPE_ERR_NONFINITE, PIPE_ERR_ACC_OVERFLOW, PIPE_ERR_TIMEOUT, PIPE_ERR_CUDA) = range(10)
+
+KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM = 0, 1, 2, 3
+
+EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
+           "pipe_quantize_act", "pipe_expanded_linear", "pipe_ensemble_forward", "pipe_select_kernel",
+           "pipe_launch_count", "pipe_poll_status", "pipe_status_string"]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("out_features", C.c_int32), ("in_features", C.c_int32), ("weight_bits", C.c_int32),
+                ("num_orders", C.c_int32), ("group_size", C.c_int32), ("keep_groups", C.c_int32),
+                ("num_branches", C.c_int32), ("branch_orders", C.c_int32 * MAX_ORDERS)]
+
+
+class LayerLayout(C.Structure):
+    _fields_ = [("num_groups", C.c_int32), ("total_rows", C.c_int32), ("canon_row_bytes", C.c_int32),
+                ("kernel_row_bytes", C.c_int32), ("rows", C.c_int32 * MAX_ORDERS),
+                ("kept_groups", C.c_int32 * MAX_ORDERS), ("branch_orders", C.c_int32 * MAX_ORDERS),
+                ("codes_off", C.c_uint64 * MAX_ORDERS), ("kcodes_off", C.c_uint64 * MAX_ORDERS),
+                ("scales_off", C.c_uint64 * MAX_ORDERS), ("kept_off", C.c_uint64 * MAX_ORDERS),
+                ("cum_off", C.c_uint64 * MAX_ORDERS), ("blob_bytes", C.c_uint64), ("expand_ws_bytes", C.c_uint64),
+                ("quantize_ws_bytes", C.c_uint64)]
+
+
+class PipeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}")
+        self.status = status
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> C.CDLL:
+    """Load libpipe.so (must have been built: ``python -m paper_2311_15806_b200.build``)."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} not found: build the CUDA library first (python -m paper_2311_15806_b200.build)")
+        L = C.CDLL(path)
+        i32, i64, p, sz = C.c_int32, C.c_int64, C.c_void_p, C.c_size_t
+        L.pipe_keep_groups_from_gamma.argtypes = [i32, C.c_double]
+        L.pipe_keep_groups_from_gamma.restype = i32
+        L.pipe_default_branches.argtypes = [i32, i32, p]
+        L.pipe_layout.argtypes = [C.POINTER(LayerDesc), C.POINTER(LayerLayout)]
+        L.pipe_expand_weights.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p, sz, p]
+        L.pipe_quantize_act.argtypes = [p, i64, i32, i64, p, p, i64, p, p, sz, p]
+        L.pipe_expanded_linear.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, p, p]
+        L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
+        L.pipe_select_kernel.argtypes = [i32]
+        L.pipe_launch_count.restype = C.c_uint64
+        L.pipe_poll_status.argtypes = [p, C.POINTER(i32)]
+        L.pipe_status_string.argtypes = [C.c_int]
+        L.pipe_status_string.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != PIPE_OK:
+        raise PipeError(status, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dp(t) -> int | None:
+    return None if t is None else int(t.data_ptr())
+
+
+def pipe_keep_groups_from_gamma(num_groups: int, gamma: float) -> int:
+    return int(lib().pipe_keep_groups_from_gamma(num_groups, float(gamma)))
+
+
+def pipe_default_branches(K: int, M: int) -> list[int]:
+    out = (C.c_int32 * MAX_ORDERS)()
+    _check(lib().pipe_default_branches(K, M, out), "pipe_default_branches")
+    return [int(out[m]) for m in range(M)]
+
+
+def make_desc(O: int, I: int, bits: int, K: int, g: int, keep_groups: int, M: int = 1,
+              branch_orders=None) -> LayerDesc:
+    d = LayerDesc()
+    d.out_features, d.in_features, d.weight_bits, d.num_orders = O, I, bits, K
+    d.group_size, d.keep_groups, d.num_branches = g, keep_groups, M
+    if branch_orders is not None:
+        for m, v in enumerate(branch_orders):
+            d.branch_orders[m] = int(v)
+    return d
+
+
+def pipe_layout(desc: LayerDesc) -> LayerLayout:
+    out = LayerLayout()
+    _check(lib().pipe_layout(C.byref(desc), C.byref(out)), "pipe_layout")
+    return out
+
+
+def pipe_expand_weights(desc: LayerDesc, W: torch.Tensor, blob: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """W: cuda float32 [O, I] (last dim contiguous); blob / ws: cuda uint8 buffers sized by pipe_layout."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.stride(1) == 1
+    _check(lib().pipe_expand_weights(C.byref(desc), _dp(W), W.stride(0), _dp(blob), blob.numel(), _dp(ws), ws.numel(),
+                                     _stream_ptr(stream)), "pipe_expand_weights")
+
+
+def pipe_quantize_act(x: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, ws: torch.Tensor,
+                      static_scale: torch.Tensor | None = None, stream=None) -> None:
+    """x: cuda float32 [T, I]; xq: cuda int8 [T, I]; sx: cuda float32 [1]; ws: cuda uint8 >= 256 bytes."""
+    assert x.is_cuda and x.dtype == torch.float32 and xq.dtype == torch.int8
+    T, I = x.shape
+    ldx = x.stride(0) if T > 1 else max(I, x.stride(0))
+    ldxq = xq.stride(0) if T > 1 else max(I, xq.stride(0))
+    _check(lib().pipe_quantize_act(_dp(x), T, I, ldx, _dp(static_scale), _dp(xq), ldxq, _dp(sx), _dp(ws), ws.numel(),
+                                   _stream_ptr(stream)), "pipe_quantize_act")
+
+
+def pipe_expanded_linear(desc: LayerDesc, blob: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, y: torch.Tensor,
+                         bias: torch.Tensor | None = None, partials: torch.Tensor | None = None, stream=None) -> None:
+    T = xq.shape[0]
+    ldxq = xq.stride(0) if T > 1 else max(xq.shape[1], xq.stride(0))
+    ldy = y.stride(0) if T > 1 else max(y.shape[1], y.stride(0))
+    _check(lib().pipe_expanded_linear(C.byref(desc), _dp(blob), _dp(xq), T, ldxq, _dp(sx), _dp(bias), _dp(y), ldy,
+                                      _dp(partials), _stream_ptr(stream)), "pipe_expanded_linear")
+
+
+def pipe_ensemble_forward(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,
+                          sum_branches: bool = False, partials: torch.Tensor | None = None, stream=None) -> None:
+    """xq_m, sx_m, y_m: sequences of M cuda tensors (xq_m entries may be the same tensor)."""
+    M = desc.num_branches
+    assert len(xq_m) == M and len(sx_m) == M and len(y_m) >= (1 if sum_branches else M)
+    T = xq_m[0].shape[0]
+    ldxq = xq_m[0].stride(0) if T > 1 else max(xq_m[0].shape[1], xq_m[0].stride(0))
+    ldy = y_m[0].stride(0) if T > 1 else max(y_m[0].shape[1], y_m[0].stride(0))
+    PA = C.c_void_p * M
+    xp = PA(*[_dp(t) for t in xq_m])
+    sp = PA(*[_dp(t) for t in sx_m])
+    yp = PA(*[(_dp(y_m[m]) if m < len(y_m) else None) for m in range(M)])
+    _check(lib().pipe_ensemble_forward(C.byref(desc), _dp(blob), xp, T, ldxq, sp, _dp(bias), yp, ldy,
+                                       1 if sum_branches else 0, _dp(partials), _stream_ptr(stream)),
+           "pipe_ensemble_forward")
+
+
+def pipe_select_kernel(which: int) -> None:
+    _check(lib().pipe_select_kernel(which), "pipe_select_kernel")
+
+
+def pipe_launch_count() -> int:
+    return int(lib().pipe_launch_count())
+
+
+def pipe_poll_status(stream=None) -> int:
+    out = C.c_int32(0)
+    _check(lib().pipe_poll_status(_stream_ptr(stream), C.byref(out)), "pipe_poll_status")
+    return int(out.value)
+
+
+def pipe_status_string(status: int) -> str:
+    return lib().pipe_status_string(status).decode()
+
+
+# ------------------------------------------------------------------------------------------------
+# Convenience: device buffers for one layer (allocation is PyTorch's job, not the library's).
+@dataclass
+class ExpandedLayer:
+    desc: LayerDesc
+    layout: LayerLayout
+    blob: torch.Tensor
+
+    def section(self, off: int, nbytes: int) -> torch.Tensor:
+        return self.blob[off:off + nbytes]
+
+    def codes(self, k: int) -> torch.Tensor:
+        n = self.layout.rows[k] * self.layout.canon_row_bytes
+        return self.section(self.layout.codes_off[k], n).view(self.layout.rows[k], self.layout.canon_row_bytes)
+
+    def kcodes(self, k: int) -> torch.Tensor:
+        n = self.layout.rows[k] * self.layout.kernel_row_bytes
+        return self.section(self.layout.kcodes_off[k], n).view(self.layout.rows[k], self.layout.kernel_row_bytes)
+
+    def scales(self, k: int) -> torch.Tensor:
+        return self.section(self.layout.scales_off[k], self.layout.rows[k] * 4).view(torch.float32)
+
+    def kept(self, k: int) -> torch.Tensor:
+        return self.section(self.layout.kept_off[k], self.layout.kept_groups[k] * 4).view(torch.int32)
+
+    def cum(self, k: int) -> torch.Tensor:
+        return self.section(self.layout.cum_off[k], (self.layout.num_groups + 1) * 4).view(torch.int32)
+
+
+def alloc_bytes(nbytes: int, device="cuda") -> torch.Tensor:
+    """uint8 device buffer whose start is aligned to BLOB_ALIGN."""
+    raw = torch.empty(int(nbytes) + BLOB_ALIGN, dtype=torch.uint8, device=device)
+    shift = (-raw.data_ptr()) % BLOB_ALIGN
+    return raw[shift:shift + int(nbytes)]
+
+
+def expand(desc: LayerDesc, W: torch.Tensor, stream=None) -> ExpandedLayer:
+    lay = pipe_layout(desc)
+    blob = alloc_bytes(lay.blob_bytes, W.device)
+    ws = alloc_bytes(lay.expand_ws_bytes, W.device)
+    pipe_expand_weights(desc, W, blob, ws, stream)
+    return ExpandedLayer(desc, lay, blob)

@@ -1,0 +1,116 @@
+"""Helpers for the GPU parity tests: run the CUDA library through its C ABI binding and compare
+with the CPU oracle.  The expected values always come from the oracle, never from the GPU."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2311_15806_b200 import binding as B
+from paper_2311_15806_b200 import build as pipe_build
+
+REL_TOL = 1e-5  # fp32 outputs: |y - y64| <= REL_TOL * sum_k |term_k|  (the stated output tolerance)
+
+
+def ensure_built():
+    pipe_build.build()
+    B.lib()
+
+
+def desc_of(O, I, bits, K, g, n_keep, M=1, branch_orders=None):
+    return B.make_desc(O, I, bits, K, g, n_keep, M, branch_orders)
+
+
+def gpu_expand(desc, W: np.ndarray) -> B.ExpandedLayer:
+    Wd = torch.from_numpy(W).cuda()
+    layer = B.expand(desc, Wd)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    return layer
+
+
+def kernel_layout_from_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """The documented streaming layout computed from int8 codes [rows, I] (see include/pipe.h)."""
+    rows, I = codes.shape
+    Ipad = (I + 127) // 128 * 128
+    c = np.zeros((rows, Ipad), np.int8)
+    c[:, :I] = codes
+    if bits == 8:
+        return c.view(np.uint8)
+    per_word = 32 // bits
+    u = (c.astype(np.int32) & ((1 << bits) - 1)).astype(np.uint32).reshape(rows, Ipad // per_word, per_word // 4, 4)
+    word = np.zeros((rows, Ipad // per_word), np.uint32)
+    for h in range(per_word // 4):
+        for j in range(4):
+            shift = (4 * (2 * j + h)) if bits == 4 else (8 * j + 2 * h)
+            word |= u[:, :, h, j] << np.uint32(shift)
+    return word.view(np.uint8).reshape(rows, -1)
+
+
+def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_layout=True):
+    """Bit-exact: kept lists, prefix counts, canonical packed codes, scales, streaming layout."""
+    lay = layer.layout
+    assert lay.total_rows == e.R_total
+    for k in range(e.K):
+        kept = layer.kept(k).cpu().numpy()
+        np.testing.assert_array_equal(kept, e.order_kept(k), err_msg=f"kept groups, order {k}")
+        flags = np.zeros(e.G, np.int32)
+        flags[e.order_kept(k)] = 1
+        np.testing.assert_array_equal(layer.cum(k).cpu().numpy(), np.concatenate([[0], np.cumsum(flags)]))
+        np.testing.assert_array_equal(layer.scales(k).cpu().numpy().view(np.uint32), e.order_scales(k).view(np.uint32),
+                                      err_msg=f"scales, order {k}")
+        np.testing.assert_array_equal(layer.codes(k).cpu().numpy(), e.packed(k), err_msg=f"codes, order {k}")
+        if check_kernel_layout:
+            np.testing.assert_array_equal(layer.kcodes(k).cpu().numpy(), kernel_layout_from_codes(e.order_codes(k), e.bits),
+                                          err_msg=f"streaming layout, order {k}")
+
+
+def gpu_quantize(x: np.ndarray, static_scale=None, xd=None):
+    xd = torch.from_numpy(x).cuda() if xd is None else xd
+    xq = torch.empty(xd.shape, dtype=torch.int8, device="cuda")
+    sx = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws = B.alloc_bytes(256)
+    ss = None if static_scale is None else torch.tensor([static_scale], dtype=torch.float32, device="cuda")
+    B.pipe_quantize_act(xd, xq, sx, ws, ss)
+    torch.cuda.synchronize()
+    return xq, sx
+
+
+def gpu_linear(layer, xq, sx, bias=None, want_partials=True, kernel=B.KERNEL_AUTO):
+    T = xq.shape[0]
+    y = torch.full((T, layer.desc.out_features), float("nan"), dtype=torch.float32, device="cuda")
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
+    bd = None if bias is None else torch.from_numpy(bias).cuda()
+    B.pipe_select_kernel(kernel)
+    try:
+        B.pipe_expanded_linear(layer.desc, layer.blob, xq, sx, y, bd, part)
+        torch.cuda.synchronize()
+    finally:
+        B.pipe_select_kernel(B.KERNEL_AUTO)
+    assert B.pipe_poll_status() == B.PIPE_OK
+    return y.cpu().numpy(), (None if part is None else part.cpu().numpy())
+
+
+def gpu_ensemble(layer, xq_m, sx_m, bias=None, sum_branches=False, want_partials=True, kernel=B.KERNEL_AUTO):
+    M = layer.desc.num_branches
+    T = xq_m[0].shape[0]
+    O = layer.desc.out_features
+    n_out = 1 if sum_branches else M
+    ys = [torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda") for _ in range(n_out)]
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
+    bd = None if bias is None else torch.from_numpy(bias).cuda()
+    B.pipe_select_kernel(kernel)
+    try:
+        B.pipe_ensemble_forward(layer.desc, layer.blob, xq_m, sx_m, ys, bd, sum_branches, part)
+        torch.cuda.synchronize()
+    finally:
+        B.pipe_select_kernel(B.KERNEL_AUTO)
+    assert B.pipe_poll_status() == B.PIPE_OK
+    return [y.cpu().numpy() for y in ys], (None if part is None else part.cpu().numpy())
+
+
+def assert_outputs_close(y_gpu: np.ndarray, f, what=""):
+    """f: oracle Forward (y, y64, yabs).  The stated tolerance, element-wise, against the binary64 sum."""
+    err = np.abs(y_gpu.astype(np.float64) - f.y64)
+    bound = REL_TOL * f.yabs + 1e-30
+    bad = err > bound
+    assert not bad.any(), f"{what}: {bad.sum()} outputs beyond 1e-5 relative; worst {np.max(err / (f.yabs + 1e-30)):.3e}"

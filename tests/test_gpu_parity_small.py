@@ -1,0 +1,207 @@
+"""GPU-vs-oracle parity on oracle-sized cases: every stage, element by element.
+Integer stages (codes, scales, kept lists, int32 partial sums, activation codes) must be bit-exact;
+fp32 outputs within 1e-5 relative of the binary64 sum (and, as a stretch, bit-equal to the oracle)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2311_15806_b200 import binding as B
+from paper_2311_15806_b200 import synth
+from tests import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_AUTO]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    H.ensure_built()
+
+
+def _w(rng, O, I, heavy=False):
+    W = (rng.standard_t(4, size=(O, I)) if heavy else rng.standard_normal((O, I))) * 0.02
+    W *= np.exp(rng.uniform(np.log(0.25), np.log(4.0), size=(O, 1)))
+    return W.astype(np.float32)
+
+
+# shapes span several tiles and ragged tails in every dimension; g in {1, 4, 8, 16}
+EXPAND_CASES = [
+    # O,   I,   bits, K, g,  n_keep
+    (256, 256, 8, 2, 8, 32),
+    (96, 200, 4, 3, 8, 3),
+    (80, 1000, 4, 4, 16, 2),
+    (64, 328, 2, 5, 4, 5),
+    (48, 130, 8, 3, 1, 7),
+    (304, 4112, 4, 3, 8, 19),
+    (40, 36, 2, 8, 8, 2),
+    (8, 8, 4, 2, 8, 1),
+]
+
+
+@pytest.mark.parametrize("O,I,bits,K,g,n_keep", EXPAND_CASES)
+def test_expand_weights_bit_exact(oracle, O, I, bits, K, g, n_keep):
+    rng = np.random.default_rng(O * 31 + I)
+    W = _w(rng, O, I, heavy=True)
+    W[O // 2] = 0.0                      # an all-zero row
+    W[1] = W[0]                          # equal rows
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep), W)
+    H.assert_expansion_matches(layer, e, oracle)
+
+
+def test_expand_weights_strided_and_tied_groups(oracle):
+    rng = np.random.default_rng(5)
+    O, I, g = 64, 72, 8
+    big = rng.standard_normal((O, I + 9)).astype(np.float32)
+    # tie the scores of several groups: copy group 1 into groups 3 and 6
+    big[3 * g:4 * g] = big[g:2 * g]
+    big[6 * g:7 * g] = big[g:2 * g]
+    Wd = torch.from_numpy(big).cuda()[:, 3:3 + I]            # pitch I+9, misaligned rows
+    W = np.ascontiguousarray(big[:, 3:3 + I])
+    d = H.desc_of(O, I, 4, 3, g, 2)
+    layer = B.expand(d, Wd)
+    torch.cuda.synchronize()
+    H.assert_expansion_matches(layer, oracle.expand(W, 4, 3, g, 2), oracle)
+
+
+def test_expand_weights_is_deterministic(oracle):
+    rng = np.random.default_rng(6)
+    W = _w(rng, 128, 512)
+    d = H.desc_of(128, 512, 4, 4, 8, 8)
+    blobs = [H.gpu_expand(d, W).blob.cpu().numpy() for _ in range(3)]
+    lay = B.pipe_layout(d)
+    for k in range(4):
+        for off, n in [(lay.codes_off[k], lay.rows[k] * lay.canon_row_bytes), (lay.scales_off[k], lay.rows[k] * 4),
+                       (lay.kcodes_off[k], lay.rows[k] * lay.kernel_row_bytes)]:
+            assert (blobs[0][off:off + n] == blobs[1][off:off + n]).all()
+            assert (blobs[0][off:off + n] == blobs[2][off:off + n]).all()
+
+
+def test_nonfinite_weights_raise_device_status():
+    W = np.ones((16, 32), np.float32)
+    W[3, 5] = np.nan
+    d = H.desc_of(16, 32, 4, 2, 8, 1)
+    B.expand(d, torch.from_numpy(W).cuda())
+    assert B.pipe_poll_status() == B.PIPE_ERR_NONFINITE
+    assert B.pipe_poll_status() == B.PIPE_OK   # cleared by the poll
+
+
+@pytest.mark.parametrize("T,I", [(64, 256), (1, 4096), (7, 33), (130, 1000), (300, 2304), (0, 64)])
+def test_quantize_act_bit_exact(oracle, T, I):
+    rng = np.random.default_rng(T * 7 + I)
+    x = (rng.standard_normal((T, I)) * 2.5).astype(np.float32)
+    if T > 2:
+        x[:, ::37] *= 20
+    xq, sx = H.gpu_quantize(x)
+    if T == 0:
+        assert float(sx.cpu()) == 0.0
+        return
+    xq_o, sx_o = oracle.quantize_act(x)
+    assert sx.cpu().numpy().view(np.uint32)[0] == np.float32(sx_o).view(np.uint32)
+    np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+
+
+def test_quantize_act_static_scale_zero_and_strided(oracle):
+    rng = np.random.default_rng(11)
+    x = (rng.standard_normal((9, 50)) * 100).astype(np.float32)
+    xq, sx = H.gpu_quantize(x, static_scale=0.5)
+    xq_o, _ = oracle.quantize_act(x, static_scale=0.5)
+    np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+    xq, sx = H.gpu_quantize(np.zeros((5, 20), np.float32))
+    assert float(sx.cpu()) == 0.0 and not xq.cpu().numpy().any()
+    big = torch.from_numpy(rng.standard_normal((12, 77)).astype(np.float32)).cuda()
+    view = big[:, 5:5 + 64]
+    xq, sx = H.gpu_quantize(None, xd=view)
+    xq_o, sx_o = oracle.quantize_act(view.cpu().numpy())
+    np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+    bad = np.ones((4, 16), np.float32)
+    bad[2, 3] = np.inf
+    H.gpu_quantize(bad)
+    assert B.pipe_poll_status() == B.PIPE_ERR_NONFINITE
+
+
+FORWARD_CASES = [
+    # O,   I,    T,  bits, K, g, n_keep, M
+    (256, 256, 64, 8, 2, 8, 32, 1),
+    (96, 200, 70, 4, 3, 8, 3, 1),
+    (192, 1000, 150, 4, 4, 8, 12, 2),
+    (128, 328, 33, 2, 8, 16, 2, 4),
+    (48, 130, 5, 8, 3, 1, 7, 3),
+    (304, 2304, 131, 4, 3, 8, 19, 1),
+    (264, 512, 1, 4, 4, 8, 17, 2),
+    (264, 512, 16, 4, 4, 8, 17, 2),
+]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", FORWARD_CASES)
+def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
+    rng = np.random.default_rng(O + 3 * I + 5 * T)
+    W = _w(rng, O, I, heavy=(bits == 2))
+    bias = rng.standard_normal(O).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    d = H.desc_of(O, I, bits, K, g, n_keep, M)
+    layer = H.gpu_expand(d, W)
+    H.assert_expansion_matches(layer, e, oracle, check_kernel_layout=False)
+    split = [layer.layout.branch_orders[m] for m in range(M)]
+    xs = [(rng.standard_normal((T, I)) * (1 + m)).astype(np.float32) for m in range(M)]
+    q = [H.gpu_quantize(x) for x in xs]
+    qo = [oracle.quantize_act(x) for x in xs]
+    for (xq, sx), (xq_o, sx_o) in zip(q, qo):
+        np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+
+    # (1) the whole expanded layer on one input
+    y, part = H.gpu_linear(layer, q[0][0], q[0][1], bias, kernel=kernel)
+    f = oracle.forward(e, qo[0][0], qo[0][1], bias=bias)
+    np.testing.assert_array_equal(part, f.partials)
+    H.assert_outputs_close(y, f, "expanded_linear")
+    np.testing.assert_array_equal(y.view(np.uint32), f.y.view(np.uint32))   # same operation order => same bits
+
+    # (2) grouped ensemble, distinct inputs, per-branch outputs
+    ys, part = H.gpu_ensemble(layer, [a for a, _ in q], [b for _, b in q], bias, kernel=kernel)
+    k0 = 0
+    want_part = np.zeros_like(part)
+    for m in range(M):
+        fm = oracle.forward(e, qo[m][0], qo[m][1], k0, k0 + split[m], bias=bias if m == 0 else None)
+        H.assert_outputs_close(ys[m], fm, f"branch {m}")
+        np.testing.assert_array_equal(ys[m].view(np.uint32), fm.y.view(np.uint32))
+        lo, hi = e.row_off(k0), e.row_off(k0 + split[m])
+        want_part[:, lo:hi] = fm.partials[:, lo:hi]
+        k0 += split[m]
+    np.testing.assert_array_equal(part, want_part)
+
+    # (3) shared input, summed after the layer: partials equal those of the un-split layer
+    ys, part = H.gpu_ensemble(layer, [q[0][0]] * M, [q[0][1]] * M, bias, sum_branches=True, kernel=kernel)
+    np.testing.assert_array_equal(part, f.partials)
+    y_o, _ = oracle.ensemble(e, np.stack([qo[0][0]] * M), [qo[0][1]] * M, split, bias=bias, sum_branches=True)
+    np.testing.assert_array_equal(ys[0].view(np.uint32), y_o.view(np.uint32))
+    assert (np.abs(ys[0] - f.y64) <= 2e-5 * f.yabs + 1e-30).all()
+
+
+def test_forward_zero_tokens_and_strided_io(oracle):
+    rng = np.random.default_rng(77)
+    O, I, T = 64, 96, 10
+    W = _w(rng, O, I)
+    e = oracle.expand(W, 4, 2, 8, 4)
+    layer = H.gpu_expand(H.desc_of(O, I, 4, 2, 8, 4), W)
+    x = rng.standard_normal((T, I)).astype(np.float32)
+    xq_o, sx_o = oracle.quantize_act(x)
+    xq_big = torch.zeros((T, I + 32), dtype=torch.int8, device="cuda")
+    xq_big[:, 16:16 + I] = torch.from_numpy(xq_o).cuda()
+    y_big = torch.zeros((T, O + 8), dtype=torch.float32, device="cuda")
+    sx = torch.tensor([sx_o], dtype=torch.float32, device="cuda")
+    B.pipe_expanded_linear(layer.desc, layer.blob, xq_big[:, 16:16 + I], sx, y_big[:, 4:4 + O])
+    torch.cuda.synchronize()
+    f = oracle.forward(e, xq_o, sx_o)
+    np.testing.assert_array_equal(y_big[:, 4:4 + O].cpu().numpy().view(np.uint32), f.y.view(np.uint32))
+    assert not y_big[:, :4].any() and not y_big[:, 4 + O:].any()
+    empty = torch.empty((0, I), dtype=torch.int8, device="cuda")
+    B.pipe_expanded_linear(layer.desc, layer.blob, empty, sx, torch.empty((0, O), dtype=torch.float32, device="cuda"))
+    assert B.pipe_poll_status() == B.PIPE_OK
+
+
+def test_launch_counter_moves():
+    before = B.pipe_launch_count()
+    H.gpu_quantize(np.ones((4, 16), np.float32))
+    assert B.pipe_launch_count() >= before + 2
