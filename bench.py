@@ -136,7 +136,6 @@ def time_oracle_sample(spec, target_seconds: float = 12.0):
     n = min(spec.T, 8)
     t_small = max(run(n), 1e-4)
     n_big = int(min(spec.T, max(n, n * target_seconds / t_small)))
-    n_big = min(n_big, 4096)
     t_big = run(n_big) if n_big > n else t_small
     per_token = t_big / n_big
     est_step = t_expand + per_token * spec.T
