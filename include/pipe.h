@@ -133,6 +133,35 @@ pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const float* d_W, i
                                 size_t blob_bytes, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
+ * pipe_expand_weights for callers that must not allocate device memory.  (The paper has no
+ * counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs after the host application has handed all of the GPU's memory
+ * to its own pool or has frozen its memory budget -- an inference-server plug-in re-expanding
+ * a layer when new weights are swapped in, say -- and code that must not stall the device:
+ * cudaMalloc and cudaFree synchronise the whole GPU, so an allocation on the weight-update path
+ * would stop the streams that are serving requests.  Such a caller cannot produce the d_ws
+ * buffer that pipe_expand_weights asks for.
+ *
+ * Here the workspace is a fixed array of PIPE_STATIC_SCRATCH_BYTES inside the library itself
+ * (every GPU that loads the library holds that much until the process exits).  The call computes
+ * exactly what pipe_expand_weights computes, into the caller's d_blob, and neither it nor
+ * anything it calls allocates or frees memory.
+ *   - Limit: the layer's expand_ws_bytes (see pipe_layout; about 4*O*I bytes) must not exceed
+ *     PIPE_STATIC_SCRATCH_BYTES, otherwise PIPE_ERR_WORKSPACE is returned and nothing is queued.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call here).  Make that first call before any stream capture begins.
+ *   - All calls share the one array.  It keeps whatever the previous call left in it; this call
+ *     overwrites every part before reading it, so nothing needs clearing.  Two calls whose GPU
+ *     work overlaps (different streams, or different host threads) race on the array: run them
+ *     one after the other on the device.
+ * Arguments, alignment rules and device-side errors are those of pipe_expand_weights.
+ */
+#define PIPE_STATIC_SCRATCH_BYTES (4u << 20)
+pipe_status pipe_expand_weights_static(const pipe_layer_desc* desc, const float* d_W, int64_t ldw, void* d_blob,
+                                       size_t blob_bytes, void* stream);
+
+/*
  * Appendix B, Eq. 9: the layer consumes Q(x) and one scale lambda_x for the whole tensor.
  * d_static_scale == NULL: lambda_x = max|x| / 127 (IEEE division); otherwise the given
  * scale is used and values are clamped.  xq = clamp(rne(x / lambda_x), -127, 127);

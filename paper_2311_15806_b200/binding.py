@@ -25,7 +25,10 @@ STATUS_NAMES = ["PIPE_OK", "PIPE_ERR_INVALID_ARG", "PIPE_ERR_SHAPE", "PIPE_ERR_A
 
 KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM = 0, 1, 2, 3
 
+STATIC_SCRATCH_BYTES = 4 << 20
+
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
+           "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_expanded_linear", "pipe_ensemble_forward", "pipe_select_kernel",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string"]
 
@@ -74,6 +77,7 @@ def lib() -> C.CDLL:
         L.pipe_default_branches.argtypes = [i32, i32, p]
         L.pipe_layout.argtypes = [C.POINTER(LayerDesc), C.POINTER(LayerLayout)]
         L.pipe_expand_weights.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p, sz, p]
+        L.pipe_expand_weights_static.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p]
         L.pipe_quantize_act.argtypes = [p, i64, i32, i64, p, p, i64, p, p, sz, p]
         L.pipe_expanded_linear.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, p, p]
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
@@ -133,6 +137,15 @@ def pipe_expand_weights(desc: LayerDesc, W: torch.Tensor, blob: torch.Tensor, ws
     assert W.is_cuda and W.dtype == torch.float32 and W.stride(1) == 1
     _check(lib().pipe_expand_weights(C.byref(desc), _dp(W), W.stride(0), _dp(blob), blob.numel(), _dp(ws), ws.numel(),
                                      _stream_ptr(stream)), "pipe_expand_weights")
+
+
+def pipe_expand_weights_static(desc: LayerDesc, W: torch.Tensor, blob: torch.Tensor, stream=None) -> None:
+    """pipe_expand_weights without a workspace argument: the library's fixed internal array
+    (STATIC_SCRATCH_BYTES) is used instead, so the call allocates nothing.  Raises PipeError
+    (PIPE_ERR_WORKSPACE) when the layer is too large for that array."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.stride(1) == 1
+    _check(lib().pipe_expand_weights_static(C.byref(desc), _dp(W), W.stride(0), _dp(blob), blob.numel(),
+                                            _stream_ptr(stream)), "pipe_expand_weights_static")
 
 
 def pipe_quantize_act(x: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, ws: torch.Tensor,

@@ -5,6 +5,8 @@
 // over the kept rows that divides, rounds, packs both code layouts, updates the residual with
 // one FMA per element and leaves the next order's row absmax behind.  All kernels are
 // HBM-bound streaming passes: 128-bit loads, warp-shuffle reductions, one block per row.
+#include <mutex>
+
 #include "pipe_common.cuh"
 
 namespace pipe {
@@ -332,4 +334,50 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     count_launch(1);
   }
   return launch_status();
+}
+
+// ------------------------------------------------------------------------------------------------
+// pipe_expand_weights_static: the same expansion for callers that cannot allocate device memory.
+// Its workspace is the fixed array below, which is part of the library image: every GPU that
+// loads the library holds PIPE_STATIC_SCRATCH_BYTES for it until the process exits.
+namespace {
+
+static __device__ __align__(256) unsigned char g_expand_scratch[PIPE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the array on the current device.  In host code the name g_expand_scratch is
+// only a handle for the runtime, not an address a kernel could use; the address has to be asked
+// for, once per device, while that device is current.
+pipe_status static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PIPE_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_expand_scratch) != cudaSuccess || !p) return PIPE_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return PIPE_OK;
+}
+
+}  // namespace
+
+extern "C" pipe_status pipe_expand_weights_static(const pipe_layer_desc* desc, const float* d_W, int64_t ldw,
+                                                  void* d_blob, size_t blob_bytes, void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  // the layer's workspace (fp32 residual + per-row and per-group arrays) must fit the fixed array
+  if (L.lay.expand_ws_bytes > static_cast<uint64_t>(PIPE_STATIC_SCRATCH_BYTES)) return PIPE_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  st = static_scratch(&scratch);
+  if (st != PIPE_OK) return st;
+  // Nothing in the workspace has to start at zero: the residual, the row maxima, the group scores
+  // and the keep flags are all written by this call before it reads them, so what an earlier
+  // call left behind is simply overwritten.
+  return pipe_expand_weights(desc, d_W, ldw, d_blob, blob_bytes, scratch, PIPE_STATIC_SCRATCH_BYTES, stream);
 }
