@@ -11,7 +11,7 @@ from tests import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_AUTO]
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_AUTO]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -131,6 +131,11 @@ FORWARD_CASES = [
     (304, 2304, 131, 4, 3, 8, 19, 1),
     (264, 512, 1, 4, 4, 8, 17, 2),
     (264, 512, 16, 4, 4, 8, 17, 2),
+    (128, 128, 128, 8, 1, 8, 16, 1),
+    (264, 1008, 700, 4, 4, 8, 17, 2),
+    (512, 272, 1000, 2, 8, 16, 8, 4),
+    (200, 144, 260, 8, 3, 8, 5, 3),
+    (640, 640, 129, 4, 6, 32, 3, 1),
 ]
 
 
@@ -152,7 +157,12 @@ def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
         np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
 
     # (1) the whole expanded layer on one input
-    y, part = H.gpu_linear(layer, q[0][0], q[0][1], bias, kernel=kernel)
+    try:
+        y, part = H.gpu_linear(layer, q[0][0], q[0][1], bias, kernel=kernel)
+    except B.PipeError as ex:
+        if ex.status == B.PIPE_ERR_UNSUPPORTED and kernel != B.KERNEL_AUTO:
+            pytest.skip("this kernel does not take this shape (the automatic choice falls back)")
+        raise
     f = oracle.forward(e, qo[0][0], qo[0][1], bias=bias)
     np.testing.assert_array_equal(part, f.partials)
     H.assert_outputs_close(y, f, "expanded_linear")
