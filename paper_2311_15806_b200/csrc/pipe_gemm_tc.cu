@@ -259,11 +259,151 @@ __device__ __forceinline__ void unpack_role(const Params& p, const UnpackCtx& u)
   }
 }
 
+struct EpiCtx {
+  uint32_t tmem_base, tfull0, tempty0;
+  volatile int* abort_flag;
+  int warp, lane;
+  int16_t* colmap;
+  int32_t* crowmap;
+  float* cscale;
+};
+
+// Epilogue role (4 warps, one TMEM lane quarter each; a lane owns one token row of the tile).
+// NKMAX = most orders a branch may have at this channel-block width (NKMAX * BN = 256).
+// Before the accumulators are ready the warp prepares, from the prefix counts, where each
+// (order, 8-channel chunk) sits in the accumulator and the products s_k * lambda_x of all stacked
+// rows, so that the drain loop has no dependent global loads.
+template <int NKMAX>
+__device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
+  constexpr int NCH = 32 / NKMAX;   // 8-channel chunks per channel block (BN / 8)
+  constexpr int CH = 8 / NKMAX;     // chunks drained per iteration (64 accumulator registers)
+  const int q = x.warp & 3;         // TMEM lane quarter this warp may read
+  const int lane = x.lane;
+  const int row_in_tile = q * 32 + lane;
+  uint32_t tcount = 0;
+  const bool y_vec = (p.f.ldy % 4 == 0);
+  for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
+    TileMeta t;
+    decode_tile(p, tile, t);
+    const BranchArgs& br = p.f.branch[t.m];
+    const int buf = tcount & 1;
+    const uint32_t aph = (tcount >> 1) & 1;
+    const float sx = __ldg(br.sx);
+    const int c0 = t.cb * p.BN;
+    const int c1 = min(c0 + p.BN, p.f.O);
+    const int nch = (c1 - c0) >> 3;
+    const int n_total = t.rowbase[kMaxClusterOrders];
+    __syncwarp();
+    {
+      const int ko = lane / NCH, cc = lane % NCH;
+      int col = -1, crow = 0;
+      if (ko < t.nk && cc < nch) {
+        int rb = 0, st = 0;
+        const int32_t* cum = nullptr;
+#pragma unroll
+        for (int u = 0; u < NKMAX; ++u)
+          if (u == ko) {
+            rb = t.rowbase[u];
+            st = t.start[u];
+            cum = p.f.order[t.k0 + u].cum;
+          }
+        const int c = c0 + 8 * cc;
+        const int j = c / p.f.g;
+        const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+        if (hi > lo) {
+          crow = lo * p.f.g + c % p.f.g;
+          col = rb + crow - st;
+        }
+      }
+      x.colmap[lane] = static_cast<int16_t>(col);
+      x.crowmap[lane] = crow;
+      for (int r = lane; r < n_total; r += 32) {
+        int rb = 0, st = t.start[0];
+        const float* sc = p.f.order[t.k0].scales;
+#pragma unroll
+        for (int u = 1; u < NKMAX; ++u)
+          if (u < t.nk && r >= t.rowbase[u]) {
+            rb = t.rowbase[u];
+            st = t.start[u];
+            sc = p.f.order[t.k0 + u].scales;
+          }
+        x.cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
+      }
+    }
+    __syncwarp();
+    if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int64_t tok = static_cast<int64_t>(t.tt) * kTileM + row_in_tile;
+    const bool tok_ok = tok < p.f.T;
+    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
+    float* yrow = br.y + tok * p.f.ldy;
+    const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
+    for (int cg = 0; cg < nch; cg += CH) {
+      int acc[CH][NKMAX][8];
+      int cols[CH][NKMAX];
+#pragma unroll
+      for (int u = 0; u < CH; ++u)
+#pragma unroll
+        for (int ko = 0; ko < NKMAX; ++ko) {
+          cols[u][ko] = (cg + u < nch) ? x.colmap[ko * NCH + cg + u] : -1;
+          if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
+        }
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int u = 0; u < CH; ++u) {
+        if (cg + u >= nch) continue;
+        const int c = c0 + 8 * (cg + u);
+        float y[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) y[e] = 0.f;
+#pragma unroll
+        for (int ko = 0; ko < NKMAX; ++ko) {
+          if (cols[u][ko] < 0) continue;
+          const float* cs = x.cscale + cols[u][ko];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
+            acc[u][ko][e] = a;
+            y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+          }
+          if (p.f.partials && tok_ok) {
+            int32_t* prow = p.f.partials + tok * p.f.total_rows + p.f.order[t.k0 + ko].row_off + x.crowmap[ko * NCH + cg + u];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
+          }
+        }
+        if (tok_ok) {
+          if (br.add_bias && p.f.bias) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], __ldg(p.f.bias + c + e));
+          }
+          if (br.accumulate) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(yrow[c + e], y[e]);
+          }
+          if (vec_ok) {
+            *reinterpret_cast<float4*>(yrow + c) = make_float4(y[0], y[1], y[2], y[3]);
+            *reinterpret_cast<float4*>(yrow + c + 4) = make_float4(y[4], y[5], y[6], y[7]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) yrow[c + e] = y[e];
+          }
+        }
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    mbar_arrive(x.tempty0 + 8u * buf);
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[4 * 8 + 4];   // full[8] ready[8] empty[8] | tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
+  __shared__ int16_t epi_colmap[4][32];     // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ int32_t epi_crowmap[4][32];    // ... and its compacted row in that order
+  __shared__ float epi_cscale[4][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
 
   volatile int* abort_flag = &abort_flag_s;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -320,11 +460,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
           if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.f.status)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), tx);
           tma_load_2d(a_tile(s), &p.tmap_a[t.m], kb * kKStep, t.tt * kTileM, full_bar(s));
-          for (int ko = 0; ko < t.nk; ++ko) {
-            const int nb = t.boxbase[ko + 1] - t.boxbase[ko];
-            for (int b = 0; b < nb; ++b)
-              tma_load_2d(stg(s) + (t.boxbase[ko] + b) * p.box_bytes, &p.tmap_b[t.k0 + ko], kb * p.packed_row_bytes,
-                          t.start[ko] + b * kBoxRows, full_bar(s));
+          int box = 0;
+#pragma unroll
+          for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
+            if (ko < t.nk) {
+              const int nb = (t.n[ko] + kBoxRows - 1) / kBoxRows;
+              for (int b = 0; b < nb; ++b, ++box)
+                tma_load_2d(stg(s) + box * p.box_bytes, &p.tmap_b[t.k0 + ko], kb * p.packed_row_bytes,
+                            t.start[ko] + b * kBoxRows, full_bar(s));
+            }
           }
         }
       }
@@ -385,88 +529,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     else unpack_role<2>(p, u);
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;               // TMEM lane quarter this warp may read
-    const int row_in_tile = q * 32 + lane;
-    uint32_t tcount = 0;
-    bool ok = true;
-    const bool y_vec = (p.f.ldy % 4 == 0);
-    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
-      TileMeta t;
-      decode_tile(p, tile, t);
-      const BranchArgs& br = p.f.branch[t.m];
-      const int buf = tcount & 1;
-      const uint32_t aph = (tcount >> 1) & 1;
-      const float sx = __ldg(br.sx);
-      if (!mbar_wait(tfull_bar(buf), aph, abort_flag, p.f.status)) { ok = false; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int64_t tok = static_cast<int64_t>(t.tt) * kTileM + row_in_tile;
-      const bool tok_ok = tok < p.f.T;
-      const int c0 = t.cb * p.BN;
-      const int c1 = min(c0 + p.BN, p.f.O);
-      const uint32_t tbase = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
-      float* yrow = br.y + tok * p.f.ldy;
-      const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
-      for (int c = c0; c < c1; c += 8) {
-        const int j = c / p.f.g, cin = c % p.f.g;
-        int acc[kMaxClusterOrders][8];
-        int crow[kMaxClusterOrders];
-#pragma unroll
-        for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
-          crow[ko] = -1;
-          if (ko < t.nk) {
-            const int32_t* cum = p.f.order[t.k0 + ko].cum;
-            const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-            if (hi > lo) {
-              crow[ko] = lo * p.f.g + cin;
-              tmem_ld8(tbase + t.rowbase[ko] + (crow[ko] - t.start[ko]), acc[ko]);
-            }
-          }
-        }
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        float y[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) y[e] = 0.f;
-#pragma unroll
-        for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
-          if (ko < t.nk && crow[ko] >= 0) {
-            const OrderView& ov = p.f.order[t.k0 + ko];
-            const float4 s0 = __ldg(reinterpret_cast<const float4*>(ov.scales + crow[ko]));
-            const float4 s1 = __ldg(reinterpret_cast<const float4*>(ov.scales + crow[ko]) + 1);
-            const float sc[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int a = acc[ko][e] >> p.shift;   // exact: the accumulator holds 2^shift times the sum
-              acc[ko][e] = a;
-              y[e] = __fmaf_rn(__int2float_rn(a), __fmul_rn(sc[e], sx), y[e]);
-            }
-            if (p.f.partials && tok_ok) {
-              int32_t* prow = p.f.partials + tok * p.f.total_rows + ov.row_off + crow[ko];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) prow[e] = acc[ko][e];
-            }
-          }
-        }
-        if (tok_ok) {
-          if (br.add_bias && p.f.bias) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], __ldg(p.f.bias + c + e));
-          }
-          if (br.accumulate) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(yrow[c + e], y[e]);
-          }
-          if (vec_ok) {
-            *reinterpret_cast<float4*>(yrow + c) = make_float4(y[0], y[1], y[2], y[3]);
-            *reinterpret_cast<float4*>(yrow + c + 4) = make_float4(y[4], y[5], y[6], y[7]);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) yrow[c + e] = y[e];
-          }
-        }
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(tempty_bar(buf));
-    }
+    EpiCtx e;
+    e.tmem_base = tmem_base;
+    e.tfull0 = tfull_bar(0);
+    e.tempty0 = tempty_bar(0);
+    e.abort_flag = abort_flag;
+    e.warp = warp;
+    e.lane = lane;
+    e.colmap = epi_colmap[warp - 6];
+    e.crowmap = epi_crowmap[warp - 6];
+    e.cscale = epi_cscale[warp - 6];
+    if (p.BN == 128) epilogue_role<2>(p, e);
+    else if (p.BN == 64) epilogue_role<4>(p, e);
+    else epilogue_role<8>(p, e);
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -544,7 +619,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int budget = smem_max - 2048 - 1024;  // static shared + alignment slack
+  const int budget = smem_max - 6144 - 1024;  // static shared + alignment slack
   p.stages = budget / p.stage_bytes;
   if (p.stages > 8) p.stages = 8;
   if (p.stages < 2) return PIPE_ERR_UNSUPPORTED;
