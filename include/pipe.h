@@ -76,12 +76,15 @@ typedef struct pipe_layer_desc {
  *   kept_off[k]   int32 [kept_groups[k]]: ascending indices of the kept groups.
  *   cum_off[k]    int32 [G + 1]: cum[j] = number of kept groups with index < j (so group j is
  *                 kept iff cum[j+1] > cum[j], and its first compacted row is cum[j] * g).
- *   kcodes_off[k] the same codes in the layout the GEMM kernels stream:
- *                 [rows[k], kernel_row_bytes], rows zero-padded to a multiple of 128 codes,
- *                 and inside every aligned 32-bit word the fields are interleaved so that
- *                 masking alone yields int8 lanes in reduction order: int4 -> code 4h+j of
- *                 the word's 8 codes sits in nibble 2j+h; ternary -> code 4h+j of the word's
- *                 16 codes sits in bits 8j+2h..8j+2h+1; int8 -> unchanged.
+ *   kcodes_off[k] the same codes in the layout the GEMM kernels stream: the reduction axis is
+ *                 zero-padded to a multiple of 128 codes and cut into blocks of 128 codes; the
+ *                 section is [I_pad/128][rows[k]][128*b/8 bytes], i.e. block-major, so that the
+ *                 rows a tile needs for one reduction block are one contiguous run of bytes
+ *                 (kernel_row_bytes is still the total per row).  Inside every aligned 32-bit
+ *                 word the fields are interleaved so that masking alone yields int8 lanes in
+ *                 reduction order: int4 -> code 4h+j of the word's 8 codes sits in nibble 2j+h;
+ *                 ternary -> code 4h+j of the word's 16 codes sits in bits 8j+2h..8j+2h+1;
+ *                 int8 -> unchanged.
  */
 typedef struct pipe_layer_layout {
   int32_t num_groups;        /* G = O / g */

@@ -174,7 +174,8 @@ struct QuantizeRowsArgs {
   float* a;              // [O] row absmax: read (this order's), overwritten (next order's) if dst
   const int32_t* kept;   // [rows/g] ascending kept groups
   uint8_t* codes;        // canonical [rows, canon_row_bytes]
-  uint8_t* kcodes;       // kernel layout [rows, kernel_row_bytes]
+  uint8_t* kcodes;       // streaming layout [ceil(I/128), rows, 128*BITS/8]
+  int rows;              // compacted rows of this order
   float* scales;         // [rows]
   int I, g, qmax;
   int canon_row_bytes, kernel_row_bytes;
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
   __syncthreads();  // every thread has read a[o] before thread 0 overwrites it at the end
   if (threadIdx.x == 0) p.scales[n] = s;
   uint8_t* crow = p.codes + static_cast<int64_t>(n) * p.canon_row_bytes;
-  uint8_t* krow = p.kcodes + static_cast<int64_t>(n) * p.kernel_row_bytes;
+  constexpr int kStepBytes = 128 * BITS / 8;  // packed bytes of one row in one 128-code reduction block
   constexpr int kChunkBytes = 16 * BITS / 8;  // bytes of 16 packed codes
   constexpr int kWords = kChunkBytes / 4;
   const int I = p.I;
@@ -240,9 +241,10 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
     uint32_t canon[4], kern[4];
     pack16<BITS>(q, canon, kern);
     const int byte0 = i0 * BITS / 8;
-    // kernel layout: rows are padded and 16-byte aligned, always whole words
+    // streaming layout: reduction-block major, [i0 / 128][row][128 codes]; padded, always whole words
+    uint8_t* kdst = p.kcodes + (static_cast<int64_t>(i0 >> 7) * p.rows + n) * kStepBytes + (i0 & 127) * BITS / 8;
 #pragma unroll
-    for (int w = 0; w < kWords; ++w) reinterpret_cast<uint32_t*>(krow + byte0)[w] = kern[w];
+    for (int w = 0; w < kWords; ++w) reinterpret_cast<uint32_t*>(kdst)[w] = kern[w];
     if (i0 < I) {
       if (full && canon_vec) {
 #pragma unroll
@@ -327,6 +329,7 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     q.I = L.I; q.g = L.g; q.qmax = L.qmax;
     q.canon_row_bytes = L.lay.canon_row_bytes;
     q.kernel_row_bytes = L.lay.kernel_row_bytes;
+    q.rows = L.lay.rows[k];
     const int rows = L.lay.rows[k];
     if (L.bits == 8) quantize_rows_kernel<8><<<rows, kRowThreads, 0, s>>>(q);
     else if (L.bits == 4) quantize_rows_kernel<4><<<rows, kRowThreads, 0, s>>>(q);

@@ -5,11 +5,15 @@
 // into one int8 B operand (order 1: BN rows; a sparse order: only its kept rows, found through
 // the prefix counts), so one chain of tcgen05.mma kind::i8 instructions (M = 128 tokens,
 // N = stacked rows, K = 32) fills one int32 accumulator region per order in TMEM while the
-// activation tile is staged once per reduction step.  Warp roles:
-//   warp 0      TMA producer: activation tile (128B-swizzled) + packed weight boxes, per stage
-//   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered)
-//   warps 2-5   unpack: packed int8/int4/ternary boxes -> int8 lanes in the swizzled B tile
+// activation tile is staged once per reduction step.  Three shared-memory rings decouple the
+// latencies: activation tiles (TMA, 128B swizzle), packed weight rows (one bulk copy per order and
+// reduction block: the streaming layout is reduction-block major, so the rows of a tile are
+// contiguous), and unpacked int8 B tiles.  Warp roles:
+//   warp 0      producer of the activation ring (TMA tensor loads)
+//   warp 10     producer of the packed-weight ring (bulk copies)
+//   warps 2-5   unpack: packed int8/int4/ternary rows -> int8 lanes in the swizzled B tile
 //               (shift + mask only; sub-byte codes arrive multiplied by 2^(8-b))
+//   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered)
 //   warps 6-9   epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
 //               s_k * lambda_x and add in ascending order with one FMA per term, store fp32
 // Every wait on an mbarrier is bounded; on expiry the CTA raises PIPE_ERR_TIMEOUT, all roles
@@ -27,26 +31,26 @@ namespace tc {
 constexpr int kTileM = 128;          // tokens per tile
 constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
-constexpr int kBoxRows = 32;         // rows per packed-weight TMA box
-constexpr int kMaxBoxes = 8;
 constexpr int kMaxClusterOrders = 8;
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kUnpackThreads = 128;
 constexpr int kEpiThreads = 128;
 constexpr int kABytes = kTileM * kKStep;       // 16 KiB
 constexpr int kBtBytes = kMaxN * kKStep;       // 32 KiB
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
+constexpr int kMaxRing = 8;
+constexpr int kBtRing = 2;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s per wait
 
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
-  CUtensorMap tmap_b[PIPE_MAX_ORDERS];  // one per order (packed streaming layout)
   ForwardArgs f;
-  int BN, ncb, ntt, num_tiles, kblocks, stages;
-  int packed_row_bytes;   // bytes of one row of one reduction step in the packed layout (128*b/8)
-  int box_bytes;          // kBoxRows * packed_row_bytes
-  int stage_bytes;
+  int BN, ncb, ntt, num_tiles, kblocks;
+  int na, ns;             // depth of the activation ring and of the packed-weight ring
+  int pk;                 // packed bytes of one row of one reduction block (128*b/8)
+  int stg_bytes;          // one packed-weight stage: kMaxN * pk
+  int a_off, s_off, bt_off;  // ring offsets in dynamic shared memory (1 KiB aligned)
   int shift;              // 8 - b
 };
 
@@ -57,7 +61,6 @@ struct TileMeta {
   int start[kMaxClusterOrders];        // first compacted row of the channel block in order k
   int n[kMaxClusterOrders];            // rows of order k in the block
   int rowbase[kMaxClusterOrders + 1];  // row offset of order k in the stacked B tile / accumulator
-  int boxbase[kMaxClusterOrders + 1];  // first staging box of order k
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -104,11 +107,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// After the last issue: wait (bounded) until the copies of the last `depth` ring slots have landed,
+// so that no copy is still writing into this CTA's shared memory when it exits.
+__device__ __forceinline__ void drain_ring(uint32_t full0, uint32_t issued, int depth) {
+  for (uint32_t j = (issued > static_cast<uint32_t>(depth) ? issued - depth : 0); j < issued; ++j) {
+    const int s = j % depth;
+    const uint32_t ph = (j / depth) & 1;
+    const uint64_t t0 = global_ns();
+    while (!mbar_try(full0 + 8u * s, ph) && global_ns() - t0 < kWaitLimitNs) {
+    }
+  }
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
+}
+
+// Contiguous global -> shared copy (both addresses 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes, stored as
@@ -159,82 +181,72 @@ __device__ __forceinline__ void decode_tile(const Params& p, int tile, TileMeta&
   const int c0 = t.cb * p.BN;
   const int c1 = min(c0 + p.BN, p.f.O);
   const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
-  int rb = 0, bb = 0;
+  int rb = 0;
 #pragma unroll
   for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
     t.rowbase[ko] = rb;
-    t.boxbase[ko] = bb;
     if (ko < t.nk) {
       const int32_t* cum = p.f.order[t.k0 + ko].cum;
       const int lo = __ldg(cum + j0), hi = __ldg(cum + j1);
       t.start[ko] = lo * p.f.g;
       t.n[ko] = (hi - lo) * p.f.g;
       rb += t.n[ko];
-      bb += (t.n[ko] + kBoxRows - 1) / kBoxRows;
     } else {
       t.start[ko] = 0;
       t.n[ko] = 0;
     }
   }
   t.rowbase[kMaxClusterOrders] = rb;
-  t.boxbase[kMaxClusterOrders] = bb;
 }
 
-struct UnpackCtx {
-  int ut, S;
-  uint32_t full0, ready0;   // shared addresses of full[0] / ready[0]; barrier s is 8*s bytes further
-  uint8_t* stage0;          // generic address of stage 0's packed staging area
-  uint8_t* bt0;             // generic address of stage 0's int8 B tile
+struct Rings {
+  uint32_t a_full0, a_empty0, s_full0, s_empty0, bt_ready0, bt_empty0, tfull0, tempty0;  // barrier i is 8*i bytes on
+  uint32_t a0, s0, bt0;   // shared addresses of slot 0 of each ring
+  uint8_t* s_gen;         // generic addresses of slot 0 of the packed-weight and B-tile rings
+  uint8_t* bt_gen;
   volatile int* abort_flag;
 };
 
-// Unpack role (128 threads): for every reduction step copy the packed weight boxes of the tile
+// Unpack role (128 threads): for every reduction block turn the packed weight rows of the tile
 // into the 128B-swizzled int8 B tile.  Work items are (stacked row, 16-byte chunk); which items a
-// thread owns depends only on the tile, so their source/destination offsets are computed once
-// per tile and kept in registers.
+// thread owns depends only on the tile, so their offsets are computed once per tile.
 template <int BITS>
-__device__ __forceinline__ void unpack_role(const Params& p, const UnpackCtx& u) {
-  constexpr int CPR = BITS;              // 16-byte chunks per packed row per step: 8, 4, 2
+__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
+  constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
   constexpr int ITEMS = 2 * CPR;         // kMaxN * CPR / kUnpackThreads
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
+  constexpr int PK = 128 * BITS / 8;
   uint32_t it = 0;
-  bool ok = true;
-  for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+  for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
     TileMeta t;
     decode_tile(p, tile, t);
     const int n_total = t.rowbase[kMaxClusterOrders];
-    int src_off[ITEMS], dst_row_off[ITEMS], chunk_sw[ITEMS];
+    int src_off[ITEMS], dst_off0[ITEMS], sw16[ITEMS];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
-      const int idx = u.ut + i * kUnpackThreads;
+      const int idx = ut + i * kUnpackThreads;
       const int r = idx >> CPR_LOG, c = idx & (CPR - 1);
-      int rb = 0, bb = 0;
-#pragma unroll
-      for (int q = 1; q < kMaxClusterOrders; ++q)
-        if (q < t.nk && r >= t.rowbase[q]) {
-          rb = t.rowbase[q];
-          bb = t.boxbase[q];
-        }
-      src_off[i] = (r < n_total) ? (bb * kBoxRows + (r - rb)) * p.packed_row_bytes + c * 16 : -1;
-      dst_row_off[i] = (r >> 3) * 1024 + (r & 7) * 128;
-      chunk_sw[i] = (c * OUT_PER_CHUNK) | ((r & 7) << 8);
+      src_off[i] = (r < n_total) ? r * PK + c * 16 : -1;
+      dst_off0[i] = (r >> 3) * 1024 + (r & 7) * 128;
+      sw16[i] = ((c * OUT_PER_CHUNK) << 8) | (r & 7);
     }
     for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-      const int s = it % u.S;
-      const uint32_t ph = (it / u.S) & 1;
-      if (!mbar_wait(u.full0 + 8u * s, ph, u.abort_flag, p.f.status)) { ok = false; break; }
-      const uint8_t* stage = u.stage0 + static_cast<size_t>(s) * p.stage_bytes;
-      uint8_t* bt = u.bt0 + static_cast<size_t>(s) * p.stage_bytes;
+      const int ss = it % p.ns, bs = it % kBtRing;
+      const uint32_t sph = (it / p.ns) & 1, bph = (it / kBtRing) & 1;
+      if (!mbar_wait(g.s_full0 + 8u * ss, sph, g.abort_flag, p.f.status)) return;
+      const uint8_t* stage = g.s_gen + static_cast<size_t>(ss) * p.stg_bytes;
       uint4 w[ITEMS];
 #pragma unroll
       for (int i = 0; i < ITEMS; ++i)
         if (src_off[i] >= 0) w[i] = *reinterpret_cast<const uint4*>(stage + src_off[i]);
+      if (!mbar_wait(g.bt_empty0 + 8u * bs, bph ^ 1, g.abort_flag, p.f.status)) return;
+      uint8_t* bt = g.bt_gen + static_cast<size_t>(bs) * kBtBytes;
 #pragma unroll
       for (int i = 0; i < ITEMS; ++i) {
         if (src_off[i] < 0) continue;
-        uint8_t* row = bt + dst_row_off[i];
-        const int c0 = chunk_sw[i] & 0xff, sw = chunk_sw[i] >> 8;
+        uint8_t* row = bt + dst_off0[i];
+        const int c0 = sw16[i] >> 8, sw = sw16[i] & 7;
         if (BITS == 8) {
           *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
         } else if (BITS == 4) {
@@ -253,8 +265,9 @@ __device__ __forceinline__ void unpack_role(const Params& p, const UnpackCtx& u)
           }
         }
       }
+      mbar_arrive(g.s_empty0 + 8u * ss);   // the packed rows are in registers / already consumed
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
-      mbar_arrive(u.ready0 + 8u * s);
+      mbar_arrive(g.bt_ready0 + 8u * bs);
     }
   }
 }
@@ -398,38 +411,47 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 
 __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bars[4 * 8 + 4];   // full[8] ready[8] empty[8] | tmem_full[2] tmem_empty[2]
+  // a_full[8] a_empty[8] s_full[8] s_empty[8] bt_ready[2] bt_empty[2] tmem_full[2] tmem_empty[2]
+  __shared__ uint64_t bars[4 * kMaxRing + 8];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int16_t epi_colmap[4][32];     // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
   __shared__ int32_t epi_crowmap[4][32];    // ... and its compacted row in that order
   __shared__ float epi_cscale[4][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
 
-  volatile int* abort_flag = &abort_flag_s;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const int S = p.stages;
-  auto a_tile = [&](int s) { return smem_base + s * p.stage_bytes; };
-  auto bt_tile = [&](int s) { return smem_base + s * p.stage_bytes + kABytes; };
-  auto stg = [&](int s) { return smem_base + s * p.stage_bytes + kABytes + kBtBytes; };
   const uint32_t bar0 = smem_u32(bars);
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto ready_bar = [&](int s) { return bar0 + 8u * (8 + s); };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (16 + s); };
-  auto tfull_bar = [&](int b) { return bar0 + 8u * (24 + b); };
-  auto tempty_bar = [&](int b) { return bar0 + 8u * (26 + b); };
+  Rings g;
+  g.a_full0 = bar0;
+  g.a_empty0 = bar0 + 8u * kMaxRing;
+  g.s_full0 = bar0 + 8u * 2 * kMaxRing;
+  g.s_empty0 = bar0 + 8u * 3 * kMaxRing;
+  g.bt_ready0 = bar0 + 8u * 4 * kMaxRing;
+  g.bt_empty0 = g.bt_ready0 + 8u * 2;
+  g.tfull0 = g.bt_ready0 + 8u * 4;
+  g.tempty0 = g.bt_ready0 + 8u * 6;
+  g.a0 = smem_base + p.a_off;
+  g.s0 = smem_base + p.s_off;
+  g.bt0 = smem_base + p.bt_off;
+  g.s_gen = smem_gen + p.s_off;
+  g.bt_gen = smem_gen + p.bt_off;
+  g.abort_flag = &abort_flag_s;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int s = 0; s < S; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(ready_bar(s), kUnpackThreads);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < kMaxRing; ++s) {
+      mbar_init(g.a_full0 + 8u * s, 1);
+      mbar_init(g.a_empty0 + 8u * s, 1);
+      mbar_init(g.s_full0 + 8u * s, 1);
+      mbar_init(g.s_empty0 + 8u * s, kUnpackThreads);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), kEpiThreads);
+      mbar_init(g.bt_ready0 + 8u * b, kUnpackThreads);
+      mbar_init(g.bt_empty0 + 8u * b, 1);
+      mbar_init(g.tfull0 + 8u * b, 1);
+      mbar_init(g.tempty0 + 8u * b, kEpiThreads);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -445,42 +467,49 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
   const uint32_t tmem_base = tmem_base_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ activation producer
     if (lane == 0) {
-      uint32_t it = 0;           // global stage counter
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        const int tt = tile % p.ntt;
+        const int m = tile / p.ntt / p.ncb;
+        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+          const int s = it % p.na;
+          const uint32_t ph = (it / p.na) & 1;
+          if (!mbar_wait(g.a_empty0 + 8u * s, ph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
+          mbar_expect_tx(g.a_full0 + 8u * s, kABytes);
+          tma_load_2d(g.a0 + s * kABytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * s);
+        }
+      }
+      drain_ring(g.a_full0, it, p.na);
+    }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------------ packed-weight producer
+    if (lane == 0) {
+      uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
         TileMeta t;
         decode_tile(p, tile, t);
-        const int nboxes = t.boxbase[kMaxClusterOrders];
-        const uint32_t tx = kABytes + nboxes * p.box_bytes;
+        const uint32_t tx = static_cast<uint32_t>(t.rowbase[kMaxClusterOrders]) * p.pk;
         for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-          const int s = it % S;
-          const uint32_t ph = (it / S) & 1;
-          if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, p.f.status)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), tx);
-          tma_load_2d(a_tile(s), &p.tmap_a[t.m], kb * kKStep, t.tt * kTileM, full_bar(s));
-          int box = 0;
+          const int s = it % p.ns;
+          const uint32_t ph = (it / p.ns) & 1;
+          if (!mbar_wait(g.s_empty0 + 8u * s, ph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
+          mbar_expect_tx(g.s_full0 + 8u * s, tx);
 #pragma unroll
           for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
-            if (ko < t.nk) {
-              const int nb = (t.n[ko] + kBoxRows - 1) / kBoxRows;
-              for (int b = 0; b < nb; ++b, ++box)
-                tma_load_2d(stg(s) + box * p.box_bytes, &p.tmap_b[t.k0 + ko], kb * p.packed_row_bytes,
-                            t.start[ko] + b * kBoxRows, full_bar(s));
+            if (ko < t.nk && t.n[ko] > 0) {
+              const OrderView& ov = p.f.order[t.k0 + ko];
+              const uint8_t* src = ov.kcodes + (static_cast<size_t>(kb) * ov.rows + t.start[ko]) * p.pk;
+              bulk_load(g.s0 + s * p.stg_bytes + t.rowbase[ko] * p.pk, src, static_cast<uint32_t>(t.n[ko]) * p.pk,
+                        g.s_full0 + 8u * s);
             }
           }
         }
       }
-      // drain: every copy this thread issued must have landed before the CTA's shared memory goes away
-      const uint32_t issued = it;
-      for (uint32_t j = (issued > static_cast<uint32_t>(S) ? issued - S : 0); j < issued; ++j) {
-        const int s = j % S;
-        const uint32_t ph = (j / S) & 1;
-        const uint64_t t0 = global_ns();
-        while (!mbar_try(full_bar(s), ph) && global_ns() - t0 < kWaitLimitNs) {
-        }
-      }
+      drain_ring(g.s_full0, it, p.ns);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -492,48 +521,42 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
         decode_tile(p, tile, t);
         const int buf = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
-        if (!mbar_wait(tempty_bar(buf), aph ^ 1, abort_flag, p.f.status)) { ok = false; break; }
+        if (!mbar_wait(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         int n = (t.rowbase[kMaxClusterOrders] + 15) & ~15;
         if (n < 16) n = 16;
         const uint32_t idesc = idesc_i8(n);
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
         for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-          const int s = it % S;
-          const uint32_t ph = (it / S) & 1;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, p.f.status)) { ok = false; break; }
-          if (!mbar_wait(ready_bar(s), ph, abort_flag, p.f.status)) { ok = false; break; }
+          const int as = it % p.na, bs = it % kBtRing;
+          const uint32_t aphs = (it / p.na) & 1, bph = (it / kBtRing) & 1;
+          if (!mbar_wait(g.a_full0 + 8u * as, aphs, g.abort_flag, p.f.status)) { ok = false; break; }
+          if (!mbar_wait(g.bt_ready0 + 8u * bs, bph, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint64_t adesc = smem_desc_sw128(a_tile(s));
-          const uint64_t bdesc = smem_desc_sw128(bt_tile(s));
+          const uint64_t adesc = smem_desc_sw128(g.a0 + as * kABytes);
+          const uint64_t bdesc = smem_desc_sw128(g.bt0 + bs * kBtBytes);
 #pragma unroll
           for (int k = 0; k < kKStep / 32; ++k)
             mma_i8(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
-          mma_commit(empty_bar(s));
+          mma_commit(g.a_empty0 + 8u * as);
+          mma_commit(g.bt_empty0 + 8u * bs);
         }
-        if (ok) mma_commit(tfull_bar(buf));
+        if (ok) mma_commit(g.tfull0 + 8u * buf);
       }
     }
   } else if (warp < 6) {
     // ------------------------------------------------------------------ unpack warps
-    UnpackCtx u;
-    u.ut = threadIdx.x - 64;
-    u.S = S;
-    u.full0 = full_bar(0);
-    u.ready0 = ready_bar(0);
-    u.stage0 = smem_gen + kABytes + kBtBytes;
-    u.bt0 = smem_gen + kABytes;
-    u.abort_flag = abort_flag;
-    if (p.f.bits == 8) unpack_role<8>(p, u);
-    else if (p.f.bits == 4) unpack_role<4>(p, u);
-    else unpack_role<2>(p, u);
+    const int ut = threadIdx.x - 64;
+    if (p.f.bits == 8) unpack_role<8>(p, g, ut);
+    else if (p.f.bits == 4) unpack_role<4>(p, g, ut);
+    else unpack_role<2>(p, g, ut);
   } else {
     // ------------------------------------------------------------------ epilogue warps
     EpiCtx e;
     e.tmem_base = tmem_base;
-    e.tfull0 = tfull_bar(0);
-    e.tempty0 = tempty_bar(0);
-    e.abort_flag = abort_flag;
+    e.tfull0 = g.tfull0;
+    e.tempty0 = g.tempty0;
+    e.abort_flag = g.abort_flag;
     e.warp = warp;
     e.lane = lane;
     e.colmap = epi_colmap[warp - 6];
@@ -611,42 +634,36 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
   p.num_tiles = static_cast<int>(tiles);
   p.kblocks = ceil_div(a.I, kKStep);
-  p.packed_row_bytes = kKStep * a.bits / 8;
-  p.box_bytes = kBoxRows * p.packed_row_bytes;
-  p.stage_bytes = kABytes + kBtBytes + kMaxBoxes * p.box_bytes;
+  p.pk = kKStep * a.bits / 8;
+  p.stg_bytes = kMaxN * p.pk;
   p.shift = 8 - a.bits;
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int budget = smem_max - 6144 - 1024;  // static shared + alignment slack
-  p.stages = budget / p.stage_bytes;
-  if (p.stages > 8) p.stages = 8;
-  if (p.stages < 2) return PIPE_ERR_UNSUPPORTED;
-  const int dyn_smem = p.stages * p.stage_bytes + 1024;
+  // dynamic shared memory: B-tile ring (2 x 32 KiB), packed-weight ring (<= 64 KiB), the rest for activations
+  int budget = smem_max - 8192 - 1024 - kBtRing * kBtBytes;  // static shared, alignment slack
+  p.ns = 65536 / p.stg_bytes;
+  if (p.ns > 6) p.ns = 6;
+  if (p.ns < 2) p.ns = 2;
+  budget -= p.ns * p.stg_bytes;
+  p.na = budget / kABytes;
+  if (p.na > kMaxRing) p.na = kMaxRing;
+  if (p.na < 2) return PIPE_ERR_UNSUPPORTED;
+  p.a_off = 0;
+  p.bt_off = p.na * kABytes;
+  p.s_off = p.bt_off + kBtRing * kBtBytes;
+  const int dyn_smem = p.s_off + p.ns * p.stg_bytes + 1024;
 
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
                      static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
   }
-  int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
-  for (int m = 0; m < a.num_branches; ++m) {
-    k_lo = min(k_lo, a.branch[m].k_begin);
-    k_hi = max(k_hi, a.branch[m].k_end);
-  }
-  for (int k = k_lo; k < k_hi; ++k) {
-    if (!make_map_2d(&p.tmap_b[k], a.order[k].kcodes, static_cast<uint64_t>(a.kernel_row_bytes),
-                     static_cast<uint64_t>(a.order[k].rows), static_cast<uint64_t>(a.kernel_row_bytes),
-                     static_cast<uint32_t>(p.packed_row_bytes), kBoxRows, CU_TENSOR_MAP_SWIZZLE_NONE))
-      return PIPE_ERR_CUDA;
-  }
-  static bool attr_set = false;
   static int attr_bytes = 0;
-  if (!attr_set || attr_bytes < dyn_smem) {
+  if (attr_bytes < dyn_smem) {
     if (cudaFuncSetAttribute(tc_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem) != cudaSuccess)
       return PIPE_ERR_CUDA;
-    attr_set = true;
     attr_bytes = dyn_smem;
   }
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;

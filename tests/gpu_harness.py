@@ -34,8 +34,13 @@ def kernel_layout_from_codes(codes: np.ndarray, bits: int) -> np.ndarray:
     Ipad = (I + 127) // 128 * 128
     c = np.zeros((rows, Ipad), np.int8)
     c[:, :I] = codes
+    nblk = Ipad // 128
+
+    def block_major(packed):   # [rows, Ipad*bits/8] -> [Ipad/128, rows, 128*bits/8] flattened back to 2-D
+        return np.ascontiguousarray(packed.reshape(rows, nblk, -1).transpose(1, 0, 2)).reshape(rows, -1)
+
     if bits == 8:
-        return c.view(np.uint8)
+        return block_major(c.view(np.uint8))
     per_word = 32 // bits
     u = (c.astype(np.int32) & ((1 << bits) - 1)).astype(np.uint32).reshape(rows, Ipad // per_word, per_word // 4, 4)
     word = np.zeros((rows, Ipad // per_word), np.uint32)
@@ -43,7 +48,7 @@ def kernel_layout_from_codes(codes: np.ndarray, bits: int) -> np.ndarray:
         for j in range(4):
             shift = (4 * (2 * j + h)) if bits == 4 else (8 * j + 2 * h)
             word |= u[:, :, h, j] << np.uint32(shift)
-    return word.view(np.uint8).reshape(rows, -1)
+    return block_major(word.view(np.uint8).reshape(rows, -1))
 
 
 def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_layout=True):
