@@ -5,19 +5,21 @@
 // into one int8 B operand (order 1: BN rows; a sparse order: only its kept rows, found through
 // the prefix counts), so one chain of tcgen05.mma kind::i8 instructions (M = 128 tokens,
 // N = stacked rows, K = 32) fills one int32 accumulator region per order in TMEM while the
-// activation tile is staged once per reduction step.  Three shared-memory rings decouple the
-// latencies: activation tiles (TMA, 128B swizzle), packed weight rows (one bulk copy per order and
-// reduction block: the streaming layout is reduction-block major, so the rows of a tile are
-// contiguous), and unpacked int8 B tiles.  Warp roles:
-//   warp 0      producer of the activation ring (TMA tensor loads)
-//   warp 10     producer of the packed-weight ring (bulk copies)
-//   warps 2-5   unpack: packed int8/int4/ternary rows -> int8 lanes in the swizzled B tile
+// activation tile is staged once per reduction step.  A ring of stages {activation tile, B tile}
+// in shared memory decouples the roles:
+//   warp 0      activation producer: TMA tensor loads (128B swizzle), several lanes issue in turn
+//   warps 2-5   unpack: read the packed int8/int4/ternary rows of the tile straight from the
+//               reduction-block-major streaming layout (coalesced 16-byte loads, prefetched one
+//               step ahead in registers) and write int8 lanes into the swizzled B tile
 //               (shift + mask only; sub-byte codes arrive multiplied by 2^(8-b))
-//   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered)
+//   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered);
+//               one tcgen05.commit per step releases the stage to both producers
 //   warps 6-9   epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
 //               s_k * lambda_x and add in ascending order with one FMA per term, store fp32
-// Every wait on an mbarrier is bounded; on expiry the CTA raises PIPE_ERR_TIMEOUT, all roles
-// leave their loops, outstanding copies are drained, TMEM is freed and the kernel returns.
+// Barrier operations cost their issuing thread on the order of a hundred cycles each, so every
+// role touches as few barriers per step as possible and ring positions are advanced without
+// divisions.  Every wait on an mbarrier is bounded; on expiry the CTA raises PIPE_ERR_TIMEOUT, all
+// roles leave their loops, outstanding copies are drained, TMEM is freed and the kernel returns.
 #include <cuda.h>
 
 #include <mutex>
@@ -32,26 +34,39 @@ constexpr int kTileM = 128;          // tokens per tile
 constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
-constexpr int kThreads = 352;
+constexpr int kThreads = 320;
 constexpr int kUnpackThreads = 128;
 constexpr int kEpiThreads = 128;
 constexpr int kABytes = kTileM * kKStep;       // 16 KiB
 constexpr int kBtBytes = kMaxN * kKStep;       // 32 KiB
+constexpr int kStageBytes = kABytes + kBtBytes;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
-constexpr int kMaxRing = 8;
-constexpr int kBtRing = 2;
-constexpr uint64_t kWaitLimitNs = 1000000000ull;  // 1 s per wait
+constexpr int kMaxRing = 4;
+constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
+constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s per wait at the maximum SM clock
+
+// Position in a ring of `depth` slots: slot index and phase parity, advanced without divisions.
+struct RingPos {
+  uint32_t slot, phase;
+  __device__ __forceinline__ void advance(uint32_t by, uint32_t depth) {  // by <= depth
+    slot += by;
+    if (slot >= depth) {
+      slot -= depth;
+      phase ^= 1u;
+    }
+  }
+};
 
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
   ForwardArgs f;
   int BN, ncb, ntt, num_tiles, kblocks;
-  int na, ns;             // depth of the activation ring and of the packed-weight ring
+  int depth;              // stages in the ring
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
-  int stg_bytes;          // one packed-weight stage: kMaxN * pk
-  int a_off, s_off, bt_off;  // ring offsets in dynamic shared memory (1 KiB aligned)
   int shift;              // 8 - b
+  const uint8_t* kbase;   // lowest address of the streaming-layout sections (16-byte aligned)
+  uint32_t koff[PIPE_MAX_ORDERS];  // (kcodes of order k - kbase) / 16
 };
 
 struct TileMeta {
@@ -64,12 +79,6 @@ struct TileMeta {
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -93,13 +102,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+// The bound is counted in SM cycles; the abort flag and the clock are looked at only every few
+// polls so that a barrier that completes soon is seen with little delay.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
+  const long long t0 = clock64();
   while (true) {
-    if (mbar_try(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) {
+    if (clock64() - t0 > kWaitLimitCycles) {
       *abort_flag = 1;
       raise_status(status, PIPE_ERR_TIMEOUT);
       return false;
@@ -113,8 +126,8 @@ __device__ __forceinline__ void drain_ring(uint32_t full0, uint32_t issued, int 
   for (uint32_t j = (issued > static_cast<uint32_t>(depth) ? issued - depth : 0); j < issued; ++j) {
     const int s = j % depth;
     const uint32_t ph = (j / depth) & 1;
-    const uint64_t t0 = global_ns();
-    while (!mbar_try(full0 + 8u * s, ph) && global_ns() - t0 < kWaitLimitNs) {
+    const long long t0 = clock64();
+    while (!mbar_try(full0 + 8u * s, ph) && clock64() - t0 < kWaitLimitCycles) {
     }
   }
 }
@@ -124,13 +137,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
-}
-
-// Contiguous global -> shared copy (both addresses 16-byte aligned, size a multiple of 16).
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-               : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes, stored as
@@ -200,53 +206,103 @@ __device__ __forceinline__ void decode_tile(const Params& p, int tile, TileMeta&
 }
 
 struct Rings {
-  uint32_t a_full0, a_empty0, s_full0, s_empty0, bt_ready0, bt_empty0, tfull0, tempty0;  // barrier i is 8*i bytes on
-  uint32_t a0, s0, bt0;   // shared addresses of slot 0 of each ring
-  uint8_t* s_gen;         // generic addresses of slot 0 of the packed-weight and B-tile rings
-  uint8_t* bt_gen;
+  uint32_t a_full0, bt_ready0, done0, tfull0, tempty0;  // barrier i of a family is 8*i bytes on
+  uint32_t stage0;        // shared address of stage 0 (activation tile, then B tile)
+  uint8_t* stage_gen;     // generic address of stage 0
   volatile int* abort_flag;
 };
 
-// Unpack role (128 threads): for every reduction block turn the packed weight rows of the tile
-// into the 128B-swizzled int8 B tile.  Work items are (stacked row, 16-byte chunk); which items a
-// thread owns depends only on the tile, so their offsets are computed once per tile.
+// Per-tile placement of one unpack work item (stacked row r, 16-byte chunk c of its packed row):
+// offset of the chunk in the streaming layout at reduction block 0 and its step per block, both
+// in 16-byte units relative to Params::kbase; 0xffffffff marks an item beyond the tile's rows.
+__device__ __forceinline__ void place_item(const Params& p, int k0, int nk, const int (&start)[kMaxClusterOrders],
+                                           const int (&rowbase)[kMaxClusterOrders + 1], int r, int c, uint32_t& off,
+                                           uint32_t& step) {
+  if (r >= rowbase[kMaxClusterOrders]) {
+    off = 0xffffffffu;
+    step = 0;
+    return;
+  }
+  int rb = 0, st = start[0], ko = 0;
+#pragma unroll
+  for (int q = 1; q < kMaxClusterOrders; ++q)
+    if (q < nk && r >= rowbase[q]) {
+      rb = rowbase[q];
+      st = start[q];
+      ko = q;
+    }
+  const OrderView& ov = p.f.order[k0 + ko];
+  const uint32_t pk16 = static_cast<uint32_t>(p.pk) >> 4;
+  off = p.koff[k0 + ko] + static_cast<uint32_t>(st + r - rb) * pk16 + static_cast<uint32_t>(c);
+  step = static_cast<uint32_t>(ov.rows) * pk16;
+}
+
+// Unpack role (128 threads).  Work items are (stacked row, 16-byte chunk); a thread owns the same
+// item indices in every tile.  The packed chunks of the NEXT step are loaded from global memory
+// (L2-resident, fully coalesced) into registers before the current step's stage is waited for,
+// also across tile boundaries.
 template <int BITS>
 __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
   constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
   constexpr int ITEMS = 2 * CPR;         // kMaxN * CPR / kUnpackThreads
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
-  constexpr int PK = 128 * BITS / 8;
-  uint32_t it = 0;
-  for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+  const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
+  const uint32_t depth = p.depth;
+  constexpr bool PREFETCH = BITS != 8;   // int8 rows need 16 chunks per thread: too many registers to double-buffer
+  const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (128 / CPR), chunk c_item
+  const int sw = r0 & 7;                                   // (128 / CPR) is a multiple of 8 for 4- and 2-bit codes
+  uint32_t off[ITEMS], step[ITEMS];
+  uint4 wn[ITEMS];
+  int tile = blockIdx.x;
+  if (tile >= p.num_tiles) return;
+  {
     TileMeta t;
     decode_tile(p, tile, t);
-    const int n_total = t.rowbase[kMaxClusterOrders];
-    int src_off[ITEMS], dst_off0[ITEMS], sw16[ITEMS];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       const int idx = ut + i * kUnpackThreads;
-      const int r = idx >> CPR_LOG, c = idx & (CPR - 1);
-      src_off[i] = (r < n_total) ? r * PK + c * 16 : -1;
-      dst_off0[i] = (r >> 3) * 1024 + (r & 7) * 128;
-      sw16[i] = ((c * OUT_PER_CHUNK) << 8) | (r & 7);
+      place_item(p, t.k0, t.nk, t.start, t.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], step[i]);
+      if (PREFETCH && off[i] != 0xffffffffu) wn[i] = __ldg(kb16 + off[i]);
     }
-    for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-      const int ss = it % p.ns, bs = it % kBtRing;
-      const uint32_t sph = (it / p.ns) & 1, bph = (it / kBtRing) & 1;
-      if (!mbar_wait(g.s_full0 + 8u * ss, sph, g.abort_flag, p.f.status)) return;
-      const uint8_t* stage = g.s_gen + static_cast<size_t>(ss) * p.stg_bytes;
+  }
+  RingPos rp{0, 0};
+  for (; tile < p.num_tiles; tile += gridDim.x) {
+    const int next_tile = tile + gridDim.x;
+    TileMeta tn;
+    decode_tile(p, next_tile < p.num_tiles ? next_tile : tile, tn);   // its loads complete during this tile's steps
+    for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
       uint4 w[ITEMS];
-#pragma unroll
-      for (int i = 0; i < ITEMS; ++i)
-        if (src_off[i] >= 0) w[i] = *reinterpret_cast<const uint4*>(stage + src_off[i]);
-      if (!mbar_wait(g.bt_empty0 + 8u * bs, bph ^ 1, g.abort_flag, p.f.status)) return;
-      uint8_t* bt = g.bt_gen + static_cast<size_t>(bs) * kBtBytes;
+      bool valid[ITEMS];
 #pragma unroll
       for (int i = 0; i < ITEMS; ++i) {
-        if (src_off[i] < 0) continue;
-        uint8_t* row = bt + dst_off0[i];
-        const int c0 = sw16[i] >> 8, sw = sw16[i] & 7;
+        valid[i] = off[i] != 0xffffffffu;
+        if (PREFETCH) w[i] = wn[i];
+        else if (valid[i]) w[i] = __ldg(kb16 + off[i]);
+      }
+      if (kb + 1 < p.kblocks) {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i)
+          if (valid[i]) {
+            off[i] += step[i];
+            if (PREFETCH) wn[i] = __ldg(kb16 + off[i]);
+          }
+      } else if (next_tile < p.num_tiles) {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+          const int idx = ut + i * kUnpackThreads;
+          place_item(p, tn.k0, tn.nk, tn.start, tn.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], step[i]);
+          if (PREFETCH && off[i] != 0xffffffffu) wn[i] = __ldg(kb16 + off[i]);
+        }
+      }
+      if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
+      uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) {
+        if (!valid[i]) continue;
+        const int r = r0 + i * (kUnpackThreads >> CPR_LOG);
+        uint8_t* row = bt + (r >> 3) * 1024 + (r & 7) * 128;
+        const int c0 = c_item * OUT_PER_CHUNK;
         if (BITS == 8) {
           *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
         } else if (BITS == 4) {
@@ -265,9 +321,9 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
           }
         }
       }
-      mbar_arrive(g.s_empty0 + 8u * ss);   // the packed rows are in registers / already consumed
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
-      mbar_arrive(g.bt_ready0 + 8u * bs);
+      __syncwarp();
+      if ((ut & 31) == 0) mbar_arrive(g.bt_ready0 + 8u * rp.slot);   // one arrival per warp
     }
   }
 }
@@ -405,14 +461,14 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    mbar_arrive(x.tempty0 + 8u * buf);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(x.tempty0 + 8u * buf);   // one arrival per warp
   }
 }
 
 __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
-  // a_full[8] a_empty[8] s_full[8] s_empty[8] bt_ready[2] bt_empty[2] tmem_full[2] tmem_empty[2]
-  __shared__ uint64_t bars[4 * kMaxRing + 8];
+  __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[4] bt_ready[4] done[4] tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int16_t epi_colmap[4][32];     // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
@@ -421,37 +477,27 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t bar0 = smem_u32(bars);
   Rings g;
   g.a_full0 = bar0;
-  g.a_empty0 = bar0 + 8u * kMaxRing;
-  g.s_full0 = bar0 + 8u * 2 * kMaxRing;
-  g.s_empty0 = bar0 + 8u * 3 * kMaxRing;
-  g.bt_ready0 = bar0 + 8u * 4 * kMaxRing;
-  g.bt_empty0 = g.bt_ready0 + 8u * 2;
-  g.tfull0 = g.bt_ready0 + 8u * 4;
-  g.tempty0 = g.bt_ready0 + 8u * 6;
-  g.a0 = smem_base + p.a_off;
-  g.s0 = smem_base + p.s_off;
-  g.bt0 = smem_base + p.bt_off;
-  g.s_gen = smem_gen + p.s_off;
-  g.bt_gen = smem_gen + p.bt_off;
+  g.bt_ready0 = bar0 + 8u * kMaxRing;
+  g.done0 = bar0 + 8u * 2 * kMaxRing;
+  g.tfull0 = bar0 + 8u * 3 * kMaxRing;
+  g.tempty0 = g.tfull0 + 8u * 2;
+  g.stage0 = smem_base;
+  g.stage_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   g.abort_flag = &abort_flag_s;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < kMaxRing; ++s) {
       mbar_init(g.a_full0 + 8u * s, 1);
-      mbar_init(g.a_empty0 + 8u * s, 1);
-      mbar_init(g.s_full0 + 8u * s, 1);
-      mbar_init(g.s_empty0 + 8u * s, kUnpackThreads);
+      mbar_init(g.bt_ready0 + 8u * s, kUnpackThreads / 32);
+      mbar_init(g.done0 + 8u * s, 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(g.bt_ready0 + 8u * b, kUnpackThreads);
-      mbar_init(g.bt_empty0 + 8u * b, 1);
       mbar_init(g.tfull0 + 8u * b, 1);
-      mbar_init(g.tempty0 + 8u * b, kEpiThreads);
+      mbar_init(g.tempty0 + 8u * b, kEpiThreads / 32);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -465,81 +511,81 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t depth = p.depth;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ activation producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+    // A copy instruction occupies its issuing thread for several hundred cycles, but copies issued
+    // by different lanes overlap.  Lane j owns the steps j, j + P, ...; every step has its own
+    // barrier pair, so the lanes need no order among themselves -- PROVIDED P does not exceed the
+    // ring depth N: a lane that issued step it - P has seen step it - P - N consumed, hence
+    // (consumption is in order) step it - 2N as well, so when it waits for the slot of step `it`
+    // that slot's barrier is at most one phase behind and the parity wait cannot be satisfied by
+    // a stale phase.
+    const int my_tiles = (p.num_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    const uint32_t total_steps = static_cast<uint32_t>(my_tiles) * p.kblocks;
+    const uint32_t P = min(static_cast<uint32_t>(kALanes), depth);
+    if (static_cast<uint32_t>(lane) < P) {
+      RingPos rp{static_cast<uint32_t>(lane), 0};
+      int tile = blockIdx.x, kb = lane;
+      for (uint32_t it = lane; it < total_steps; it += P, rp.advance(P, depth), kb += P) {
+        while (kb >= p.kblocks) {
+          kb -= p.kblocks;
+          tile += gridDim.x;
+        }
         const int tt = tile % p.ntt;
         const int m = tile / p.ntt / p.ncb;
-        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-          const int s = it % p.na;
-          const uint32_t ph = (it / p.na) & 1;
-          if (!mbar_wait(g.a_empty0 + 8u * s, ph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
-          mbar_expect_tx(g.a_full0 + 8u * s, kABytes);
-          tma_load_2d(g.a0 + s * kABytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * s);
-        }
+        if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
+        mbar_expect_tx(g.a_full0 + 8u * rp.slot, kABytes);
+        tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * rp.slot);
       }
-      drain_ring(g.a_full0, it, p.na);
     }
-  } else if (warp == 10) {
-    // ------------------------------------------------------------------ packed-weight producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-        TileMeta t;
-        decode_tile(p, tile, t);
-        const uint32_t tx = static_cast<uint32_t>(t.rowbase[kMaxClusterOrders]) * p.pk;
-        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-          const int s = it % p.ns;
-          const uint32_t ph = (it / p.ns) & 1;
-          if (!mbar_wait(g.s_empty0 + 8u * s, ph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
-          mbar_expect_tx(g.s_full0 + 8u * s, tx);
-#pragma unroll
-          for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
-            if (ko < t.nk && t.n[ko] > 0) {
-              const OrderView& ov = p.f.order[t.k0 + ko];
-              const uint8_t* src = ov.kcodes + (static_cast<size_t>(kb) * ov.rows + t.start[ko]) * p.pk;
-              bulk_load(g.s0 + s * p.stg_bytes + t.rowbase[ko] * p.pk, src, static_cast<uint32_t>(t.n[ko]) * p.pk,
-                        g.s_full0 + 8u * s);
-            }
-          }
-        }
-      }
-      drain_ring(g.s_full0, it, p.ns);
-    }
+    __syncwarp();
+    if (lane == 0) drain_ring(g.a_full0, total_steps, p.depth);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t it = 0, tcount = 0;
+      RingPos rp{0, 0};
+      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kABytes);
+      uint32_t tcount = 0;
       bool ok = true;
+      // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
+      auto stacked_rows = [&](int tile) {
+        const int cb = (tile / p.ntt) % p.ncb, m = tile / p.ntt / p.ncb;
+        const BranchArgs& br = p.f.branch[m];
+        const int c0 = cb * p.BN, c1 = min(c0 + p.BN, p.f.O);
+        const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
+        int n = 0;
+        for (int k = br.k_begin; k < br.k_end; ++k) {
+          const int32_t* cum = p.f.order[k].cum;
+          n += (__ldg(cum + j1) - __ldg(cum + j0)) * p.f.g;
+        }
+        return n;
+      };
+      int n_next = blockIdx.x < p.num_tiles ? stacked_rows(blockIdx.x) : 0;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
-        TileMeta t;
-        decode_tile(p, tile, t);
+        const int n_total = n_next;
+        if (tile + static_cast<int>(gridDim.x) < p.num_tiles) n_next = stacked_rows(tile + gridDim.x);
         const int buf = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
         if (!mbar_wait(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        int n = (t.rowbase[kMaxClusterOrders] + 15) & ~15;
+        int n = (n_total + 15) & ~15;
         if (n < 16) n = 16;
         const uint32_t idesc = idesc_i8(n);
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
-        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-          const int as = it % p.na, bs = it % kBtRing;
-          const uint32_t aphs = (it / p.na) & 1, bph = (it / kBtRing) & 1;
-          if (!mbar_wait(g.a_full0 + 8u * as, aphs, g.abort_flag, p.f.status)) { ok = false; break; }
-          if (!mbar_wait(g.bt_ready0 + 8u * bs, bph, g.abort_flag, p.f.status)) { ok = false; break; }
+        for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
+          // both barriers are polled before either result is tested so that the two polls overlap
+          const bool r1 = mbar_try(g.a_full0 + 8u * rp.slot, rp.phase);
+          const bool r2 = mbar_try(g.bt_ready0 + 8u * rp.slot, rp.phase);
+          if (!r1 && !mbar_wait(g.a_full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
+          if (!r2 && !mbar_wait(g.bt_ready0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint64_t adesc = smem_desc_sw128(g.a0 + as * kABytes);
-          const uint64_t bdesc = smem_desc_sw128(g.bt0 + bs * kBtBytes);
+          const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
+          const uint64_t adesc = adesc0 + so, bdesc = bdesc0 + so;
 #pragma unroll
           for (int k = 0; k < kKStep / 32; ++k)
             mma_i8(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
-          mma_commit(g.a_empty0 + 8u * as);
-          mma_commit(g.bt_empty0 + 8u * bs);
+          mma_commit(g.done0 + 8u * rp.slot);   // frees the stage for the activation producer AND the unpack warps
         }
         if (ok) mma_commit(g.tfull0 + 8u * buf);
       }
@@ -635,25 +681,29 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   p.num_tiles = static_cast<int>(tiles);
   p.kblocks = ceil_div(a.I, kKStep);
   p.pk = kKStep * a.bits / 8;
-  p.stg_bytes = kMaxN * p.pk;
   p.shift = 8 - a.bits;
+  int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
+  for (int m = 0; m < a.num_branches; ++m) {
+    k_lo = min(k_lo, a.branch[m].k_begin);
+    k_hi = max(k_hi, a.branch[m].k_end);
+  }
+  const uint8_t* kbase = a.order[k_lo].kcodes;
+  for (int k = k_lo; k < k_hi; ++k) kbase = a.order[k].kcodes < kbase ? a.order[k].kcodes : kbase;
+  p.kbase = kbase;
+  for (int k = k_lo; k < k_hi; ++k) {
+    const uint64_t d = static_cast<uint64_t>(a.order[k].kcodes - kbase);
+    const uint64_t end = (d + static_cast<uint64_t>(a.order[k].rows) * a.kernel_row_bytes) >> 4;
+    if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
+    p.koff[k] = static_cast<uint32_t>(d >> 4);
+  }
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  // dynamic shared memory: B-tile ring (2 x 32 KiB), packed-weight ring (<= 64 KiB), the rest for activations
-  int budget = smem_max - 8192 - 1024 - kBtRing * kBtBytes;  // static shared, alignment slack
-  p.ns = 65536 / p.stg_bytes;
-  if (p.ns > 6) p.ns = 6;
-  if (p.ns < 2) p.ns = 2;
-  budget -= p.ns * p.stg_bytes;
-  p.na = budget / kABytes;
-  if (p.na > kMaxRing) p.na = kMaxRing;
-  if (p.na < 2) return PIPE_ERR_UNSUPPORTED;
-  p.a_off = 0;
-  p.bt_off = p.na * kABytes;
-  p.s_off = p.bt_off + kBtRing * kBtBytes;
-  const int dyn_smem = p.s_off + p.ns * p.stg_bytes + 1024;
+  p.depth = (smem_max - 8192 - 1024) / kStageBytes;  // static shared, alignment slack
+  if (p.depth > kMaxRing) p.depth = kMaxRing;
+  if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
+  const int dyn_smem = p.depth * kStageBytes + 1024;
 
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
