@@ -11,7 +11,7 @@ from tests import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_AUTO]
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_STREAM, B.KERNEL_AUTO]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -136,6 +136,11 @@ FORWARD_CASES = [
     (512, 272, 1000, 2, 8, 16, 8, 4),
     (200, 144, 260, 8, 3, 8, 5, 3),
     (640, 640, 129, 4, 6, 32, 3, 1),
+    (128, 328, 7, 2, 8, 16, 2, 4),
+    (256, 256, 9, 8, 2, 8, 32, 1),
+    (304, 2304, 16, 4, 3, 8, 19, 1),
+    (72, 4112, 3, 4, 5, 8, 4, 2),
+    (136, 1000, 12, 2, 4, 8, 9, 1),
 ]
 
 
