@@ -253,6 +253,48 @@ def run_ours(args):
     tokens_per_s = world * T * args.steps / (total_ms * 1e-3)
     macs = run.macs_per_token() * T
 
+    # ---- the GEMM kernel alone: back-to-back launches (one CUDA graph when capture works, so that
+    # the host does not pace ~10 us kernels), rotating over copies of the blob whose total size
+    # exceeds L2 so that weights are streamed from HBM every launch
+    reps = 20
+    blobs = run.blob_copies(0 if flush is None else 2 * L2_BYTES)
+    blobs = blobs[:reps]
+    def launch_all():
+        for r in range(reps):
+            run.forward(blob=blobs[r % len(blobs)])
+    for _ in range(2):
+        launch_all()
+    torch.cuda.synchronize()
+    graph = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                launch_all()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = g
+    except Exception:
+        graph = None
+        torch.cuda.synchronize()
+    launch_ms = []
+    for _ in range(5):
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        k0.record()
+        if graph is not None:
+            graph.replay()
+        else:
+            launch_all()
+        k1.record()
+        torch.cuda.synchronize()
+        launch_ms.append(k0.elapsed_time(k1) / reps)
+    fwd_launch_ms = statistics.median(launch_ms)
+    del blobs
+    st = B.pipe_poll_status()
+    if st != B.PIPE_OK:
+        raise SystemExit(f"device status after the kernel timing loop: {B.pipe_status_string(st)}")
+
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region ------------
     hW = run.W.cpu().pin_memory()
     hx = [x.cpu().pin_memory() for x in run.x]
@@ -290,7 +332,7 @@ def run_ours(args):
     dominant = max(phases, key=phases.get)
     int8_peak_burst = 2.0 * peaks["bf16_tflops"]
     int8_peak_sust = 2.0 * peaks["bf16_tflops_sustained"]
-    fwd_s = phases["forward"] * 1e-3
+    fwd_s = fwd_launch_ms * 1e-3   # per-launch duration of the GEMM kernel, back-to-back launches
     fwd_tops = 2.0 * macs / fwd_s / 1e12
     fwd_gbs = run.forward_bytes() / fwd_s / 1e9
     ai = 2.0 * macs / run.forward_bytes()
@@ -322,7 +364,9 @@ def run_ours(args):
             "config": dict(config_of(spec), l2="flush_between_steps" if flush is not None else "inputs_exceed_l2",
                            distinct_branch_inputs=run.distinct_inputs, multi_gpu="independent replicas"),
             "effective_tops_whole_step": 2.0 * macs * world / (ms_per_step * 1e-3) / 1e12,
-            "forward": {"ms": phases["forward"], "effective_tops": fwd_tops, "gbs": fwd_gbs,
+            "forward": {"ms": fwd_launch_ms, "timing": ("cuda graph of 20 launches" if graph is not None else "20 back-to-back launches")
+                        + (", blob copies rotated (> 2 x L2)" if flush is not None else ""),
+                        "ms_in_step": phases["forward"], "effective_tops": fwd_tops, "gbs": fwd_gbs,
                         "frac_int8_peak_sustained": fwd_tops / int8_peak_sust, "frac_int8_peak_burst": fwd_tops / int8_peak_burst,
                         "frac_int8_nominal_4500": fwd_tops / 4500.0, "frac_hbm": fwd_gbs / peaks["hbm_gbs"],
                         "arithmetic_intensity": ai},

@@ -1,41 +1,84 @@
 // Small-token kernel of the expanded layer (Appendix B, Eq. 9; Sec. 3.2 for the branches), T <= 16.
 //
 // With a handful of tokens the layer is bound by streaming the packed weight codes from HBM once.
-// The kernel therefore moves weights global -> registers with coalesced 16-byte loads (many in
-// flight per warp), unpacks them in registers with the shift-and-mask layout and feeds legacy
-// warp-level integer MMAs (mma.sync m16n8k32, weights as the 16-row operand, tokens as the
-// 8-column operand): the tensor pipe is nowhere near a limit here, the byte stream is.
+// The kernel therefore moves weights global -> registers with coalesced 16-byte loads (the loads of
+// the next batch are always in flight while the current batch is consumed), unpacks them in
+// registers with the shift-and-mask layout and feeds legacy warp-level integer MMAs
+// (mma.sync m16n8k32, weights as the 16-row operand, tokens as the 8-column operand): the tensor
+// pipe is nowhere near a limit here, the byte stream is.
 //
 // Work unit: a "slab" = 8 consecutive output channels of one branch.  In every order of the branch
 // that keeps the slab's group, the slab is 8 consecutive compacted rows.  Two such 8-row chunks
 // (two orders, ascending) form one 16-row MMA tile, so both orders of a pair accumulate in the same
-// thread and the fixed-order fp32 epilogue is thread-local.  A CTA of 16 warps works on 4 slabs at a
-// time; the 4 warps of a slab split the reduction axis and add their exact int32 partial sums
-// through shared memory.  The quantized activations sit in shared memory in MMA-fragment order.
+// thread and the fixed-order fp32 epilogue is thread-local.  A persistent CTA walks groups of 2
+// slabs: 8 streaming warps (4 per slab, each owning a range of the reduction axis) drop their exact
+// int32 partial sums into a double-buffered shared-memory area; 2 epilogue warps (one per slab)
+// add the four ranges, apply the scales in ascending order and store, while the streaming warps
+// are already on the next group.  The quantized activations sit in shared memory in MMA-fragment
+// order; all slab metadata of the CTA is gathered once, up front, with independent loads.
 #include "pipe_common.cuh"
 
 namespace pipe {
 
 namespace st {
 
-constexpr int kThreads = 512;
-constexpr int kSlabsPerCta = 4;
-constexpr int kSlices = 4;        // warps per slab, each owns a contiguous range of macro steps
+constexpr int kStreamWarps = 8;
+constexpr int kEpiWarps = 2;
+constexpr int kThreads = 32 * (kStreamWarps + kEpiWarps);
+constexpr int kSlabsPerGroup = 2;
+constexpr int kSlices = 4;        // streaming warps per slab
 constexpr int kMaxPairs = 4;      // up to 8 orders per branch
 constexpr int kBatch = 8;         // macro steps whose loads are issued together
+constexpr int kMaxGroups = 128;   // groups one CTA may own (metadata table size)
+constexpr int kMetaInts = 2 + 4 * kMaxPairs;   // nchunks, branch, then (order, row0) per chunk
+constexpr long long kWaitLimitCycles = 4000000000ll;
 
 struct Params {
   ForwardArgs f;
-  int nt;            // 8-token MMA column tiles: 1 (T <= 8) or 2
-  int chk;           // codes per 16-byte chunk: 16 (int8), 32 (int4), 64 (ternary)
-  int nmma;          // MMAs per macro step = chk / 8
-  int nms;           // macro steps: ceil(I_pad / (4 * chk))
+  int nms;           // macro steps: ceil(I_pad / (4 * codes per 16-byte chunk))
   int kblocks;       // I_pad / 128
   int pk;            // packed bytes of one row of one 128-code block
   int shift;         // 8 - b
-  int slabs_per_branch, total_slabs;
-  int xs_bytes, red_bytes;
+  int slabs_per_branch;   // padded to a multiple of kSlabsPerGroup
+  int groups;
+  int xs_bytes;
+  int np;            // pairs of orders per slab the partial-sum buffers are sized for
 };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      raise_status(status, PIPE_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
 
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -67,206 +110,305 @@ __device__ __forceinline__ void unpack_chunk(const uint4& w, uint32_t (&reg)[16]
   }
 }
 
+// One batch of a streaming warp: kBatch macro steps of one pair of one slab.
+struct Batch {
+  int gi;        // index into the CTA's own group list (-1: none)
+  int q;         // pair
+  int ms0;       // first macro step
+};
+
 template <int BITS, int NT>
 __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Params p) {
   constexpr int CHK = 128 / BITS;        // codes per 16-byte chunk
   constexpr int NMMA = CHK / 8;          // MMAs per macro step
+  const int RED_INTS = kSlabsPerGroup * kSlices * p.np * 32 * 4 * NT;   // one buffer of partial sums
   extern __shared__ uint4 smem_u4[];
-  uint2* xs = reinterpret_cast<uint2*>(smem_u4);                                  // [nms][NMMA][NT][32] 8-byte fragments
-  int* red = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(smem_u4) + p.xs_bytes);  // [slab][slice-1][pair][lane][4*NT]
-  __shared__ int slab_meta[kSlabsPerCta][2 + 2 * kMaxPairs * 2];  // per slab: branch, npairs, then (order, row0) per chunk
+  uint2* xs = reinterpret_cast<uint2*>(smem_u4);                                             // [nms][NMMA][NT][32]
+  int* red = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(smem_u4) + p.xs_bytes);      // [2][slab][slice][pair][lane][4*NT]
+  int* meta = red + 2 * RED_INTS;                                                            // [own groups][slab][kMetaInts]
+  __shared__ uint64_t bars[6];   // full[2] empty[2] stage[2]
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
-  const int slab_local = warp / kSlices, slice = warp % kSlices;
   const int I = p.f.I;
-  int cur_branch_loaded = -1;
+  const int my_groups = (p.groups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  const uint32_t bar0 = smem_u32(bars);
+  const uint32_t full0 = bar0, empty0 = bar0 + 16, stage0 = bar0 + 32;
 
-  const int groups = (p.total_slabs + kSlabsPerCta - 1) / kSlabsPerCta;
-  for (int grp = blockIdx.x; grp < groups; grp += gridDim.x) {
-    const int slab = grp * kSlabsPerCta + slab_local;
-    // slabs_per_branch is padded to a multiple of 4, so a group never straddles two branches; the
-    // padding slabs (channels beyond O) do nothing.
-    const int branch = (grp * kSlabsPerCta) / p.slabs_per_branch;
-    const bool slab_ok = (slab - branch * p.slabs_per_branch) * 8 < p.f.O;
-    const BranchArgs& br = p.f.branch[branch];
-
-    // ---- stage the activations of this branch in fragment order (once per branch change)
-    if (branch != cur_branch_loaded) {
-      __syncthreads();
-      const int units = p.nms * NMMA * NT * 32;
-      for (int u = threadIdx.x; u < units; u += kThreads) {
-        const int l = u & 31;
-        const int nt = (u >> 5) % NT;
-        const int m = ((u >> 5) / NT) % NMMA;
-        const int ms = (u >> 5) / NT / NMMA;
-        const int n = (l >> 2) + 8 * nt;
-        const int k0 = ms * 4 * CHK + (l & 3) * CHK + 8 * m;
-        uint32_t lo = 0, hi = 0;
-        if (n < p.f.T) {
-          const int8_t* xr = br.xq + static_cast<int64_t>(n) * p.f.ldxq;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            if (k0 + e < I) lo |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + e])) << (8 * e);
-            if (k0 + 4 + e < I) hi |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + 4 + e])) << (8 * e);
-          }
-        }
-        xs[u] = make_uint2(lo, hi);
-      }
-      cur_branch_loaded = branch;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(full0 + 8u * b, kStreamWarps);
+      mbar_init(empty0 + 8u * b, kEpiWarps);
+      mbar_init(stage0 + 8u * b, kStreamWarps);
     }
-    // ---- slab metadata: which orders keep this slab's group, and where its 8 rows start
-    if (slice == 0 && lane == 0) {
-      int nchunks = 0;
-      if (slab_ok) {
-        const int c0 = (slab - branch * p.slabs_per_branch) * 8;
-        const int j = c0 / p.f.g;
-        for (int k = br.k_begin; k < br.k_end; ++k) {
-          const int32_t* cum = p.f.order[k].cum;
-          const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-          if (hi > lo) {
-            slab_meta[slab_local][2 + 2 * nchunks] = k;
-            slab_meta[slab_local][3 + 2 * nchunks] = lo * p.f.g + c0 % p.f.g;
-            ++nchunks;
-          }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // ---- metadata of every slab this CTA owns: which orders keep its group, where its 8 rows start
+  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup; e += kThreads) {
+    const int gi = e / kSlabsPerGroup, sl = e % kSlabsPerGroup;
+    const int grp = blockIdx.x + gi * gridDim.x;
+    const int slab = grp * kSlabsPerGroup + sl;
+    const int branch = slab / p.slabs_per_branch;
+    const int c0 = (slab - branch * p.slabs_per_branch) * 8;
+    int* m = meta + e * kMetaInts;
+    int nchunks = 0;
+    if (c0 < p.f.O) {
+      const BranchArgs& br = p.f.branch[branch];
+      const int j = c0 / p.f.g;
+      for (int k = br.k_begin; k < br.k_end; ++k) {
+        const int32_t* cum = p.f.order[k].cum;
+        const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+        if (hi > lo) {
+          m[2 + 2 * nchunks] = k;
+          m[3 + 2 * nchunks] = lo * p.f.g + c0 % p.f.g;
+          ++nchunks;
         }
       }
-      slab_meta[slab_local][0] = branch;
-      slab_meta[slab_local][1] = nchunks;
     }
-    __syncthreads();
-    const int nchunks = slab_meta[slab_local][1];
-    const int npairs = (nchunks + 1) >> 1;
+    m[0] = c0 < p.f.O ? nchunks : -1;   // -1: padding slab, nothing to store
+    m[1] = branch;
+  }
+  __syncthreads();
 
-    int acc[kMaxPairs][NT][4];
-#pragma unroll
-    for (int q = 0; q < kMaxPairs; ++q)
-#pragma unroll
-      for (int t = 0; t < NT; ++t)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[q][t][e] = 0;
-
-    // macro steps of this warp's slice
+  if (warp < kStreamWarps) {
+    // ================================================================== streaming warps
+    const int sl = warp / kSlices, slice = warp % kSlices;
     const int per = (p.nms + kSlices - 1) / kSlices;
     const int ms_begin = min(slice * per, p.nms), ms_end = min(ms_begin + per, p.nms);
+    const bool has_range = ms_begin < ms_end;
 
+    auto pairs_of = [&](int gi) {
+      const int nch = meta[(gi * kSlabsPerGroup + sl) * kMetaInts];
+      return nch > 0 ? (nch + 1) >> 1 : 0;
+    };
+    // first batch at or after (gi, q = 0)
+    auto first_batch = [&](int gi) {
+      Batch b{-1, 0, 0};
+      if (!has_range) return b;
+      while (gi < my_groups && pairs_of(gi) == 0) ++gi;
+      if (gi < my_groups) b = Batch{gi, 0, ms_begin};
+      return b;
+    };
+    auto next_batch = [&](const Batch& c) {
+      if (c.ms0 + kBatch < ms_end) return Batch{c.gi, c.q, c.ms0 + kBatch};
+      if (c.q + 1 < pairs_of(c.gi)) return Batch{c.gi, c.q + 1, ms_begin};
+      return first_batch(c.gi + 1);
+    };
+    auto issue = [&](const Batch& b, uint4 (&wa)[kBatch], uint4 (&wb)[kBatch]) {
+      if (b.gi < 0) return;
+      const int* m = meta + (b.gi * kSlabsPerGroup + sl) * kMetaInts;
+      const int nch = m[0];
+      const int k_a = m[2 + 4 * b.q], row_a = m[3 + 4 * b.q];
+      const bool has_b = 2 * b.q + 1 < nch;
+      const int k_b = has_b ? m[4 + 4 * b.q] : k_a;
+      const int row_b = has_b ? m[5 + 4 * b.q] : row_a;
+      const uint8_t* base_a = p.f.order[k_a].kcodes + static_cast<size_t>(row_a + gid) * p.pk;
+      const uint8_t* base_b = p.f.order[k_b].kcodes + static_cast<size_t>(row_b + gid) * p.pk;
+      const size_t blk_a = static_cast<size_t>(p.f.order[k_a].rows) * p.pk;
+      const size_t blk_b = static_cast<size_t>(p.f.order[k_b].rows) * p.pk;
 #pragma unroll
-    for (int q = 0; q < kMaxPairs; ++q) {
-      if (q >= npairs) break;
-      const int k_a = slab_meta[slab_local][2 + 4 * q], row_a = slab_meta[slab_local][3 + 4 * q];
-      const bool has_b = 2 * q + 1 < nchunks;
-      const int k_b = has_b ? slab_meta[slab_local][4 + 4 * q] : k_a;
-      const int row_b = has_b ? slab_meta[slab_local][5 + 4 * q] : row_a;
-      const OrderView& oa = p.f.order[k_a];
-      const OrderView& ob = p.f.order[k_b];
-      for (int ms0 = ms_begin; ms0 < ms_end; ms0 += kBatch) {
-        uint4 wa[kBatch], wb[kBatch];
-#pragma unroll
-        for (int s = 0; s < kBatch; ++s) {
-          const int ms = ms0 + s;
-          wa[s] = make_uint4(0, 0, 0, 0);
-          wb[s] = make_uint4(0, 0, 0, 0);
-          if (ms < ms_end) {
-            // byte position of this thread's chunk: reduction offset ms*4*CHK + tig*CHK
-            const int kcode = ms * 4 * CHK + tig * CHK;
-            const int kb = kcode >> 7;
-            if (kb < p.kblocks) {
-              const int inblk = ((kcode & 127) * BITS) >> 3;
-              const size_t oa_off = (static_cast<size_t>(kb) * oa.rows + row_a + gid) * p.pk + inblk;
-              wa[s] = __ldg(reinterpret_cast<const uint4*>(oa.kcodes + oa_off));
-              if (has_b) {
-                const size_t ob_off = (static_cast<size_t>(kb) * ob.rows + row_b + gid) * p.pk + inblk;
-                wb[s] = __ldg(reinterpret_cast<const uint4*>(ob.kcodes + ob_off));
-              }
-            }
-          }
-        }
-#pragma unroll
-        for (int s = 0; s < kBatch; ++s) {
-          const int ms = ms0 + s;
-          if (ms >= ms_end) break;
-          uint32_t ra[16], rb[16];
-          unpack_chunk<BITS>(wa[s], ra);
-          unpack_chunk<BITS>(wb[s], rb);
-          const uint2* xf = xs + static_cast<size_t>(ms) * NMMA * NT * 32 + lane;
-#pragma unroll
-          for (int m = 0; m < NMMA; ++m)
-#pragma unroll
-            for (int t = 0; t < NT; ++t) {
-              const uint2 b = xf[(m * NT + t) * 32];
-              // tile rows 0-7: order k_a, rows 8-15: order k_b
-              mma_s8(acc[q][t], ra[2 * m], rb[2 * m], ra[2 * m + 1], rb[2 * m + 1], b.x, b.y);
-            }
+      for (int s = 0; s < kBatch; ++s) {
+        const int ms = b.ms0 + s;
+        wa[s] = make_uint4(0, 0, 0, 0);
+        wb[s] = make_uint4(0, 0, 0, 0);
+        // this thread's chunk starts at reduction offset ms*4*CHK + tig*CHK
+        const int kcode = ms * 4 * CHK + tig * CHK;
+        const int kb = kcode >> 7;
+        if (ms < ms_end && kb < p.kblocks) {
+          const int inblk = ((kcode & 127) * BITS) >> 3;
+          wa[s] = __ldg(reinterpret_cast<const uint4*>(base_a + kb * blk_a + inblk));
+          if (has_b) wb[s] = __ldg(reinterpret_cast<const uint4*>(base_b + kb * blk_b + inblk));
         }
       }
-    }
+    };
 
-    // ---- add the slices' exact partial sums; slice 0 keeps the total
-    if (slice != 0) {
+    uint4 na[kBatch], nb[kBatch];
+    Batch nxt = first_batch(0);
+    issue(nxt, na, nb);
+
+    int staged_branch = -1;
+    uint32_t stage_uses = 0;
+    for (int gi = 0; gi < my_groups; ++gi) {
+      const int* m = meta + (gi * kSlabsPerGroup + sl) * kMetaInts;
+      const int branch = meta[(gi * kSlabsPerGroup) * kMetaInts + 1];   // the group's branch (slab 0 of the group)
+      // ---- (re)stage the activations in fragment order when the branch changes
+      if (branch != staged_branch) {
+        // everybody has finished reading the old fragments ...
+        __syncwarp();
+        if (lane == 0) mbar_arrive(stage0);
+        if (!mbar_wait(stage0, stage_uses & 1, abort_flag, p.f.status)) break;
+        const BranchArgs& br = p.f.branch[branch];
+        const int units = p.nms * NMMA * NT * 32;
+        for (int u = threadIdx.x; u < units; u += 32 * kStreamWarps) {
+          const int l = u & 31;
+          const int nt = (u >> 5) % NT;
+          const int mm = ((u >> 5) / NT) % NMMA;
+          const int ms = (u >> 5) / NT / NMMA;
+          const int n = (l >> 2) + 8 * nt;
+          const int k0 = ms * 4 * CHK + (l & 3) * CHK + 8 * mm;
+          uint32_t lo = 0, hi = 0;
+          if (n < p.f.T) {
+            const int8_t* xr = br.xq + static_cast<int64_t>(n) * p.f.ldxq;
 #pragma unroll
-      for (int q = 0; q < kMaxPairs; ++q) {
-        if (q >= npairs) break;
-        int* dst = red + ((((slab_local * (kSlices - 1) + slice - 1) * kMaxPairs + q) * 32 + lane) * (4 * NT));
+            for (int e = 0; e < 4; ++e) {
+              if (k0 + e < I) lo |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + e])) << (8 * e);
+              if (k0 + 4 + e < I) hi |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + 4 + e])) << (8 * e);
+            }
+          }
+          xs[u] = make_uint2(lo, hi);
+        }
+        // ... and everybody sees the new ones
+        __syncwarp();
+        if (lane == 0) mbar_arrive(stage0 + 8);
+        if (!mbar_wait(stage0 + 8, stage_uses & 1, abort_flag, p.f.status)) break;
+        ++stage_uses;
+        staged_branch = branch;
+      }
+      const int nch = m[0];
+      const int npairs = nch > 0 ? (nch + 1) >> 1 : 0;
+      const int buf = gi & 1;
+      // the epilogue warps must have drained this buffer (group gi - 2)
+      if (!mbar_wait(empty0 + 8u * buf, ((gi >> 1) & 1) ^ 1, abort_flag, p.f.status)) break;
+      int* dst_base = red + buf * RED_INTS + ((sl * kSlices + slice) * p.np * 32 + lane) * (4 * NT);
+      for (int q = 0; q < npairs; ++q) {
+        int acc[NT][4];
 #pragma unroll
         for (int t = 0; t < NT; ++t)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) dst[t * 4 + e] = acc[q][t][e];
-      }
-    }
-    __syncthreads();
-    if (slice == 0 && slab_ok) {
-      const float sx = __ldg(br.sx);
-      const int c = (slab - branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
-      float y[NT][2];
+          for (int e = 0; e < 4; ++e) acc[t][e] = 0;
+        if (has_range) {
+          for (int ms0 = ms_begin; ms0 < ms_end; ms0 += kBatch) {
+            // the loads of this batch were issued one batch ago; issue the next batch now
+            uint4 wa[kBatch], wb[kBatch];
 #pragma unroll
-      for (int t = 0; t < NT; ++t) y[t][0] = y[t][1] = 0.f;
-#pragma unroll
-      for (int q = 0; q < kMaxPairs; ++q) {
-        if (q >= npairs) break;
-#pragma unroll
-        for (int sl = 1; sl < kSlices; ++sl) {
-          const int* src = red + ((((slab_local * (kSlices - 1) + sl - 1) * kMaxPairs + q) * 32 + lane) * (4 * NT));
-#pragma unroll
-          for (int t = 0; t < NT; ++t)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[q][t][e] += src[t * 4 + e];
-        }
-        // accumulator registers 0,1: tile row gid (order k_a); 2,3: tile row gid + 8 (order k_b);
-        // columns 2*tig, 2*tig + 1 of token tile t.  Ascending order: k_a first, then k_b.
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          if (2 * q + half >= nchunks) break;
-          const int k = slab_meta[slab_local][2 + 2 * (2 * q + half)];
-          const int row = slab_meta[slab_local][3 + 2 * (2 * q + half)] + gid;
-          const OrderView& ov = p.f.order[k];
-          const float cs = __fmul_rn(__ldg(ov.scales + row), sx);
-#pragma unroll
-          for (int t = 0; t < NT; ++t)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int a = acc[q][t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
-              y[t][e] = __fmaf_rn(__int2float_rn(a), cs, y[t][e]);
-              const int tok = 8 * t + 2 * tig + e;
-              if (p.f.partials && tok < p.f.T) p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + ov.row_off + row] = a;
+            for (int s = 0; s < kBatch; ++s) {
+              wa[s] = na[s];
+              wb[s] = nb[s];
             }
+            nxt = next_batch(Batch{gi, q, ms0});
+            issue(nxt, na, nb);
+#pragma unroll
+            for (int s = 0; s < kBatch; ++s) {
+              const int ms = ms0 + s;
+              if (ms >= ms_end) break;
+              uint32_t ra[16], rb[16];
+              unpack_chunk<BITS>(wa[s], ra);
+              unpack_chunk<BITS>(wb[s], rb);
+              const uint2* xf = xs + static_cast<size_t>(ms) * NMMA * NT * 32 + lane;
+#pragma unroll
+              for (int mm = 0; mm < NMMA; ++mm)
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                  const uint2 b = xf[(mm * NT + t) * 32];
+                  // tile rows 0-7: first order of the pair, rows 8-15: second order
+                  mma_s8(acc[t], ra[2 * mm], rb[2 * mm], ra[2 * mm + 1], rb[2 * mm + 1], b.x, b.y);
+                }
+            }
+          }
+        }
+        int* dst = dst_base + q * 32 * (4 * NT);
+#pragma unroll
+        for (int t = 0; t < NT; ++t)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) dst[t * 4 + e] = acc[t][e];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full0 + 8u * buf);
+    }
+  } else {
+    // ================================================================== epilogue warps (one per slab)
+    const int sl = warp - kStreamWarps;
+    for (int gi = 0; gi < my_groups; ++gi) {
+      const int* m = meta + (gi * kSlabsPerGroup + sl) * kMetaInts;
+      const int nch = m[0];
+      const int branch = m[1];
+      const int npairs = nch > 0 ? (nch + 1) >> 1 : 0;
+      const int buf = gi & 1;
+      const int grp = blockIdx.x + gi * gridDim.x;
+      const int slab = grp * kSlabsPerGroup + sl;
+      const int c = (slab - branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
+      // scale products of this thread's rows, fetched before the partial sums are waited for
+      float cs[2 * kMaxPairs];
+      int rows[2 * kMaxPairs], roff[2 * kMaxPairs];
+      float sx = 0.f, bv = 0.f;
+      bool bias = false;
+      if (nch >= 0) {
+        const BranchArgs& br = p.f.branch[branch];
+        sx = __ldg(br.sx);
+        bias = br.add_bias && p.f.bias;
+        if (bias) bv = __ldg(p.f.bias + c);
+      }
+#pragma unroll
+      for (int ci = 0; ci < 2 * kMaxPairs; ++ci) {
+        cs[ci] = 0.f;
+        rows[ci] = 0;
+        roff[ci] = 0;
+        if (ci < nch) {
+          const OrderView& ov = p.f.order[m[2 + 2 * ci]];
+          rows[ci] = m[3 + 2 * ci] + gid;
+          roff[ci] = ov.row_off;
+          cs[ci] = __fmul_rn(__ldg(ov.scales + rows[ci]), sx);
         }
       }
-      const bool bias = br.add_bias && p.f.bias;
-      const float bv = bias ? __ldg(p.f.bias + c) : 0.f;
+      if (!mbar_wait(full0 + 8u * buf, (gi >> 1) & 1, abort_flag, p.f.status)) break;
+      if (nch >= 0) {
+        const BranchArgs& br = p.f.branch[branch];
+        float y[NT][2];
 #pragma unroll
-      for (int t = 0; t < NT; ++t)
+        for (int t = 0; t < NT; ++t) y[t][0] = y[t][1] = 0.f;
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int tok = 8 * t + 2 * tig + e;
-          if (tok >= p.f.T) continue;
-          float v = y[t][e];
-          if (bias) v = __fadd_rn(v, bv);
-          float* dst = br.y + static_cast<int64_t>(tok) * p.f.ldy + c;
-          if (br.accumulate) v = __fadd_rn(*dst, v);
-          *dst = v;
+        for (int q = 0; q < kMaxPairs; ++q) {
+          if (q >= npairs) break;
+          int acc[NT][4];
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[t][e] = 0;
+#pragma unroll
+          for (int s = 0; s < kSlices; ++s) {
+            const int* src = red + buf * RED_INTS + (((sl * kSlices + s) * p.np + q) * 32 + lane) * (4 * NT);
+#pragma unroll
+            for (int t = 0; t < NT; ++t)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) acc[t][e] += src[t * 4 + e];
+          }
+          // accumulator registers 0,1: tile row gid (first order of the pair); 2,3: tile row gid + 8
+          // (second order); columns 2*tig, 2*tig + 1 of token tile t.  Ascending order.
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int ci = 2 * q + half;
+            if (ci >= nch) break;
+#pragma unroll
+            for (int t = 0; t < NT; ++t)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const int a = acc[t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
+                y[t][e] = __fmaf_rn(__int2float_rn(a), cs[ci], y[t][e]);
+                const int tok = 8 * t + 2 * tig + e;
+                if (p.f.partials && tok < p.f.T)
+                  p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff[ci] + rows[ci]] = a;
+              }
+          }
         }
+#pragma unroll
+        for (int t = 0; t < NT; ++t)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int tok = 8 * t + 2 * tig + e;
+            if (tok >= p.f.T) continue;
+            float v = y[t][e];
+            if (bias) v = __fadd_rn(v, bv);
+            float* dst = br.y + static_cast<int64_t>(tok) * p.f.ldy + c;
+            if (br.accumulate) v = __fadd_rn(*dst, v);
+            *dst = v;
+          }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * buf);
     }
-    __syncthreads();   // red[] and slab_meta[] are reused by the next group
   }
 }
 
@@ -280,31 +422,33 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   if (max_cluster > 2 * kMaxPairs) return PIPE_ERR_UNSUPPORTED;
   Params p;
   p.f = a;
-  p.nt = a.T <= 8 ? 1 : 2;
-  p.chk = 128 / a.bits;
-  p.nmma = p.chk / 8;
+  const int nt = a.T <= 8 ? 1 : 2;
+  const int chk = 128 / a.bits;
   p.kblocks = ceil_div(a.I, 128);
-  p.nms = ceil_div(p.kblocks * 128, 4 * p.chk);
+  p.nms = ceil_div(p.kblocks * 128, 4 * chk);
   p.pk = 128 * a.bits / 8;
   p.shift = 8 - a.bits;
-  // groups of 4 slabs must not straddle branches: pad every branch to a multiple of 4 slabs
-  p.slabs_per_branch = round_up(a.O / 8, kSlabsPerCta);
-  p.total_slabs = p.slabs_per_branch * a.num_branches;
-  p.xs_bytes = round_up(p.nms * p.nmma * p.nt * 32 * 8, 16);
-  p.red_bytes = kSlabsPerCta * (kSlices - 1) * kMaxPairs * 32 * 4 * p.nt * 4;
-  const int dyn = p.xs_bytes + p.red_bytes;
+  // groups of slabs must not straddle branches: pad every branch to a multiple of the group size
+  p.slabs_per_branch = round_up(a.O / 8, kSlabsPerGroup);
+  p.groups = p.slabs_per_branch * a.num_branches / kSlabsPerGroup;
+  p.xs_bytes = round_up(p.nms * (chk / 8) * nt * 32 * 8, 16);
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (dyn + 2048 > smem_max) return PIPE_ERR_UNSUPPORTED;
-  const int groups = p.total_slabs / kSlabsPerCta;
-  const int grid = groups < sms ? groups : sms;
+  const int grid = p.groups < sms ? p.groups : sms;
+  const int own = ceil_div(p.groups, grid);
+  if (own > kMaxGroups) return PIPE_ERR_UNSUPPORTED;
+  p.np = (max_cluster + 1) / 2;
+  const int red_bytes = 2 * kSlabsPerGroup * kSlices * p.np * 32 * 4 * nt * 4;
+  const int meta_bytes = own * kSlabsPerGroup * kMetaInts * 4;
+  const int dyn = p.xs_bytes + red_bytes + meta_bytes;
+  if (dyn + 1024 > smem_max) return PIPE_ERR_UNSUPPORTED;
 
   void (*kern)(const Params) = nullptr;
-  if (a.bits == 8) kern = p.nt == 1 ? stream_forward_kernel<8, 1> : stream_forward_kernel<8, 2>;
-  else if (a.bits == 4) kern = p.nt == 1 ? stream_forward_kernel<4, 1> : stream_forward_kernel<4, 2>;
-  else kern = p.nt == 1 ? stream_forward_kernel<2, 1> : stream_forward_kernel<2, 2>;
+  if (a.bits == 8) kern = nt == 1 ? stream_forward_kernel<8, 1> : stream_forward_kernel<8, 2>;
+  else if (a.bits == 4) kern = nt == 1 ? stream_forward_kernel<4, 1> : stream_forward_kernel<4, 2>;
+  else kern = nt == 1 ? stream_forward_kernel<2, 1> : stream_forward_kernel<2, 2>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess) return PIPE_ERR_CUDA;
   kern<<<grid, kThreads, dyn, stream>>>(p);
   count_launch(1);

@@ -91,14 +91,26 @@ class LayerRunner:
         for m in range(len(self.x)):
             B.pipe_quantize_act(self.x[m], self.xq[m], self.sx[m], self.quant_ws[m])
 
-    def forward(self, partials: torch.Tensor | None = None) -> None:
+    def forward(self, partials: torch.Tensor | None = None, blob: torch.Tensor | None = None) -> None:
+        blob = self.blob if blob is None else blob
         if self.M == 1:
-            B.pipe_expanded_linear(self.desc, self.blob, self.xq[0], self.sx[0], self.y[0], None, partials)
+            B.pipe_expanded_linear(self.desc, blob, self.xq[0], self.sx[0], self.y[0], None, partials)
         else:
             n = len(self.xq)
             xq = [self.xq[m if n > 1 else 0] for m in range(self.M)]
             sx = [self.sx[m if n > 1 else 0] for m in range(self.M)]
-            B.pipe_ensemble_forward(self.desc, self.blob, xq, sx, self.y, None, False, partials)
+            B.pipe_ensemble_forward(self.desc, blob, xq, sx, self.y, None, False, partials)
+
+    def blob_copies(self, min_total_bytes: int) -> list:
+        """The expanded blob plus enough byte copies of it that together they exceed
+        ``min_total_bytes`` (for timing loops that must not re-read weights from L2)."""
+        n = max(1, -(-int(min_total_bytes) // int(self.layout.blob_bytes)))
+        out = [self.blob]
+        for _ in range(n - 1):
+            c = B.alloc_bytes(self.layout.blob_bytes, self.device)
+            c.copy_(self.blob)
+            out.append(c)
+        return out
 
     def step(self) -> None:
         self.expand()
