@@ -10,9 +10,9 @@
 // Work unit: a "slab" = 8 consecutive output channels of one branch.  In every order of the branch
 // that keeps the slab's group, the slab is 8 consecutive compacted rows.  Two such 8-row chunks
 // (two orders, ascending) form one 16-row MMA tile, so both orders of a pair accumulate in the same
-// thread and the fixed-order fp32 epilogue is thread-local.  A persistent CTA walks groups of 2
-// slabs: 8 streaming warps (4 per slab, each owning a range of the reduction axis) drop their exact
-// int32 partial sums into a double-buffered shared-memory area; 2 epilogue warps (one per slab)
+// thread and the fixed-order fp32 epilogue is thread-local.  A persistent CTA walks groups of 4
+// slabs: 16 streaming warps (4 per slab, each owning a range of the reduction axis) drop their exact
+// int32 partial sums into a double-buffered shared-memory area; 4 epilogue warps (one per slab)
 // add the four ranges, apply the scales in ascending order and store, while the streaming warps
 // are already on the next group.  The quantized activations sit in shared memory in MMA-fragment
 // order; all slab metadata of the CTA is gathered once, up front, with independent loads.
@@ -22,13 +22,13 @@ namespace pipe {
 
 namespace st {
 
-constexpr int kStreamWarps = 8;
-constexpr int kEpiWarps = 2;
+constexpr int kStreamWarps = 16;
+constexpr int kEpiWarps = 4;
 constexpr int kThreads = 32 * (kStreamWarps + kEpiWarps);
-constexpr int kSlabsPerGroup = 2;
+constexpr int kSlabsPerGroup = 4;
 constexpr int kSlices = 4;        // streaming warps per slab
 constexpr int kMaxPairs = 4;      // up to 8 orders per branch
-constexpr int kBatch = 8;         // macro steps whose loads are issued together
+constexpr int kBatch = 4;         // macro steps whose loads are issued together
 constexpr int kMaxGroups = 128;   // groups one CTA may own (metadata table size)
 constexpr int kMetaInts = 2 + 4 * kMaxPairs;   // nchunks, branch, then (order, row0) per chunk
 constexpr long long kWaitLimitCycles = 4000000000ll;
@@ -241,6 +241,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
         if (lane == 0) mbar_arrive(stage0);
         if (!mbar_wait(stage0, stage_uses & 1, abort_flag, p.f.status)) break;
         const BranchArgs& br = p.f.branch[branch];
+        const bool x_vec = ((reinterpret_cast<uintptr_t>(br.xq) | static_cast<uintptr_t>(p.f.ldxq)) & 7) == 0;
         const int units = p.nms * NMMA * NT * 32;
         for (int u = threadIdx.x; u < units; u += 32 * kStreamWarps) {
           const int l = u & 31;
@@ -252,10 +253,16 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
           uint32_t lo = 0, hi = 0;
           if (n < p.f.T) {
             const int8_t* xr = br.xq + static_cast<int64_t>(n) * p.f.ldxq;
+            if (x_vec && k0 + 8 <= I) {
+              const uint2 v = __ldg(reinterpret_cast<const uint2*>(xr + k0));
+              lo = v.x;
+              hi = v.y;
+            } else {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              if (k0 + e < I) lo |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + e])) << (8 * e);
-              if (k0 + 4 + e < I) hi |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + 4 + e])) << (8 * e);
+              for (int e = 0; e < 4; ++e) {
+                if (k0 + e < I) lo |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + e])) << (8 * e);
+                if (k0 + 4 + e < I) hi |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + 4 + e])) << (8 * e);
+              }
             }
           }
           xs[u] = make_uint2(lo, hi);
