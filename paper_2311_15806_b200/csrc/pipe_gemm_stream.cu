@@ -14,8 +14,9 @@
 // slabs: 16 streaming warps (4 per slab, each owning a range of the reduction axis) drop their exact
 // int32 partial sums into a double-buffered shared-memory area; 4 epilogue warps (one per slab)
 // add the four ranges, apply the scales in ascending order and store, while the streaming warps
-// are already on the next group.  The quantized activations sit in shared memory in MMA-fragment
-// order; all slab metadata of the CTA is gathered once, up front, with independent loads.
+// are already on the next group.  The quantized activations (at most 16 rows) are read as MMA
+// fragments straight from global memory: they stay resident in L1.  All slab metadata and scale
+// products of the CTA are gathered once, up front, with independent loads.
 #include "pipe_common.cuh"
 
 namespace pipe {
@@ -123,10 +124,12 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
   constexpr int NMMA = CHK / 8;          // MMAs per macro step
   const int RED_INTS = kSlabsPerGroup * kSlices * p.np * 32 * 4 * NT;   // one buffer of partial sums
   extern __shared__ uint4 smem_u4[];
-  uint2* xs = reinterpret_cast<uint2*>(smem_u4);                                             // [nms][NMMA][NT][32]
-  int* red = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(smem_u4) + p.xs_bytes);      // [2][slab][slice][pair][lane][4*NT]
-  int* meta = red + 2 * RED_INTS;                                                            // [own groups][slab][kMetaInts]
-  __shared__ uint64_t bars[6];   // full[2] empty[2] stage[2]
+  int* red = reinterpret_cast<int*>(smem_u4);                    // [2][slab][slice][pair][lane][4*NT]
+  int* meta = red + 2 * RED_INTS;                                // [own slabs][kMetaInts]
+  const int my_groups_ = (p.groups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  float* cstab = reinterpret_cast<float*>(meta + my_groups_ * kSlabsPerGroup * kMetaInts);   // [own slabs][2*np][8] s_k * lambda_x
+  float* biastab = cstab + my_groups_ * kSlabsPerGroup * 2 * p.np * 8;                        // [own slabs][8]
+  __shared__ uint64_t bars[4];   // full[2] empty[2]
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
 
@@ -135,14 +138,13 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
   const int I = p.f.I;
   const int my_groups = (p.groups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
   const uint32_t bar0 = smem_u32(bars);
-  const uint32_t full0 = bar0, empty0 = bar0 + 16, stage0 = bar0 + 32;
+  const uint32_t full0 = bar0, empty0 = bar0 + 16;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int b = 0; b < 2; ++b) {
       mbar_init(full0 + 8u * b, kStreamWarps);
       mbar_init(empty0 + 8u * b, kEpiWarps);
-      mbar_init(stage0 + 8u * b, kStreamWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -170,6 +172,29 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
     }
     m[0] = c0 < p.f.O ? nchunks : -1;   // -1: padding slab, nothing to store
     m[1] = branch;
+  }
+  __syncthreads();
+  // ---- scale products s_k * lambda_x of every row this CTA will finish, and its bias values
+  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup * 2 * p.np * 8; e += kThreads) {
+    const int r = e & 7, ci = (e >> 3) % (2 * p.np), slab_i = (e >> 3) / (2 * p.np);
+    const int* m = meta + slab_i * kMetaInts;
+    float v = 0.f;
+    if (ci < m[0]) {
+      const BranchArgs& br = p.f.branch[m[1]];
+      v = __fmul_rn(__ldg(p.f.order[m[2 + 2 * ci]].scales + m[3 + 2 * ci] + r), __ldg(br.sx));
+    }
+    cstab[e] = v;
+  }
+  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup * 8; e += kThreads) {
+    const int r = e & 7, slab_i = e >> 3;
+    const int* m = meta + slab_i * kMetaInts;
+    float v = 0.f;
+    if (m[0] >= 0 && p.f.bias && p.f.branch[m[1]].add_bias) {
+      const int gi = slab_i / kSlabsPerGroup, sl = slab_i % kSlabsPerGroup;
+      const int slab = (blockIdx.x + gi * gridDim.x) * kSlabsPerGroup + sl;
+      v = __ldg(p.f.bias + (slab - m[1] * p.slabs_per_branch) * 8 + r);
+    }
+    biastab[e] = v;
   }
   __syncthreads();
 
@@ -229,50 +254,17 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
     Batch nxt = first_batch(0);
     issue(nxt, na, nb);
 
-    int staged_branch = -1;
-    uint32_t stage_uses = 0;
     for (int gi = 0; gi < my_groups; ++gi) {
       const int* m = meta + (gi * kSlabsPerGroup + sl) * kMetaInts;
       const int branch = meta[(gi * kSlabsPerGroup) * kMetaInts + 1];   // the group's branch (slab 0 of the group)
-      // ---- (re)stage the activations in fragment order when the branch changes
-      if (branch != staged_branch) {
-        // everybody has finished reading the old fragments ...
-        __syncwarp();
-        if (lane == 0) mbar_arrive(stage0);
-        if (!mbar_wait(stage0, stage_uses & 1, abort_flag, p.f.status)) break;
-        const BranchArgs& br = p.f.branch[branch];
-        const bool x_vec = ((reinterpret_cast<uintptr_t>(br.xq) | static_cast<uintptr_t>(p.f.ldxq)) & 7) == 0;
-        const int units = p.nms * NMMA * NT * 32;
-        for (int u = threadIdx.x; u < units; u += 32 * kStreamWarps) {
-          const int l = u & 31;
-          const int nt = (u >> 5) % NT;
-          const int mm = ((u >> 5) / NT) % NMMA;
-          const int ms = (u >> 5) / NT / NMMA;
-          const int n = (l >> 2) + 8 * nt;
-          const int k0 = ms * 4 * CHK + (l & 3) * CHK + 8 * mm;
-          uint32_t lo = 0, hi = 0;
-          if (n < p.f.T) {
-            const int8_t* xr = br.xq + static_cast<int64_t>(n) * p.f.ldxq;
-            if (x_vec && k0 + 8 <= I) {
-              const uint2 v = __ldg(reinterpret_cast<const uint2*>(xr + k0));
-              lo = v.x;
-              hi = v.y;
-            } else {
+      const BranchArgs& br = p.f.branch[branch];
+      // this thread's activation rows (token gid of each 8-token tile); aligned rows take 16-byte loads
+      const int8_t* xrow[NT];
+      bool xok[NT];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                if (k0 + e < I) lo |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + e])) << (8 * e);
-                if (k0 + 4 + e < I) hi |= static_cast<uint32_t>(static_cast<uint8_t>(xr[k0 + 4 + e])) << (8 * e);
-              }
-            }
-          }
-          xs[u] = make_uint2(lo, hi);
-        }
-        // ... and everybody sees the new ones
-        __syncwarp();
-        if (lane == 0) mbar_arrive(stage0 + 8);
-        if (!mbar_wait(stage0 + 8, stage_uses & 1, abort_flag, p.f.status)) break;
-        ++stage_uses;
-        staged_branch = branch;
+      for (int t = 0; t < NT; ++t) {
+        xok[t] = gid + 8 * t < p.f.T;
+        xrow[t] = br.xq + static_cast<int64_t>(xok[t] ? gid + 8 * t : 0) * p.f.ldxq;
       }
       const int nch = m[0];
       const int npairs = nch > 0 ? (nch + 1) >> 1 : 0;
@@ -304,15 +296,26 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
               uint32_t ra[16], rb[16];
               unpack_chunk<BITS>(wa[s], ra);
               unpack_chunk<BITS>(wb[s], rb);
-              const uint2* xf = xs + static_cast<size_t>(ms) * NMMA * NT * 32 + lane;
+              // B fragments: CHK consecutive activation codes of this thread's token, from
+              // reduction offset ms*4*CHK + tig*CHK (register 2m covers 8m..8m+3, 2m+1 covers 8m+4..8m+7)
+              const int kx = ms * 4 * CHK + tig * CHK;
 #pragma unroll
-              for (int mm = 0; mm < NMMA; ++mm)
+              for (int t = 0; t < NT; ++t) {
+                uint32_t xb[2 * NMMA];
 #pragma unroll
-                for (int t = 0; t < NT; ++t) {
-                  const uint2 b = xf[(mm * NT + t) * 32];
-                  // tile rows 0-7: first order of the pair, rows 8-15: second order
-                  mma_s8(acc[t], ra[2 * mm], rb[2 * mm], ra[2 * mm + 1], rb[2 * mm + 1], b.x, b.y);
+                for (int v = 0; v < NMMA / 2; ++v) {
+                  uint4 xv = make_uint4(0, 0, 0, 0);
+                  if (xok[t]) {
+                    const int k16 = kx + 16 * v;
+                    if (k16 < I) xv = __ldg(reinterpret_cast<const uint4*>(xrow[t] + k16));   // I % 16 == 0 (host check)
+                  }
+                  xb[4 * v] = xv.x; xb[4 * v + 1] = xv.y; xb[4 * v + 2] = xv.z; xb[4 * v + 3] = xv.w;
                 }
+#pragma unroll
+                for (int mm = 0; mm < NMMA; ++mm)
+                  // tile rows 0-7: first order of the pair, rows 8-15: second order
+                  mma_s8(acc[t], ra[2 * mm], rb[2 * mm], ra[2 * mm + 1], rb[2 * mm + 1], xb[2 * mm], xb[2 * mm + 1]);
+              }
             }
           }
         }
@@ -337,29 +340,9 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
       const int grp = blockIdx.x + gi * gridDim.x;
       const int slab = grp * kSlabsPerGroup + sl;
       const int c = (slab - branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
-      // scale products of this thread's rows, fetched before the partial sums are waited for
-      float cs[2 * kMaxPairs];
-      int rows[2 * kMaxPairs], roff[2 * kMaxPairs];
-      float sx = 0.f, bv = 0.f;
-      bool bias = false;
-      if (nch >= 0) {
-        const BranchArgs& br = p.f.branch[branch];
-        sx = __ldg(br.sx);
-        bias = br.add_bias && p.f.bias;
-        if (bias) bv = __ldg(p.f.bias + c);
-      }
-#pragma unroll
-      for (int ci = 0; ci < 2 * kMaxPairs; ++ci) {
-        cs[ci] = 0.f;
-        rows[ci] = 0;
-        roff[ci] = 0;
-        if (ci < nch) {
-          const OrderView& ov = p.f.order[m[2 + 2 * ci]];
-          rows[ci] = m[3 + 2 * ci] + gid;
-          roff[ci] = ov.row_off;
-          cs[ci] = __fmul_rn(__ldg(ov.scales + rows[ci]), sx);
-        }
-      }
+      const float* cs_slab = cstab + (gi * kSlabsPerGroup + sl) * 2 * p.np * 8;
+      const float bv = biastab[(gi * kSlabsPerGroup + sl) * 8 + gid];
+      const bool bias = nch >= 0 && p.f.bias && p.f.branch[branch].add_bias;
       if (!mbar_wait(full0 + 8u * buf, (gi >> 1) & 1, abort_flag, p.f.status)) break;
       if (nch >= 0) {
         const BranchArgs& br = p.f.branch[branch];
@@ -388,15 +371,17 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
           for (int half = 0; half < 2; ++half) {
             const int ci = 2 * q + half;
             if (ci >= nch) break;
+            const float cs = cs_slab[ci * 8 + gid];
+            const int row = m[3 + 2 * ci] + gid, roff = p.f.order[m[2 + 2 * ci]].row_off;
 #pragma unroll
             for (int t = 0; t < NT; ++t)
 #pragma unroll
               for (int e = 0; e < 2; ++e) {
                 const int a = acc[t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
-                y[t][e] = __fmaf_rn(__int2float_rn(a), cs[ci], y[t][e]);
+                y[t][e] = __fmaf_rn(__int2float_rn(a), cs, y[t][e]);
                 const int tok = 8 * t + 2 * tig + e;
                 if (p.f.partials && tok < p.f.T)
-                  p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff[ci] + rows[ci]] = a;
+                  p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff + row] = a;
               }
           }
         }
@@ -424,6 +409,10 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
 static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   using namespace st;
   if (a.T > 16 || a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
+  // activation fragments are fetched with 16-byte loads
+  if (a.I % 16 != 0 || a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
+  for (int m = 0; m < a.num_branches; ++m)
+    if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
   if (max_cluster > 2 * kMaxPairs) return PIPE_ERR_UNSUPPORTED;
@@ -438,7 +427,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   // groups of slabs must not straddle branches: pad every branch to a multiple of the group size
   p.slabs_per_branch = round_up(a.O / 8, kSlabsPerGroup);
   p.groups = p.slabs_per_branch * a.num_branches / kSlabsPerGroup;
-  p.xs_bytes = round_up(p.nms * (chk / 8) * nt * 32 * 8, 16);
+  p.xs_bytes = 0;
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -448,8 +437,8 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   if (own > kMaxGroups) return PIPE_ERR_UNSUPPORTED;
   p.np = (max_cluster + 1) / 2;
   const int red_bytes = 2 * kSlabsPerGroup * kSlices * p.np * 32 * 4 * nt * 4;
-  const int meta_bytes = own * kSlabsPerGroup * kMetaInts * 4;
-  const int dyn = p.xs_bytes + red_bytes + meta_bytes;
+  const int meta_bytes = own * kSlabsPerGroup * (kMetaInts + 2 * p.np * 8 + 8) * 4;
+  const int dyn = red_bytes + meta_bytes;
   if (dyn + 1024 > smem_max) return PIPE_ERR_UNSUPPORTED;
 
   void (*kern)(const Params) = nullptr;
