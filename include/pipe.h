@@ -205,6 +205,29 @@ pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blo
                                   float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials,
                                   void* stream);
 
+/*
+ * The expanded layer as a stride-1 "same" convolution (Appendix H counts a d x d convolution as
+ * d^2 * n_i * n_o multiplications per output pixel: the same contraction with the reduction
+ * index running over (tap, input channel)).  Implicit GEMM: the quantized NHWC input is read in
+ * place, tap by tap, with zero padding supplied by the copy engine; no im2col matrix exists.
+ * Output row t = (n*H + h)*W + w, reduction index (dh*kernel_w + dw)*C + c, i.e. the weight
+ * tensor [O, kernel_h, kernel_w, C] flattened to [O, I] with I = kernel_h*kernel_w*C = in_features.
+ * All K orders act on the one input (as in pipe_expanded_linear).
+ * d_xq: int8 [N, H, W, C], dense, 16-byte aligned (quantize it with pipe_quantize_act as a
+ * [N*H*W, C] matrix).  d_y: float [N*H*W, O] pitch ldy.  d_partials as in pipe_expanded_linear.
+ * This build takes kernel 2*pad + 1 square or not, stride 1, C a multiple of 128 and H, W
+ * multiples of 8; anything else returns PIPE_ERR_UNSUPPORTED.
+ */
+typedef struct pipe_conv_geom {
+  int32_t batch, height, width, channels; /* N, H, W, C of the input (= of the output, stride 1) */
+  int32_t kernel_h, kernel_w;             /* odd */
+  int32_t pad_h, pad_w;                   /* (kernel - 1) / 2 */
+} pipe_conv_geom;
+
+pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                 const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y, int64_t ldy,
+                                 int32_t* d_partials, void* stream);
+
 /* Which GEMM kernel the two forward calls use (process-wide, for tests and measurements):
  * 0 = automatic, 1 = CUDA-core reference kernel, 2 = tcgen05 tensor-core kernel,
  * 3 = small-token weight-streaming kernel.  A forced kernel that cannot run the request

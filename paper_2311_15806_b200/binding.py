@@ -29,7 +29,8 @@ STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
            "pipe_expand_weights_static",
-           "pipe_quantize_act", "pipe_expanded_linear", "pipe_ensemble_forward", "pipe_select_kernel",
+           "pipe_quantize_act", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
+           "pipe_select_kernel",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string"]
 
 
@@ -37,6 +38,11 @@ class LayerDesc(C.Structure):
     _fields_ = [("out_features", C.c_int32), ("in_features", C.c_int32), ("weight_bits", C.c_int32),
                 ("num_orders", C.c_int32), ("group_size", C.c_int32), ("keep_groups", C.c_int32),
                 ("num_branches", C.c_int32), ("branch_orders", C.c_int32 * MAX_ORDERS)]
+
+
+class ConvGeom(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("height", C.c_int32), ("width", C.c_int32), ("channels", C.c_int32),
+                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
 
 
 class LayerLayout(C.Structure):
@@ -80,6 +86,7 @@ def lib() -> C.CDLL:
         L.pipe_expand_weights_static.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p]
         L.pipe_quantize_act.argtypes = [p, i64, i32, i64, p, p, i64, p, p, sz, p]
         L.pipe_expanded_linear.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, p, p]
+        L.pipe_expanded_conv2d.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, p, i64, p, p]
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
         L.pipe_select_kernel.argtypes = [i32]
         L.pipe_launch_count.restype = C.c_uint64
@@ -166,6 +173,15 @@ def pipe_expanded_linear(desc: LayerDesc, blob: torch.Tensor, xq: torch.Tensor, 
     ldy = y.stride(0) if T > 1 else max(y.shape[1], y.stride(0))
     _check(lib().pipe_expanded_linear(C.byref(desc), _dp(blob), _dp(xq), T, ldxq, _dp(sx), _dp(bias), _dp(y), ldy,
                                       _dp(partials), _stream_ptr(stream)), "pipe_expanded_linear")
+
+
+def pipe_expanded_conv2d(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_nhwc: torch.Tensor, sx: torch.Tensor,
+                         y: torch.Tensor, bias: torch.Tensor | None = None, partials: torch.Tensor | None = None,
+                         stream=None) -> None:
+    """xq_nhwc: cuda int8 [N, H, W, C] contiguous; y: cuda float32 [N*H*W, O]."""
+    assert xq_nhwc.is_contiguous() and xq_nhwc.dtype == torch.int8
+    _check(lib().pipe_expanded_conv2d(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias), _dp(y),
+                                      y.stride(0), _dp(partials), _stream_ptr(stream)), "pipe_expanded_conv2d")
 
 
 def pipe_ensemble_forward(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,

@@ -89,6 +89,8 @@ struct ForwardArgs {
   int total_rows;
   int kernel_row_bytes, canon_row_bytes;
   int* status;
+  // implicit convolution (conv_on != 0): branch[0].xq is the NHWC input, T = N*H*W
+  int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
 };
 
 // GEMM back ends (each returns PIPE_ERR_UNSUPPORTED when it cannot take the request).

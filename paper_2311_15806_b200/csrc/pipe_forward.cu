@@ -42,6 +42,8 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   a.canon_row_bytes = L.lay.canon_row_bytes;
   a.status = device_status_word();
   if (!a.status) return PIPE_ERR_CUDA;
+  a.conv_on = 0;
+  a.cN = a.cH = a.cW = a.cC = a.ckh = a.ckw = a.cph = a.cpw = 0;
 
   const int choice = kernel_choice();
   if (choice == 1) return forward_reference(a, stream);
@@ -84,4 +86,51 @@ extern "C" pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const 
   }
   return run_forward(L, d_blob, L.M, h_xq_m, h_sx_m, h_y_m, kb, ke, T, ldxq, ldy, d_bias, sum_branches ? 1 : 0,
                      d_partials, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                            const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y,
+                                            int64_t ldy, int32_t* d_partials, void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  if (!geom || !d_blob || !d_xq || !d_sx || !d_y) return PIPE_ERR_INVALID_ARG;
+  if (geom->batch < 1 || geom->height < 1 || geom->width < 1 || geom->channels < 1 || geom->kernel_h < 1 ||
+      geom->kernel_w < 1)
+    return PIPE_ERR_INVALID_ARG;
+  if (2 * geom->pad_h + 1 != geom->kernel_h || 2 * geom->pad_w + 1 != geom->kernel_w) return PIPE_ERR_SHAPE;
+  if (static_cast<int64_t>(geom->kernel_h) * geom->kernel_w * geom->channels != L.I) return PIPE_ERR_SHAPE;
+  if (ldy < L.O) return PIPE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_xq) & 15) ||
+      (reinterpret_cast<uintptr_t>(d_sx) & 3) || (reinterpret_cast<uintptr_t>(d_y) & 3) ||
+      (reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3))
+    return PIPE_ERR_ALIGNMENT;
+  if (geom->channels % 128 != 0 || geom->height % 8 != 0 || geom->width % 8 != 0) return PIPE_ERR_UNSUPPORTED;
+
+  ForwardArgs a;
+  for (int k = 0; k < L.K; ++k) a.order[k] = order_view(L, d_blob, k);
+  a.num_branches = 1;
+  BranchArgs& b = a.branch[0];
+  b.xq = d_xq;
+  b.sx = d_sx;
+  b.y = d_y;
+  b.k_begin = 0;
+  b.k_end = L.K;
+  b.add_bias = 1;
+  b.accumulate = 0;
+  a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
+  a.T = static_cast<int64_t>(geom->batch) * geom->height * geom->width;
+  a.ldxq = geom->channels;
+  a.ldy = ldy;
+  a.bias = d_bias;
+  a.partials = d_partials;
+  a.total_rows = L.lay.total_rows;
+  a.kernel_row_bytes = L.lay.kernel_row_bytes;
+  a.canon_row_bytes = L.lay.canon_row_bytes;
+  a.status = device_status_word();
+  if (!a.status) return PIPE_ERR_CUDA;
+  a.conv_on = 1;
+  a.cN = geom->batch; a.cH = geom->height; a.cW = geom->width; a.cC = geom->channels;
+  a.ckh = geom->kernel_h; a.ckw = geom->kernel_w; a.cph = geom->pad_h; a.cpw = geom->pad_w;
+  return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
 }

@@ -65,6 +65,7 @@ struct Params {
   int depth;              // stages in the ring
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
   int shift;              // 8 - b
+  int conv_pw, conv_pp, conv_np, conv_chunks;   // patches per image row / per image / in total; 128-channel chunks per tap
   const uint8_t* kbase;   // lowest address of the streaming-layout sections (16-byte aligned)
   uint32_t koff[PIPE_MAX_ORDERS];  // (kcodes of order k - kbase) / 16
 };
@@ -139,6 +140,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Four-dimensional tile of an NHWC tensor (coordinates innermost first: channel, x, y, image);
+// coordinates outside the tensor read zeros, which is the convolution's padding.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
+// Implicit convolution: a token tile is two 8 x 8 pixel patches (64 rows each); patch p lies in
+// image p / pp at patch coordinates ((p % pp) / pw, (p % pp) % pw).
+__device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n, int& h0, int& w0);
+
 // Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes, stored as
 // 8-row atoms of 1024 bytes with the 128-byte swizzle (the layout TMA writes with SWIZZLE_128B).
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
@@ -203,6 +217,13 @@ __device__ __forceinline__ void decode_tile(const Params& p, int tile, TileMeta&
     }
   }
   t.rowbase[kMaxClusterOrders] = rb;
+}
+
+__device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n, int& h0, int& w0) {
+  n = patch / p.conv_pp;
+  const int rem = patch - n * p.conv_pp;
+  h0 = (rem / p.conv_pw) * 8;
+  w0 = (rem % p.conv_pw) * 8;
 }
 
 struct Rings {
@@ -402,8 +423,15 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     __syncwarp();
     if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int64_t tok = static_cast<int64_t>(t.tt) * kTileM + row_in_tile;
-    const bool tok_ok = tok < p.f.T;
+    int64_t tok = static_cast<int64_t>(t.tt) * kTileM + row_in_tile;
+    bool tok_ok = tok < p.f.T;
+    if (p.f.conv_on) {
+      const int patch = 2 * t.tt + (row_in_tile >> 6);
+      int n, h0, w0;
+      patch_origin(p, patch, n, h0, w0);
+      tok = (static_cast<int64_t>(n) * p.f.cH + h0 + ((row_in_tile >> 3) & 7)) * p.f.cW + w0 + (row_in_tile & 7);
+      tok_ok = patch < p.conv_np;
+    }
     const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
     float* yrow = br.y + tok * p.f.ldy;
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
@@ -537,7 +565,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
         const int m = tile / p.ntt / p.ncb;
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
         mbar_expect_tx(g.a_full0 + 8u * rp.slot, kABytes);
-        tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * rp.slot);
+        if (!p.f.conv_on) {
+          tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * rp.slot);
+        } else {
+          // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
+          const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
+          const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            int n, h0, w0;
+            patch_origin(p, 2 * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
+            tma_load_4d(g.stage0 + rp.slot * kStageBytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, w0 + dw, h0 + dh,
+                        n, g.a_full0 + 8u * rp.slot);
+          }
+        }
       }
     }
     __syncwarp();
@@ -653,6 +694,21 @@ static bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner_bytes
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// NHWC int8 tensor as a 4-D map; one box = 128 channels x 8 x 8 pixels of one image (64 rows of 128 bytes).
+static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int W, int C) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                              static_cast<cuuint64_t>(N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W) * C,
+                                 static_cast<cuuint64_t>(H) * W * C};
+  const cuuint32_t box[4] = {128, 8, 8, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tc
 
 static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
@@ -667,6 +723,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   const int BN = max_cluster <= 2 ? 128 : (max_cluster <= 4 ? 64 : 32);
   if (a.g % 8 != 0 || a.g > BN || BN % a.g != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.conv_on && (a.cC % kKStep != 0 || a.cH % 8 != 0 || a.cW % 8 != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
     if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   }
@@ -676,6 +733,14 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   p.BN = BN;
   p.ncb = ceil_div(a.O, BN);
   p.ntt = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
+  p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
+  if (a.conv_on) {
+    p.conv_pw = a.cW / 8;
+    p.conv_pp = (a.cH / 8) * p.conv_pw;
+    p.conv_np = p.conv_pp * a.cN;
+    p.conv_chunks = a.cC / kKStep;
+    p.ntt = ceil_div(p.conv_np, 2);
+  }
   const int64_t tiles = static_cast<int64_t>(p.ncb) * p.ntt * a.num_branches;
   if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
   p.num_tiles = static_cast<int>(tiles);
@@ -705,6 +770,9 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
   const int dyn_smem = p.depth * kStageBytes + 1024;
 
+  if (a.conv_on) {
+    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC)) return PIPE_ERR_CUDA;
+  } else
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
                      static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))

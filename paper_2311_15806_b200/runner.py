@@ -14,7 +14,8 @@ from . import synth
 
 
 class LayerRunner:
-    def __init__(self, spec: synth.LayerSpec, device="cuda", distinct_inputs: bool = True, second_layer: bool = False):
+    def __init__(self, spec: synth.LayerSpec, device="cuda", distinct_inputs: bool = True, second_layer: bool = False,
+                 implicit_conv: bool = True):
         self.spec = spec
         self.device = torch.device(device)
         G = spec.O // spec.g
@@ -22,6 +23,15 @@ class LayerRunner:
         self.desc = B.make_desc(spec.O, spec.I, spec.bits, spec.K, spec.g, self.n_keep, spec.M)
         self.layout = B.pipe_layout(self.desc)
         self.second_layer = second_layer
+        # a convolution workload runs as implicit GEMM on the NHWC tensor when the library takes its shape
+        self.geom = None
+        if spec.conv is not None and implicit_conv:
+            N, H, W_, C, kh, kw, pad = spec.conv
+            if C % 128 == 0 and H % 8 == 0 and W_ % 8 == 0 and spec.M == 1:
+                g = B.ConvGeom()
+                g.batch, g.height, g.width, g.channels = N, H, W_, C
+                g.kernel_h, g.kernel_w, g.pad_h, g.pad_w = kh, kw, pad, pad
+                self.geom = g
         self.M = spec.M
         self.distinct_inputs = distinct_inputs and spec.M > 1
         self.blob = B.alloc_bytes(self.layout.blob_bytes, self.device)
@@ -58,13 +68,16 @@ class LayerRunner:
         for m in range(n):
             if xs is not None and xs[m] is not None:
                 self.x.append(torch.from_numpy(xs[m]).to(self.device))
+            elif spec.conv is not None and self.geom is not None:
+                N, H, W_, C = spec.conv[:4]
+                self.x.append(torch.from_numpy(synth.make_conv_input(spec, m)).to(self.device).view(N * H * W_, C))
             elif spec.conv is not None:
                 self.x.append(self._lower_conv_on_device(synth.make_conv_input(spec, m)))
             else:
                 self.x.append(torch.from_numpy(synth.make_activations(spec, m)).to(self.device))
         T = self.x[0].shape[0]
         self.T = T
-        self.xq = [torch.empty((T, spec.I), dtype=torch.int8, device=self.device) for _ in range(n)]
+        self.xq = [torch.empty(tuple(self.x[0].shape), dtype=torch.int8, device=self.device) for _ in range(n)]
         self.sx = [torch.zeros(1, dtype=torch.float32, device=self.device) for _ in range(n)]
         self.y = [torch.empty((T, spec.O), dtype=torch.float32, device=self.device) for _ in range(self.M)]
 
@@ -93,7 +106,11 @@ class LayerRunner:
 
     def forward(self, partials: torch.Tensor | None = None, blob: torch.Tensor | None = None) -> None:
         blob = self.blob if blob is None else blob
-        if self.M == 1:
+        if self.geom is not None:
+            N, H, W_, C = self.spec.conv[:4]
+            B.pipe_expanded_conv2d(self.desc, self.geom, blob, self.xq[0].view(N, H, W_, C), self.sx[0], self.y[0], None,
+                                   partials)
+        elif self.M == 1:
             B.pipe_expanded_linear(self.desc, blob, self.xq[0], self.sx[0], self.y[0], None, partials)
         else:
             n = len(self.xq)
@@ -131,7 +148,7 @@ class LayerRunner:
         lay, s = self.layout, self.spec
         codes = sum(lay.rows[k] * lay.kernel_row_bytes for k in range(s.K))
         scales = 4 * self.total_rows + 4 * (lay.num_groups + 1) * s.K
-        return codes + scales + len(self.xq) * self.T * s.I + 4 * self.M * self.T * s.O
+        return codes + scales + sum(x.numel() for x in self.xq) + 4 * self.M * self.T * s.O
 
     def expand_bytes(self) -> int:
         """Algorithmic bytes of the expansion: every processed row is read and (except at the last
@@ -145,4 +162,4 @@ class LayerRunner:
 
     def quantize_bytes(self) -> int:
         """absmax pass reads fp32 once, quantize pass reads it again and writes int8."""
-        return len(self.x) * self.T * self.spec.I * (4 + 4 + 1)
+        return sum(x.numel() for x in self.x) * (4 + 4 + 1)

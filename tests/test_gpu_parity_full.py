@@ -62,7 +62,11 @@ def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_chec
             i = m if len(xs_rows) > 1 else 0
             assert run.sx[i].cpu().numpy().view(np.uint32)[0] == np.float32(sx_full[i]).view(np.uint32)
             xq_o, _ = oracle.quantize_act(xs_rows[i], static_scale=float(sx_full[i]))
-            np.testing.assert_array_equal(run.xq[i][rows_t].cpu().numpy(), xq_o)
+            if run.geom is None:
+                np.testing.assert_array_equal(run.xq[i][rows_t].cpu().numpy(), xq_o)
+            else:   # implicit convolution: the quantized tensor is the NHWC input itself
+                x_nhwc = x4[i].reshape(-1, x4[i].shape[-1])
+                np.testing.assert_array_equal(run.xq[i].cpu().numpy(), oracle.quantize_act(x_nhwc)[0])
             f = oracle.forward(e, xq_o, sx_full[i], k0, k0 + split[m])
             lo, hi = e.row_off(k0), e.row_off(k0 + split[m])
             np.testing.assert_array_equal(part[rows_t][:, lo:hi].cpu().numpy(), f.partials[:, lo:hi])
@@ -70,6 +74,22 @@ def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_chec
             H.assert_outputs_close(y, f, f"{sp.name} T={run.T} branch {m}")
             np.testing.assert_array_equal(y.view(np.uint32), f.y.view(np.uint32))
             k0 += split[m]
+        if run.geom is not None:
+            # implicit GEMM vs the same layer on explicitly lowered rows (and that one vs the CUDA-core kernel)
+            y_conv = run.y[0].clone()
+            part_conv = part.clone()
+            del run
+            torch.cuda.empty_cache()
+            run = LayerRunner(sp, implicit_conv=False)
+            run.load(W)
+            run.expand()
+            run.quantize()
+            part.zero_()
+            run.forward(part)
+            torch.cuda.synchronize()
+            assert torch.equal(y_conv.view(torch.int32), run.y[0].view(torch.int32))
+            assert torch.equal(part_conv, part)
+            del y_conv, part_conv
         if cross_check:
             # the whole output, tensor-core/streaming kernel vs CUDA-core kernel, bit for bit
             y_auto = [y.clone() for y in run.y]

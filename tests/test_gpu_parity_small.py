@@ -216,6 +216,71 @@ def test_forward_zero_tokens_and_strided_io(oracle):
     assert B.pipe_poll_status() == B.PIPE_OK
 
 
+CONV_CASES = [
+    # N, H,  W,  C,   O,  kh, kw, bits, K, g, n_keep
+    (2, 16, 8, 128, 64, 3, 3, 4, 3, 8, 2),
+    (1, 8, 24, 128, 72, 3, 3, 8, 2, 8, 3),      # odd number of 8x8 patches: the last tile is half empty
+    (3, 8, 8, 256, 136, 1, 1, 2, 4, 8, 5),      # 1x1: no halo
+    (1, 24, 16, 128, 40, 5, 3, 4, 2, 8, 5),     # rectangular filter, two rows/columns of padding
+]
+
+
+@pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep", CONV_CASES)
+def test_implicit_convolution_matches_oracle(oracle, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep):
+    """pipe_expanded_conv2d on the NHWC tensor == the oracle on explicitly lowered im2col rows."""
+    rng = np.random.default_rng(N * 1000 + Hh * 10 + Cc)
+    I = kh * kw * Cc
+    W = _w(rng, O, I, heavy=(bits == 2))
+    bias = rng.standard_normal(O).astype(np.float32)
+    x4 = np.maximum(rng.standard_normal((N, Hh, Ww, Cc)), 0).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep), W)
+    xq4, sx = H.gpu_quantize(x4.reshape(-1, Cc))
+    xq_o, sx_o = oracle.quantize_act(x4.reshape(-1, Cc))
+    np.testing.assert_array_equal(xq4.cpu().numpy(), xq_o)
+    # explicit lowering on the host (pad_h may differ from pad_w: lower by hand)
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    xp = np.zeros((N, Hh + 2 * ph, Ww + 2 * pw, Cc), np.int8)
+    xp[:, ph:ph + Hh, pw:pw + Ww] = xq_o.reshape(N, Hh, Ww, Cc)
+    rows = np.zeros((N, Hh, Ww, kh * kw * Cc), np.int8)
+    for dh in range(kh):
+        for dw in range(kw):
+            tap = dh * kw + dw
+            rows[..., tap * Cc:(tap + 1) * Cc] = xp[:, dh:dh + Hh, dw:dw + Ww]
+    f = oracle.forward(e, rows.reshape(-1, I), sx_o, bias=bias)
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, ph, pw
+    T = N * Hh * Ww
+    y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
+    B.pipe_expanded_conv2d(layer.desc, geom, layer.blob, xq4.view(N, Hh, Ww, Cc), sx, y, torch.from_numpy(bias).cuda(), part)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    np.testing.assert_array_equal(part.cpu().numpy(), f.partials)
+    H.assert_outputs_close(y.cpu().numpy(), f, "conv2d")
+    np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), f.y.view(np.uint32))
+
+
+def test_convolution_shapes_outside_the_fast_path_are_refused():
+    layer_desc = H.desc_of(64, 9 * 96, 4, 2, 8, 2)
+    lay = B.pipe_layout(layer_desc)
+    blob = B.alloc_bytes(lay.blob_bytes)
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = 1, 8, 8, 96
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = 3, 3, 1, 1
+    xq = torch.zeros((1, 8, 8, 96), dtype=torch.int8, device="cuda")
+    sx = torch.ones(1, device="cuda")
+    y = torch.zeros((64, 64), device="cuda")
+    with pytest.raises(B.PipeError) as ei:
+        B.pipe_expanded_conv2d(layer_desc, geom, blob, xq, sx, y)
+    assert ei.value.status == B.PIPE_ERR_UNSUPPORTED
+    geom.pad_h = 0
+    with pytest.raises(B.PipeError) as ei:
+        B.pipe_expanded_conv2d(layer_desc, geom, blob, xq, sx, y)
+    assert ei.value.status == B.PIPE_ERR_SHAPE
+
+
 def test_launch_counter_moves():
     before = B.pipe_launch_count()
     H.gpu_quantize(np.ones((4, 16), np.float32))
