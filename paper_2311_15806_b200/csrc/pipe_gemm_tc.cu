@@ -62,6 +62,7 @@ struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
   ForwardArgs f;
   int BN, ncb, ntt, num_tiles, kblocks;
+  int nkmax;              // most orders any branch has
   int depth;              // stages in the ring
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
   int shift;              // 8 - b
@@ -359,13 +360,13 @@ struct EpiCtx {
 };
 
 // Epilogue role (4 warps, one TMEM lane quarter each; a lane owns one token row of the tile).
-// NKMAX = most orders a branch may have at this channel-block width (NKMAX * BN = 256).
+// NKMAX bounds the orders of a branch (2, 4 or 8); the channel block is BN = 8 * nch_max channels.
 // Before the accumulators are ready the warp prepares, from the prefix counts, where each
 // (order, 8-channel chunk) sits in the accumulator and the products s_k * lambda_x of all stacked
 // rows, so that the drain loop has no dependent global loads.
 template <int NKMAX>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
-  constexpr int NCH = 32 / NKMAX;   // 8-channel chunks per channel block (BN / 8)
+  constexpr int NCH = 16;           // row pitch of the (order, 8-channel chunk) tables (BN <= 128)
   constexpr int CH = 8 / NKMAX;     // chunks drained per iteration (64 accumulator registers)
   const int q = x.warp & 3;         // TMEM lane quarter this warp may read
   const int lane = x.lane;
@@ -385,28 +386,30 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     const int n_total = t.rowbase[kMaxClusterOrders];
     __syncwarp();
     {
-      const int ko = lane / NCH, cc = lane % NCH;
-      int col = -1, crow = 0;
-      if (ko < t.nk && cc < nch) {
-        int rb = 0, st = 0;
-        const int32_t* cum = nullptr;
+      for (int e = lane; e < NKMAX * NCH; e += 32) {
+        const int ko = e / NCH, cc = e % NCH;
+        int col = -1, crow = 0;
+        if (ko < t.nk && cc < nch) {
+          int rb = 0, st = 0;
+          const int32_t* cum = nullptr;
 #pragma unroll
-        for (int u = 0; u < NKMAX; ++u)
-          if (u == ko) {
-            rb = t.rowbase[u];
-            st = t.start[u];
-            cum = p.f.order[t.k0 + u].cum;
+          for (int u = 0; u < NKMAX; ++u)
+            if (u == ko) {
+              rb = t.rowbase[u];
+              st = t.start[u];
+              cum = p.f.order[t.k0 + u].cum;
+            }
+          const int c = c0 + 8 * cc;
+          const int j = c / p.f.g;
+          const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+          if (hi > lo) {
+            crow = lo * p.f.g + c % p.f.g;
+            col = rb + crow - st;
           }
-        const int c = c0 + 8 * cc;
-        const int j = c / p.f.g;
-        const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-        if (hi > lo) {
-          crow = lo * p.f.g + c % p.f.g;
-          col = rb + crow - st;
         }
+        x.colmap[e] = static_cast<int16_t>(col);
+        x.crowmap[e] = crow;
       }
-      x.colmap[lane] = static_cast<int16_t>(col);
-      x.crowmap[lane] = crow;
       for (int r = lane; r < n_total; r += 32) {
         int rb = 0, st = t.start[0];
         const float* sc = p.f.order[t.k0].scales;
@@ -499,8 +502,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
   __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[4] bt_ready[4] done[4] tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ int16_t epi_colmap[4][32];     // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
-  __shared__ int32_t epi_crowmap[4][32];    // ... and its compacted row in that order
+  __shared__ int16_t epi_colmap[4][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ int32_t epi_crowmap[4][128];   // ... and its compacted row in that order
   __shared__ float epi_cscale[4][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -649,8 +652,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     e.colmap = epi_colmap[warp - 6];
     e.crowmap = epi_crowmap[warp - 6];
     e.cscale = epi_cscale[warp - 6];
-    if (p.BN == 128) epilogue_role<2>(p, e);
-    else if (p.BN == 64) epilogue_role<4>(p, e);
+    if (p.nkmax <= 2) epilogue_role<2>(p, e);
+    else if (p.nkmax <= 4) epilogue_role<4>(p, e);
     else epilogue_role<8>(p, e);
   }
 
@@ -720,8 +723,19 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
   if (max_cluster > kMaxClusterOrders) return PIPE_ERR_UNSUPPORTED;
-  const int BN = max_cluster <= 2 ? 128 : (max_cluster <= 4 ? 64 : 32);
-  if (a.g % 8 != 0 || a.g > BN || BN % a.g != 0) return PIPE_ERR_UNSUPPORTED;
+  // Widest channel block whose stacked rows fit the 256 accumulator columns in the worst case:
+  // order 1 contributes BN rows, a sparse order at most min(BN, rows it keeps in the whole layer).
+  int BN = 0;
+  for (int cand = 128; cand >= 32 && BN == 0; cand >>= 1) {
+    int worst = 0;
+    for (int m = 0; m < a.num_branches; ++m) {
+      int w = 0;
+      for (int k = a.branch[m].k_begin; k < a.branch[m].k_end; ++k) w += min(cand, a.order[k].rows);
+      worst = max(worst, w);
+    }
+    if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand;
+  }
+  if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.conv_on && (a.cC % kKStep != 0 || a.cH % 8 != 0 || a.cW % 8 != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
@@ -731,6 +745,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
 
   p.f = a;
   p.BN = BN;
+  p.nkmax = max_cluster;
   p.ncb = ceil_div(a.O, BN);
   p.ntt = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
   p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
