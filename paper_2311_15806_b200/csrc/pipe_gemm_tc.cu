@@ -8,13 +8,13 @@
 // activation tile is staged once per reduction step.  A ring of stages {activation tile, B tile}
 // in shared memory decouples the roles:
 //   warp 0      activation producer: TMA tensor loads (128B swizzle), several lanes issue in turn
-//   warps 2-5   unpack: read the packed int8/int4/ternary rows of the tile straight from the
+//   warps 2-9   unpack: read the packed int8/int4/ternary rows of the tile straight from the
 //               reduction-block-major streaming layout (coalesced 16-byte loads, prefetched one
 //               step ahead in registers) and write int8 lanes into the swizzled B tile
 //               (shift + mask only; sub-byte codes arrive multiplied by 2^(8-b))
 //   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered);
 //               one tcgen05.commit per step releases the stage to both producers
-//   warps 6-9   epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
+//   warps 10-13 epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
 //               s_k * lambda_x and add in ascending order with one FMA per term, store fp32
 // Barrier operations cost their issuing thread on the order of a hundred cycles each, so every
 // role touches as few barriers per step as possible and ring positions are advanced without
@@ -34,8 +34,9 @@ constexpr int kTileM = 128;          // tokens per tile
 constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
-constexpr int kThreads = 320;
-constexpr int kUnpackThreads = 128;
+constexpr int kUnpackWarps = 8;
+constexpr int kThreads = 32 * (2 + kUnpackWarps + 4);
+constexpr int kUnpackThreads = 32 * kUnpackWarps;
 constexpr int kEpiThreads = 128;
 constexpr int kABytes = kTileM * kKStep;       // 16 KiB
 constexpr int kBtBytes = kMaxN * kKStep;       // 32 KiB
@@ -267,13 +268,13 @@ template <int BITS>
 __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
   constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
-  constexpr int ITEMS = 2 * CPR;         // kMaxN * CPR / kUnpackThreads
+  constexpr int ITEMS = kMaxN * CPR / kUnpackThreads;
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
   const uint32_t depth = p.depth;
   constexpr bool PREFETCH = BITS != 8;   // int8 rows need 16 chunks per thread: too many registers to double-buffer
   const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (128 / CPR), chunk c_item
-  const int sw = r0 & 7;                                   // (128 / CPR) is a multiple of 8 for 4- and 2-bit codes
+  const int sw = r0 & 7;                                   // the row step between items is a multiple of 8
   uint32_t off[ITEMS], step[ITEMS];
   uint4 wn[ITEMS];
   int tile = blockIdx.x;
@@ -634,7 +635,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
         if (ok) mma_commit(g.tfull0 + 8u * buf);
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 + kUnpackWarps) {
     // ------------------------------------------------------------------ unpack warps
     const int ut = threadIdx.x - 64;
     if (p.f.bits == 8) unpack_role<8>(p, g, ut);
@@ -649,9 +650,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     e.abort_flag = g.abort_flag;
     e.warp = warp;
     e.lane = lane;
-    e.colmap = epi_colmap[warp - 6];
-    e.crowmap = epi_crowmap[warp - 6];
-    e.cscale = epi_cscale[warp - 6];
+    e.colmap = epi_colmap[warp - 2 - kUnpackWarps];
+    e.crowmap = epi_crowmap[warp - 2 - kUnpackWarps];
+    e.cscale = epi_cscale[warp - 2 - kUnpackWarps];
     if (p.nkmax <= 2) epilogue_role<2>(p, e);
     else if (p.nkmax <= 4) epilogue_role<4>(p, e);
     else epilogue_role<8>(p, e);
