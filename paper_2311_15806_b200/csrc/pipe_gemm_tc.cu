@@ -260,94 +260,116 @@ __device__ __forceinline__ void place_item(const Params& p, int k0, int nk, cons
   step = static_cast<uint32_t>(ov.rows) * pk16;
 }
 
-// Unpack role (128 threads).  Work items are (stacked row, 16-byte chunk); a thread owns the same
-// item indices in every tile.  The packed chunks of the NEXT step are loaded from global memory
-// (L2-resident, fully coalesced) into registers before the current step's stage is waited for,
-// also across tile boundaries.
+// Unpack role.  Work items are (stacked row, 16-byte chunk); a thread owns the same item indices
+// in every tile.  A load cursor runs two reduction steps ahead of the step being written (also
+// across tile boundaries): the packed chunks travel global memory (L2-resident, fully coalesced)
+// -> registers -> swizzled B tile, and a step never waits for the latency of its own loads.
 template <int BITS>
 __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
   constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
   constexpr int ITEMS = kMaxN * CPR / kUnpackThreads;
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
+  constexpr int AHEAD = (BITS == 8) ? 1 : 2;   // int8 rows carry 8 chunks per thread: one step ahead only
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
   const uint32_t depth = p.depth;
-  constexpr bool PREFETCH = BITS != 8;   // int8 rows need 16 chunks per thread: too many registers to double-buffer
-  const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (128 / CPR), chunk c_item
+  const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (threads / CPR), chunk c_item
   const int sw = r0 & 7;                                   // the row step between items is a multiple of 8
-  uint32_t off[ITEMS], step[ITEMS];
-  uint4 wn[ITEMS];
-  int tile = blockIdx.x;
-  if (tile >= p.num_tiles) return;
+  const int my_tiles = (p.num_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  if (my_tiles <= 0) return;
+  const uint32_t total_steps = static_cast<uint32_t>(my_tiles) * p.kblocks;
+
+  // ---- load cursor
+  uint32_t off[ITEMS], stp[ITEMS];
+  int cur_tile = blockIdx.x, cur_kb = 0;
+  uint32_t issued = 0;
+  TileMeta tn;   // metadata of the tile after the cursor's tile, fetched when the cursor enters a tile
   {
     TileMeta t;
-    decode_tile(p, tile, t);
+    decode_tile(p, cur_tile, t);
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       const int idx = ut + i * kUnpackThreads;
-      place_item(p, t.k0, t.nk, t.start, t.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], step[i]);
-      if (PREFETCH && off[i] != 0xffffffffu) wn[i] = __ldg(kb16 + off[i]);
+      place_item(p, t.k0, t.nk, t.start, t.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
     }
+    const int nt = cur_tile + gridDim.x;
+    decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
   }
-  RingPos rp{0, 0};
-  for (; tile < p.num_tiles; tile += gridDim.x) {
-    const int next_tile = tile + gridDim.x;
-    TileMeta tn;
-    decode_tile(p, next_tile < p.num_tiles ? next_tile : tile, tn);   // its loads complete during this tile's steps
-    for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
-      uint4 w[ITEMS];
-      bool valid[ITEMS];
+  auto fetch = [&](uint4 (&w)[ITEMS], uint32_t& mask) {
+    mask = 0;
+    if (issued >= total_steps) return;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+      if (off[i] != 0xffffffffu) {
+        w[i] = __ldg(kb16 + off[i]);
+        mask |= 1u << i;
+      }
+    ++issued;
+    if (++cur_kb < p.kblocks) {
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i)
+        if (off[i] != 0xffffffffu) off[i] += stp[i];
+    } else if (issued < total_steps) {
+      cur_kb = 0;
+      cur_tile += gridDim.x;
 #pragma unroll
       for (int i = 0; i < ITEMS; ++i) {
-        valid[i] = off[i] != 0xffffffffu;
-        if (PREFETCH) w[i] = wn[i];
-        else if (valid[i]) w[i] = __ldg(kb16 + off[i]);
+        const int idx = ut + i * kUnpackThreads;
+        place_item(p, tn.k0, tn.nk, tn.start, tn.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
       }
-      if (kb + 1 < p.kblocks) {
-#pragma unroll
-        for (int i = 0; i < ITEMS; ++i)
-          if (valid[i]) {
-            off[i] += step[i];
-            if (PREFETCH) wn[i] = __ldg(kb16 + off[i]);
-          }
-      } else if (next_tile < p.num_tiles) {
-#pragma unroll
-        for (int i = 0; i < ITEMS; ++i) {
-          const int idx = ut + i * kUnpackThreads;
-          place_item(p, tn.k0, tn.nk, tn.start, tn.rowbase, idx >> CPR_LOG, idx & (CPR - 1), off[i], step[i]);
-          if (PREFETCH && off[i] != 0xffffffffu) wn[i] = __ldg(kb16 + off[i]);
-        }
-      }
-      if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
-      uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
-#pragma unroll
-      for (int i = 0; i < ITEMS; ++i) {
-        if (!valid[i]) continue;
-        const int r = r0 + i * (kUnpackThreads >> CPR_LOG);
-        uint8_t* row = bt + (r >> 3) * 1024 + (r & 7) * 128;
-        const int c0 = c_item * OUT_PER_CHUNK;
-        if (BITS == 8) {
-          *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
-        } else if (BITS == 4) {
-          const uint32_t m4 = 0xF0F0F0F0u;
-          const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
-          const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
-          *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = v0;
-          *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ sw) << 4)) = v1;
-        } else {
-          const uint32_t m2 = 0xC0C0C0C0u;
-          const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
-#pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            const uint4 v = make_uint4((ww[h] << 6) & m2, (ww[h] << 4) & m2, (ww[h] << 2) & m2, ww[h] & m2);
-            *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
-          }
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
-      __syncwarp();
-      if ((ut & 31) == 0) mbar_arrive(g.bt_ready0 + 8u * rp.slot);   // one arrival per warp
+      const int nt = cur_tile + gridDim.x;
+      decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
     }
+  };
+
+  uint4 q1[ITEMS], q2[ITEMS];
+  uint32_t m1 = 0, m2 = 0;
+  fetch(q1, m1);
+  if (AHEAD == 2) fetch(q2, m2);
+
+  RingPos rp{0, 0};
+  for (uint32_t it = 0; it < total_steps; ++it, rp.advance(1, depth)) {
+    uint4 w[ITEMS];
+    const uint32_t mask = m1;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) w[i] = q1[i];
+    if (AHEAD == 2) {
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) q1[i] = q2[i];
+      m1 = m2;
+      fetch(q2, m2);
+    } else {
+      fetch(q1, m1);
+    }
+    if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
+    uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      if (!((mask >> i) & 1u)) continue;
+      const int r = r0 + i * (kUnpackThreads >> CPR_LOG);
+      uint8_t* row = bt + (r >> 3) * 1024 + (r & 7) * 128;
+      const int c0 = c_item * OUT_PER_CHUNK;
+      if (BITS == 8) {
+        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
+      } else if (BITS == 4) {
+        const uint32_t m4 = 0xF0F0F0F0u;
+        const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
+        const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
+        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = v0;
+        *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ sw) << 4)) = v1;
+      } else {
+        const uint32_t m2c = 0xC0C0C0C0u;
+        const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const uint4 v = make_uint4((ww[h] << 6) & m2c, (ww[h] << 4) & m2c, (ww[h] << 2) & m2c, ww[h] & m2c);
+          *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
+        }
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
+    __syncwarp();
+    if ((ut & 31) == 0) mbar_arrive(g.bt_ready0 + 8u * rp.slot);   // one arrival per warp
   }
 }
 
