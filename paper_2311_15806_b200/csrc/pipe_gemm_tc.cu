@@ -35,14 +35,13 @@ constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
 constexpr int kUnpackWarps = 8;
-constexpr int kThreads = 32 * (2 + kUnpackWarps + 4);
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
 constexpr int kUnpackThreads = 32 * kUnpackWarps;
-constexpr int kEpiThreads = 128;
-constexpr int kABytes = kTileM * kKStep;       // 16 KiB
+constexpr int kABytes = kTileM * kKStep;       // 16 KiB per token tile
 constexpr int kBtBytes = kMaxN * kKStep;       // 32 KiB
-constexpr int kStageBytes = kABytes + kBtBytes;
+constexpr int kMaxTokTiles = 2;                // token tiles that share one B tile
 constexpr int kTmemCols = 512;
-constexpr int kAccCols = 256;
 constexpr int kMaxRing = 4;
 constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
 constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s per wait at the maximum SM clock
@@ -62,7 +61,14 @@ struct RingPos {
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
   ForwardArgs f;
-  int BN, ncb, ntt, num_tiles, kblocks;
+  int BN, ncb, ntt, num_tiles, kblocks;   // ntt: token-tile groups
+  int tpt;                // token tiles (128 tokens each) per CTA tile: 1 or 2; they share every B tile
+  int ntok_tiles;         // token tiles in total
+  int a_bytes;            // activation bytes per stage: tpt * 16 KiB
+  int stage_bytes;        // a_bytes + 32 KiB
+  int nbuf;               // accumulator buffers in TMEM: 2 (epilogue overlaps the next tile) or 1
+  int buf_stride;         // TMEM columns between buffers
+  int acc_stride;         // TMEM columns between the accumulators of the token tiles of one buffer
   int nkmax;              // most orders any branch has
   int depth;              // stages in the ring
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
@@ -73,7 +79,7 @@ struct Params {
 };
 
 struct TileMeta {
-  int m, cb, tt;
+  int m, cb, tt;                       // branch, channel block, token-tile group
   int nk;                              // orders in this branch
   int k0;                              // first order
   int start[kMaxClusterOrders];        // first compacted row of the channel block in order k
@@ -342,7 +348,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
       fetch(q1, m1);
     }
     if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
-    uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
+    uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * p.stage_bytes + p.a_bytes;
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       if (!((mask >> i) & 1u)) continue;
@@ -377,31 +383,39 @@ struct EpiCtx {
   uint32_t tmem_base, tfull0, tempty0;
   volatile int* abort_flag;
   int warp, lane;
+  int jt;            // token tile of the group this warp drains
+  int part, nparts;  // share of the 16-channel groups this warp drains (two warps split a lone token tile)
   int16_t* colmap;
-  int32_t* crowmap;
   float* cscale;
+  float* stg;        // 32 rows x 16 floats, swizzled
 };
 
-// Epilogue role (4 warps, one TMEM lane quarter each; a lane owns one token row of the tile).
+// Epilogue role (8 warps, one TMEM lane quarter each; a lane owns one token row of a token tile).
+// With two token tiles per CTA tile each tile has its own four warps; a lone token tile is split
+// by channel groups between the two warps of a lane quarter.
 // NKMAX bounds the orders of a branch (2, 4 or 8); the channel block is BN = 8 * nch_max channels.
 // Before the accumulators are ready the warp prepares, from the prefix counts, where each
 // (order, 8-channel chunk) sits in the accumulator and the products s_k * lambda_x of all stacked
 // rows, so that the drain loop has no dependent global loads.
+// A lane computes 16 channels of its own token row at a time; the 32 x 16 block is then turned
+// through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
+// (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
+// which is what bounds the drain otherwise).
 template <int NKMAX>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
-  constexpr int NCH = 16;           // row pitch of the (order, 8-channel chunk) tables (BN <= 128)
-  constexpr int CH = 8 / NKMAX;     // chunks drained per iteration (64 accumulator registers)
-  const int q = x.warp & 3;         // TMEM lane quarter this warp may read
+  constexpr int NCH = 16;                    // row pitch of the (order, 8-channel chunk) table (BN <= 128)
+  constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
+  const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
   const int lane = x.lane;
-  const int row_in_tile = q * 32 + lane;
   uint32_t tcount = 0;
   const bool y_vec = (p.f.ldy % 4 == 0);
+  const int wsw = (lane >> 1) & 3;           // swizzle of this lane's row in the staging block
   for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
     TileMeta t;
     decode_tile(p, tile, t);
     const BranchArgs& br = p.f.branch[t.m];
-    const int buf = tcount & 1;
-    const uint32_t aph = (tcount >> 1) & 1;
+    const int buf = (p.nbuf == 2) ? (tcount & 1) : 0;
+    const uint32_t aph = ((p.nbuf == 2) ? (tcount >> 1) : tcount) & 1;
     const float sx = __ldg(br.sx);
     const int c0 = t.cb * p.BN;
     const int c1 = min(c0 + p.BN, p.f.O);
@@ -411,7 +425,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     {
       for (int e = lane; e < NKMAX * NCH; e += 32) {
         const int ko = e / NCH, cc = e % NCH;
-        int col = -1, crow = 0;
+        int col = -1;
         if (ko < t.nk && cc < nch) {
           int rb = 0, st = 0;
           const int32_t* cum = nullptr;
@@ -425,13 +439,9 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
           const int c = c0 + 8 * cc;
           const int j = c / p.f.g;
           const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-          if (hi > lo) {
-            crow = lo * p.f.g + c % p.f.g;
-            col = rb + crow - st;
-          }
+          if (hi > lo) col = rb + lo * p.f.g + c % p.f.g - st;
         }
         x.colmap[e] = static_cast<int16_t>(col);
-        x.crowmap[e] = crow;
       }
       for (int r = lane; r < n_total; r += 32) {
         int rb = 0, st = t.start[0];
@@ -449,70 +459,98 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     __syncwarp();
     if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    int64_t tok = static_cast<int64_t>(t.tt) * kTileM + row_in_tile;
-    bool tok_ok = tok < p.f.T;
+    // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
+    // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
+    const int ttile = t.tt * p.tpt + x.jt;
+    bool tile_ok = ttile < p.ntok_tiles;
+    int64_t tok_base = static_cast<int64_t>(ttile) * kTileM + q * 32;
+    int row_pitch = 0;   // tokens between image rows (convolution only)
     if (p.f.conv_on) {
-      const int patch = 2 * t.tt + (row_in_tile >> 6);
+      const int patch = 2 * ttile + (q >> 1);
       int n, h0, w0;
       patch_origin(p, patch, n, h0, w0);
-      tok = (static_cast<int64_t>(n) * p.f.cH + h0 + ((row_in_tile >> 3) & 7)) * p.f.cW + w0 + (row_in_tile & 7);
-      tok_ok = patch < p.conv_np;
+      tok_base = (static_cast<int64_t>(n) * p.f.cH + h0 + (q & 1) * 4) * p.f.cW + w0;
+      row_pitch = p.f.cW;
+      tile_ok = patch < p.conv_np;
     }
-    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
-    float* yrow = br.y + tok * p.f.ldy;
+    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * row_pitch + (r & 7) : tok_base + r; };
+    const int64_t tok_own = token_of(lane);
+    const bool own_ok = tile_ok && (p.f.conv_on || tok_own < p.f.T);
+    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * p.buf_stride + x.jt * p.acc_stride;
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
-    for (int cg = 0; cg < nch; cg += CH) {
-      int acc[CH][NKMAX][8];
-      int cols[CH][NKMAX];
+    const bool add_bias = br.add_bias && p.f.bias;
+    const int ngrp = (nch + 1) >> 1;
+    for (int grp = x.part; grp < ngrp && tile_ok; grp += x.nparts) {
+      // ---- this lane's row: 16 channels into the staging block
 #pragma unroll
-      for (int u = 0; u < CH; ++u)
+      for (int sub = 0; sub < 2; sub += CH) {
+        int acc[CH][NKMAX][8];
+        int cols[CH][NKMAX];
 #pragma unroll
-        for (int ko = 0; ko < NKMAX; ++ko) {
-          cols[u][ko] = (cg + u < nch) ? x.colmap[ko * NCH + cg + u] : -1;
-          if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
-        }
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        for (int u = 0; u < CH; ++u)
 #pragma unroll
-      for (int u = 0; u < CH; ++u) {
-        if (cg + u >= nch) continue;
-        const int c = c0 + 8 * (cg + u);
-        float y[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) y[e] = 0.f;
-#pragma unroll
-        for (int ko = 0; ko < NKMAX; ++ko) {
-          if (cols[u][ko] < 0) continue;
-          const float* cs = x.cscale + cols[u][ko];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
-            acc[u][ko][e] = a;
-            y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+          for (int ko = 0; ko < NKMAX; ++ko) {
+            const int chunk = 2 * grp + sub + u;
+            cols[u][ko] = (chunk < nch) ? x.colmap[ko * NCH + chunk] : -1;
+            if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
           }
-          if (p.f.partials && tok_ok) {
-            int32_t* prow = p.f.partials + tok * p.f.total_rows + p.f.order[t.k0 + ko].row_off + x.crowmap[ko * NCH + cg + u];
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
+        for (int u = 0; u < CH; ++u) {
+          const int chunk = 2 * grp + sub + u;
+          if (chunk >= nch) continue;
+          const int c = c0 + 8 * chunk;
+          float y[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) y[e] = 0.f;
+#pragma unroll
+          for (int ko = 0; ko < NKMAX; ++ko) {
+            if (cols[u][ko] < 0) continue;
+            const float* cs = x.cscale + cols[u][ko];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
+              acc[u][ko][e] = a;
+              y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+            }
+            if (p.f.partials && own_ok) {
+              const int crow = cols[u][ko] - t.rowbase[ko] + t.start[ko];   // compacted row of the chunk's first channel
+              int32_t* prow = p.f.partials + tok_own * p.f.total_rows + p.f.order[t.k0 + ko].row_off + crow;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
+            }
           }
-        }
-        if (tok_ok) {
-          if (br.add_bias && p.f.bias) {
+          if (add_bias) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], __ldg(p.f.bias + c + e));
           }
-          if (br.accumulate) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(yrow[c + e], y[e]);
-          }
-          if (vec_ok) {
-            *reinterpret_cast<float4*>(yrow + c) = make_float4(y[0], y[1], y[2], y[3]);
-            *reinterpret_cast<float4*>(yrow + c + 4) = make_float4(y[4], y[5], y[6], y[7]);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) yrow[c + e] = y[e];
-          }
+          const int j0 = 2 * (sub + u);
+          *reinterpret_cast<float4*>(x.stg + lane * 16 + ((j0 ^ wsw) << 2)) = make_float4(y[0], y[1], y[2], y[3]);
+          *reinterpret_cast<float4*>(x.stg + lane * 16 + (((j0 + 1) ^ wsw) << 2)) = make_float4(y[4], y[5], y[6], y[7]);
         }
       }
+      __syncwarp();
+      // ---- 8 rows x 64 bytes per store instruction
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int r = i * 8 + (lane >> 2), pp = lane & 3;
+        const int j = pp ^ ((r >> 1) & 3);
+        const int64_t tok = token_of(r);
+        if (2 * grp + (j >> 1) >= nch || (!p.f.conv_on && tok >= p.f.T)) continue;
+        float4 v = *reinterpret_cast<const float4*>(x.stg + r * 16 + (pp << 2));
+        float* dst = br.y + tok * p.f.ldy + c0 + 16 * grp + 4 * j;
+        if (vec_ok) {
+          if (br.accumulate) {
+            const float4 o = *reinterpret_cast<const float4*>(dst);
+            v = make_float4(__fadd_rn(o.x, v.x), __fadd_rn(o.y, v.y), __fadd_rn(o.z, v.z), __fadd_rn(o.w, v.w));
+          }
+          *reinterpret_cast<float4*>(dst) = v;
+        } else {
+          if (br.accumulate) v = make_float4(__fadd_rn(dst[0], v.x), __fadd_rn(dst[1], v.y), __fadd_rn(dst[2], v.z), __fadd_rn(dst[3], v.w));
+          dst[0] = v.x, dst[1] = v.y, dst[2] = v.z, dst[3] = v.w;
+        }
+      }
+      __syncwarp();
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncwarp();
@@ -525,9 +563,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
   __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[4] bt_ready[4] done[4] tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ int16_t epi_colmap[4][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
-  __shared__ int32_t epi_crowmap[4][128];   // ... and its compacted row in that order
-  __shared__ float epi_cscale[4][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
+  __shared__ int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
+  __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -551,7 +589,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
-      mbar_init(g.tempty0 + 8u * b, kEpiThreads / 32);
+      mbar_init(g.tempty0 + 8u * b, kEpiWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -590,18 +628,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
         const int tt = tile % p.ntt;
         const int m = tile / p.ntt / p.ncb;
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
-        mbar_expect_tx(g.a_full0 + 8u * rp.slot, kABytes);
+        mbar_expect_tx(g.a_full0 + 8u * rp.slot, p.a_bytes);
         if (!p.f.conv_on) {
-          tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, tt * kTileM, g.a_full0 + 8u * rp.slot);
+          // one box of tpt * 128 token rows; rows beyond T read zeros
+          tma_load_2d(g.stage0 + rp.slot * p.stage_bytes, &p.tmap_a[m], kb * kKStep, tt * p.tpt * kTileM, g.a_full0 + 8u * rp.slot);
         } else {
           // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
           const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
           const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          for (int half = 0; half < 2 * p.tpt; ++half) {
             int n, h0, w0;
-            patch_origin(p, 2 * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-            tma_load_4d(g.stage0 + rp.slot * kStageBytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, w0 + dw, h0 + dh,
+            patch_origin(p, 2 * p.tpt * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
+            tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, w0 + dw, h0 + dh,
                         n, g.a_full0 + 8u * rp.slot);
           }
         }
@@ -613,7 +651,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       RingPos rp{0, 0};
-      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kABytes);
+      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + p.a_bytes);
       uint32_t tcount = 0;
       bool ok = true;
       // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
@@ -633,13 +671,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
         const int n_total = n_next;
         if (tile + static_cast<int>(gridDim.x) < p.num_tiles) n_next = stacked_rows(tile + gridDim.x);
-        const int buf = tcount & 1;
-        const uint32_t aph = (tcount >> 1) & 1;
+        const int buf = (p.nbuf == 2) ? (tcount & 1) : 0;
+        const uint32_t aph = ((p.nbuf == 2) ? (tcount >> 1) : tcount) & 1;
+        // token tiles of this group that exist (the last group may hold one only)
+        const int jn = min(p.tpt, p.ntok_tiles - (tile % p.ntt) * p.tpt);
         if (!mbar_wait(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
         int n = (n_total + 15) & ~15;
         if (n < 16) n = 16;
         const uint32_t idesc = idesc_i8(n);
-        const uint32_t d_tmem = tmem_base + buf * kAccCols;
+        const uint32_t d_tmem = tmem_base + buf * p.buf_stride;
         for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
           // both barriers are polled before either result is tested so that the two polls overlap
           const bool r1 = mbar_try(g.a_full0 + 8u * rp.slot, rp.phase);
@@ -647,11 +687,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
           if (!r1 && !mbar_wait(g.a_full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           if (!r2 && !mbar_wait(g.bt_ready0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
+          const uint64_t so = static_cast<uint64_t>(rp.slot * (p.stage_bytes >> 4));
           const uint64_t adesc = adesc0 + so, bdesc = bdesc0 + so;
+          for (int j = 0; j < jn; ++j) {
 #pragma unroll
-          for (int k = 0; k < kKStep / 32; ++k)
-            mma_i8(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
+            for (int k = 0; k < kKStep / 32; ++k)
+              mma_i8(d_tmem + j * p.acc_stride, adesc + static_cast<uint64_t>(j * (kABytes >> 4) + k * 2),
+                     bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
+          }
           mma_commit(g.done0 + 8u * rp.slot);   // frees the stage for the activation producer AND the unpack warps
         }
         if (ok) mma_commit(g.tfull0 + 8u * buf);
@@ -672,9 +715,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     e.abort_flag = g.abort_flag;
     e.warp = warp;
     e.lane = lane;
-    e.colmap = epi_colmap[warp - 2 - kUnpackWarps];
-    e.crowmap = epi_crowmap[warp - 2 - kUnpackWarps];
-    e.cscale = epi_cscale[warp - 2 - kUnpackWarps];
+    const int ew = warp - 2 - kUnpackWarps;
+    e.jt = (p.tpt == 2) ? (ew >> 2) : 0;
+    e.part = (p.tpt == 2) ? 0 : (ew >> 2);
+    e.nparts = (p.tpt == 2) ? 1 : 2;
+    e.colmap = epi_colmap[ew];
+    e.cscale = epi_cscale[ew];
+    e.stg = epi_stage[ew];
     if (p.nkmax <= 2) epilogue_role<2>(p, e);
     else if (p.nkmax <= 4) epilogue_role<4>(p, e);
     else epilogue_role<8>(p, e);
@@ -748,7 +795,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   if (max_cluster > kMaxClusterOrders) return PIPE_ERR_UNSUPPORTED;
   // Widest channel block whose stacked rows fit the 256 accumulator columns in the worst case:
   // order 1 contributes BN rows, a sparse order at most min(BN, rows it keeps in the whole layer).
-  int BN = 0;
+  int BN = 0, worst_rows = 0;
   for (int cand = 128; cand >= 32 && BN == 0; cand >>= 1) {
     int worst = 0;
     for (int m = 0; m < a.num_branches; ++m) {
@@ -756,7 +803,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
       for (int k = a.branch[m].k_begin; k < a.branch[m].k_end; ++k) w += min(cand, a.order[k].rows);
       worst = max(worst, w);
     }
-    if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand;
+    if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand, worst_rows = worst;
   }
   if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
@@ -770,14 +817,31 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   p.BN = BN;
   p.nkmax = max_cluster;
   p.ncb = ceil_div(a.O, BN);
-  p.ntt = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
+  p.ntok_tiles = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
   p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
   if (a.conv_on) {
     p.conv_pw = a.cW / 8;
     p.conv_pp = (a.cH / 8) * p.conv_pw;
     p.conv_np = p.conv_pp * a.cN;
     p.conv_chunks = a.cC / kKStep;
-    p.ntt = ceil_div(p.conv_np, 2);
+    p.ntok_tiles = ceil_div(p.conv_np, 2);
+  }
+  int dev = 0, smem_max = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
+  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  // Two token tiles per CTA tile halve the unpack work per multiply-accumulate; worth it once the
+  // paired tiles still fill the machine a few times over.
+  p.tpt = (static_cast<int64_t>(p.ncb) * ceil_div(p.ntok_tiles, 2) * a.num_branches >= 2ll * sms) ? 2 : 1;
+  p.ntt = ceil_div(p.ntok_tiles, p.tpt);
+  p.a_bytes = p.tpt * kABytes;
+  p.stage_bytes = p.a_bytes + kBtBytes;
+  if (p.tpt == 1) {
+    p.nbuf = 2, p.buf_stride = 256, p.acc_stride = 0;
+  } else if (worst_rows <= 128) {
+    p.nbuf = 2, p.buf_stride = 256, p.acc_stride = 128;
+  } else {
+    p.nbuf = 1, p.buf_stride = 0, p.acc_stride = 256;
   }
   const int64_t tiles = static_cast<int64_t>(p.ncb) * p.ntt * a.num_branches;
   if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
@@ -799,21 +863,19 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
     if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
     p.koff[k] = static_cast<uint32_t>(d >> 4);
   }
-  int dev = 0, smem_max = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
-  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  p.depth = (smem_max - 8192 - 1024) / kStageBytes;  // static shared, alignment slack
+  cudaFuncAttributes fattr;
+  if (cudaFuncGetAttributes(&fattr, tc_forward_kernel) != cudaSuccess) return PIPE_ERR_CUDA;
+  p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / p.stage_bytes;  // static shared, alignment slack
   if (p.depth > kMaxRing) p.depth = kMaxRing;
   if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
-  const int dyn_smem = p.depth * kStageBytes + 1024;
+  const int dyn_smem = p.depth * p.stage_bytes + 1024;
 
   if (a.conv_on) {
     if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC)) return PIPE_ERR_CUDA;
   } else
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
-                     static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
+                     static_cast<uint64_t>(a.ldxq), kKStep, p.tpt * kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
   }
   static int attr_bytes = 0;
