@@ -401,15 +401,20 @@ struct EpiCtx {
 // through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
 // (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
 // which is what bounds the drain otherwise).
-template <int NKMAX>
+template <int NKMAX, bool PARTIALS>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
-  constexpr int NCH = 16;                    // row pitch of the (order, 8-channel chunk) table (BN <= 128)
   constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
   const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
   const int lane = x.lane;
   uint32_t tcount = 0;
   const bool y_vec = (p.f.ldy % 4 == 0);
   const int wsw = (lane >> 1) & 3;           // swizzle of this lane's row in the staging block
+  // store phase: this lane writes channel quad sj of rows sr0, sr0 + 8, sr0 + 16, sr0 + 24
+  const int sr0 = lane >> 2, spp = lane & 3;
+  const int sj = spp ^ ((sr0 >> 1) & 3);     // the same for all four rows (they differ by multiples of 8)
+  const uint32_t stg_w = smem_u32(x.stg) + static_cast<uint32_t>(lane * 64);
+  const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
+  const uint32_t colmap_s = smem_u32(x.colmap), cscale_s = smem_u32(x.cscale);
   for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
     TileMeta t;
     decode_tile(p, tile, t);
@@ -423,8 +428,9 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     const int n_total = t.rowbase[kMaxClusterOrders];
     __syncwarp();
     {
-      for (int e = lane; e < NKMAX * NCH; e += 32) {
-        const int ko = e / NCH, cc = e % NCH;
+      // accumulator column of (8-channel chunk, order), or -1: entry [chunk][order]
+      for (int e = lane; e < NKMAX * 16; e += 32) {
+        const int cc = e / NKMAX, ko = e % NKMAX;
         int col = -1;
         if (ko < t.nk && cc < nch) {
           int rb = 0, st = 0;
@@ -456,98 +462,130 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
         x.cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
       }
     }
-    __syncwarp();
-    if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
     // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
     const int ttile = t.tt * p.tpt + x.jt;
     bool tile_ok = ttile < p.ntok_tiles;
     int64_t tok_base = static_cast<int64_t>(ttile) * kTileM + q * 32;
-    int row_pitch = 0;   // tokens between image rows (convolution only)
     if (p.f.conv_on) {
       const int patch = 2 * ttile + (q >> 1);
       int n, h0, w0;
       patch_origin(p, patch, n, h0, w0);
       tok_base = (static_cast<int64_t>(n) * p.f.cH + h0 + (q & 1) * 4) * p.f.cW + w0;
-      row_pitch = p.f.cW;
       tile_ok = patch < p.conv_np;
     }
-    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * row_pitch + (r & 7) : tok_base + r; };
+    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * p.f.cW + (r & 7) : tok_base + r; };
     const int64_t tok_own = token_of(lane);
     const bool own_ok = tile_ok && (p.f.conv_on || tok_own < p.f.T);
-    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * p.buf_stride + x.jt * p.acc_stride;
+    float* srow[4];        // the four rows this lane stores, at channel c0 + 4 * sj
+    uint32_t srow_ok = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t tok = token_of(sr0 + 8 * i);
+      srow[i] = br.y + tok * p.f.ldy + c0 + 4 * sj;
+      if (tile_ok && (p.f.conv_on || tok < p.f.T)) srow_ok |= 1u << i;
+    }
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
     const bool add_bias = br.add_bias && p.f.bias;
+    const float* bias_q = add_bias ? p.f.bias + c0 + 4 * sj : nullptr;
     const int ngrp = (nch + 1) >> 1;
+    __syncwarp();
+    if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * p.buf_stride + x.jt * p.acc_stride;
     for (int grp = x.part; grp < ngrp && tile_ok; grp += x.nparts) {
+      // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
+      const bool quad_ok = 2 * grp + (sj >> 1) < nch;
+      float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (add_bias && quad_ok) {
+        const float* bp = bias_q + 16 * grp;
+        bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
+      }
       // ---- this lane's row: 16 channels into the staging block
 #pragma unroll
       for (int sub = 0; sub < 2; sub += CH) {
         int acc[CH][NKMAX][8];
         int cols[CH][NKMAX];
+        {
+          // CH * NKMAX int16 entries, contiguous
+          constexpr int W = CH * NKMAX / 2;   // 32-bit words: 2, 2 or 4
+          uint32_t cw[W];
+          const uint32_t addr = colmap_s + static_cast<uint32_t>((2 * grp + sub) * NKMAX * 2);
+          if constexpr (W == 2) {
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(cw[0]), "=r"(cw[1]) : "r"(addr));
+          } else {
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(cw[0]), "=r"(cw[1]), "=r"(cw[2]), "=r"(cw[3]) : "r"(addr));
+          }
+#pragma unroll
+          for (int u = 0; u < CH; ++u)
+#pragma unroll
+            for (int ko = 0; ko < NKMAX; ++ko) {
+              const int idx = u * NKMAX + ko;
+              cols[u][ko] = static_cast<int16_t>((cw[idx >> 1] >> (16 * (idx & 1))) & 0xffffu);
+            }
+        }
 #pragma unroll
         for (int u = 0; u < CH; ++u)
 #pragma unroll
-          for (int ko = 0; ko < NKMAX; ++ko) {
-            const int chunk = 2 * grp + sub + u;
-            cols[u][ko] = (chunk < nch) ? x.colmap[ko * NCH + chunk] : -1;
+          for (int ko = 0; ko < NKMAX; ++ko)
             if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
-          }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
         for (int u = 0; u < CH; ++u) {
           const int chunk = 2 * grp + sub + u;
           if (chunk >= nch) continue;
-          const int c = c0 + 8 * chunk;
           float y[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) y[e] = 0.f;
 #pragma unroll
           for (int ko = 0; ko < NKMAX; ++ko) {
             if (cols[u][ko] < 0) continue;
-            const float* cs = x.cscale + cols[u][ko];
+            float cs[8];
+            const uint32_t ca = cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[0]), "=f"(cs[1]), "=f"(cs[2]), "=f"(cs[3]) : "r"(ca));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[4]), "=f"(cs[5]), "=f"(cs[6]), "=f"(cs[7]) : "r"(ca + 16));
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
               acc[u][ko][e] = a;
               y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
             }
-            if (p.f.partials && own_ok) {
+            if (PARTIALS && own_ok) {
               const int crow = cols[u][ko] - t.rowbase[ko] + t.start[ko];   // compacted row of the chunk's first channel
               int32_t* prow = p.f.partials + tok_own * p.f.total_rows + p.f.order[t.k0 + ko].row_off + crow;
 #pragma unroll
               for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
             }
           }
-          if (add_bias) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], __ldg(p.f.bias + c + e));
-          }
           const int j0 = 2 * (sub + u);
-          *reinterpret_cast<float4*>(x.stg + lane * 16 + ((j0 ^ wsw) << 2)) = make_float4(y[0], y[1], y[2], y[3]);
-          *reinterpret_cast<float4*>(x.stg + lane * 16 + (((j0 + 1) ^ wsw) << 2)) = make_float4(y[4], y[5], y[6], y[7]);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>((j0 ^ wsw) << 4)), "f"(y[0]),
+                       "f"(y[1]), "f"(y[2]), "f"(y[3])
+                       : "memory");
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>(((j0 + 1) ^ wsw) << 4)), "f"(y[4]),
+                       "f"(y[5]), "f"(y[6]), "f"(y[7])
+                       : "memory");
         }
       }
       __syncwarp();
-      // ---- 8 rows x 64 bytes per store instruction
+      // ---- 8 rows x 64 bytes per store instruction; the bias joins here, after the whole chain
+      if (quad_ok) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int r = i * 8 + (lane >> 2), pp = lane & 3;
-        const int j = pp ^ ((r >> 1) & 3);
-        const int64_t tok = token_of(r);
-        if (2 * grp + (j >> 1) >= nch || (!p.f.conv_on && tok >= p.f.T)) continue;
-        float4 v = *reinterpret_cast<const float4*>(x.stg + r * 16 + (pp << 2));
-        float* dst = br.y + tok * p.f.ldy + c0 + 16 * grp + 4 * j;
-        if (vec_ok) {
-          if (br.accumulate) {
-            const float4 o = *reinterpret_cast<const float4*>(dst);
-            v = make_float4(__fadd_rn(o.x, v.x), __fadd_rn(o.y, v.y), __fadd_rn(o.z, v.z), __fadd_rn(o.w, v.w));
+        for (int i = 0; i < 4; ++i) {
+          if (!((srow_ok >> i) & 1u)) continue;
+          float4 v;
+          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg_r + static_cast<uint32_t>(i * 8 * 64)));
+          if (add_bias) v = make_float4(__fadd_rn(v.x, bq.x), __fadd_rn(v.y, bq.y), __fadd_rn(v.z, bq.z), __fadd_rn(v.w, bq.w));
+          float* dst = srow[i] + 16 * grp;
+          if (vec_ok) {
+            if (br.accumulate) {
+              const float4 o = *reinterpret_cast<const float4*>(dst);
+              v = make_float4(__fadd_rn(o.x, v.x), __fadd_rn(o.y, v.y), __fadd_rn(o.z, v.z), __fadd_rn(o.w, v.w));
+            }
+            *reinterpret_cast<float4*>(dst) = v;
+          } else {
+            if (br.accumulate) v = make_float4(__fadd_rn(dst[0], v.x), __fadd_rn(dst[1], v.y), __fadd_rn(dst[2], v.z), __fadd_rn(dst[3], v.w));
+            dst[0] = v.x, dst[1] = v.y, dst[2] = v.z, dst[3] = v.w;
           }
-          *reinterpret_cast<float4*>(dst) = v;
-        } else {
-          if (br.accumulate) v = make_float4(__fadd_rn(dst[0], v.x), __fadd_rn(dst[1], v.y), __fadd_rn(dst[2], v.z), __fadd_rn(dst[3], v.w));
-          dst[0] = v.x, dst[1] = v.y, dst[2] = v.z, dst[3] = v.w;
         }
       }
       __syncwarp();
@@ -563,8 +601,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
   __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[4] bt_ready[4] done[4] tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
-  __shared__ float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
+  __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ __align__(16) float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
   __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -722,9 +760,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     e.colmap = epi_colmap[ew];
     e.cscale = epi_cscale[ew];
     e.stg = epi_stage[ew];
-    if (p.nkmax <= 2) epilogue_role<2>(p, e);
-    else if (p.nkmax <= 4) epilogue_role<4>(p, e);
-    else epilogue_role<8>(p, e);
+    if (p.f.partials) {   // verification output: every integer accumulator is also written out
+      if (p.nkmax <= 2) epilogue_role<2, true>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true>(p, e);
+      else epilogue_role<8, true>(p, e);
+    } else {
+      if (p.nkmax <= 2) epilogue_role<2, false>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false>(p, e);
+      else epilogue_role<8, false>(p, e);
+    }
   }
 
   // ---------------------------------------------------------------------- teardown
