@@ -875,8 +875,8 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   // Two token tiles per CTA tile halve the unpack work per multiply-accumulate; worth it once the
-  // paired tiles still fill the machine a few times over.
-  p.tpt = (static_cast<int64_t>(p.ncb) * ceil_div(p.ntok_tiles, 2) * a.num_branches >= 2ll * sms) ? 2 : 1;
+  // paired tiles still give every SM a tile.
+  p.tpt = (static_cast<int64_t>(p.ncb) * ceil_div(p.ntok_tiles, 2) * a.num_branches >= sms) ? 2 : 1;
   p.ntt = ceil_div(p.ntok_tiles, p.tpt);
   p.a_bytes = p.tpt * kABytes;
   p.stage_bytes = p.a_bytes + kBtBytes;
