@@ -102,6 +102,12 @@ def workload_spec(name: str):
 
 
 # ------------------------------------------------------------------------------------------------
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    ("cfg2", "forward"): 28.380928e6 + 51.302400e6,      # profiles/ncu_tc_forward_kernel_cfg2.txt
+    ("cfg4a_t16", "forward"): 56.969216e6 + 0.482048e6,  # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
+}
+
+
 def time_oracle_sample(spec, target_seconds: float = 12.0):
     """The CPU oracle, as it stands, on a bounded sample of the workload: full weight expansion,
     then activation quantization + forward of every branch on the first `n` token rows."""
@@ -352,7 +358,9 @@ def run_ours(args):
         gbs = nbytes / (phases[dominant] * 1e-3) / 1e9
         roof = {"kernel": f"{dominant} kernels", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_note": f"copy bandwidth of {peaks['source']}"}
-    roof["traffic"] = None
+    # DRAM read + write bytes per launch of the dominant kernel from one ncu capture of this same
+    # command line (summaries under profiles/); None where no capture of the current kernel exists.
+    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get((spec.name, dominant))
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
