@@ -108,6 +108,22 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
 }
 
 
+def max_over_ranks(value_ms: float, world: int, device) -> float:
+    """Replicas run independently; the job's time is that of its slowest rank."""
+    if world <= 1:
+        return float(value_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, tokens_per_replica: int, steps: int, total_ms: float) -> float:
+    """Aggregate over all replicas: every rank processes its own `tokens_per_replica` per step."""
+    return world * tokens_per_replica * steps / (total_ms * 1e-3)
+
+
 def time_oracle_sample(spec, target_seconds: float = 12.0):
     """The CPU oracle, as it stands, on a bounded sample of the workload: full weight expansion,
     then activation quantization + forward of every branch on the first `n` token rows."""
@@ -251,12 +267,9 @@ def run_ours(args):
     t_quant = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
     t_fwd = [ev[i][2].elapsed_time(ev[i][3]) for i in range(args.steps)]
     total_ms = sum(ev[i][0].elapsed_time(ev[i][3]) for i in range(args.steps))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
-    tokens_per_s = world * T * args.steps / (total_ms * 1e-3)
+    tokens_per_s = whole_job_tokens_per_s(world, T, args.steps, total_ms)
     macs = run.macs_per_token() * T
 
     # ---- the GEMM kernel alone: back-to-back launches (one CUDA graph when capture works, so that
@@ -321,10 +334,7 @@ def run_ours(args):
     e1.record()
     sync_all()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     h2d = hW.numel() * 4 + sum(x.numel() * 4 for x in hx)
     d2h = sum(y.numel() * 4 for y in hy)
 
@@ -387,7 +397,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
@@ -396,7 +406,11 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--kernel", type=int, default=None, help="force a GEMM kernel (see pipe_select_kernel)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    return ap.parse_args(argv)
+
+
+def main():
+    args = parse_args()
     if args.impl == "reference":
         run_reference(args)
     else:
