@@ -1,6 +1,7 @@
 // Shared host/device helpers of libpipe (internal; the public surface is include/pipe.h).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -92,6 +93,12 @@ struct ForwardArgs {
   // implicit convolution (conv_on != 0): branch[0].xq is the NHWC input, T = N*H*W
   int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
 };
+
+// Tensor map of a row-major byte matrix [rows, inner_bytes] with row pitch pitch_bytes (a multiple of 16) and
+// a box of box_inner x box_rows bytes; swizzle128 selects the 128-byte swizzle.  False when the driver entry
+// point is missing or the encoding fails.
+bool make_tensor_map_2d_u8(CUtensorMap* map, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+                           uint32_t box_inner, uint32_t box_rows, bool swizzle128);
 
 // GEMM back ends (each returns PIPE_ERR_UNSUPPORTED when it cannot take the request).
 pipe_status forward_reference(const ForwardArgs& a, cudaStream_t stream);

@@ -1,49 +1,60 @@
 // Small-token kernel of the expanded layer (Appendix B, Eq. 9; Sec. 3.2 for the branches), T <= 16.
 //
-// With a handful of tokens the layer is bound by streaming the packed weight codes from HBM once.
-// The kernel therefore moves weights global -> registers with coalesced 16-byte loads (the loads of
-// the next batch are always in flight while the current batch is consumed), unpacks them in
-// registers with the shift-and-mask layout and feeds legacy warp-level integer MMAs
-// (mma.sync m16n8k32, weights as the 16-row operand, tokens as the 8-column operand): the tensor
-// pipe is nowhere near a limit here, the byte stream is.
+// With a handful of tokens the layer is bound by streaming the packed weight codes from HBM once,
+// so the kernel is built around the byte stream.  A "slab" is 8 consecutive output channels of
+// one branch; in every order of the branch that keeps the slab's group the slab is 8 consecutive
+// compacted rows.  Every CTA (one per SM) owns one contiguous range of slabs.  Because the
+// streaming section of the codes is reduction-block-major, the rows a CTA needs from one order
+// and one 128-code reduction block are ONE contiguous run, which a producer warp brings into a
+// deep ring of shared-memory stages with bulk asynchronous copies (a stage = one reduction block
+// of every order of the branch for up to 32 slabs, plus the matching 16 x 128-byte tile of the
+// quantized activations as a swizzled TMA box).  Nothing on the load path costs registers, and the
+// ring keeps far more bytes in flight than the bandwidth-delay product of the memory system.
 //
-// Work unit: a "slab" = 8 consecutive output channels of one branch.  In every order of the branch
-// that keeps the slab's group, the slab is 8 consecutive compacted rows.  Two such 8-row chunks
-// (two orders, ascending) form one 16-row MMA tile, so both orders of a pair accumulate in the same
-// thread and the fixed-order fp32 epilogue is thread-local.  A persistent CTA walks groups of 4
-// slabs: 16 streaming warps (4 per slab, each owning a range of the reduction axis) drop their exact
-// int32 partial sums into a double-buffered shared-memory area; 4 epilogue warps (one per slab)
-// add the four ranges, apply the scales in ascending order and store, while the streaming warps
-// are already on the next group.  The quantized activations (at most 16 rows) are read as MMA
-// fragments straight from global memory: they stay resident in L1.  All slab metadata and scale
-// products of the CTA are gathered once, up front, with independent loads.
+// 16 consumer warps each own one or two slabs of the pass for the WHOLE reduction axis: they read
+// their 8 rows of a stage from shared memory, widen sub-byte codes with the shift-and-mask layout
+// and feed warp-level integer MMAs (mma.sync m16n8k32: weights as the 16-row operand -- two orders
+// of the slab, ascending, share a tile -- tokens as the 8-column operand).  The int32 sums stay in
+// registers until the reduction axis is done, so the fixed-order fp32 epilogue is thread-local and
+// needs neither a cross-warp reduction nor extra memory.  Every mbarrier wait is bounded.
+#include <mutex>
+
 #include "pipe_common.cuh"
 
 namespace pipe {
 
 namespace st {
 
-constexpr int kStreamWarps = 16;
-constexpr int kEpiWarps = 4;
-constexpr int kThreads = 32 * (kStreamWarps + kEpiWarps);
-constexpr int kSlabsPerGroup = 4;
-constexpr int kSlices = 4;        // streaming warps per slab
-constexpr int kMaxPairs = 4;      // up to 8 orders per branch
-constexpr int kBatch = 4;         // macro steps whose loads are issued together
-constexpr int kMaxGroups = 128;   // groups one CTA may own (metadata table size)
-constexpr int kMetaInts = 2 + 4 * kMaxPairs;   // nchunks, branch, then (order, row0) per chunk
+constexpr int kConsWarps = 16;
+constexpr int kProdWarps = 4;
+constexpr int kThreads = 32 * (kConsWarps + kProdWarps);
+constexpr int kMaxOrd = 8;          // orders per branch
+constexpr int kMaxPasses = 32;      // passes (<= 32 slabs of one branch) a CTA may need
+constexpr int kMaxDepth = 16;
+constexpr int kXTile = 16 * 128;    // 16 token rows x 128 reduction bytes
 constexpr long long kWaitLimitCycles = 4000000000ll;
 
 struct Params {
+  CUtensorMap tmap_x[PIPE_MAX_ORDERS];   // per branch input: [T rows, I bytes], box 128 x 16, 128-byte swizzle
   ForwardArgs f;
-  int nms;           // macro steps: ceil(I_pad / (4 * codes per 16-byte chunk))
-  int kblocks;       // I_pad / 128
-  int pk;            // packed bytes of one row of one 128-code block
-  int shift;         // 8 - b
-  int slabs_per_branch;   // padded to a multiple of kSlabsPerGroup
-  int groups;
-  int xs_bytes;
-  int np;            // pairs of orders per slab the partial-sum buffers are sized for
+  int kblocks;            // reduction blocks of 128 codes
+  int pk;                 // packed bytes of one row of one reduction block
+  int shift;              // 8 - b
+  int slabs_per_branch;   // O / 8
+  int total_slabs;
+  int pass_slabs;         // slabs per pass: 16 * slabs per warp
+  int depth, stage_bytes;
+  int kbps;               // reduction blocks per stage (2 for 2-bit codes, else 1)
+  int nstages;            // stages per pass
+  int nkmax;              // most orders any branch has
+  int own_max;            // most slabs any CTA owns
+  int ctas_per_branch;    // every branch has its own CTAs, so no CTA's range crosses a branch boundary
+};
+
+struct Pass {
+  int branch, lb, le;                 // local slab range [lb, le) of the CTA's own slabs
+  int seg_row0[kMaxOrd], seg_rows[kMaxOrd], seg_off[kMaxOrd];
+  int wbytes;                         // weight bytes of one reduction block of this pass
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -52,6 +63,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -81,6 +95,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
   asm volatile(
@@ -89,302 +120,354 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, ui
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// int8 lanes (times 2^(8-b)) of the codes held by 16 packed bytes: reg[2m] covers reduction
-// offsets 8m..8m+3 of the chunk, reg[2m+1] covers 8m+4..8m+7 (see the streaming layout).
+// int8 lanes (times 2^(8-b)) of MMA number mm of a 16-byte packed chunk: r0 covers the chunk's
+// reduction offsets 8mm..8mm+3, r1 covers 8mm+4..8mm+7 (see the streaming layout).
 template <int BITS>
-__device__ __forceinline__ void unpack_chunk(const uint4& w, uint32_t (&reg)[16]) {
+__device__ __forceinline__ void frag(const uint4& w, int mm, uint32_t& r0, uint32_t& r1) {
   const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
   if (BITS == 8) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) reg[j] = ww[j];
+    r0 = ww[2 * mm];
+    r1 = ww[2 * mm + 1];
   } else if (BITS == 4) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      reg[2 * j] = (ww[j] << 4) & 0xF0F0F0F0u;
-      reg[2 * j + 1] = ww[j] & 0xF0F0F0F0u;
-    }
+    r0 = (ww[mm] << 4) & 0xF0F0F0F0u;
+    r1 = ww[mm] & 0xF0F0F0F0u;
   } else {
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int h = 0; h < 4; ++h) reg[4 * j + h] = (ww[j] << (6 - 2 * h)) & 0xC0C0C0C0u;
+    const uint32_t x = ww[mm >> 1];
+    const int h = 2 * (mm & 1);
+    r0 = (x << (6 - 2 * h)) & 0xC0C0C0C0u;
+    r1 = (x << (4 - 2 * h)) & 0xC0C0C0C0u;
   }
 }
 
-// One batch of a streaming warp: kBatch macro steps of one pair of one slab.
-struct Batch {
-  int gi;        // index into the CTA's own group list (-1: none)
-  int q;         // pair
-  int ms0;       // first macro step
-};
+// Number of compacted rows of an order before channel c of the branch (c a multiple of 8, c <= O).
+__device__ __forceinline__ int rows_before(const int32_t* cum, int c, int O, int g) {
+  if (c >= O) return __ldg(cum + O / g) * g;
+  const int j = c / g;
+  const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+  return lo * g + (hi > lo ? c - j * g : 0);
+}
 
-template <int BITS, int NT>
-__global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Params p) {
-  constexpr int CHK = 128 / BITS;        // codes per 16-byte chunk
-  constexpr int NMMA = CHK / 8;          // MMAs per macro step
-  const int RED_INTS = kSlabsPerGroup * kSlices * p.np * 32 * 4 * NT;   // one buffer of partial sums
-  extern __shared__ uint4 smem_u4[];
-  int* red = reinterpret_cast<int*>(smem_u4);                    // [2][slab][slice][pair][lane][4*NT]
-  int* meta = red + 2 * RED_INTS;                                // [own slabs][kMetaInts]
-  const int my_groups_ = (p.groups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
-  float* cstab = reinterpret_cast<float*>(meta + my_groups_ * kSlabsPerGroup * kMetaInts);   // [own slabs][2*np][8] s_k * lambda_x
-  float* biastab = cstab + my_groups_ * kSlabsPerGroup * 2 * p.np * 8;                        // [own slabs][8]
-  __shared__ uint64_t bars[4];   // full[2] empty[2]
+template <int BITS, int NT, int NP>
+__global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __grid_constant__ Params p) {
+  constexpr int SPW = (NP * NT <= 2) ? 2 : 1;   // slabs per consumer warp and pass
+  constexpr int CHK = 128 / BITS;               // codes per 16-byte chunk
+  constexpr int KBPS = (BITS == 2) ? 2 : 1;     // reduction blocks per stage
+  constexpr int MS = KBPS * 128 / (4 * CHK);    // macro steps (4 chunks per row of 8 lanes x 4) per stage
+  constexpr int XCH = CHK / 16;                 // 16-byte activation chunks per macro step and token
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bars[2 * kMaxDepth];      // full[depth] empty[depth]
+  __shared__ Pass passes[kMaxPasses];
+  __shared__ int npass_s;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
-  const int I = p.f.I;
-  const int my_groups = (p.groups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
-  const uint32_t bar0 = smem_u32(bars);
-  const uint32_t full0 = bar0, empty0 = bar0 + 16;
+  const uint32_t stage0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tables = smem_raw + (stage0 - smem_u32(smem_raw)) + static_cast<size_t>(p.depth) * p.stage_bytes;
+  int* slabmeta = reinterpret_cast<int*>(tables);                                   // [own][nkmax] first row or -1
+  float* cstab = reinterpret_cast<float*>(slabmeta + p.own_max * p.nkmax);          // [own][nkmax][8] s_k * lambda_x
+  float* biastab = cstab + p.own_max * p.nkmax * 8;                                 // [own][8]
+  int* chunktab = reinterpret_cast<int*>(biastab + p.own_max * 8);                  // [warp][SPW][1 + 3 * nkmax]
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8u * kMaxDepth;
+  const int depth = p.depth;
+
+  // this CTA's slabs: [s0, s0 + cnt), all of one branch
+  const int my_branch = static_cast<int>(blockIdx.x) / p.ctas_per_branch, cib = static_cast<int>(blockIdx.x) % p.ctas_per_branch;
+  const int base = p.slabs_per_branch / p.ctas_per_branch, rem = p.slabs_per_branch % p.ctas_per_branch;
+  const int s0 = my_branch * p.slabs_per_branch + cib * base + min(cib, rem);
+  const int cnt = base + (cib < rem ? 1 : 0);
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(full0 + 8u * b, kStreamWarps);
-      mbar_init(empty0 + 8u * b, kEpiWarps);
+    for (int s = 0; s < depth; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // passes: at most pass_slabs slabs, never across a branch boundary
+    int np = 0;
+    for (int cur = 0; cur < cnt && np < kMaxPasses; ++np) {
+      const int br = (s0 + cur) / p.slabs_per_branch;
+      const int br_end = (br + 1) * p.slabs_per_branch - s0;
+      const int le = min(min(cnt, br_end), cur + p.pass_slabs);
+      passes[np].branch = br;
+      passes[np].lb = cur;
+      passes[np].le = le;
+      cur = le;
+    }
+    npass_s = np;
   }
-  // ---- metadata of every slab this CTA owns: which orders keep its group, where its 8 rows start
-  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup; e += kThreads) {
-    const int gi = e / kSlabsPerGroup, sl = e % kSlabsPerGroup;
-    const int grp = blockIdx.x + gi * gridDim.x;
-    const int slab = grp * kSlabsPerGroup + sl;
+  // ---- which orders keep each own slab, and where its 8 rows start
+  for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
+    const int li = e / p.nkmax, ko = e % p.nkmax;
+    const int slab = s0 + li;
     const int branch = slab / p.slabs_per_branch;
     const int c0 = (slab - branch * p.slabs_per_branch) * 8;
-    int* m = meta + e * kMetaInts;
-    int nchunks = 0;
-    if (c0 < p.f.O) {
-      const BranchArgs& br = p.f.branch[branch];
+    const BranchArgs& br = p.f.branch[branch];
+    int row0 = -1;
+    if (br.k_begin + ko < br.k_end) {
+      const int32_t* cum = p.f.order[br.k_begin + ko].cum;
       const int j = c0 / p.f.g;
-      for (int k = br.k_begin; k < br.k_end; ++k) {
-        const int32_t* cum = p.f.order[k].cum;
-        const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-        if (hi > lo) {
-          m[2 + 2 * nchunks] = k;
-          m[3 + 2 * nchunks] = lo * p.f.g + c0 % p.f.g;
-          ++nchunks;
-        }
-      }
+      const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+      if (hi > lo) row0 = lo * p.f.g + c0 % p.f.g;
     }
-    m[0] = c0 < p.f.O ? nchunks : -1;   // -1: padding slab, nothing to store
-    m[1] = branch;
+    slabmeta[e] = row0;
   }
   __syncthreads();
-  // ---- scale products s_k * lambda_x of every row this CTA will finish, and its bias values
-  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup * 2 * p.np * 8; e += kThreads) {
-    const int r = e & 7, ci = (e >> 3) % (2 * p.np), slab_i = (e >> 3) / (2 * p.np);
-    const int* m = meta + slab_i * kMetaInts;
-    float v = 0.f;
-    if (ci < m[0]) {
-      const BranchArgs& br = p.f.branch[m[1]];
-      v = __fmul_rn(__ldg(p.f.order[m[2 + 2 * ci]].scales + m[3 + 2 * ci] + r), __ldg(br.sx));
+  const int npass = npass_s;
+  // ---- the contiguous run of rows every pass needs from every order
+  for (int e = threadIdx.x; e < npass * kMaxOrd; e += kThreads) {
+    const int pi = e / kMaxOrd, ko = e % kMaxOrd;
+    Pass& P = passes[pi];
+    const BranchArgs& br = p.f.branch[P.branch];
+    int r0 = 0, rows = 0;
+    if (br.k_begin + ko < br.k_end) {
+      const int32_t* cum = p.f.order[br.k_begin + ko].cum;
+      const int cb = (s0 + P.lb - P.branch * p.slabs_per_branch) * 8, ce = (s0 + P.le - P.branch * p.slabs_per_branch) * 8;
+      r0 = rows_before(cum, cb, p.f.O, p.f.g);
+      rows = rows_before(cum, ce, p.f.O, p.f.g) - r0;
     }
-    cstab[e] = v;
-  }
-  for (int e = threadIdx.x; e < my_groups * kSlabsPerGroup * 8; e += kThreads) {
-    const int r = e & 7, slab_i = e >> 3;
-    const int* m = meta + slab_i * kMetaInts;
-    float v = 0.f;
-    if (m[0] >= 0 && p.f.bias && p.f.branch[m[1]].add_bias) {
-      const int gi = slab_i / kSlabsPerGroup, sl = slab_i % kSlabsPerGroup;
-      const int slab = (blockIdx.x + gi * gridDim.x) * kSlabsPerGroup + sl;
-      v = __ldg(p.f.bias + (slab - m[1] * p.slabs_per_branch) * 8 + r);
-    }
-    biastab[e] = v;
+    P.seg_row0[ko] = r0;
+    P.seg_rows[ko] = rows;
   }
   __syncthreads();
+  if (threadIdx.x < npass) {
+    Pass& P = passes[threadIdx.x];
+    int off = KBPS * kXTile;
+    int wb = 0;
+    for (int ko = 0; ko < kMaxOrd; ++ko) {
+      P.seg_off[ko] = off;
+      off += KBPS * P.seg_rows[ko] * p.pk;
+      wb += P.seg_rows[ko] * p.pk;
+    }
+    P.wbytes = wb;
+  }
+  __syncthreads();
+  const uint32_t total_stages = static_cast<uint32_t>(npass) * p.nstages;
 
-  if (warp < kStreamWarps) {
-    // ================================================================== streaming warps
-    const int sl = warp / kSlices, slice = warp % kSlices;
-    const int per = (p.nms + kSlices - 1) / kSlices;
-    const int ms_begin = min(slice * per, p.nms), ms_end = min(ms_begin + per, p.nms);
-    const bool has_range = ms_begin < ms_end;
-
-    auto pairs_of = [&](int gi) {
-      const int nch = meta[(gi * kSlabsPerGroup + sl) * kMetaInts];
-      return nch > 0 ? (nch + 1) >> 1 : 0;
-    };
-    // first batch at or after (gi, q = 0)
-    auto first_batch = [&](int gi) {
-      Batch b{-1, 0, 0};
-      if (!has_range) return b;
-      while (gi < my_groups && pairs_of(gi) == 0) ++gi;
-      if (gi < my_groups) b = Batch{gi, 0, ms_begin};
-      return b;
-    };
-    auto next_batch = [&](const Batch& c) {
-      if (c.ms0 + kBatch < ms_end) return Batch{c.gi, c.q, c.ms0 + kBatch};
-      if (c.q + 1 < pairs_of(c.gi)) return Batch{c.gi, c.q + 1, ms_begin};
-      return first_batch(c.gi + 1);
-    };
-    auto issue = [&](const Batch& b, uint4 (&wa)[kBatch], uint4 (&wb)[kBatch]) {
-      if (b.gi < 0) return;
-      const int* m = meta + (b.gi * kSlabsPerGroup + sl) * kMetaInts;
-      const int nch = m[0];
-      const int k_a = m[2 + 4 * b.q], row_a = m[3 + 4 * b.q];
-      const bool has_b = 2 * b.q + 1 < nch;
-      const int k_b = has_b ? m[4 + 4 * b.q] : k_a;
-      const int row_b = has_b ? m[5 + 4 * b.q] : row_a;
-      const uint8_t* base_a = p.f.order[k_a].kcodes + static_cast<size_t>(row_a + gid) * p.pk;
-      const uint8_t* base_b = p.f.order[k_b].kcodes + static_cast<size_t>(row_b + gid) * p.pk;
-      const size_t blk_a = static_cast<size_t>(p.f.order[k_a].rows) * p.pk;
-      const size_t blk_b = static_cast<size_t>(p.f.order[k_b].rows) * p.pk;
+  if (warp >= kConsWarps) {
+    // ================================================================== producer warps
+    // A copy instruction keeps its issuing thread busy for a hundred cycles or more, but the
+    // copies of different lanes of ONE warp instruction, and of different warps, overlap.  So each
+    // producer warp issues stages in batches: lane = (stage of the batch, job), a job being one
+    // copy of the stage (the activation tile or one order's rows, per reduction block); job-0
+    // lanes first wait until the consumers have released their slot, then all lanes issue in
+    // step.  Producer warp j owns the batches j, j + W, ... and with them a FIXED subset of the
+    // ring's slots (the ring is cut to W batches), so the uses of a slot are issued in order by
+    // one warp and the barrier a lane waits for is at most one phase behind.
+    constexpr int kJobLanes = 4;
+    const uint32_t SB = static_cast<uint32_t>(depth) / kProdWarps;   // depth = SB * kProdWarps (host)
+    const int st_in_batch = lane / kJobLanes, job0 = lane % kJobLanes;
+    for (uint32_t it0 = (warp - kConsWarps) * SB; it0 < total_stages; it0 += SB * kProdWarps) {
+      const uint32_t it = it0 + st_in_batch;
+      const bool valid = static_cast<uint32_t>(st_in_batch) < SB && it < total_stages;
+      const uint32_t use = valid ? it / depth : 0, slot = valid ? it - use * depth : 0;
+      const int pi = valid ? it / p.nstages : 0, ks = valid ? it - pi * p.nstages : 0;
+      const Pass& P = passes[pi];
+      const BranchArgs& br = p.f.branch[P.branch];
+      const int nk = br.k_end - br.k_begin;
+      const uint32_t sbase = stage0 + slot * p.stage_bytes;
+      const uint32_t bar = full0 + 8u * slot;
+      if (valid && job0 == 0) {
+        if (mbar_wait(empty0 + 8u * slot, (use & 1u) ^ 1u, abort_flag, p.f.status)) {
+          int nkb = 0;
 #pragma unroll
-      for (int s = 0; s < kBatch; ++s) {
-        const int ms = b.ms0 + s;
-        wa[s] = make_uint4(0, 0, 0, 0);
-        wb[s] = make_uint4(0, 0, 0, 0);
-        // this thread's chunk starts at reduction offset ms*4*CHK + tig*CHK
-        const int kcode = ms * 4 * CHK + tig * CHK;
-        const int kb = kcode >> 7;
-        if (ms < ms_end && kb < p.kblocks) {
-          const int inblk = ((kcode & 127) * BITS) >> 3;
-          wa[s] = __ldg(reinterpret_cast<const uint4*>(base_a + kb * blk_a + inblk));
-          if (has_b) wb[s] = __ldg(reinterpret_cast<const uint4*>(base_b + kb * blk_b + inblk));
+          for (int kbs = 0; kbs < KBPS; ++kbs) nkb += (ks * KBPS + kbs < p.kblocks) ? 1 : 0;
+          mbar_expect_tx(bar, static_cast<uint32_t>(nkb * (kXTile + P.wbytes)));
         }
       }
-    };
-
-    uint4 na[kBatch], nb[kBatch];
-    Batch nxt = first_batch(0);
-    issue(nxt, na, nb);
-
-    for (int gi = 0; gi < my_groups; ++gi) {
-      const int* m = meta + (gi * kSlabsPerGroup + sl) * kMetaInts;
-      const int branch = meta[(gi * kSlabsPerGroup) * kMetaInts + 1];   // the group's branch (slab 0 of the group)
-      const BranchArgs& br = p.f.branch[branch];
-      // this thread's activation rows (token gid of each 8-token tile); aligned rows take 16-byte loads
-      const int8_t* xrow[NT];
-      bool xok[NT];
-#pragma unroll
-      for (int t = 0; t < NT; ++t) {
-        xok[t] = gid + 8 * t < p.f.T;
-        xrow[t] = br.xq + static_cast<int64_t>(xok[t] ? gid + 8 * t : 0) * p.f.ldxq;
-      }
-      const int nch = m[0];
-      const int npairs = nch > 0 ? (nch + 1) >> 1 : 0;
-      const int buf = gi & 1;
-      // the epilogue warps must have drained this buffer (group gi - 2)
-      if (!mbar_wait(empty0 + 8u * buf, ((gi >> 1) & 1) ^ 1, abort_flag, p.f.status)) break;
-      int* dst_base = red + buf * RED_INTS + ((sl * kSlices + slice) * p.np * 32 + lane) * (4 * NT);
-      for (int q = 0; q < npairs; ++q) {
-        int acc[NT][4];
-#pragma unroll
-        for (int t = 0; t < NT; ++t)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[t][e] = 0;
-        if (has_range) {
-          for (int ms0 = ms_begin; ms0 < ms_end; ms0 += kBatch) {
-            // the loads of this batch were issued one batch ago; issue the next batch now
-            uint4 wa[kBatch], wb[kBatch];
-#pragma unroll
-            for (int s = 0; s < kBatch; ++s) {
-              wa[s] = na[s];
-              wb[s] = nb[s];
-            }
-            nxt = next_batch(Batch{gi, q, ms0});
-            issue(nxt, na, nb);
-#pragma unroll
-            for (int s = 0; s < kBatch; ++s) {
-              const int ms = ms0 + s;
-              if (ms >= ms_end) break;
-              uint32_t ra[16], rb[16];
-              unpack_chunk<BITS>(wa[s], ra);
-              unpack_chunk<BITS>(wb[s], rb);
-              // B fragments: CHK consecutive activation codes of this thread's token, from
-              // reduction offset ms*4*CHK + tig*CHK (register 2m covers 8m..8m+3, 2m+1 covers 8m+4..8m+7)
-              const int kx = ms * 4 * CHK + tig * CHK;
-#pragma unroll
-              for (int t = 0; t < NT; ++t) {
-                uint32_t xb[2 * NMMA];
-#pragma unroll
-                for (int v = 0; v < NMMA / 2; ++v) {
-                  uint4 xv = make_uint4(0, 0, 0, 0);
-                  if (xok[t]) {
-                    const int k16 = kx + 16 * v;
-                    if (k16 < I) xv = __ldg(reinterpret_cast<const uint4*>(xrow[t] + k16));   // I % 16 == 0 (host check)
-                  }
-                  xb[4 * v] = xv.x; xb[4 * v + 1] = xv.y; xb[4 * v + 2] = xv.z; xb[4 * v + 3] = xv.w;
-                }
-#pragma unroll
-                for (int mm = 0; mm < NMMA; ++mm)
-                  // tile rows 0-7: first order of the pair, rows 8-15: second order
-                  mma_s8(acc[t], ra[2 * mm], rb[2 * mm], ra[2 * mm + 1], rb[2 * mm + 1], xb[2 * mm], xb[2 * mm + 1]);
-              }
+      __syncwarp();
+      if (*abort_flag) break;
+      // jobs of a stage: per reduction block, the activation tile and then one run of rows per order
+      const int njobs = KBPS * (1 + nk);
+      for (int j0 = 0; j0 < KBPS * (1 + p.nkmax); j0 += kJobLanes) {   // same trip count in every lane; lanes without a job idle
+        const int j = j0 + job0;
+        if (valid && j < njobs) {
+          const int kbs = j / (1 + nk), idx = j - kbs * (1 + nk);
+          const int kb = ks * KBPS + kbs;
+          if (kb < p.kblocks) {
+            if (idx == 0) {
+              // activations: token rows beyond T and reduction bytes beyond I come back as zeros
+              tma_load_2d(sbase + kbs * kXTile, &p.tmap_x[P.branch], kb * 128, 0, bar);
+            } else if (P.seg_rows[idx - 1] > 0) {
+              const int ko = idx - 1;
+              const OrderView& ov = p.f.order[br.k_begin + ko];
+              const uint8_t* src = ov.kcodes + (static_cast<size_t>(kb) * ov.rows + P.seg_row0[ko]) * p.pk;
+              bulk_load(sbase + P.seg_off[ko] + kbs * P.seg_rows[ko] * p.pk, src, static_cast<uint32_t>(P.seg_rows[ko] * p.pk), bar);
             }
           }
         }
-        int* dst = dst_base + q * 32 * (4 * NT);
-#pragma unroll
-        for (int t = 0; t < NT; ++t)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) dst[t * 4 + e] = acc[t][e];
+        __syncwarp();
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(full0 + 8u * buf);
+    }
+    __syncwarp();
+    // no copy may still be writing into this CTA's shared memory when it exits
+    if (warp == kConsWarps && lane == 0) {
+      for (uint32_t j = (total_stages > static_cast<uint32_t>(depth) ? total_stages - depth : 0); j < total_stages; ++j) {
+        const long long t0 = clock64();
+        while (!mbar_try(full0 + 8u * (j % depth), (j / depth) & 1) && clock64() - t0 < kWaitLimitCycles) {
+        }
+      }
     }
   } else {
-    // ================================================================== epilogue warps (one per slab)
-    const int sl = warp - kStreamWarps;
-    for (int gi = 0; gi < my_groups; ++gi) {
-      const int* m = meta + (gi * kSlabsPerGroup + sl) * kMetaInts;
-      const int nch = m[0];
-      const int branch = m[1];
-      const int npairs = nch > 0 ? (nch + 1) >> 1 : 0;
-      const int buf = gi & 1;
-      const int grp = blockIdx.x + gi * gridDim.x;
-      const int slab = grp * kSlabsPerGroup + sl;
-      const int c = (slab - branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
-      const float* cs_slab = cstab + (gi * kSlabsPerGroup + sl) * 2 * p.np * 8;
-      const float bv = biastab[(gi * kSlabsPerGroup + sl) * 8 + gid];
-      const bool bias = nch >= 0 && p.f.bias && p.f.branch[branch].add_bias;
-      if (!mbar_wait(full0 + 8u * buf, (gi >> 1) & 1, abort_flag, p.f.status)) break;
-      if (nch >= 0) {
-        const BranchArgs& br = p.f.branch[branch];
+    // ================================================================== consumer warps
+    // scale products s_k * lambda_x and bias of every own slab (needed at the end of a pass only;
+    // the loads overlap the first copies)
+    for (int e = threadIdx.x; e < cnt * p.nkmax * 8; e += 32 * kConsWarps) {
+      const int r = e & 7, ko = (e >> 3) % p.nkmax, li = (e >> 3) / p.nkmax;
+      const int branch = (s0 + li) / p.slabs_per_branch;
+      const BranchArgs& br = p.f.branch[branch];
+      const int row0 = slabmeta[li * p.nkmax + ko];
+      float v = 0.f;
+      if (row0 >= 0) v = __fmul_rn(__ldg(p.f.order[br.k_begin + ko].scales + row0 + r), __ldg(br.sx));
+      cstab[e] = v;
+    }
+    for (int e = threadIdx.x; e < cnt * 8; e += 32 * kConsWarps) {
+      const int r = e & 7, li = e >> 3;
+      const int branch = (s0 + li) / p.slabs_per_branch;
+      float v = 0.f;
+      if (p.f.bias && p.f.branch[branch].add_bias) v = __ldg(p.f.bias + (s0 + li - branch * p.slabs_per_branch) * 8 + r);
+      biastab[e] = v;
+    }
+    asm volatile("bar.sync 1, %0;" ::"r"(32 * kConsWarps) : "memory");   // every consumer warp arrives here unconditionally
+
+    const int centries = 1 + 3 * p.nkmax;
+    int* mychunks = chunktab + warp * SPW * centries;
+    uint32_t slot = 0, phase = 0;
+    bool ok = true;
+    for (int pi = 0; pi < npass && ok; ++pi) {
+      const Pass& P = passes[pi];
+      const BranchArgs& br = p.f.branch[P.branch];
+      const int nk = br.k_end - br.k_begin;
+      // kept orders of this warp's slabs, ascending: (order index in branch, byte offset of the 8 rows in a
+      // stage, bytes between the two reduction blocks of a stage)
+      __syncwarp();
+      if (lane < SPW) {
+        int* ct = mychunks + lane * centries;
+        const int li = P.lb + warp + kConsWarps * lane;
+        int n = 0;
+        if (li < P.le) {
+          for (int ko = 0; ko < nk; ++ko) {
+            const int row0 = slabmeta[li * p.nkmax + ko];
+            if (row0 < 0) continue;
+            ct[1 + 3 * n] = ko;
+            ct[2 + 3 * n] = P.seg_off[ko] + (row0 - P.seg_row0[ko]) * p.pk;
+            ct[3 + 3 * n] = P.seg_rows[ko] * p.pk;
+            ++n;
+          }
+        }
+        ct[0] = n;
+      }
+      __syncwarp();
+      int acc[SPW][NP][NT][4];
+#pragma unroll
+      for (int s = 0; s < SPW; ++s)
+#pragma unroll
+        for (int q = 0; q < NP; ++q)
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[s][q][t][e] = 0;
+      int nchunks[SPW];
+#pragma unroll
+      for (int s = 0; s < SPW; ++s) nchunks[s] = mychunks[s * centries];
+
+      for (int ks = 0; ks < p.nstages; ++ks) {
+        if (!mbar_wait(full0 + 8u * slot, phase, abort_flag, p.f.status)) {
+          ok = false;
+          break;
+        }
+        const uint32_t sbase = stage0 + slot * p.stage_bytes;
+#pragma unroll
+        for (int ms = 0; ms < MS; ++ms) {
+          // this lane's chunk: CHK codes from reduction offset kc of the stage
+          const int kc = ms * 4 * CHK + tig * CHK;
+          const int kbs = kc >> 7, within = kc & 127;
+          if (ks * KBPS + kbs >= p.kblocks) continue;   // the stage's second block lies beyond the reduction axis
+          const uint32_t wbyte = static_cast<uint32_t>(gid * p.pk + ((within * BITS) >> 3));
+          uint4 wa[SPW][NP], wb[SPW][NP];
+#pragma unroll
+          for (int s = 0; s < SPW; ++s)
+#pragma unroll
+            for (int q = 0; q < NP; ++q) {
+              wa[s][q] = make_uint4(0, 0, 0, 0);
+              wb[s][q] = make_uint4(0, 0, 0, 0);
+              const int* ct = mychunks + s * centries;
+              if (2 * q < nchunks[s]) wa[s][q] = lds128(sbase + ct[2 + 6 * q] + kbs * ct[3 + 6 * q] + wbyte);
+              if (2 * q + 1 < nchunks[s]) wb[s][q] = lds128(sbase + ct[5 + 6 * q] + kbs * ct[6 + 6 * q] + wbyte);
+            }
+#pragma unroll
+          for (int v = 0; v < XCH; ++v) {
+            uint4 xv[NT];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) {
+              const int r = gid + 8 * t;
+              const int c16 = (within >> 4) + v;
+              xv[t] = lds128(sbase + kbs * kXTile + r * 128 + ((c16 ^ (r & 7)) << 4));
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int mm = 2 * v + h;
+#pragma unroll
+              for (int s = 0; s < SPW; ++s)
+#pragma unroll
+                for (int q = 0; q < NP; ++q) {
+                  if (2 * q >= nchunks[s]) continue;
+                  uint32_t a0, a1, b0, b1;
+                  frag<BITS>(wa[s][q], mm, a0, a1);
+                  frag<BITS>(wb[s][q], mm, b0, b1);
+#pragma unroll
+                  for (int t = 0; t < NT; ++t) {
+                    const uint32_t xw[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
+                    // tile rows 0-7: first order of the pair, rows 8-15: second order
+                    mma_s8(acc[s][q][t], a0, b0, a1, b1, xw[2 * h], xw[2 * h + 1]);
+                  }
+                }
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * slot);
+        if (++slot == static_cast<uint32_t>(depth)) {
+          slot = 0;
+          phase ^= 1u;
+        }
+      }
+      if (!ok) break;
+      // ---- fixed-order epilogue, thread-local: accumulator registers 0,1 belong to tile row gid (first
+      // order of the pair), 2,3 to row gid + 8 (second order); columns 2*tig, 2*tig + 1 of token tile t
+#pragma unroll
+      for (int s = 0; s < SPW; ++s) {
+        const int li = P.lb + warp + kConsWarps * s;
+        if (li >= P.le) continue;
+        const int* ct = mychunks + s * centries;
+        const int c = (s0 + li - P.branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
         float y[NT][2];
 #pragma unroll
         for (int t = 0; t < NT; ++t) y[t][0] = y[t][1] = 0.f;
 #pragma unroll
-        for (int q = 0; q < kMaxPairs; ++q) {
-          if (q >= npairs) break;
-          int acc[NT][4];
-#pragma unroll
-          for (int t = 0; t < NT; ++t)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[t][e] = 0;
-#pragma unroll
-          for (int s = 0; s < kSlices; ++s) {
-            const int* src = red + buf * RED_INTS + (((sl * kSlices + s) * p.np + q) * 32 + lane) * (4 * NT);
-#pragma unroll
-            for (int t = 0; t < NT; ++t)
-#pragma unroll
-              for (int e = 0; e < 4; ++e) acc[t][e] += src[t * 4 + e];
-          }
-          // accumulator registers 0,1: tile row gid (first order of the pair); 2,3: tile row gid + 8
-          // (second order); columns 2*tig, 2*tig + 1 of token tile t.  Ascending order.
+        for (int q = 0; q < NP; ++q) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const int ci = 2 * q + half;
-            if (ci >= nch) break;
-            const float cs = cs_slab[ci * 8 + gid];
-            const int row = m[3 + 2 * ci] + gid, roff = p.f.order[m[2 + 2 * ci]].row_off;
+            if (ci >= nchunks[s]) continue;
+            const int ko = ct[1 + 3 * ci];
+            const float cs = cstab[(li * p.nkmax + ko) * 8 + gid];
+            const int row = slabmeta[li * p.nkmax + ko] + gid, roff = p.f.order[br.k_begin + ko].row_off;
 #pragma unroll
             for (int t = 0; t < NT; ++t)
 #pragma unroll
               for (int e = 0; e < 2; ++e) {
-                const int a = acc[t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
+                const int a = acc[s][q][t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
                 y[t][e] = __fmaf_rn(__int2float_rn(a), cs, y[t][e]);
                 const int tok = 8 * t + 2 * tig + e;
-                if (p.f.partials && tok < p.f.T)
-                  p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff + row] = a;
+                if (p.f.partials && tok < p.f.T) p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff + row] = a;
               }
           }
         }
+        const bool bias = p.f.bias && br.add_bias;
+        const float bv = biastab[li * 8 + gid];
 #pragma unroll
         for (int t = 0; t < NT; ++t)
 #pragma unroll
@@ -398,8 +481,6 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
             *dst = v;
           }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8u * buf);
     }
   }
 }
@@ -408,43 +489,65 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const Param
 
 static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   using namespace st;
-  if (a.T > 16 || a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
-  // activation fragments are fetched with 16-byte loads
-  if (a.I % 16 != 0 || a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.T > 16 || a.g % 8 != 0 || a.O % 8 != 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // tensor-map row pitch
   for (int m = 0; m < a.num_branches; ++m)
     if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
-  if (max_cluster > 2 * kMaxPairs) return PIPE_ERR_UNSUPPORTED;
-  Params p;
+  if (max_cluster > kMaxOrd) return PIPE_ERR_UNSUPPORTED;
+  static Params p;   // large; filled per call under the lock
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   p.f = a;
   const int nt = a.T <= 8 ? 1 : 2;
-  const int chk = 128 / a.bits;
+  const int np = max_cluster <= 2 ? 1 : (max_cluster <= 4 ? 2 : 4);
+  const int spw = (np * nt <= 2) ? 2 : 1;
   p.kblocks = ceil_div(a.I, 128);
-  p.nms = ceil_div(p.kblocks * 128, 4 * chk);
   p.pk = 128 * a.bits / 8;
   p.shift = 8 - a.bits;
-  // groups of slabs must not straddle branches: pad every branch to a multiple of the group size
-  p.slabs_per_branch = round_up(a.O / 8, kSlabsPerGroup);
-  p.groups = p.slabs_per_branch * a.num_branches / kSlabsPerGroup;
-  p.xs_bytes = 0;
+  p.kbps = a.bits == 2 ? 2 : 1;
+  p.nstages = ceil_div(p.kblocks, p.kbps);
+  p.nkmax = max_cluster;
+  p.slabs_per_branch = a.O / 8;
+  p.total_slabs = p.slabs_per_branch * a.num_branches;
+  p.pass_slabs = kConsWarps * spw;
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int grid = p.groups < sms ? p.groups : sms;
-  const int own = ceil_div(p.groups, grid);
-  if (own > kMaxGroups) return PIPE_ERR_UNSUPPORTED;
-  p.np = (max_cluster + 1) / 2;
-  const int red_bytes = 2 * kSlabsPerGroup * kSlices * p.np * 32 * 4 * nt * 4;
-  const int meta_bytes = own * kSlabsPerGroup * (kMetaInts + 2 * p.np * 8 + 8) * 4;
-  const int dyn = red_bytes + meta_bytes;
-  if (dyn + 1024 > smem_max) return PIPE_ERR_UNSUPPORTED;
-
+  p.ctas_per_branch = sms / a.num_branches;
+  if (p.ctas_per_branch < 1) return PIPE_ERR_UNSUPPORTED;
+  if (p.ctas_per_branch > p.slabs_per_branch) p.ctas_per_branch = p.slabs_per_branch;
+  const int grid = p.ctas_per_branch * a.num_branches;
+  p.own_max = ceil_div(p.slabs_per_branch, p.ctas_per_branch);
+  // passes a CTA may need: its range cut into pieces of pass_slabs
+  if (ceil_div(p.own_max, p.pass_slabs) > kMaxPasses) return PIPE_ERR_UNSUPPORTED;
+  // a stage holds one reduction block (two for 2-bit codes) of every order for the slabs of a pass, all kept
+  const int pass_cap = p.pass_slabs < p.own_max ? p.pass_slabs : p.own_max;
+  p.stage_bytes = round_up(p.kbps * (kXTile + pass_cap * 8 * max_cluster * p.pk), 1024);
+  const int table_bytes = p.own_max * (max_cluster * 4 + max_cluster * 32 + 32) + kConsWarps * spw * (1 + 3 * max_cluster) * 4;
   void (*kern)(const Params) = nullptr;
-  if (a.bits == 8) kern = nt == 1 ? stream_forward_kernel<8, 1> : stream_forward_kernel<8, 2>;
-  else if (a.bits == 4) kern = nt == 1 ? stream_forward_kernel<4, 1> : stream_forward_kernel<4, 2>;
-  else kern = nt == 1 ? stream_forward_kernel<2, 1> : stream_forward_kernel<2, 2>;
+#define PIPE_ST_PICK(B)                                                                     \
+  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1> : (np == 2 ? stream_forward_kernel<B, 1, 2> : stream_forward_kernel<B, 1, 4>); \
+  else kern = np == 1 ? stream_forward_kernel<B, 2, 1> : (np == 2 ? stream_forward_kernel<B, 2, 2> : stream_forward_kernel<B, 2, 4>);
+  if (a.bits == 8) { PIPE_ST_PICK(8) } else if (a.bits == 4) { PIPE_ST_PICK(4) } else { PIPE_ST_PICK(2) }
+#undef PIPE_ST_PICK
+  cudaFuncAttributes fattr;
+  if (cudaFuncGetAttributes(&fattr, kern) != cudaSuccess) return PIPE_ERR_CUDA;
+  const int avail = smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024 - round_up(table_bytes, 16);
+  p.depth = avail / p.stage_bytes;
+  if (p.depth > kMaxDepth) p.depth = kMaxDepth;
+  // no more ring than the stages a CTA will ever fill
+  const int most_stages = ceil_div(p.own_max, p.pass_slabs) * p.nstages;
+  if (p.depth > round_up(most_stages, kProdWarps)) p.depth = round_up(most_stages, kProdWarps);
+  p.depth -= p.depth % kProdWarps;   // every producer warp owns depth / kProdWarps slots
+  if (p.depth < kProdWarps) return PIPE_ERR_UNSUPPORTED;
+  const int dyn = 1024 + p.depth * p.stage_bytes + round_up(table_bytes, 16);
+  for (int m = 0; m < a.num_branches; ++m)
+    if (!make_tensor_map_2d_u8(&p.tmap_x[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
+                               static_cast<uint64_t>(a.ldxq), 128, 16, true))
+      return PIPE_ERR_CUDA;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess) return PIPE_ERR_CUDA;
   kern<<<grid, kThreads, dyn, stream>>>(p);
   count_launch(1);

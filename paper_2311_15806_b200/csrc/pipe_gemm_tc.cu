@@ -828,6 +828,12 @@ static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int 
 
 }  // namespace tc
 
+bool make_tensor_map_2d_u8(CUtensorMap* map, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+                           uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
+  return tc::make_map_2d(map, base, inner_bytes, rows, pitch_bytes, box_inner, box_rows,
+                         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
 static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   using namespace tc;
   static Params p;  // large; filled per call under the lock
