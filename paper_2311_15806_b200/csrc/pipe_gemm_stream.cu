@@ -11,12 +11,14 @@
 // quantized activations as a swizzled TMA box).  Nothing on the load path costs registers, and the
 // ring keeps far more bytes in flight than the bandwidth-delay product of the memory system.
 //
-// 16 consumer warps each own one or two slabs of the pass for the WHOLE reduction axis: they read
-// their 8 rows of a stage from shared memory, widen sub-byte codes with the shift-and-mask layout
-// and feed warp-level integer MMAs (mma.sync m16n8k32: weights as the 16-row operand -- two orders
-// of the slab, ascending, share a tile -- tokens as the 8-column operand).  The int32 sums stay in
-// registers until the reduction axis is done, so the fixed-order fp32 epilogue is thread-local and
-// needs neither a cross-warp reduction nor extra memory.  Every mbarrier wait is bounded.
+// 16 consumer warps form 4 groups; group j handles the stages j, j + 4, ... (so a stage is read by 4
+// warps, each of which covers up to 5 slabs of it: enough independent work per visit to hide the
+// latency of the barrier wait, the shared-memory loads and the chain of dependent MMAs).  A warp
+// reads its slabs' 8 rows from the stage, widens sub-byte codes with the shift-and-mask layout and
+// feeds warp-level integer MMAs (mma.sync m16n8k32: weights as the 16-row operand -- two orders of
+// the slab, ascending, share a tile -- tokens as the 8-column operand).  At the end of a pass the
+// four groups add their exact int32 sums in a small shared-memory array, and the fixed-order fp32
+// epilogue runs once per slab.  Every mbarrier wait is bounded.
 #include <mutex>
 
 #include "pipe_common.cuh"
@@ -27,6 +29,8 @@ namespace st {
 
 constexpr int kConsWarps = 16;
 constexpr int kProdWarps = 4;
+constexpr int kGroups = 4;                       // consumer groups = slices of the reduction axis
+constexpr int kGroupWarps = kConsWarps / kGroups;
 constexpr int kThreads = 32 * (kConsWarps + kProdWarps);
 constexpr int kMaxOrd = 8;          // orders per branch
 constexpr int kMaxPasses = 32;      // passes (<= 32 slabs of one branch) a CTA may need
@@ -42,7 +46,7 @@ struct Params {
   int shift;              // 8 - b
   int slabs_per_branch;   // O / 8
   int total_slabs;
-  int pass_slabs;         // slabs per pass: 16 * slabs per warp
+  int pass_slabs;         // slabs per pass: warps of a group * slabs per warp
   int depth, stage_bytes;
   int kbps;               // reduction blocks per stage (2 for 2-bit codes, else 1)
   int nstages;            // stages per pass
@@ -106,10 +110,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
+// Ordinary loads (not volatile asm), so that the compiler may schedule them between the MMAs; the
+// barrier wait before them is a volatile asm with a memory clobber, which they cannot cross.
+__device__ __forceinline__ uint4 lds128(const uint8_t* stage, uint32_t off) {
+  return *reinterpret_cast<const uint4*>(stage + off);
 }
 
 __device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -149,13 +153,13 @@ __device__ __forceinline__ int rows_before(const int32_t* cum, int c, int O, int
 
 template <int BITS, int NT, int NP>
 __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __grid_constant__ Params p) {
-  constexpr int SPW = (NP * NT <= 2) ? 2 : 1;   // slabs per consumer warp and pass
+  constexpr int SPW = (NP * NT <= 2) ? 5 : (NP * NT == 4 ? 2 : 1);   // slabs per consumer warp and pass
   constexpr int CHK = 128 / BITS;               // codes per 16-byte chunk
   constexpr int KBPS = (BITS == 2) ? 2 : 1;     // reduction blocks per stage
   constexpr int MS = KBPS * 128 / (4 * CHK);    // macro steps (4 chunks per row of 8 lanes x 4) per stage
   constexpr int XCH = CHK / 16;                 // 16-byte activation chunks per macro step and token
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bars[2 * kMaxDepth];      // full[depth] empty[depth]
+  __shared__ uint64_t bars[2 * kMaxDepth + 2];  // full[depth] empty[depth] sums_ready sums_free
   __shared__ Pass passes[kMaxPasses];
   __shared__ int npass_s;
   __shared__ int abort_flag_s;
@@ -169,7 +173,10 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   float* cstab = reinterpret_cast<float*>(slabmeta + p.own_max * p.nkmax);          // [own][nkmax][8] s_k * lambda_x
   float* biastab = cstab + p.own_max * p.nkmax * 8;                                 // [own][8]
   int* chunktab = reinterpret_cast<int*>(biastab + p.own_max * 8);                  // [warp][SPW][1 + 3 * nkmax]
+  int* sums = chunktab + kConsWarps * SPW * (1 + 3 * p.nkmax);                          // [pass slab][NP][NT * 4][32 lanes]
+  const uint8_t* stage_gen = smem_raw + (stage0 - smem_u32(smem_raw));
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8u * kMaxDepth;
+  const uint32_t sums_ready = empty0 + 8u * kMaxDepth, sums_free = sums_ready + 8u;
   const int depth = p.depth;
 
   // this CTA's slabs: [s0, s0 + cnt), all of one branch
@@ -182,8 +189,10 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     abort_flag_s = 0;
     for (int s = 0; s < depth; ++s) {
       mbar_init(full0 + 8u * s, 1);
-      mbar_init(empty0 + 8u * s, kConsWarps);
+      mbar_init(empty0 + 8u * s, kGroupWarps);   // slot s is only ever read by group s % kGroups
     }
+    mbar_init(sums_ready, kConsWarps);
+    mbar_init(sums_free, kConsWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // passes: at most pass_slabs slabs, never across a branch boundary
     int np = 0;
@@ -198,6 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     }
     npass_s = np;
   }
+  for (int e = threadIdx.x; e < p.pass_slabs * NP * NT * 4 * 32; e += kThreads) sums[e] = 0;
   // ---- which orders keep each own slab, and where its 8 rows start
   for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
     const int li = e / p.nkmax, ko = e % p.nkmax;
@@ -333,25 +343,27 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     asm volatile("bar.sync 1, %0;" ::"r"(32 * kConsWarps) : "memory");   // every consumer warp arrives here unconditionally
 
     const int centries = 1 + 3 * p.nkmax;
-    int* mychunks = chunktab + warp * SPW * centries;
-    uint32_t slot = 0, phase = 0;
+    const int grp = warp / kGroupWarps, wg = warp % kGroupWarps;
     bool ok = true;
     for (int pi = 0; pi < npass && ok; ++pi) {
       const Pass& P = passes[pi];
       const BranchArgs& br = p.f.branch[P.branch];
       const int nk = br.k_end - br.k_begin;
-      // kept orders of this warp's slabs, ascending: (order index in branch, byte offset of the 8 rows in a
-      // stage, bytes between the two reduction blocks of a stage)
+      const int nsl = P.le - P.lb;
+      // the sums of the previous pass have been read and cleared by every warp
+      if (pi > 0 && !mbar_wait(sums_free, (pi - 1) & 1, abort_flag, p.f.status)) break;
+      // This warp's slabs in every stage it visits: wg, wg + 4, ...  Their kept orders, ascending: (byte offset
+      // of the 8 rows in a stage, bytes between the reduction blocks of a stage), in a table private to the warp.
+      int* mychunks = chunktab + warp * SPW * centries;
       __syncwarp();
       if (lane < SPW) {
         int* ct = mychunks + lane * centries;
-        const int li = P.lb + warp + kConsWarps * lane;
+        const int sl = wg + kGroupWarps * lane;
         int n = 0;
-        if (li < P.le) {
+        if (sl < nsl) {
           for (int ko = 0; ko < nk; ++ko) {
-            const int row0 = slabmeta[li * p.nkmax + ko];
+            const int row0 = slabmeta[(P.lb + sl) * p.nkmax + ko];
             if (row0 < 0) continue;
-            ct[1 + 3 * n] = ko;
             ct[2 + 3 * n] = P.seg_off[ko] + (row0 - P.seg_row0[ko]) * p.pk;
             ct[3 + 3 * n] = P.seg_rows[ko] * p.pk;
             ++n;
@@ -360,6 +372,17 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
         ct[0] = n;
       }
       __syncwarp();
+      int nchunks[SPW];
+      uint32_t woff[SPW][2 * NP], wstr[SPW][2 * NP];
+#pragma unroll
+      for (int s = 0; s < SPW; ++s) {
+        nchunks[s] = mychunks[s * centries];
+#pragma unroll
+        for (int ci = 0; ci < 2 * NP; ++ci) {
+          woff[s][ci] = ci < nchunks[s] ? mychunks[s * centries + 2 + 3 * ci] : 0;
+          wstr[s][ci] = ci < nchunks[s] ? mychunks[s * centries + 3 + 3 * ci] : 0;
+        }
+      }
       int acc[SPW][NP][NT][4];
 #pragma unroll
       for (int s = 0; s < SPW; ++s)
@@ -369,97 +392,121 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
           for (int t = 0; t < NT; ++t)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[s][q][t][e] = 0;
-      int nchunks[SPW];
-#pragma unroll
-      for (int s = 0; s < SPW; ++s) nchunks[s] = mychunks[s * centries];
 
-      for (int ks = 0; ks < p.nstages; ++ks) {
-        if (!mbar_wait(full0 + 8u * slot, phase, abort_flag, p.f.status)) {
+      // stages of this pass that belong to this warp's group
+      const uint32_t it_begin = static_cast<uint32_t>(pi) * p.nstages, it_end = it_begin + p.nstages;
+      uint32_t it = it_begin + ((grp + kGroups - it_begin % kGroups) % kGroups);
+      for (; it < it_end; it += kGroups) {
+        const uint32_t use = it / depth, slot = it - use * depth;
+        const int ks = it - it_begin;
+        if (!mbar_wait(full0 + 8u * slot, use & 1u, abort_flag, p.f.status)) {
           ok = false;
           break;
         }
-        const uint32_t sbase = stage0 + slot * p.stage_bytes;
+        const uint8_t* sgen = stage_gen + static_cast<size_t>(slot) * p.stage_bytes;
 #pragma unroll
         for (int ms = 0; ms < MS; ++ms) {
           // this lane's chunk: CHK codes from reduction offset kc of the stage
           const int kc = ms * 4 * CHK + tig * CHK;
           const int kbs = kc >> 7, within = kc & 127;
-          if (ks * KBPS + kbs >= p.kblocks) continue;   // the stage's second block lies beyond the reduction axis
+          if (ks * KBPS + kbs >= p.kblocks) continue;   // a stage's later blocks may lie beyond the reduction axis
           const uint32_t wbyte = static_cast<uint32_t>(gid * p.pk + ((within * BITS) >> 3));
-          uint4 wa[SPW][NP], wb[SPW][NP];
+          uint4 xv[XCH][NT];
 #pragma unroll
-          for (int s = 0; s < SPW; ++s)
-#pragma unroll
-            for (int q = 0; q < NP; ++q) {
-              wa[s][q] = make_uint4(0, 0, 0, 0);
-              wb[s][q] = make_uint4(0, 0, 0, 0);
-              const int* ct = mychunks + s * centries;
-              if (2 * q < nchunks[s]) wa[s][q] = lds128(sbase + ct[2 + 6 * q] + kbs * ct[3 + 6 * q] + wbyte);
-              if (2 * q + 1 < nchunks[s]) wb[s][q] = lds128(sbase + ct[5 + 6 * q] + kbs * ct[6 + 6 * q] + wbyte);
-            }
-#pragma unroll
-          for (int v = 0; v < XCH; ++v) {
-            uint4 xv[NT];
+          for (int v = 0; v < XCH; ++v)
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
               const int r = gid + 8 * t;
               const int c16 = (within >> 4) + v;
-              xv[t] = lds128(sbase + kbs * kXTile + r * 128 + ((c16 ^ (r & 7)) << 4));
+              xv[v][t] = lds128(sgen, kbs * kXTile + r * 128 + ((c16 ^ (r & 7)) << 4));
             }
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const int mm = 2 * v + h;
+          for (int s = 0; s < SPW; ++s) {
 #pragma unroll
-              for (int s = 0; s < SPW; ++s)
+            for (int q = 0; q < NP; ++q) {
+              if (2 * q >= nchunks[s]) continue;
+              const uint4 wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
+              uint4 wb = make_uint4(0, 0, 0, 0);
+              if (2 * q + 1 < nchunks[s]) wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
 #pragma unroll
-                for (int q = 0; q < NP; ++q) {
-                  if (2 * q >= nchunks[s]) continue;
-                  uint32_t a0, a1, b0, b1;
-                  frag<BITS>(wa[s][q], mm, a0, a1);
-                  frag<BITS>(wb[s][q], mm, b0, b1);
+              for (int mm = 0; mm < 2 * XCH; ++mm) {
+                uint32_t a0, a1, b0, b1;
+                frag<BITS>(wa, mm, a0, a1);
+                frag<BITS>(wb, mm, b0, b1);
 #pragma unroll
-                  for (int t = 0; t < NT; ++t) {
-                    const uint32_t xw[4] = {xv[t].x, xv[t].y, xv[t].z, xv[t].w};
-                    // tile rows 0-7: first order of the pair, rows 8-15: second order
-                    mma_s8(acc[s][q][t], a0, b0, a1, b1, xw[2 * h], xw[2 * h + 1]);
-                  }
+                for (int t = 0; t < NT; ++t) {
+                  const uint32_t xw[4] = {xv[mm >> 1][t].x, xv[mm >> 1][t].y, xv[mm >> 1][t].z, xv[mm >> 1][t].w};
+                  // tile rows 0-7: first order of the pair, rows 8-15: second order
+                  mma_s8(acc[s][q][t], a0, b0, a1, b1, xw[2 * (mm & 1)], xw[2 * (mm & 1) + 1]);
                 }
+              }
             }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
-        if (++slot == static_cast<uint32_t>(depth)) {
-          slot = 0;
-          phase ^= 1u;
-        }
       }
       if (!ok) break;
-      // ---- fixed-order epilogue, thread-local: accumulator registers 0,1 belong to tile row gid (first
-      // order of the pair), 2,3 to row gid + 8 (second order); columns 2*tig, 2*tig + 1 of token tile t
+      // ---- the four groups add their exact partial sums
 #pragma unroll
       for (int s = 0; s < SPW; ++s) {
-        const int li = P.lb + warp + kConsWarps * s;
-        if (li >= P.le) continue;
-        const int* ct = mychunks + s * centries;
+        const int sl = wg + kGroupWarps * s;
+        if (sl >= nsl) continue;
+#pragma unroll
+        for (int q = 0; q < NP; ++q) {
+          if (2 * q >= nchunks[s]) continue;
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) atomicAdd(sums + ((sl * NP + q) * NT * 4 + t * 4 + e) * 32 + lane, acc[s][q][t][e]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sums_ready);
+      if (!mbar_wait(sums_ready, pi & 1, abort_flag, p.f.status)) break;
+      // ---- fixed-order epilogue, one warp per slab: accumulator registers 0,1 belong to tile row gid (first
+      // order of the pair), 2,3 to row gid + 8 (second order); columns 2*tig, 2*tig + 1 of token tile t
+      for (int sl = warp; sl < nsl; sl += kConsWarps) {
+        const int li = P.lb + sl;
+        // kept orders of the slab, ascending (at most 2 * NP)
+        int kos[2 * NP];
+        int nch = 0;
+#pragma unroll
+        for (int ko = 0; ko < kMaxOrd; ++ko)
+          if (ko < nk && slabmeta[li * p.nkmax + ko] >= 0) {
+#pragma unroll
+            for (int ci = 0; ci < 2 * NP; ++ci)
+              if (ci == nch) kos[ci] = ko;
+            ++nch;
+          }
         const int c = (s0 + li - P.branch * p.slabs_per_branch) * 8 + gid;   // this thread's output channel
         float y[NT][2];
 #pragma unroll
         for (int t = 0; t < NT; ++t) y[t][0] = y[t][1] = 0.f;
 #pragma unroll
         for (int q = 0; q < NP; ++q) {
+          if (2 * q >= nch) continue;
+          int a4[NT][4];
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              int* cell = sums + ((sl * NP + q) * NT * 4 + t * 4 + e) * 32 + lane;
+              a4[t][e] = *cell;
+              *cell = 0;   // ready for the next pass
+            }
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const int ci = 2 * q + half;
-            if (ci >= nchunks[s]) continue;
-            const int ko = ct[1 + 3 * ci];
+            if (ci >= nch) continue;
+            const int ko = kos[ci];
             const float cs = cstab[(li * p.nkmax + ko) * 8 + gid];
             const int row = slabmeta[li * p.nkmax + ko] + gid, roff = p.f.order[br.k_begin + ko].row_off;
 #pragma unroll
             for (int t = 0; t < NT; ++t)
 #pragma unroll
               for (int e = 0; e < 2; ++e) {
-                const int a = acc[s][q][t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
+                const int a = a4[t][2 * half + e] >> p.shift;   // exact: the sum carries a factor 2^shift
                 y[t][e] = __fmaf_rn(__int2float_rn(a), cs, y[t][e]);
                 const int tok = 8 * t + 2 * tig + e;
                 if (p.f.partials && tok < p.f.T) p.f.partials[static_cast<int64_t>(tok) * p.f.total_rows + roff + row] = a;
@@ -481,6 +528,8 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
             *dst = v;
           }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sums_free);
     }
   }
 }
@@ -502,7 +551,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   p.f = a;
   const int nt = a.T <= 8 ? 1 : 2;
   const int np = max_cluster <= 2 ? 1 : (max_cluster <= 4 ? 2 : 4);
-  const int spw = (np * nt <= 2) ? 2 : 1;
+  const int spw = (np * nt <= 2) ? 5 : (np * nt == 4 ? 2 : 1);
   p.kblocks = ceil_div(a.I, 128);
   p.pk = 128 * a.bits / 8;
   p.shift = 8 - a.bits;
@@ -511,7 +560,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   p.nkmax = max_cluster;
   p.slabs_per_branch = a.O / 8;
   p.total_slabs = p.slabs_per_branch * a.num_branches;
-  p.pass_slabs = kConsWarps * spw;
+  p.pass_slabs = kGroupWarps * spw;
   int dev = 0, smem_max = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
   cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -526,7 +575,8 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   // a stage holds one reduction block (two for 2-bit codes) of every order for the slabs of a pass, all kept
   const int pass_cap = p.pass_slabs < p.own_max ? p.pass_slabs : p.own_max;
   p.stage_bytes = round_up(p.kbps * (kXTile + pass_cap * 8 * max_cluster * p.pk), 1024);
-  const int table_bytes = p.own_max * (max_cluster * 4 + max_cluster * 32 + 32) + kConsWarps * spw * (1 + 3 * max_cluster) * 4;
+  const int table_bytes = p.own_max * (max_cluster * 4 + max_cluster * 32 + 32) + kConsWarps * spw * (1 + 3 * max_cluster) * 4 +
+                          p.pass_slabs * np * nt * 4 * 32 * 4;
   void (*kern)(const Params) = nullptr;
 #define PIPE_ST_PICK(B)                                                                     \
   if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1> : (np == 2 ? stream_forward_kernel<B, 1, 2> : stream_forward_kernel<B, 1, 4>); \
