@@ -161,7 +161,6 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxDepth + 2];  // full[depth] empty[depth] sums_ready sums_free
   __shared__ Pass passes[kMaxPasses];
-  __shared__ int npass_s;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
 
@@ -194,19 +193,9 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     mbar_init(sums_ready, kConsWarps);
     mbar_init(sums_free, kConsWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // passes: at most pass_slabs slabs, never across a branch boundary
-    int np = 0;
-    for (int cur = 0; cur < cnt && np < kMaxPasses; ++np) {
-      const int br = (s0 + cur) / p.slabs_per_branch;
-      const int br_end = (br + 1) * p.slabs_per_branch - s0;
-      const int le = min(min(cnt, br_end), cur + p.pass_slabs);
-      passes[np].branch = br;
-      passes[np].lb = cur;
-      passes[np].le = le;
-      cur = le;
-    }
-    npass_s = np;
   }
+  // passes: pieces of at most pass_slabs slabs of the CTA's range (which lies in one branch)
+  const int npass = min((cnt + p.pass_slabs - 1) / p.pass_slabs, kMaxPasses);
   for (int e = threadIdx.x; e < p.pass_slabs * NP * NT * 4 * 32; e += kThreads) sums[e] = 0;
   // ---- which orders keep each own slab, and where its 8 rows start
   for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
@@ -224,22 +213,27 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     }
     slabmeta[e] = row0;
   }
-  __syncthreads();
-  const int npass = npass_s;
-  // ---- the contiguous run of rows every pass needs from every order
-  for (int e = threadIdx.x; e < npass * kMaxOrd; e += kThreads) {
+  // ---- the contiguous run of rows every pass needs from every order (the last threads take this, so that
+  // its loads run beside those above)
+  for (int e = kThreads - 1 - threadIdx.x; e < npass * kMaxOrd; e += kThreads) {
     const int pi = e / kMaxOrd, ko = e % kMaxOrd;
     Pass& P = passes[pi];
-    const BranchArgs& br = p.f.branch[P.branch];
+    const BranchArgs& br = p.f.branch[my_branch];
+    const int lb = pi * p.pass_slabs, le = min(cnt, lb + p.pass_slabs);
     int r0 = 0, rows = 0;
     if (br.k_begin + ko < br.k_end) {
       const int32_t* cum = p.f.order[br.k_begin + ko].cum;
-      const int cb = (s0 + P.lb - P.branch * p.slabs_per_branch) * 8, ce = (s0 + P.le - P.branch * p.slabs_per_branch) * 8;
+      const int cb = (s0 + lb - my_branch * p.slabs_per_branch) * 8, ce = (s0 + le - my_branch * p.slabs_per_branch) * 8;
       r0 = rows_before(cum, cb, p.f.O, p.f.g);
       rows = rows_before(cum, ce, p.f.O, p.f.g) - r0;
     }
     P.seg_row0[ko] = r0;
     P.seg_rows[ko] = rows;
+    if (ko == 0) {
+      P.branch = my_branch;
+      P.lb = lb;
+      P.le = le;
+    }
   }
   __syncthreads();
   if (threadIdx.x < npass) {
