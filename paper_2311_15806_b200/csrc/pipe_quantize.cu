@@ -100,6 +100,97 @@ __global__ void __launch_bounds__(kQThreads) act_quantize_kernel(const QuantArgs
   }
 }
 
+// ---- contiguous tensors (ldx == ldxq == I, I a multiple of 4, 16-byte aligned input): the tensor is one
+// flat array, a thread takes one float4 per trip (a warp reads 512 and writes 128 contiguous bytes per
+// instruction) and keeps four trips in flight.
+constexpr int kFlatUnroll = 4;
+
+__global__ void __launch_bounds__(kQThreads) act_absmax_flat_kernel(const float4* __restrict__ x, int64_t n4, uint32_t* ws) {
+  uint32_t m = 0;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+  for (; i + (kFlatUnroll - 1) * stride < n4; i += kFlatUnroll * stride) {
+    float4 f[kFlatUnroll];
+#pragma unroll
+    for (int u = 0; u < kFlatUnroll; ++u) f[u] = __ldg(x + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < kFlatUnroll; ++u)
+      m = max(max(m, max(q_abs_key(f[u].x), q_abs_key(f[u].y))), max(q_abs_key(f[u].z), q_abs_key(f[u].w)));
+  }
+  for (; i < n4; i += stride) {
+    const float4 f = __ldg(x + i);
+    m = max(max(m, max(q_abs_key(f.x), q_abs_key(f.y))), max(q_abs_key(f.z), q_abs_key(f.w)));
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, d));
+  __shared__ uint32_t part[kQThreads / 32];
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kQThreads / 32; ++w) m = max(m, part[w]);
+    if (m) atomicMax(ws, m);
+  }
+}
+
+// clamp(rne(v / s)) as an int8 lane.  The IEEE quotient is what defines the code (Eq. 1 with true
+// division), but a division costs an order of magnitude more than a multiplication, so the quotient is
+// first estimated as t = v * r with r = rn(1 / s): t is within a relative 2^-22.9 of the real quotient,
+// as is the IEEE quotient itself (2^-24), so both round to the same integer unless the estimate lies
+// within |t| * 2^-21 of a rounding boundary (an odd multiple of one half) -- only then, a few times in a
+// hundred thousand, is the division carried out.  Beyond +-130 both clamp.
+__device__ __forceinline__ uint32_t quant_lane(float v, float s, float r) {
+  const float t = __fmul_rn(v, r);
+  float q = rintf(t);
+  const float at = fabsf(t);
+  if (at > 130.f) {
+    q = copysignf(127.f, t);
+  } else if (0.5f - fabsf(__fsub_rn(t, q)) <= at * 4.76837158203125e-07f) {
+    q = rintf(__fdiv_rn(v, s));
+  }
+  q = fminf(fmaxf(q, -127.f), 127.f);
+  return static_cast<uint32_t>(static_cast<int>(q)) & 0xffu;
+}
+
+__device__ __forceinline__ uint32_t quant4(const float4& f, float s, float r, bool fast) {
+  if (fast) return quant_lane(f.x, s, r) | (quant_lane(f.y, s, r) << 8) | (quant_lane(f.z, s, r) << 16) | (quant_lane(f.w, s, r) << 24);
+  uint32_t w = 0;
+  const float v[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float q = 0.f;
+    if (s != 0.f) q = fminf(fmaxf(rintf(__fdiv_rn(v[e], s)), -127.f), 127.f);
+    w |= (static_cast<uint32_t>(static_cast<int>(q)) & 0xffu) << (8 * e);
+  }
+  return w;
+}
+
+__global__ void __launch_bounds__(kQThreads) act_quantize_flat_kernel(const float4* __restrict__ x, int64_t n4,
+                                                                      uint32_t* __restrict__ xq, const uint32_t* ws,
+                                                                      const float* static_scale, float* sx_out, int* status) {
+  const uint32_t mbits = ws[0];
+  float s;
+  if (static_scale) s = *static_scale;
+  else s = __fdiv_rn(__uint_as_float(mbits), 127.f);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *sx_out = s;
+    if (mbits >= 0x7f800000u) raise_status(status, PIPE_ERR_NONFINITE);
+    if (static_scale && !(s >= 0.f && s < __uint_as_float(0x7f800000u))) raise_status(status, PIPE_ERR_INVALID_ARG);
+  }
+  // the estimate needs a reciprocal that neither overflows nor is subnormal
+  const bool fast = s >= 1e-30f && s <= 1e30f;
+  const float r = fast ? __frcp_rn(s) : 0.f;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+  for (; i + (kFlatUnroll - 1) * stride < n4; i += kFlatUnroll * stride) {
+    float4 f[kFlatUnroll];
+#pragma unroll
+    for (int u = 0; u < kFlatUnroll; ++u) f[u] = __ldg(x + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < kFlatUnroll; ++u) xq[i + u * stride] = quant4(f[u], s, r, fast);
+  }
+  for (; i < n4; i += stride) xq[i] = quant4(__ldg(x + i), s, r, fast);
+}
+
 __global__ void act_empty_kernel(const float* static_scale, float* sx_out) {
   if (threadIdx.x == 0) *sx_out = static_scale ? *static_scale : 0.f;
 }
@@ -125,6 +216,17 @@ pipe_status quantize_act_impl(const float* d_x, int64_t T, int32_t I, int64_t ld
   const int64_t want = ceil_div<int64_t>(p.total_chunks, kQThreads);
   const int grid = static_cast<int>(want < static_cast<int64_t>(sms) * 8 ? want : static_cast<int64_t>(sms) * 8);
   if (cudaMemsetAsync(d_scratch, 0, 16, s) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (ldx == I && ldxq == I && I % 4 == 0 && p.vec_in && (reinterpret_cast<uintptr_t>(d_xq) & 3) == 0) {
+    const int64_t n4 = T * (I / 4);
+    const int64_t want4 = ceil_div<int64_t>(n4, kQThreads * kFlatUnroll);
+    const int g4 = static_cast<int>(want4 < static_cast<int64_t>(sms) * 8 ? want4 : static_cast<int64_t>(sms) * 8);
+    // (with a static scale the first pass still serves the non-finite check of the input)
+    act_absmax_flat_kernel<<<g4, kQThreads, 0, s>>>(reinterpret_cast<const float4*>(d_x), n4, d_scratch);
+    act_quantize_flat_kernel<<<g4, kQThreads, 0, s>>>(reinterpret_cast<const float4*>(d_x), n4, reinterpret_cast<uint32_t*>(d_xq),
+                                                      d_scratch, d_static_scale, d_sx, status);
+    count_launch(2);
+    return launch_status();
+  }
   if (!d_static_scale) {
     act_absmax_kernel<<<grid, kQThreads, 0, s>>>(p, d_scratch);
     count_launch(1);

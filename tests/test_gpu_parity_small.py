@@ -102,6 +102,38 @@ def test_quantize_act_bit_exact(oracle, T, I):
     np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
 
 
+def test_quantize_act_at_rounding_boundaries(oracle):
+    """Values placed on, and one or two ulps beside, the rounding boundaries (k + 1/2) * lambda_x: the code is
+    defined by the IEEE quotient, so a kernel that estimates the quotient must fall back to the true
+    division there (Eq. 1 with the division reading)."""
+    rng = np.random.default_rng(5)
+    for amax in (127.0, 3.1415927, 1e-3, 77.7):
+        s = np.float32(np.float32(amax) / np.float32(127.0))
+        ks = np.arange(-127, 127, dtype=np.float64) + 0.5
+        base = (ks * np.float64(s)).astype(np.float32)
+        cols = [base]
+        v = base.copy()
+        for _ in range(3):
+            v = np.nextafter(v, np.float32(np.inf), dtype=np.float32)
+            cols.append(v.copy())
+        v = base.copy()
+        for _ in range(3):
+            v = np.nextafter(v, np.float32(-np.inf), dtype=np.float32)
+            cols.append(v.copy())
+        x = np.stack(cols).astype(np.float32)                     # [7, 254]
+        x = np.concatenate([x, (rng.standard_normal((5, 254)) * amax / 3).astype(np.float32).clip(-amax, amax)])
+        x = np.concatenate([x, np.zeros((12, 2), np.float32)], axis=1)   # 256 columns: the contiguous fast path
+        x[0, -1] = np.float32(amax)                                # pins the tensor's absmax
+        xq, sx = H.gpu_quantize(x)
+        xq_o, sx_o = oracle.quantize_act(x)
+        assert sx.cpu().numpy().view(np.uint32)[0] == np.float32(sx_o).view(np.uint32)
+        np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+        # the same through a static scale that is not absmax / 127 (clamping and large quotients)
+        xq, _ = H.gpu_quantize(x, static_scale=float(s) / 3)
+        xq_o, _ = oracle.quantize_act(x, static_scale=float(s) / 3)
+        np.testing.assert_array_equal(xq.cpu().numpy(), xq_o)
+
+
 def test_quantize_act_static_scale_zero_and_strided(oracle):
     rng = np.random.default_rng(11)
     x = (rng.standard_normal((9, 50)) * 100).astype(np.float32)
