@@ -50,6 +50,33 @@ def test_expand_weights_bit_exact(oracle, O, I, bits, K, g, n_keep):
     H.assert_expansion_matches(layer, e, oracle)
 
 
+@pytest.mark.parametrize("bits", [8, 4, 2])
+def test_expand_weights_at_rounding_boundaries(oracle, bits):
+    """Rows whose entries sit on, and a few ulps beside, the boundaries (k + 1/2) * s of their own scale: the
+    codes are defined by the IEEE quotient, whatever shortcut the kernel takes elsewhere (Eq. 1)."""
+    qmax = (1 << (bits - 1)) - 1
+    rows = []
+    for amax in (1.0, 0.0372, 3e-5, 911.0):
+        s = np.float32(np.float32(amax) / np.float32(qmax))
+        ks = np.arange(-qmax, qmax, dtype=np.float64) + 0.5
+        base = (ks * np.float64(s)).astype(np.float32)
+        for shift in range(-3, 4):
+            v = base.copy()
+            for _ in range(abs(shift)):
+                v = np.nextafter(v, np.float32(np.inf if shift > 0 else -np.inf), dtype=np.float32)
+            row = np.zeros(256, np.float32)
+            reps = -(-255 // len(v))
+            row[:255] = np.tile(v, reps)[:255]
+            row[255] = np.float32(amax)            # pins the row's absmax
+            rows.append(row)
+    W = np.stack(rows).astype(np.float32)
+    W = np.concatenate([W, np.zeros((32 - len(W) % 32 if len(W) % 32 else 0, 256), np.float32)])
+    O = W.shape[0]
+    e = oracle.expand(W, bits, 3, 8, O // 8)
+    layer = H.gpu_expand(H.desc_of(O, 256, bits, 3, 8, O // 8), W)
+    H.assert_expansion_matches(layer, e, oracle)
+
+
 def test_expand_weights_strided_and_tied_groups(oracle):
     rng = np.random.default_rng(5)
     O, I, g = 64, 72, 8
