@@ -230,7 +230,8 @@ pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_ge
 
 /* Which GEMM kernel the two forward calls use (process-wide, for tests and measurements):
  * 0 = automatic, 1 = CUDA-core reference kernel, 2 = tcgen05 tensor-core kernel,
- * 3 = small-token weight-streaming kernel.  A forced kernel that cannot run the request
+ * 3 = small-token weight-streaming kernel, 4 = two-SM form of the tcgen05 kernel (clusters of
+ * two CTAs).  A forced kernel that cannot run the request
  * makes the forward call return PIPE_ERR_UNSUPPORTED. */
 pipe_status pipe_select_kernel(int32_t which);
 

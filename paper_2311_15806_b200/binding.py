@@ -23,7 +23,7 @@ STATUS_NAMES = ["PIPE_OK", "PIPE_ERR_INVALID_ARG", "PIPE_ERR_SHAPE", "PIPE_ERR_A
 (PIPE_OK, PIPE_ERR_INVALID_ARG, PIPE_ERR_SHAPE, PIPE_ERR_ALIGNMENT, PIPE_ERR_UNSUPPORTED, PIPE_ERR_WORKSPACE,
  PIPE_ERR_NONFINITE, PIPE_ERR_ACC_OVERFLOW, PIPE_ERR_TIMEOUT, PIPE_ERR_CUDA) = range(10)
 
-KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM, KERNEL_TCGEN05_PAIR = 0, 1, 2, 3, 4
 
 STATIC_SCRATCH_BYTES = 4 << 20
 

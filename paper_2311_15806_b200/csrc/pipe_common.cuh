@@ -103,6 +103,7 @@ bool make_tensor_map_2d_u8(CUtensorMap* map, const void* base, uint64_t inner_by
 // GEMM back ends (each returns PIPE_ERR_UNSUPPORTED when it cannot take the request).
 pipe_status forward_reference(const ForwardArgs& a, cudaStream_t stream);
 pipe_status forward_tcgen05(const ForwardArgs& a, cudaStream_t stream);
+pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream);   // two-SM form (clusters of two CTAs)
 pipe_status forward_stream(const ForwardArgs& a, cudaStream_t stream);
 
 }  // namespace pipe

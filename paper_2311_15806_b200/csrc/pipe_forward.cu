@@ -49,6 +49,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   if (choice == 1) return forward_reference(a, stream);
   if (choice == 2) return forward_tcgen05(a, stream);
   if (choice == 3) return forward_stream(a, stream);
+  if (choice == 4) return forward_tcgen05_pair(a, stream);
   pipe_status st = PIPE_ERR_UNSUPPORTED;
   if (T <= 16) st = forward_stream(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05(a, stream);
@@ -132,5 +133,6 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   a.conv_on = 1;
   a.cN = geom->batch; a.cH = geom->height; a.cW = geom->width; a.cC = geom->channels;
   a.ckh = geom->kernel_h; a.ckw = geom->kernel_w; a.cph = geom->pad_h; a.cpw = geom->pad_w;
+  if (kernel_choice() == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
   return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
 }

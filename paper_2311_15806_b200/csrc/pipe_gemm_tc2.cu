@@ -1,0 +1,1040 @@
+// Two-SM form of the tcgen05 kernel of the expanded layer (Appendix B, Eq. 9; Sec. 3.2 for the branches).
+//
+// CTAs run as clusters of two (one SM pair).  A pair walks tiles (branch, block of BN output channels,
+// 256 tokens): each CTA stages the 128 token rows that will land in ITS tensor memory and unpacks HALF
+// of the stacked weight rows of the tile (the rows of all orders of the branch in the channel block,
+// see the one-SM kernel), and one thread of the pair's first CTA issues tcgen05.mma.cta_group::2
+// (M = 256 over the two SMs, N = stacked rows, K = 32), which reads both halves of B.  Compared with
+// the one-SM kernel this halves the unpack work and the B-tile traffic per multiply-accumulate and
+// leaves room for two accumulator buffers of up to 256 columns per SM, so the epilogue of a tile
+// always overlaps the MMAs of the next.  Roles per CTA:
+//   warp 0      activation producer (TMA, several lanes in turn); in the second CTA two more lanes
+//               forward "both operands of the stage are in place" and "accumulators drained" to the
+//               first CTA's barriers (one signal across the pair per event, not one per warp)
+//   warps 2-9   unpack half of the B tile
+//   warp 1      first CTA: MMA issuer (one lane); both: owner of the tensor-memory allocation.
+//               tcgen05.commit with a two-CTA multicast returns a stage to the producers of both
+//               CTAs and hands the accumulators to the epilogue warps of both
+//   warps 10-17 epilogue of the CTA's own 128 token rows (as in the one-SM kernel)
+// Every mbarrier wait is bounded; the pair leaves through a cluster barrier so that neither CTA's
+// shared memory or barriers disappear while its peer may still signal them.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "pipe_common.cuh"
+
+namespace pipe {
+
+namespace tc2 {
+
+constexpr int kTileM = 128;          // tokens per tile
+constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
+constexpr int kMaxN = 256;           // stacked weight rows per tile
+constexpr int kMaxClusterOrders = 8;
+constexpr int kUnpackWarps = 8;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
+constexpr int kUnpackThreads = 32 * kUnpackWarps;
+constexpr int kABytes = kTileM * kKStep;       // 16 KiB per token tile
+constexpr int kBtBytes = (kMaxN / 2) * kKStep;   // 16 KiB: this CTA's half of the stacked rows
+constexpr int kStageBytes = kABytes + kBtBytes;
+constexpr int kTmemCols = 512;
+constexpr int kAccCols = 256;
+constexpr int kMaxRing = 6;
+constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
+constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s per wait at the maximum SM clock
+
+// Position in a ring of `depth` slots: slot index and phase parity, advanced without divisions.
+struct RingPos {
+  uint32_t slot, phase;
+  __device__ __forceinline__ void advance(uint32_t by, uint32_t depth) {  // by <= depth
+    slot += by;
+    if (slot >= depth) {
+      slot -= depth;
+      phase ^= 1u;
+    }
+  }
+};
+
+struct Params {
+  CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
+  ForwardArgs f;
+  int BN, ncb, ntt, num_tiles, kblocks;   // ntt: pairs of token tiles
+  int ntok_tiles;         // token tiles (128 tokens) in total
+  int nkmax;              // most orders any branch has
+  int depth;              // stages in the ring
+  int pk;                 // packed bytes of one row of one reduction block (128*b/8)
+  int shift;              // 8 - b
+  int conv_pw, conv_pp, conv_np, conv_chunks;   // patches per image row / per image / in total; 128-channel chunks per tap
+  const uint8_t* kbase;   // lowest address of the streaming-layout sections (16-byte aligned)
+  uint32_t koff[PIPE_MAX_ORDERS];  // (kcodes of order k - kbase) / 16
+};
+
+struct TileMeta {
+  int m, cb, tt;                       // branch, channel block, token-tile group
+  int nk;                              // orders in this branch
+  int k0;                              // first order
+  int start[kMaxClusterOrders];        // first compacted row of the channel block in order k
+  int n[kMaxClusterOrders];            // rows of order k in the block
+  int rowbase[kMaxClusterOrders + 1];  // row offset of order k in the stacked B tile / accumulator
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// For barriers that the peer CTA signals: the wait acquires at cluster scope.
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in the CTA of the given cluster rank.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// Arrival on a barrier of the peer CTA.  The default semantics (release at CTA scope) are enough: what
+// the peer's MMA issuer learns from the signal is that this CTA's operands are in place, and those were
+// made visible to this SM's own tensor core by the writers' proxy fences / by the copy engine; a release
+// at cluster scope costs the signalling thread several hundred cycles more.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+// The bound is counted in SM cycles; the abort flag and the clock are looked at only every few
+// polls so that a barrier that completes soon is seen with little delay.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      raise_status(status, PIPE_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+// The same for a barrier that the peer CTA signals.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      raise_status(status, PIPE_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+// After the last issue: wait (bounded) until the copies of the last `depth` ring slots have landed,
+// so that no copy is still writing into this CTA's shared memory when it exits.
+__device__ __forceinline__ void drain_ring(uint32_t full0, uint32_t issued, int depth) {
+  for (uint32_t j = (issued > static_cast<uint32_t>(depth) ? issued - depth : 0); j < issued; ++j) {
+    const int s = j % depth;
+    const uint32_t ph = (j / depth) & 1;
+    const long long t0 = clock64();
+    while (!mbar_try(full0 + 8u * s, ph) && clock64() - t0 < kWaitLimitCycles) {
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+// Four-dimensional tile of an NHWC tensor (coordinates innermost first: channel, x, y, image);
+// coordinates outside the tensor read zeros, which is the convolution's padding.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
+// Implicit convolution: a token tile is two 8 x 8 pixel patches (64 rows each); patch p lies in
+// image p / pp at patch coordinates ((p % pp) / pw, (p % pp) % pw).
+__device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n, int& h0, int& w0);
+
+// Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes, stored as
+// 8-row atoms of 1024 bytes with the 128-byte swizzle (the layout TMA writes with SWIZZLE_128B).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);  // start address
+  d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset: next 8-row atom
+  d |= static_cast<uint64_t>(1) << 46;                 // descriptor version of this architecture
+  d |= static_cast<uint64_t>(2) << 61;                 // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D = int32, A and B = signed int8, both K-major, M = 256 (two SMs), N = n.
+__device__ __forceinline__ uint32_t idesc_i8(int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>((2 * kTileM) >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate ? 1u : 0u)
+      : "memory");
+}
+
+// Arrives, once the MMAs issued so far have completed in both SMs, on the barrier at this
+// shared-memory offset in BOTH CTAs of the pair.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(static_cast<uint16_t>(3))
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+
+__device__ __forceinline__ void decode_tile(const Params& p, int tile, TileMeta& t) {
+  t.tt = tile % p.ntt;
+  const int rest = tile / p.ntt;
+  t.cb = rest % p.ncb;
+  t.m = rest / p.ncb;
+  const BranchArgs& br = p.f.branch[t.m];
+  t.k0 = br.k_begin;
+  t.nk = br.k_end - br.k_begin;
+  const int c0 = t.cb * p.BN;
+  const int c1 = min(c0 + p.BN, p.f.O);
+  const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
+  int rb = 0;
+#pragma unroll
+  for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
+    t.rowbase[ko] = rb;
+    if (ko < t.nk) {
+      const int32_t* cum = p.f.order[t.k0 + ko].cum;
+      const int lo = __ldg(cum + j0), hi = __ldg(cum + j1);
+      t.start[ko] = lo * p.f.g;
+      t.n[ko] = (hi - lo) * p.f.g;
+      rb += t.n[ko];
+    } else {
+      t.start[ko] = 0;
+      t.n[ko] = 0;
+    }
+  }
+  t.rowbase[kMaxClusterOrders] = rb;
+}
+
+__device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n, int& h0, int& w0) {
+  n = patch / p.conv_pp;
+  const int rem = patch - n * p.conv_pp;
+  h0 = (rem / p.conv_pw) * 8;
+  w0 = (rem % p.conv_pw) * 8;
+}
+
+struct Rings {
+  uint32_t a_full0, bt_ready0, done0, tfull0, tempty0;  // barrier i of a family is 8*i bytes on
+  uint32_t bt_ready_lead0, tempty_lead0;   // the same barriers in the pair's first CTA (cluster addresses)
+  int rank, pair, npairs;                  // this CTA's rank in the pair; tiles go round the pairs
+  uint32_t stage0;        // shared address of stage 0 (activation tile, then B tile)
+  uint8_t* stage_gen;     // generic address of stage 0
+  volatile int* abort_flag;
+};
+
+// Per-tile placement of one unpack work item (stacked row r, 16-byte chunk c of its packed row):
+// offset of the chunk in the streaming layout at reduction block 0 and its step per block, both
+// in 16-byte units relative to Params::kbase; 0xffffffff marks an item beyond the tile's rows.
+// The CTA of rank q unpacks the stacked rows [q * half, (q + 1) * half), half = half of the row count
+// rounded up to the MMA's granularity of 16; r_local counts from the start of that range.
+__device__ __forceinline__ void place_item(const Params& p, int k0, int nk, const int (&start)[kMaxClusterOrders],
+                                           const int (&rowbase)[kMaxClusterOrders + 1], int rank, int r_local, int c, uint32_t& off,
+                                           uint32_t& step) {
+  const int half = ((rowbase[kMaxClusterOrders] + 15) & ~15) >> 1;
+  const int r = rank * half + r_local;
+  if (r_local >= half || r >= rowbase[kMaxClusterOrders]) {
+    off = 0xffffffffu;
+    step = 0;
+    return;
+  }
+  int rb = 0, st = start[0], ko = 0;
+#pragma unroll
+  for (int q = 1; q < kMaxClusterOrders; ++q)
+    if (q < nk && r >= rowbase[q]) {
+      rb = rowbase[q];
+      st = start[q];
+      ko = q;
+    }
+  const OrderView& ov = p.f.order[k0 + ko];
+  const uint32_t pk16 = static_cast<uint32_t>(p.pk) >> 4;
+  off = p.koff[k0 + ko] + static_cast<uint32_t>(st + r - rb) * pk16 + static_cast<uint32_t>(c);
+  step = static_cast<uint32_t>(ov.rows) * pk16;
+}
+
+// Unpack role.  Work items are (stacked row, 16-byte chunk); a thread owns the same item indices
+// in every tile.  A load cursor runs two reduction steps ahead of the step being written (also
+// across tile boundaries): the packed chunks travel global memory (L2-resident, fully coalesced)
+// -> registers -> swizzled B tile, and a step never waits for the latency of its own loads.
+template <int BITS>
+__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
+  constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
+  constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
+  constexpr int ITEMS = (kMaxN / 2) * CPR / kUnpackThreads;
+  constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
+  constexpr int AHEAD = 2;
+  const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
+  const uint32_t depth = p.depth;
+  const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (threads / CPR), chunk c_item
+  const int sw = r0 & 7;                                   // the row step between items is a multiple of 8
+  const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
+  if (my_tiles <= 0) return;
+  const uint32_t total_steps = static_cast<uint32_t>(my_tiles) * p.kblocks;
+
+  // ---- load cursor
+  uint32_t off[ITEMS], stp[ITEMS];
+  int cur_tile = g.pair, cur_kb = 0;
+  uint32_t issued = 0;
+  TileMeta tn;   // metadata of the tile after the cursor's tile, fetched when the cursor enters a tile
+  {
+    TileMeta t;
+    decode_tile(p, cur_tile, t);
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      const int idx = ut + i * kUnpackThreads;
+      place_item(p, t.k0, t.nk, t.start, t.rowbase, g.rank, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
+    }
+    const int nt = cur_tile + g.npairs;
+    decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
+  }
+  auto fetch = [&](uint4 (&w)[ITEMS], uint32_t& mask) {
+    mask = 0;
+    if (issued >= total_steps) return;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+      if (off[i] != 0xffffffffu) {
+        w[i] = __ldg(kb16 + off[i]);
+        mask |= 1u << i;
+      }
+    ++issued;
+    if (++cur_kb < p.kblocks) {
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i)
+        if (off[i] != 0xffffffffu) off[i] += stp[i];
+    } else if (issued < total_steps) {
+      cur_kb = 0;
+      cur_tile += g.npairs;
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) {
+        const int idx = ut + i * kUnpackThreads;
+        place_item(p, tn.k0, tn.nk, tn.start, tn.rowbase, g.rank, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
+      }
+      const int nt = cur_tile + g.npairs;
+      decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
+    }
+  };
+
+  uint4 q1[ITEMS], q2[ITEMS];
+  uint32_t m1 = 0, m2 = 0;
+  fetch(q1, m1);
+  if (AHEAD == 2) fetch(q2, m2);
+
+  RingPos rp{0, 0};
+  for (uint32_t it = 0; it < total_steps; ++it, rp.advance(1, depth)) {
+    uint4 w[ITEMS];
+    const uint32_t mask = m1;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) w[i] = q1[i];
+    if (AHEAD == 2) {
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) q1[i] = q2[i];
+      m1 = m2;
+      fetch(q2, m2);
+    } else {
+      fetch(q1, m1);
+    }
+    if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
+    uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      if (!((mask >> i) & 1u)) continue;
+      const int r = r0 + i * (kUnpackThreads >> CPR_LOG);
+      uint8_t* row = bt + (r >> 3) * 1024 + (r & 7) * 128;
+      const int c0 = c_item * OUT_PER_CHUNK;
+      if (BITS == 8) {
+        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
+      } else if (BITS == 4) {
+        const uint32_t m4 = 0xF0F0F0F0u;
+        const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
+        const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
+        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = v0;
+        *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ sw) << 4)) = v1;
+      } else {
+        const uint32_t m2c = 0xC0C0C0C0u;
+        const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const uint4 v = make_uint4((ww[h] << 6) & m2c, (ww[h] << 4) & m2c, (ww[h] << 2) & m2c, ww[h] & m2c);
+          *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
+        }
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
+    __syncwarp();
+    if ((ut & 31) == 0) mbar_arrive(g.bt_ready0 + 8u * rp.slot);   // one arrival per warp, on this CTA's barrier
+  }
+}
+
+struct EpiCtx {
+  uint32_t tmem_base, tfull0, tempty0;
+  volatile int* abort_flag;
+  int warp, lane;
+  int rank, pair, npairs;
+  uint32_t tempty_lead0;   // the accumulator-released barriers of the pair's first CTA (cluster address)
+  int part, nparts;  // share of the 16-channel groups this warp drains (two warps per lane quarter)
+  int16_t* colmap;
+  float* cscale;
+  float* stg;        // 32 rows x 16 floats, swizzled
+};
+
+// Epilogue role (8 warps, one TMEM lane quarter each; a lane owns one token row of a token tile).
+// The CTA drains the 128 token rows held by its own tensor memory; the channel groups are split
+// between the two warps of a lane quarter.
+// NKMAX bounds the orders of a branch (2, 4 or 8); the channel block is BN = 8 * nch_max channels.
+// Before the accumulators are ready the warp prepares, from the prefix counts, where each
+// (order, 8-channel chunk) sits in the accumulator and the products s_k * lambda_x of all stacked
+// rows, so that the drain loop has no dependent global loads.
+// A lane computes 16 channels of its own token row at a time; the 32 x 16 block is then turned
+// through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
+// (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
+// which is what bounds the drain otherwise).
+template <int NKMAX, bool PARTIALS>
+__device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
+  constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
+  const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
+  const int lane = x.lane;
+  uint32_t tcount = 0;
+  const bool y_vec = (p.f.ldy % 4 == 0);
+  const int wsw = (lane >> 1) & 3;           // swizzle of this lane's row in the staging block
+  // store phase: this lane writes channel quad sj of rows sr0, sr0 + 8, sr0 + 16, sr0 + 24
+  const int sr0 = lane >> 2, spp = lane & 3;
+  const int sj = spp ^ ((sr0 >> 1) & 3);     // the same for all four rows (they differ by multiples of 8)
+  const uint32_t stg_w = smem_u32(x.stg) + static_cast<uint32_t>(lane * 64);
+  const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
+  const uint32_t colmap_s = smem_u32(x.colmap), cscale_s = smem_u32(x.cscale);
+  for (int tile = x.pair; tile < p.num_tiles; tile += x.npairs, ++tcount) {
+    TileMeta t;
+    decode_tile(p, tile, t);
+    const BranchArgs& br = p.f.branch[t.m];
+    const int buf = tcount & 1;
+    const uint32_t aph = (tcount >> 1) & 1;
+    const float sx = __ldg(br.sx);
+    const int c0 = t.cb * p.BN;
+    const int c1 = min(c0 + p.BN, p.f.O);
+    const int nch = (c1 - c0) >> 3;
+    const int n_total = t.rowbase[kMaxClusterOrders];
+    __syncwarp();
+    {
+      // accumulator column of (8-channel chunk, order), or -1: entry [chunk][order]
+      for (int e = lane; e < NKMAX * 16; e += 32) {
+        const int cc = e / NKMAX, ko = e % NKMAX;
+        int col = -1;
+        if (ko < t.nk && cc < nch) {
+          int rb = 0, st = 0;
+          const int32_t* cum = nullptr;
+#pragma unroll
+          for (int u = 0; u < NKMAX; ++u)
+            if (u == ko) {
+              rb = t.rowbase[u];
+              st = t.start[u];
+              cum = p.f.order[t.k0 + u].cum;
+            }
+          const int c = c0 + 8 * cc;
+          const int j = c / p.f.g;
+          const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
+          if (hi > lo) col = rb + lo * p.f.g + c % p.f.g - st;
+        }
+        x.colmap[e] = static_cast<int16_t>(col);
+      }
+      for (int r = lane; r < n_total; r += 32) {
+        int rb = 0, st = t.start[0];
+        const float* sc = p.f.order[t.k0].scales;
+#pragma unroll
+        for (int u = 1; u < NKMAX; ++u)
+          if (u < t.nk && r >= t.rowbase[u]) {
+            rb = t.rowbase[u];
+            st = t.start[u];
+            sc = p.f.order[t.k0 + u].scales;
+          }
+        x.cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
+      }
+    }
+    // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
+    // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
+    const int ttile = 2 * t.tt + x.rank;
+    bool tile_ok = ttile < p.ntok_tiles;
+    int64_t tok_base = static_cast<int64_t>(ttile) * kTileM + q * 32;
+    if (p.f.conv_on) {
+      const int patch = 2 * ttile + (q >> 1);
+      int n, h0, w0;
+      patch_origin(p, patch, n, h0, w0);
+      tok_base = (static_cast<int64_t>(n) * p.f.cH + h0 + (q & 1) * 4) * p.f.cW + w0;
+      tile_ok = patch < p.conv_np;
+    }
+    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * p.f.cW + (r & 7) : tok_base + r; };
+    const int64_t tok_own = token_of(lane);
+    const bool own_ok = tile_ok && (p.f.conv_on || tok_own < p.f.T);
+    float* srow[4];        // the four rows this lane stores, at channel c0 + 4 * sj
+    uint32_t srow_ok = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t tok = token_of(sr0 + 8 * i);
+      srow[i] = br.y + tok * p.f.ldy + c0 + 4 * sj;
+      if (tile_ok && (p.f.conv_on || tok < p.f.T)) srow_ok |= 1u << i;
+    }
+    const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
+    const bool add_bias = br.add_bias && p.f.bias;
+    const float* bias_q = add_bias ? p.f.bias + c0 + 4 * sj : nullptr;
+    const int ngrp = (nch + 1) >> 1;
+    __syncwarp();
+    if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
+    for (int grp = x.part; grp < ngrp && tile_ok; grp += x.nparts) {
+      // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
+      const bool quad_ok = 2 * grp + (sj >> 1) < nch;
+      float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (add_bias && quad_ok) {
+        const float* bp = bias_q + 16 * grp;
+        bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
+      }
+      // ---- this lane's row: 16 channels into the staging block
+#pragma unroll
+      for (int sub = 0; sub < 2; sub += CH) {
+        int acc[CH][NKMAX][8];
+        int cols[CH][NKMAX];
+        {
+          // CH * NKMAX int16 entries, contiguous
+          constexpr int W = CH * NKMAX / 2;   // 32-bit words: 2, 2 or 4
+          uint32_t cw[W];
+          const uint32_t addr = colmap_s + static_cast<uint32_t>((2 * grp + sub) * NKMAX * 2);
+          if constexpr (W == 2) {
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(cw[0]), "=r"(cw[1]) : "r"(addr));
+          } else {
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(cw[0]), "=r"(cw[1]), "=r"(cw[2]), "=r"(cw[3]) : "r"(addr));
+          }
+#pragma unroll
+          for (int u = 0; u < CH; ++u)
+#pragma unroll
+            for (int ko = 0; ko < NKMAX; ++ko) {
+              const int idx = u * NKMAX + ko;
+              cols[u][ko] = static_cast<int16_t>((cw[idx >> 1] >> (16 * (idx & 1))) & 0xffffu);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < CH; ++u)
+#pragma unroll
+          for (int ko = 0; ko < NKMAX; ++ko)
+            if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int u = 0; u < CH; ++u) {
+          const int chunk = 2 * grp + sub + u;
+          if (chunk >= nch) continue;
+          float y[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) y[e] = 0.f;
+#pragma unroll
+          for (int ko = 0; ko < NKMAX; ++ko) {
+            if (cols[u][ko] < 0) continue;
+            float cs[8];
+            const uint32_t ca = cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[0]), "=f"(cs[1]), "=f"(cs[2]), "=f"(cs[3]) : "r"(ca));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[4]), "=f"(cs[5]), "=f"(cs[6]), "=f"(cs[7]) : "r"(ca + 16));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
+              acc[u][ko][e] = a;
+              y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+            }
+            if (PARTIALS && own_ok) {
+              const int crow = cols[u][ko] - t.rowbase[ko] + t.start[ko];   // compacted row of the chunk's first channel
+              int32_t* prow = p.f.partials + tok_own * p.f.total_rows + p.f.order[t.k0 + ko].row_off + crow;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
+            }
+          }
+          const int j0 = 2 * (sub + u);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>((j0 ^ wsw) << 4)), "f"(y[0]),
+                       "f"(y[1]), "f"(y[2]), "f"(y[3])
+                       : "memory");
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>(((j0 + 1) ^ wsw) << 4)), "f"(y[4]),
+                       "f"(y[5]), "f"(y[6]), "f"(y[7])
+                       : "memory");
+        }
+      }
+      __syncwarp();
+      // ---- 8 rows x 64 bytes per store instruction; the bias joins here, after the whole chain
+      if (quad_ok) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (!((srow_ok >> i) & 1u)) continue;
+          float4 v;
+          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(stg_r + static_cast<uint32_t>(i * 8 * 64)));
+          if (add_bias) v = make_float4(__fadd_rn(v.x, bq.x), __fadd_rn(v.y, bq.y), __fadd_rn(v.z, bq.z), __fadd_rn(v.w, bq.w));
+          float* dst = srow[i] + 16 * grp;
+          if (vec_ok) {
+            if (br.accumulate) {
+              const float4 o = *reinterpret_cast<const float4*>(dst);
+              v = make_float4(__fadd_rn(o.x, v.x), __fadd_rn(o.y, v.y), __fadd_rn(o.z, v.z), __fadd_rn(o.w, v.w));
+            }
+            *reinterpret_cast<float4*>(dst) = v;
+          } else {
+            if (br.accumulate) v = make_float4(__fadd_rn(dst[0], v.x), __fadd_rn(dst[1], v.y), __fadd_rn(dst[2], v.z), __fadd_rn(dst[3], v.w));
+            dst[0] = v.x, dst[1] = v.y, dst[2] = v.z, dst[3] = v.w;
+          }
+        }
+      }
+      __syncwarp();
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) mbar_arrive(x.tempty0 + 8u * buf);   // one arrival per warp, on this CTA's barrier
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[6] bt_ready[6] done[6] tmem_full[2] tmem_empty[2]
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ __align__(16) float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
+  __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = smem_u32(bars);
+  Rings g;
+  g.a_full0 = bar0;
+  g.bt_ready0 = bar0 + 8u * kMaxRing;
+  g.done0 = bar0 + 8u * 2 * kMaxRing;
+  g.tfull0 = bar0 + 8u * 3 * kMaxRing;
+  g.tempty0 = g.tfull0 + 8u * 2;
+  g.rank = static_cast<int>(cluster_rank());
+  g.pair = static_cast<int>(blockIdx.x >> 1);
+  g.npairs = static_cast<int>(gridDim.x >> 1);
+  g.bt_ready_lead0 = map_to_cta(g.bt_ready0, 0);
+  g.tempty_lead0 = map_to_cta(g.tempty0, 0);
+  g.stage0 = smem_base;
+  g.stage_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  g.abort_flag = &abort_flag_s;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < kMaxRing; ++s) {
+      mbar_init(g.a_full0 + 8u * s, 1);
+      // own unpack warps; in the first CTA also the peer's "both of my operands are in place"
+      mbar_init(g.bt_ready0 + 8u * s, kUnpackWarps + (g.rank == 0 ? 1 : 0));
+      mbar_init(g.done0 + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(g.tfull0 + 8u * b, 1);
+      // own epilogue warps; in the first CTA also the peer's "my accumulators are drained"
+      mbar_init(g.tempty0 + 8u * b, kEpiWarps + (g.rank == 0 ? 1 : 0));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();   // both CTAs' barriers are initialised before either signals the other
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t depth = p.depth;
+  const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
+  const uint32_t total_steps = static_cast<uint32_t>(my_tiles > 0 ? my_tiles : 0) * p.kblocks;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ activation producer
+    // Lane j < P owns the steps j, j + P, ... (P <= ring depth, see the one-SM kernel for why).  In
+    // the second CTA lane P forwards every "tile landed" to the first CTA's stage barrier, where
+    // the MMA issuer waits for both CTAs' operands.
+    const uint32_t P = min(static_cast<uint32_t>(kALanes), depth);
+    if (static_cast<uint32_t>(lane) < P) {
+      RingPos rp{static_cast<uint32_t>(lane), 0};
+      int tile = g.pair, kb = lane;
+      for (uint32_t it = lane; it < total_steps; it += P, rp.advance(P, depth), kb += P) {
+        while (kb >= p.kblocks) {
+          kb -= p.kblocks;
+          tile += g.npairs;
+        }
+        const int ttile = 2 * (tile % p.ntt) + g.rank;   // this CTA's 128 token rows of the pair's tile
+        const int m = tile / p.ntt / p.ncb;
+        if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
+        mbar_expect_tx(g.a_full0 + 8u * rp.slot, kABytes);
+        if (!p.f.conv_on) {
+          // rows beyond T read zeros
+          tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, ttile * kTileM, g.a_full0 + 8u * rp.slot);
+        } else {
+          // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
+          const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
+          const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            int n, h0, w0;
+            patch_origin(p, 2 * ttile + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
+            tma_load_4d(g.stage0 + rp.slot * kStageBytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, w0 + dw, h0 + dh,
+                        n, g.a_full0 + 8u * rp.slot);
+          }
+        }
+      }
+    } else if (static_cast<uint32_t>(lane) < P + depth && g.rank == 1) {
+      // stage relays: one signal per step across the pair instead of one per warp.  A signal to the
+      // peer keeps its thread busy for a couple of thousand cycles, so every ring slot has its own
+      // relay lane (slot s <-> lane P + s; the steps of one slot stay in order).
+      const uint32_t slot = static_cast<uint32_t>(lane) - P;
+      uint32_t phase = 0;
+      for (uint32_t it = slot; it < total_steps; it += depth, phase ^= 1u) {
+        if (!mbar_wait(g.a_full0 + 8u * slot, phase, g.abort_flag, p.f.status)) break;
+        if (!mbar_wait(g.bt_ready0 + 8u * slot, phase, g.abort_flag, p.f.status)) break;
+        mbar_arrive_cluster(g.bt_ready_lead0 + 8u * slot);
+      }
+    } else if (static_cast<uint32_t>(lane) == P + depth && g.rank == 1) {
+      // accumulator relay: this CTA's epilogue warps have drained a buffer
+      for (int n = 0; n < my_tiles; ++n) {
+        if (!mbar_wait(g.tempty0 + 8u * (n & 1), (n >> 1) & 1, g.abort_flag, p.f.status)) break;
+        mbar_arrive_cluster(g.tempty_lead0 + 8u * (n & 1));
+      }
+    }
+    __syncwarp();
+    if (lane == 0) drain_ring(g.a_full0, total_steps, p.depth);
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (first CTA of the pair)
+    if (lane == 0 && g.rank == 0) {
+      RingPos rp{0, 0};
+      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kABytes);
+      uint32_t tcount = 0;
+      bool ok = true;
+      // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
+      auto stacked_rows = [&](int tile) {
+        const int cb = (tile / p.ntt) % p.ncb, m = tile / p.ntt / p.ncb;
+        const BranchArgs& br = p.f.branch[m];
+        const int c0 = cb * p.BN, c1 = min(c0 + p.BN, p.f.O);
+        const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
+        int n = 0;
+        for (int k = br.k_begin; k < br.k_end; ++k) {
+          const int32_t* cum = p.f.order[k].cum;
+          n += (__ldg(cum + j1) - __ldg(cum + j0)) * p.f.g;
+        }
+        return n;
+      };
+      int n_next = g.pair < p.num_tiles ? stacked_rows(g.pair) : 0;
+      for (int tile = g.pair; ok && tile < p.num_tiles; tile += g.npairs, ++tcount) {
+        const int n_total = n_next;
+        if (tile + g.npairs < p.num_tiles) n_next = stacked_rows(tile + g.npairs);
+        const int buf = tcount & 1;
+        const uint32_t aph = (tcount >> 1) & 1;
+        if (!mbar_wait(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
+        int n = (n_total + 15) & ~15;
+        if (n < 16) n = 16;
+        const uint32_t idesc = idesc_i8(n);
+        const uint32_t d_tmem = tmem_base + buf * kAccCols;
+        for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
+          // both barriers are polled before either result is tested so that the two polls overlap
+          const bool r1 = mbar_try(g.a_full0 + 8u * rp.slot, rp.phase);
+          const bool r2 = mbar_try(g.bt_ready0 + 8u * rp.slot, rp.phase);
+          if (!r1 && !mbar_wait(g.a_full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
+          if (!r2 && !mbar_wait(g.bt_ready0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
+          const uint64_t adesc = adesc0 + so, bdesc = bdesc0 + so;
+#pragma unroll
+          for (int k = 0; k < kKStep / 32; ++k)
+            mma_i8(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
+          mma_commit_pair(g.done0 + 8u * rp.slot);   // frees the stage for the producers of both CTAs
+        }
+        if (ok) mma_commit_pair(g.tfull0 + 8u * buf);
+      }
+    }
+  } else if (warp < 2 + kUnpackWarps) {
+    // ------------------------------------------------------------------ unpack warps
+    const int ut = threadIdx.x - 64;
+    if (p.f.bits == 8) unpack_role<8>(p, g, ut);
+    else if (p.f.bits == 4) unpack_role<4>(p, g, ut);
+    else unpack_role<2>(p, g, ut);
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    EpiCtx e;
+    e.tmem_base = tmem_base;
+    e.tfull0 = g.tfull0;
+    e.tempty0 = g.tempty0;
+    e.tempty_lead0 = g.tempty_lead0;
+    e.rank = g.rank;
+    e.pair = g.pair;
+    e.npairs = g.npairs;
+    e.abort_flag = g.abort_flag;
+    e.warp = warp;
+    e.lane = lane;
+    const int ew = warp - 2 - kUnpackWarps;
+    e.part = ew >> 2;
+    e.nparts = 2;
+    e.colmap = epi_colmap[ew];
+    e.cscale = epi_cscale[ew];
+    e.stg = epi_stage[ew];
+    if (p.f.partials) {   // verification output: every integer accumulator is also written out
+      if (p.nkmax <= 2) epilogue_role<2, true>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true>(p, e);
+      else epilogue_role<8, true>(p, e);
+    } else {
+      if (p.nkmax <= 2) epilogue_role<2, false>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false>(p, e);
+      else epilogue_role<8, false>(p, e);
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  // Neither CTA may free its tensor memory or leave while the peer can still signal its barriers or
+  // the pair's MMAs can still read its shared memory: both meet at a cluster barrier first.
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn encode_fn() {
+  static std::once_flag once;
+  static EncodeFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(p);
+  });
+  return fn;
+}
+
+static bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+                        uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {inner_bytes, rows};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// NHWC int8 tensor as a 4-D map; one box = 128 channels x 8 x 8 pixels of one image (64 rows of 128 bytes).
+static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int W, int C) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                              static_cast<cuuint64_t>(N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W) * C,
+                                 static_cast<cuuint64_t>(H) * W * C};
+  const cuuint32_t box[4] = {128, 8, 8, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tc2
+
+static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
+  using namespace tc2;
+  static Params p;  // large; filled per call under the lock
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+
+  int max_cluster = 0;
+  for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
+  if (max_cluster > kMaxClusterOrders) return PIPE_ERR_UNSUPPORTED;
+  // Widest channel block whose stacked rows fit the 256 accumulator columns in the worst case:
+  // order 1 contributes BN rows, a sparse order at most min(BN, rows it keeps in the whole layer).
+  int BN = 0;
+  for (int cand = 128; cand >= 32 && BN == 0; cand >>= 1) {
+    int worst = 0;
+    for (int m = 0; m < a.num_branches; ++m) {
+      int w = 0;
+      for (int k = a.branch[m].k_begin; k < a.branch[m].k_end; ++k) w += min(cand, a.order[k].rows);
+      worst = max(worst, w);
+    }
+    if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand;
+  }
+  if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.conv_on && (a.cC % kKStep != 0 || a.cH % 8 != 0 || a.cW % 8 != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
+  for (int m = 0; m < a.num_branches; ++m) {
+    if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
+  }
+  if (a.T > (1ll << 30)) return PIPE_ERR_UNSUPPORTED;
+
+  p.f = a;
+  p.BN = BN;
+  p.nkmax = max_cluster;
+  p.ncb = ceil_div(a.O, BN);
+  p.ntok_tiles = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
+  p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
+  if (a.conv_on) {
+    p.conv_pw = a.cW / 8;
+    p.conv_pp = (a.cH / 8) * p.conv_pw;
+    p.conv_np = p.conv_pp * a.cN;
+    p.conv_chunks = a.cC / kKStep;
+    p.ntok_tiles = ceil_div(p.conv_np, 2);
+  }
+  if (p.ntok_tiles < 2) return PIPE_ERR_UNSUPPORTED;   // a pair needs two token tiles; the one-SM kernel takes these
+  p.ntt = ceil_div(p.ntok_tiles, 2);
+  const int64_t tiles = static_cast<int64_t>(p.ncb) * p.ntt * a.num_branches;
+  if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
+  p.num_tiles = static_cast<int>(tiles);
+  p.kblocks = ceil_div(a.I, kKStep);
+  p.pk = kKStep * a.bits / 8;
+  p.shift = 8 - a.bits;
+  int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
+  for (int m = 0; m < a.num_branches; ++m) {
+    k_lo = min(k_lo, a.branch[m].k_begin);
+    k_hi = max(k_hi, a.branch[m].k_end);
+  }
+  const uint8_t* kbase = a.order[k_lo].kcodes;
+  for (int k = k_lo; k < k_hi; ++k) kbase = a.order[k].kcodes < kbase ? a.order[k].kcodes : kbase;
+  p.kbase = kbase;
+  for (int k = k_lo; k < k_hi; ++k) {
+    const uint64_t d = static_cast<uint64_t>(a.order[k].kcodes - kbase);
+    const uint64_t end = (d + static_cast<uint64_t>(a.order[k].rows) * a.kernel_row_bytes) >> 4;
+    if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
+    p.koff[k] = static_cast<uint32_t>(d >> 4);
+  }
+  int dev = 0, smem_max = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
+  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaFuncAttributes fattr;
+  if (cudaFuncGetAttributes(&fattr, tc2_forward_kernel) != cudaSuccess) return PIPE_ERR_CUDA;
+  p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / kStageBytes;  // static shared, alignment slack
+  if (p.depth > kMaxRing) p.depth = kMaxRing;
+  if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
+  const int dyn_smem = p.depth * kStageBytes + 1024;
+
+  if (a.conv_on) {
+    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC)) return PIPE_ERR_CUDA;
+  } else
+  for (int m = 0; m < a.num_branches; ++m) {
+    if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
+                     static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
+      return PIPE_ERR_CUDA;
+  }
+  static int attr_bytes = 0;
+  if (attr_bytes < dyn_smem) {
+    if (cudaFuncSetAttribute(tc2_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem) != cudaSuccess)
+      return PIPE_ERR_CUDA;
+    attr_bytes = dyn_smem;
+  }
+  // one cluster of two CTAs per SM pair; how many pairs can be resident is asked of the runtime once
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = dyn_smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
+    cfg.gridDim = dim3(sms & ~1, 1, 1);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel, &cfg) != cudaSuccess || n < 1) return PIPE_ERR_UNSUPPORTED;
+    max_pairs = n;
+  }
+  const int pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  if (cudaLaunchKernelEx(&cfg, tc2_forward_kernel, p) != cudaSuccess) return PIPE_ERR_CUDA;
+  count_launch(1);
+  return launch_status();
+}
+
+pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream) {
+  if (a.T == 0) return PIPE_OK;
+  const bool sum_mode = a.num_branches > 1 && a.branch[1].accumulate;
+  if (!sum_mode) return launch_tc2(a, stream);
+  // Summed ensemble: one launch per branch, in order, so that y = ((y_1 + y_2) + ...) is formed
+  // by the same thread in a fixed order.
+  for (int m = 0; m < a.num_branches; ++m) {
+    ForwardArgs one = a;
+    one.num_branches = 1;
+    one.branch[0] = a.branch[m];
+    pipe_status st = launch_tc2(one, stream);
+    if (st != PIPE_OK) return st;
+  }
+  return PIPE_OK;
+}
+
+}  // namespace pipe

@@ -136,7 +136,7 @@ pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
 }
 
 pipe_status pipe_select_kernel(int32_t which) {
-  if (which < 0 || which > 3) return PIPE_ERR_INVALID_ARG;
+  if (which < 0 || which > 4) return PIPE_ERR_INVALID_ARG;
   g_kernel_choice.store(which);
   return PIPE_OK;
 }
