@@ -103,8 +103,8 @@ def workload_spec(name: str):
 
 # ------------------------------------------------------------------------------------------------
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("cfg2", "forward"): 28.380928e6 + 51.302400e6,      # profiles/ncu_tc_forward_kernel_cfg2.txt
-    ("cfg4a_t16", "forward"): 56.969216e6 + 0.482048e6,  # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
+    ("cfg2", "forward"): 28.445440e6 + 50.608640e6,      # profiles/ncu_tc_forward_kernel_cfg2.txt
+    ("cfg4a_t16", "forward"): 56.671744e6 + 0.155136e6,  # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
 }
 
 
