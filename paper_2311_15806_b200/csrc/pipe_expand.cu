@@ -1,9 +1,9 @@
 // pipe_expand_weights: residual expansion of a weight matrix (Sec. 3.1, Eq. 2-3 and the masked
 // form), with the per-channel symmetric quantizer of Eq. 1.
 //
-// Per order: [row absmax, only for order 1] -> [group select, orders >= 2] -> one fused pass
-// over the kept rows that divides, rounds, packs both code layouts, updates the residual with
-// one FMA per element and leaves the next order's row absmax behind.  All kernels are
+// Per order: [group select, orders >= 2] -> one fused pass over the kept rows that (order 1: finds the
+// row maximum,) divides, rounds, packs both code layouts, updates the residual with one FMA per
+// element and leaves the next order's row absmax behind.  All kernels are
 // HBM-bound streaming passes: 128-bit loads, warp-shuffle reductions, one block per row.
 #include <mutex>
 
@@ -41,31 +41,6 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v) {
 // |v| as an ordered unsigned key: for finite floats the order of the keys is the order of the
 // magnitudes, and every Inf/NaN maps to a key >= 0x7f800000.
 __device__ __forceinline__ uint32_t abs_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
-
-// a[o] = max_i |src[o,i]|   (one block per row)
-__global__ void __launch_bounds__(kRowThreads) row_absmax_kernel(const float* __restrict__ src, int64_t ld, int I,
-                                                                 float* __restrict__ a, int* status) {
-  const int o = blockIdx.x;
-  const float* row = src + static_cast<int64_t>(o) * ld;
-  uint32_t m = 0;
-  const bool vec = ((reinterpret_cast<uintptr_t>(row) & 15) == 0);
-  int i0 = 0;
-  if (vec) {
-    const int n4 = I >> 2;
-    const float4* r4 = reinterpret_cast<const float4*>(row);
-    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-      const float4 v = __ldg(r4 + i);
-      m = max(max(m, abs_key(v.x)), max(abs_key(v.y), max(abs_key(v.z), abs_key(v.w))));
-    }
-    i0 = n4 << 2;
-  }
-  for (int i = i0 + threadIdx.x; i < I; i += blockDim.x) m = max(m, abs_key(row[i]));
-  m = block_max_u32(m);
-  if (threadIdx.x == 0) {
-    a[o] = __uint_as_float(m);
-    if (m >= 0x7f800000u) raise_status(status, PIPE_ERR_NONFINITE);
-  }
-}
 
 // score[j] = max over the g rows of group j of a[] ; one thread per group.
 __global__ void group_score_kernel(const float* __restrict__ a, int G, int g, float* __restrict__ score) {
@@ -125,6 +100,51 @@ __global__ void __launch_bounds__(1024) group_compact_kernel(const int32_t* __re
   if (threadIdx.x == blockDim.x - 1) cum[G] = chunk_sum[blockDim.x - 1];
 }
 
+// Group selection of one order in ONE block, for layers of up to kFusedGroups groups: scores, ranks and
+// the compacted list stay in shared memory (three tiny launches less per sparse order).  Same rule and
+// same exact comparisons as the three kernels above.
+constexpr int kFusedGroups = 512;   // one group per thread: the ranking is G comparisons per thread
+__global__ void __launch_bounds__(kFusedGroups) group_select_kernel(const float* __restrict__ a, int G, int g, int n_keep,
+                                                            int32_t* __restrict__ cum, int32_t* __restrict__ kept) {
+  __shared__ float score[kFusedGroups];
+  __shared__ int32_t flag[kFusedGroups];
+  __shared__ int32_t chunk_sum[kFusedGroups];
+  for (int j = threadIdx.x; j < G; j += blockDim.x) {
+    float m = 0.f;
+    for (int u = 0; u < g; ++u) m = fmaxf(m, a[static_cast<int64_t>(j) * g + u]);
+    score[j] = m;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < G; j += blockDim.x) {
+    const float sj = score[j];
+    int rank = 0;
+    for (int t = 0; t < G; ++t) {
+      const float si = score[t];
+      rank += (si > sj) || (si == sj && t < j);
+    }
+    flag[j] = rank < n_keep ? 1 : 0;
+  }
+  __syncthreads();
+  const int per = (G + blockDim.x - 1) / blockDim.x;
+  const int b = threadIdx.x * per, e = min(G, b + per);
+  int32_t sum = 0;
+  for (int j = b; j < e; ++j) sum += flag[j];
+  chunk_sum[threadIdx.x] = sum;
+  __syncthreads();
+  for (int d = 1; d < blockDim.x; d <<= 1) {
+    int32_t v = threadIdx.x >= d ? chunk_sum[threadIdx.x - d] : 0;
+    __syncthreads();
+    chunk_sum[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int32_t run = threadIdx.x == 0 ? 0 : chunk_sum[threadIdx.x - 1];
+  for (int j = b; j < e; ++j) {
+    cum[j] = run;
+    if (flag[j]) kept[run++] = j;
+  }
+  if (threadIdx.x == blockDim.x - 1) cum[G] = chunk_sum[blockDim.x - 1];
+}
+
 // Pack 16 codes (each already in [-qmax, qmax]) into the canonical and the kernel layout.
 // canonical: field e at bit e*b of the stream; kernel: see include/pipe.h.
 template <int BITS>
@@ -172,6 +192,8 @@ struct QuantizeRowsArgs {
   float* dst;            // residual leaving this order ([O, ld_dst]) or nullptr (last order)
   int64_t ld_dst;
   float* a;              // [O] row absmax: read (this order's), overwritten (next order's) if dst
+  int first;             // order 1: the row maximum is not in a[] yet, the block finds it itself
+  int* status;
   const int32_t* kept;   // [rows/g] ascending kept groups
   uint8_t* codes;        // canonical [rows, canon_row_bytes]
   uint8_t* kcodes;       // streaming layout [ceil(I/128), rows, 128*BITS/8]
@@ -189,7 +211,28 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
   const float* src = p.src + static_cast<int64_t>(o) * p.ld_src;
   float* dst = p.dst ? p.dst + static_cast<int64_t>(o) * p.ld_dst : nullptr;
   const float fq = static_cast<float>(p.qmax);
-  const float s = __fdiv_rn(p.a[o], fq);
+  float amax;
+  if (p.first) {
+    // order 1 (Eq. 1 on W itself): one more pass over the row, which the second pass then finds in cache
+    uint32_t mk = 0;
+    if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+      const int n4 = p.I >> 2;
+      const float4* r4 = reinterpret_cast<const float4*>(src);
+      for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+        const float4 v = r4[i];
+        mk = max(max(mk, abs_key(v.x)), max(abs_key(v.y), max(abs_key(v.z), abs_key(v.w))));
+      }
+      for (int i = (n4 << 2) + threadIdx.x; i < p.I; i += blockDim.x) mk = max(mk, abs_key(src[i]));
+    } else {
+      for (int i = threadIdx.x; i < p.I; i += blockDim.x) mk = max(mk, abs_key(src[i]));
+    }
+    mk = block_max_u32(mk);
+    if (threadIdx.x == 0 && mk >= 0x7f800000u) raise_status(p.status, PIPE_ERR_NONFINITE);
+    amax = __uint_as_float(mk);
+  } else {
+    amax = p.a[o];
+  }
+  const float s = __fdiv_rn(amax, fq);
   __syncthreads();  // every thread has read a[o] before thread 0 overwrites it at the end
   if (threadIdx.x == 0) p.scales[n] = s;
   uint8_t* crow = p.codes + static_cast<int64_t>(n) * p.canon_row_bytes;
@@ -303,25 +346,31 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
   uint8_t* blob = static_cast<uint8_t*>(d_blob);
 
   write_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<uint32_t*>(blob), *desc);
-  row_absmax_kernel<<<L.O, kRowThreads, 0, s>>>(d_W, ldw, L.I, a, status);
-  count_launch(2);
+  count_launch(1);
   for (int k = 0; k < L.K; ++k) {
     int32_t* kept = reinterpret_cast<int32_t*>(blob + L.lay.kept_off[k]);
     int32_t* cum = reinterpret_cast<int32_t*>(blob + L.lay.cum_off[k]);
     const bool dense = (k == 0) || (L.n_keep == L.G);
-    if (!dense) {
-      group_score_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(a, L.G, L.g, score);
-      group_rank_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
-      count_launch(2);
+    if (!dense && L.G <= kFusedGroups) {
+      group_select_kernel<<<1, kFusedGroups, 0, s>>>(a, L.G, L.g, L.n_keep, cum, kept);
+      count_launch(1);
+    } else {
+      if (!dense) {
+        group_score_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(a, L.G, L.g, score);
+        group_rank_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
+        count_launch(2);
+      }
+      group_compact_kernel<<<1, 1024, 0, s>>>(dense ? nullptr : keep, L.G, cum, kept);
+      count_launch(1);
     }
-    group_compact_kernel<<<1, 1024, 0, s>>>(dense ? nullptr : keep, L.G, cum, kept);
-    count_launch(1);
     QuantizeRowsArgs q;
     q.src = (k == 0) ? d_W : resid;
     q.ld_src = (k == 0) ? ldw : I4;
     q.dst = (k + 1 < L.K) ? resid : nullptr;
     q.ld_dst = I4;
     q.a = a;
+    q.first = (k == 0) ? 1 : 0;
+    q.status = status;
     q.kept = kept;
     q.codes = blob + L.lay.codes_off[k];
     q.kcodes = blob + L.lay.kcodes_off[k];
