@@ -36,7 +36,7 @@ typedef enum {
   PIPE_ERR_INVALID_ARG = 1,  /* null pointer, negative size, value out of range */
   PIPE_ERR_SHAPE = 2,        /* group size does not divide out_features, K/M inconsistent, ... */
   PIPE_ERR_ALIGNMENT = 3,    /* pointer or pitch not aligned as documented */
-  PIPE_ERR_UNSUPPORTED = 4,  /* valid request this build has no kernel for */
+  PIPE_ERR_UNSUPPORTED = 4,  /* valid request the library has no kernel for */
   PIPE_ERR_WORKSPACE = 5,    /* blob / workspace smaller than pipe_layout says */
   PIPE_ERR_NONFINITE = 6,    /* device saw NaN or Inf in weights or activations */
   PIPE_ERR_ACC_OVERFLOW = 7, /* in_features so large that an int32 partial sum could overflow */
