@@ -403,7 +403,11 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
           // this lane's chunk: CHK codes from reduction offset kc of the stage
           const int kc = ms * 4 * CHK + tig * CHK;
           const int kbs = kc >> 7, within = kc & 127;
-          if (ks * KBPS + kbs >= p.kblocks) continue;   // a stage's later blocks may lie beyond the reduction axis
+          // A stage's later blocks may lie beyond the reduction axis.  With 2-bit codes that differs from lane
+          // to lane, and the MMAs below are warp-wide instructions that every lane must execute: such a lane
+          // contributes zero weights instead of leaving the loop (its activation words are stale but finite
+          // integers, and zero times anything is zero).
+          const bool live = ks * KBPS + kbs < p.kblocks;
           const uint32_t wbyte = static_cast<uint32_t>(gid * p.pk + ((within * BITS) >> 3));
           uint4 xv[XCH][NT];
 #pragma unroll
@@ -419,9 +423,9 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
 #pragma unroll
             for (int q = 0; q < NP; ++q) {
               if (2 * q >= nchunks[s]) continue;
-              const uint4 wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
-              uint4 wb = make_uint4(0, 0, 0, 0);
-              if (2 * q + 1 < nchunks[s]) wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
+              uint4 wa = make_uint4(0, 0, 0, 0), wb = make_uint4(0, 0, 0, 0);
+              if (live) wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
+              if (live && 2 * q + 1 < nchunks[s]) wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
 #pragma unroll
               for (int mm = 0; mm < 2 * XCH; ++mm) {
                 uint32_t a0, a1, b0, b1;

@@ -200,6 +200,12 @@ FORWARD_CASES = [
     (304, 2304, 16, 4, 3, 8, 19, 1),
     (72, 4112, 3, 4, 5, 8, 4, 2),
     (136, 1000, 12, 2, 4, 8, 9, 1),
+    # decode kernel: int8 codes; eight orders in one branch (four order pairs per slab); ternary with an odd
+    # number of reduction blocks; more slabs per CTA than one pass holds
+    (256, 384, 9, 8, 2, 8, 16, 1),
+    (320, 1024, 7, 2, 8, 8, 10, 1),
+    (200, 1152, 16, 2, 3, 8, 11, 1),
+    (24832, 128, 5, 4, 2, 8, 1552, 1),
 ]
 
 
