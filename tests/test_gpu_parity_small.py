@@ -290,8 +290,9 @@ CONV_CASES = [
 ]
 
 
+@pytest.mark.parametrize("kernel", [B.KERNEL_AUTO, B.KERNEL_TCGEN05_PAIR])
 @pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep", CONV_CASES)
-def test_implicit_convolution_matches_oracle(oracle, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep):
+def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep):
     """pipe_expanded_conv2d on the NHWC tensor == the oracle on explicitly lowered im2col rows."""
     rng = np.random.default_rng(N * 1000 + Hh * 10 + Cc)
     I = kh * kw * Cc
@@ -319,7 +320,15 @@ def test_implicit_convolution_matches_oracle(oracle, N, Hh, Ww, Cc, O, kh, kw, b
     T = N * Hh * Ww
     y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
-    B.pipe_expanded_conv2d(layer.desc, geom, layer.blob, xq4.view(N, Hh, Ww, Cc), sx, y, torch.from_numpy(bias).cuda(), part)
+    B.pipe_select_kernel(kernel)
+    try:
+        B.pipe_expanded_conv2d(layer.desc, geom, layer.blob, xq4.view(N, Hh, Ww, Cc), sx, y, torch.from_numpy(bias).cuda(), part)
+    except B.PipeError as ex:
+        if ex.status == B.PIPE_ERR_UNSUPPORTED and kernel != B.KERNEL_AUTO:
+            pytest.skip("the two-SM kernel needs at least two token tiles")
+        raise
+    finally:
+        B.pipe_select_kernel(B.KERNEL_AUTO)
     torch.cuda.synchronize()
     assert B.pipe_poll_status() == B.PIPE_OK
     np.testing.assert_array_equal(part.cpu().numpy(), f.partials)
