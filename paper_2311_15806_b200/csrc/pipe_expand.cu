@@ -245,6 +245,57 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
   const bool dst_vec = dst && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
   const bool canon_vec = (reinterpret_cast<uintptr_t>(crow) & 3) == 0;
   uint32_t m = 0;
+  constexpr int CPW = 32 / BITS;   // codes per packed 32-bit word
+  constexpr int LPW = CPW / 4;     // lanes that share one word when a lane holds 4 consecutive codes
+  const bool lanewise = (I % CPW == 0) && src_vec && (!dst || dst_vec) && canon_vec && (p.canon_row_bytes % 4 == 0);
+  if (lanewise) {
+    // Lane-contiguous form: per trip a warp covers 512 consecutive elements, lane L holding the four quads at
+    // offsets w * 128 + 4 L (w = 0..3), so every load and store instruction of the warp touches one contiguous
+    // run.  A packed word then takes its fields from LPW neighbouring lanes; each lane shifts its four codes
+    // to their places in both layouts and the lanes OR their parts together.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int h = lane & (LPW - 1);
+    const uint32_t fmask = (1u << BITS) - 1u;
+    for (int base = warp * 512; base < I_pad; base += nwarps * 512) {
+      float4 v[4];
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const int e0 = base + w * 128 + lane * 4;
+        v[w] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 < I) v[w] = *reinterpret_cast<const float4*>(src + e0);   // plain load: src may alias dst
+      }
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const int e0 = base + w * 128 + lane * 4;
+        float x[4] = {v[w].x, v[w].y, v[w].z, v[w].w};
+        uint32_t cc = 0, ck = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float c = 0.f;
+          if (s != 0.f) {
+            c = rintf(__fdiv_rn(x[j], s));         // round half to even
+            c = fminf(fmaxf(c, -fq), fq);
+            x[j] = __fmaf_rn(-s, c, x[j]);         // exact new residual, rounded once
+          }
+          m = max(m, abs_key(x[j]));
+          const uint32_t f = static_cast<uint32_t>(static_cast<int>(c)) & fmask;
+          cc |= f << (BITS * (4 * h + j));          // canonical: field e at bit e * b of the stream
+          ck |= f << (8 * j + BITS * h);            // streaming layout: see include/pipe.h
+        }
+        if (dst && e0 < I) *reinterpret_cast<float4*>(dst + e0) = make_float4(x[0], x[1], x[2], x[3]);
+#pragma unroll
+        for (int d = 1; d < LPW; d <<= 1) {
+          cc |= __shfl_xor_sync(0xffffffffu, cc, d);
+          ck |= __shfl_xor_sync(0xffffffffu, ck, d);
+        }
+        if (h == 0 && e0 < I_pad) {
+          uint8_t* kdst = p.kcodes + (static_cast<int64_t>(e0 >> 7) * p.rows + n) * kStepBytes + (e0 & 127) * BITS / 8;
+          *reinterpret_cast<uint32_t*>(kdst) = ck;
+          if (e0 < I) *reinterpret_cast<uint32_t*>(crow + e0 * BITS / 8) = cc;
+        }
+      }
+    }
+  } else
   for (int i0 = threadIdx.x * 16; i0 < I_pad; i0 += blockDim.x * 16) {
     float v[16];
     const bool full = i0 + 16 <= I;
