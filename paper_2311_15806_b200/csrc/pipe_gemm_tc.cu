@@ -8,13 +8,13 @@
 // activation tile is staged once per reduction step.  A ring of stages {activation tile, B tile}
 // in shared memory decouples the roles:
 //   warp 0      activation producer: TMA tensor loads (128B swizzle), several lanes issue in turn
-//   warps 2-9   unpack: read the packed int8/int4/ternary rows of the tile straight from the
+//   warps 2-7   unpack: read the packed int8/int4/ternary rows of the tile straight from the
 //               reduction-block-major streaming layout (coalesced 16-byte loads, prefetched one
 //               step ahead in registers) and write int8 lanes into the swizzled B tile
 //               (shift + mask only; sub-byte codes arrive multiplied by 2^(8-b))
 //   warp 1      MMA issuer (one lane), owns the TMEM allocation (2 x 256 columns, double buffered);
 //               one tcgen05.commit per step releases the stage to both producers
-//   warps 10-13 epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
+//   warps 8-15  epilogue: tcgen05.ld the accumulators of each order, shift back, scale by
 //               s_k * lambda_x and add in ascending order with one FMA per term, store fp32
 // Barrier operations cost their issuing thread on the order of a hundred cycles each, so every
 // role touches as few barriers per step as possible and ring positions are advanced without
@@ -34,7 +34,9 @@ constexpr int kTileM = 128;          // tokens per tile
 constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
-constexpr int kUnpackWarps = 8;
+// 2 + 6 + 8 = 16 warps: four per scheduler, so every thread may hold 128 registers and neither the unpack
+// nor the epilogue role spills; measured faster than 8 unpack warps at 96 registers on every workload.
+constexpr int kUnpackWarps = 6;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
 constexpr int kUnpackThreads = 32 * kUnpackWarps;
@@ -274,7 +276,7 @@ template <int BITS>
 __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
   constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
-  constexpr int ITEMS = kMaxN * CPR / kUnpackThreads;
+  constexpr int ITEMS = (kMaxN * CPR + kUnpackThreads - 1) / kUnpackThreads;   // items past the last row are masked
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
   constexpr int AHEAD = (BITS == 8) ? 1 : 2;   // int8 rows carry 8 chunks per thread: one step ahead only
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
