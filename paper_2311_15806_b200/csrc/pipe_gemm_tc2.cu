@@ -11,11 +11,11 @@
 //   warp 0      activation producer (TMA, several lanes in turn); in the second CTA two more lanes
 //               forward "both operands of the stage are in place" and "accumulators drained" to the
 //               first CTA's barriers (one signal across the pair per event, not one per warp)
-//   warps 2-9   unpack half of the B tile
+//   warps 2-7   unpack half of the B tile
 //   warp 1      first CTA: MMA issuer (one lane); both: owner of the tensor-memory allocation.
 //               tcgen05.commit with a two-CTA multicast returns a stage to the producers of both
 //               CTAs and hands the accumulators to the epilogue warps of both
-//   warps 10-17 epilogue of the CTA's own 128 token rows (as in the one-SM kernel)
+//   warps 8-15  epilogue of the CTA's own 128 token rows (as in the one-SM kernel)
 // Every mbarrier wait is bounded; the pair leaves through a cluster barrier so that neither CTA's
 // shared memory or barriers disappear while its peer may still signal them.
 #include <cuda.h>
@@ -32,7 +32,7 @@ constexpr int kTileM = 128;          // tokens per tile
 constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
-constexpr int kUnpackWarps = 8;
+constexpr int kUnpackWarps = 6;   // 16 warps per CTA: 128 registers per thread (see the one-SM kernel)
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
 constexpr int kUnpackThreads = 32 * kUnpackWarps;
@@ -328,7 +328,7 @@ template <int BITS>
 __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
   constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
-  constexpr int ITEMS = (kMaxN / 2) * CPR / kUnpackThreads;
+  constexpr int ITEMS = ((kMaxN / 2) * CPR + kUnpackThreads - 1) / kUnpackThreads;   // items past the last row are masked
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
   constexpr int AHEAD = 2;
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
