@@ -261,7 +261,6 @@ def run_ours(args):
         ev[i][3].record()
     sync_all()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop()
     launches = B.pipe_launch_count() - launches0
     t_expand = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
     t_quant = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
@@ -297,8 +296,11 @@ def run_ours(args):
     except Exception:
         graph = None
         torch.cuda.synchronize()
+    # The clock sampler (one nvidia-smi sample per 100 ms) keeps running through this loop, which therefore
+    # goes on for at least half a second: the timed steps above are over within a few milliseconds.
     launch_ms = []
-    for _ in range(5):
+    t_loop = time.perf_counter()
+    while len(launch_ms) < 5 or (time.perf_counter() - t_loop < 0.6 and len(launch_ms) < 20000):
         k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         k0.record()
         if graph is not None:
@@ -309,6 +311,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         launch_ms.append(k0.elapsed_time(k1) / reps)
     fwd_launch_ms = statistics.median(launch_ms)
+    clocks = sampler.stop()
     del blobs
     st = B.pipe_poll_status()
     if st != B.PIPE_OK:
