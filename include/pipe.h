@@ -206,22 +206,27 @@ pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blo
                                   void* stream);
 
 /*
- * The expanded layer as a stride-1 "same" convolution (Appendix H counts a d x d convolution as
+ * The expanded layer as a two-dimensional convolution (Appendix H counts a d x d convolution as
  * d^2 * n_i * n_o multiplications per output pixel: the same contraction with the reduction
  * index running over (tap, input channel)).  Implicit GEMM: the quantized NHWC input is read in
- * place, tap by tap, with zero padding supplied by the copy engine; no im2col matrix exists.
- * Output row t = (n*H + h)*W + w, reduction index (dh*kernel_w + dw)*C + c, i.e. the weight
- * tensor [O, kernel_h, kernel_w, C] flattened to [O, I] with I = kernel_h*kernel_w*C = in_features.
+ * place, tap by tap, at the convolution's stride, with zero padding supplied by the copy engine;
+ * no im2col matrix exists.
+ * Output size Ho = (H + 2*pad_h - kernel_h) / stride_h + 1, Wo likewise.  Output row
+ * t = (n*Ho + ho)*Wo + wo, input pixel (stride_h*ho + dh - pad_h, stride_w*wo + dw - pad_w),
+ * reduction index (dh*kernel_w + dw)*C + c, i.e. the weight tensor [O, kernel_h, kernel_w, C]
+ * flattened to [O, I] with I = kernel_h*kernel_w*C = in_features.
  * All K orders act on the one input (as in pipe_expanded_linear).
  * d_xq: int8 [N, H, W, C], dense, 16-byte aligned (quantize it with pipe_quantize_act as a
- * [N*H*W, C] matrix).  d_y: float [N*H*W, O] pitch ldy.  d_partials as in pipe_expanded_linear.
- * This build takes kernel 2*pad + 1 square or not, stride 1, C a multiple of 128 and H, W
- * multiples of 8; anything else returns PIPE_ERR_UNSUPPORTED.
+ * [N*H*W, C] matrix).  d_y: float [N*Ho*Wo, O] pitch ldy.  d_partials as in pipe_expanded_linear
+ * with T = N*Ho*Wo.
+ * The library takes C a multiple of 128, strides 1..8 (0 means 1), 0 <= pad < kernel; anything else
+ * returns PIPE_ERR_UNSUPPORTED (PIPE_ERR_SHAPE if the geometry contradicts itself or the layer).
  */
 typedef struct pipe_conv_geom {
-  int32_t batch, height, width, channels; /* N, H, W, C of the input (= of the output, stride 1) */
-  int32_t kernel_h, kernel_w;             /* odd */
-  int32_t pad_h, pad_w;                   /* (kernel - 1) / 2 */
+  int32_t batch, height, width, channels; /* N, H, W, C of the input */
+  int32_t kernel_h, kernel_w;
+  int32_t pad_h, pad_w;                   /* zeros on each side */
+  int32_t stride_h, stride_w;             /* 0 is read as 1 */
 } pipe_conv_geom;
 
 pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,

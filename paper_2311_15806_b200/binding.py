@@ -42,7 +42,8 @@ class LayerDesc(C.Structure):
 
 class ConvGeom(C.Structure):
     _fields_ = [("batch", C.c_int32), ("height", C.c_int32), ("width", C.c_int32), ("channels", C.c_int32),
-                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
+                ("kernel_h", C.c_int32), ("kernel_w", C.c_int32), ("pad_h", C.c_int32), ("pad_w", C.c_int32),
+                ("stride_h", C.c_int32), ("stride_w", C.c_int32)]
 
 
 class LayerLayout(C.Structure):
@@ -178,7 +179,7 @@ def pipe_expanded_linear(desc: LayerDesc, blob: torch.Tensor, xq: torch.Tensor, 
 def pipe_expanded_conv2d(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_nhwc: torch.Tensor, sx: torch.Tensor,
                          y: torch.Tensor, bias: torch.Tensor | None = None, partials: torch.Tensor | None = None,
                          stream=None) -> None:
-    """xq_nhwc: cuda int8 [N, H, W, C] contiguous; y: cuda float32 [N*H*W, O]."""
+    """xq_nhwc: cuda int8 [N, H, W, C] contiguous; y: cuda float32 [N*Ho*Wo, O]."""
     assert xq_nhwc.is_contiguous() and xq_nhwc.dtype == torch.int8
     _check(lib().pipe_expanded_conv2d(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias), _dp(y),
                                       y.stride(0), _dp(partials), _stream_ptr(stream)), "pipe_expanded_conv2d")

@@ -92,6 +92,7 @@ struct ForwardArgs {
   int* status;
   // implicit convolution (conv_on != 0): branch[0].xq is the NHWC input, T = N*H*W
   int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
+  int cHo, cWo, csh, csw;   // output height / width and the strides
 };
 
 // Tensor map of a row-major byte matrix [rows, inner_bytes] with row pitch pitch_bytes (a multiple of 16) and

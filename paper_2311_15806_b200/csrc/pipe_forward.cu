@@ -99,14 +99,19 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   if (geom->batch < 1 || geom->height < 1 || geom->width < 1 || geom->channels < 1 || geom->kernel_h < 1 ||
       geom->kernel_w < 1)
     return PIPE_ERR_INVALID_ARG;
-  if (2 * geom->pad_h + 1 != geom->kernel_h || 2 * geom->pad_w + 1 != geom->kernel_w) return PIPE_ERR_SHAPE;
+  const int sh = geom->stride_h > 0 ? geom->stride_h : 1, sw = geom->stride_w > 0 ? geom->stride_w : 1;
+  if (geom->stride_h < 0 || geom->stride_w < 0 || geom->pad_h < 0 || geom->pad_w < 0) return PIPE_ERR_INVALID_ARG;
+  if (geom->pad_h >= geom->kernel_h || geom->pad_w >= geom->kernel_w) return PIPE_ERR_SHAPE;
+  if (geom->height + 2 * geom->pad_h < geom->kernel_h || geom->width + 2 * geom->pad_w < geom->kernel_w) return PIPE_ERR_SHAPE;
+  const int Ho = (geom->height + 2 * geom->pad_h - geom->kernel_h) / sh + 1;
+  const int Wo = (geom->width + 2 * geom->pad_w - geom->kernel_w) / sw + 1;
   if (static_cast<int64_t>(geom->kernel_h) * geom->kernel_w * geom->channels != L.I) return PIPE_ERR_SHAPE;
   if (ldy < L.O) return PIPE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_xq) & 15) ||
       (reinterpret_cast<uintptr_t>(d_sx) & 3) || (reinterpret_cast<uintptr_t>(d_y) & 3) ||
       (reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3))
     return PIPE_ERR_ALIGNMENT;
-  if (geom->channels % 128 != 0 || geom->height % 8 != 0 || geom->width % 8 != 0) return PIPE_ERR_UNSUPPORTED;
+  if (geom->channels % 128 != 0 || sh > 8 || sw > 8) return PIPE_ERR_UNSUPPORTED;
 
   ForwardArgs a;
   for (int k = 0; k < L.K; ++k) a.order[k] = order_view(L, d_blob, k);
@@ -120,7 +125,7 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   b.add_bias = 1;
   b.accumulate = 0;
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
-  a.T = static_cast<int64_t>(geom->batch) * geom->height * geom->width;
+  a.T = static_cast<int64_t>(geom->batch) * Ho * Wo;
   a.ldxq = geom->channels;
   a.ldy = ldy;
   a.bias = d_bias;
@@ -133,6 +138,7 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   a.conv_on = 1;
   a.cN = geom->batch; a.cH = geom->height; a.cW = geom->width; a.cC = geom->channels;
   a.ckh = geom->kernel_h; a.ckw = geom->kernel_w; a.cph = geom->pad_h; a.cpw = geom->pad_w;
+  a.cHo = Ho; a.cWo = Wo; a.csh = sh; a.csw = sw;
   if (kernel_choice() == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
   return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
 }

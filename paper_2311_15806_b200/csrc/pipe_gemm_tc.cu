@@ -469,23 +469,28 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     const int ttile = t.tt * p.tpt + x.jt;
     bool tile_ok = ttile < p.ntok_tiles;
     int64_t tok_base = static_cast<int64_t>(ttile) * kTileM + q * 32;
+    int eh = 4, ew = 8;
     if (p.f.conv_on) {
       const int patch = 2 * ttile + (q >> 1);
       int n, h0, w0;
       patch_origin(p, patch, n, h0, w0);
-      tok_base = (static_cast<int64_t>(n) * p.f.cH + h0 + (q & 1) * 4) * p.f.cW + w0;
+      tok_base = (static_cast<int64_t>(n) * p.f.cHo + h0 + (q & 1) * 4) * p.f.cWo + w0;
       tile_ok = patch < p.conv_np;
+      eh = p.f.cHo - (h0 + (q & 1) * 4);   // rows (of 8 pixels) and pixels of this half patch that lie inside the output
+      ew = p.f.cWo - w0;
     }
-    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * p.f.cW + (r & 7) : tok_base + r; };
+    auto token_of = [&](int r) -> int64_t { return p.f.conv_on ? tok_base + (r >> 3) * p.f.cWo + (r & 7) : tok_base + r; };
+    // a patch on the right or lower edge of the output may hang over it
+    auto inside = [&](int r) -> bool { return (r >> 3) < eh && (r & 7) < ew; };
     const int64_t tok_own = token_of(lane);
-    const bool own_ok = tile_ok && (p.f.conv_on || tok_own < p.f.T);
+    const bool own_ok = tile_ok && (p.f.conv_on ? inside(lane) : tok_own < p.f.T);
     float* srow[4];        // the four rows this lane stores, at channel c0 + 4 * sj
     uint32_t srow_ok = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int64_t tok = token_of(sr0 + 8 * i);
       srow[i] = br.y + tok * p.f.ldy + c0 + 4 * sj;
-      if (tile_ok && (p.f.conv_on || tok < p.f.T)) srow_ok |= 1u << i;
+      if (tile_ok && (p.f.conv_on ? inside(sr0 + 8 * i) : tok < p.f.T)) srow_ok |= 1u << i;
     }
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
     const bool add_bias = br.add_bias && p.f.bias;
@@ -679,7 +684,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
           for (int half = 0; half < 2 * p.tpt; ++half) {
             int n, h0, w0;
             patch_origin(p, 2 * p.tpt * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-            tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, w0 + dw, h0 + dh,
+            tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
                         n, g.a_full0 + 8u * rp.slot);
           }
         }
@@ -814,15 +819,17 @@ static bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner_bytes
 }
 
 // NHWC int8 tensor as a 4-D map; one box = 128 channels x 8 x 8 pixels of one image (64 rows of 128 bytes).
-static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int W, int C) {
+static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int W, int C, int sh, int sw) {
   EncodeFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
                               static_cast<cuuint64_t>(N)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W) * C,
                                  static_cast<cuuint64_t>(H) * W * C};
-  const cuuint32_t box[4] = {128, 8, 8, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  // 8 x 8 pixels at the convolution's stride: the box spans 8 * stride positions and the copy takes every
+  // stride-th of them
+  const cuuint32_t box[4] = {128, static_cast<cuuint32_t>(8 * sw), static_cast<cuuint32_t>(8 * sh), 1};
+  const cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(sw), static_cast<cuuint32_t>(sh), 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -859,7 +866,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   }
   if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
-  if (a.conv_on && (a.cC % kKStep != 0 || a.cH % 8 != 0 || a.cW % 8 != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
+  if (a.conv_on && (a.cC % kKStep != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
     if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   }
@@ -872,8 +879,8 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   p.ntok_tiles = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
   p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
   if (a.conv_on) {
-    p.conv_pw = a.cW / 8;
-    p.conv_pp = (a.cH / 8) * p.conv_pw;
+    p.conv_pw = ceil_div(a.cWo, 8);
+    p.conv_pp = ceil_div(a.cHo, 8) * p.conv_pw;
     p.conv_np = p.conv_pp * a.cN;
     p.conv_chunks = a.cC / kKStep;
     p.ntok_tiles = ceil_div(p.conv_np, 2);
@@ -923,7 +930,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   const int dyn_smem = p.depth * p.stage_bytes + 1024;
 
   if (a.conv_on) {
-    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC)) return PIPE_ERR_CUDA;
+    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
   } else
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),

@@ -282,17 +282,22 @@ def test_forward_zero_tokens_and_strided_io(oracle):
 
 
 CONV_CASES = [
-    # N, H,  W,  C,   O,  kh, kw, bits, K, g, n_keep
-    (2, 16, 8, 128, 64, 3, 3, 4, 3, 8, 2),
-    (1, 8, 24, 128, 72, 3, 3, 8, 2, 8, 3),      # odd number of 8x8 patches: the last tile is half empty
-    (3, 8, 8, 256, 136, 1, 1, 2, 4, 8, 5),      # 1x1: no halo
-    (1, 24, 16, 128, 40, 5, 3, 4, 2, 8, 5),     # rectangular filter, two rows/columns of padding
+    # N, H,  W,  C,   O,  kh, kw, bits, K, g, n_keep, stride, pad (None: (k - 1) / 2)
+    (2, 16, 8, 128, 64, 3, 3, 4, 3, 8, 2, 1, None),
+    (1, 8, 24, 128, 72, 3, 3, 8, 2, 8, 3, 1, None),      # odd number of 8x8 patches: the last tile is half empty
+    (3, 8, 8, 256, 136, 1, 1, 2, 4, 8, 5, 1, None),      # 1x1: no halo
+    (1, 24, 16, 128, 40, 5, 3, 4, 2, 8, 5, 1, None),     # rectangular filter, two rows/columns of padding
+    (2, 14, 14, 128, 64, 3, 3, 4, 3, 8, 2, 1, None),     # output not a multiple of the 8x8 patch: edge patches hang over
+    (1, 15, 9, 128, 40, 3, 3, 4, 2, 8, 5, 2, None),      # stride 2, odd sizes: 8 x 5 outputs
+    (2, 16, 16, 256, 72, 1, 1, 8, 2, 8, 3, 2, None),     # strided 1x1 (a downsampling shortcut)
+    (1, 28, 28, 128, 64, 3, 3, 4, 3, 8, 2, 2, None),     # 28 -> 14
+    (1, 12, 20, 128, 48, 3, 3, 2, 3, 8, 2, 1, (0, 0)),   # no padding: 10 x 18 outputs
 ]
 
 
 @pytest.mark.parametrize("kernel", [B.KERNEL_AUTO, B.KERNEL_TCGEN05_PAIR])
-@pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep", CONV_CASES)
-def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep):
+@pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep,stride,pad", CONV_CASES)
+def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep, stride, pad):
     """pipe_expanded_conv2d on the NHWC tensor == the oracle on explicitly lowered im2col rows."""
     rng = np.random.default_rng(N * 1000 + Hh * 10 + Cc)
     I = kh * kw * Cc
@@ -305,19 +310,21 @@ def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, k
     xq_o, sx_o = oracle.quantize_act(x4.reshape(-1, Cc))
     np.testing.assert_array_equal(xq4.cpu().numpy(), xq_o)
     # explicit lowering on the host (pad_h may differ from pad_w: lower by hand)
-    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    ph, pw = ((kh - 1) // 2, (kw - 1) // 2) if pad is None else pad
+    Ho, Wo = (Hh + 2 * ph - kh) // stride + 1, (Ww + 2 * pw - kw) // stride + 1
     xp = np.zeros((N, Hh + 2 * ph, Ww + 2 * pw, Cc), np.int8)
     xp[:, ph:ph + Hh, pw:pw + Ww] = xq_o.reshape(N, Hh, Ww, Cc)
-    rows = np.zeros((N, Hh, Ww, kh * kw * Cc), np.int8)
+    rows = np.zeros((N, Ho, Wo, kh * kw * Cc), np.int8)
     for dh in range(kh):
         for dw in range(kw):
             tap = dh * kw + dw
-            rows[..., tap * Cc:(tap + 1) * Cc] = xp[:, dh:dh + Hh, dw:dw + Ww]
+            rows[..., tap * Cc:(tap + 1) * Cc] = xp[:, dh:dh + stride * (Ho - 1) + 1:stride, dw:dw + stride * (Wo - 1) + 1:stride]
     f = oracle.forward(e, rows.reshape(-1, I), sx_o, bias=bias)
     geom = B.ConvGeom()
     geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
     geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, ph, pw
-    T = N * Hh * Ww
+    geom.stride_h = geom.stride_w = stride
+    T = N * Ho * Wo
     y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
     B.pipe_select_kernel(kernel)
@@ -349,7 +356,7 @@ def test_convolution_shapes_outside_the_fast_path_are_refused():
     with pytest.raises(B.PipeError) as ei:
         B.pipe_expanded_conv2d(layer_desc, geom, blob, xq, sx, y)
     assert ei.value.status == B.PIPE_ERR_UNSUPPORTED
-    geom.pad_h = 0
+    geom.pad_h = 3   # as much padding as the filter is high: no output row would see the image
     with pytest.raises(B.PipeError) as ei:
         B.pipe_expanded_conv2d(layer_desc, geom, blob, xq, sx, y)
     assert ei.value.status == B.PIPE_ERR_SHAPE
