@@ -206,6 +206,25 @@ pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blo
                                   void* stream);
 
 /*
+ * An INNER layer of the M predictors (Sec. 3.2, Fig. 2; Appendix B, Eq. 9 with its activation
+ * function): predictor m's output never leaves the integer pipeline as floats.  Per predictor
+ *     y_m            as in pipe_ensemble_forward (same order of operations, bias with predictor 1),
+ *     a_m[t,o]       = relu != 0 ? max(y_m[t,o], 0) : y_m[t,o]           (sigma of Eq. 9)
+ *     yq_m[t,o]      = clamp(rne(a_m[t,o] / s_m), -127, 127)             (Eq. 1 as the next layer's Q,
+ *                                                                         IEEE binary32 quotient, ties to even)
+ * so that yq_m and s_m are the next layer's xq_m and lambda_{x_m}.  s_m is a static step the caller
+ * calibrated: h_out_scale_m is a HOST array of M device pointers to one float each (s_m >= 0 and
+ * finite, else PIPE_ERR_INVALID_ARG through the device status; s_m = 0 gives all-zero codes).
+ * h_yq_m: HOST array of M device pointers, int8 [T, O] pitch ldyq (>= O); no float output is
+ * written.  The other arguments are those of pipe_ensemble_forward; M = 1 is the plain expanded
+ * layer with this epilogue.  The two-SM kernel (choice 4) answers PIPE_ERR_UNSUPPORTED.
+ */
+pipe_status pipe_ensemble_forward_q8(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                     int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
+                                     int32_t relu, const float* const* h_out_scale_m, int8_t* const* h_yq_m,
+                                     int64_t ldyq, int32_t* d_partials, void* stream);
+
+/*
  * The expanded layer as a two-dimensional convolution (Appendix H counts a d x d convolution as
  * d^2 * n_i * n_o multiplications per output pixel: the same contraction with the reduction
  * index running over (tap, input channel)).  Implicit GEMM: the quantized NHWC input is read in
@@ -232,6 +251,17 @@ typedef struct pipe_conv_geom {
 pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
                                  const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y, int64_t ldy,
                                  int32_t* d_partials, void* stream);
+
+/*
+ * The convolution as an inner layer: pipe_expanded_conv2d with the epilogue of
+ * pipe_ensemble_forward_q8 (sigma of Eq. 9, then Eq. 1 as the next layer's input quantizer with
+ * the static step *d_out_scale).  d_yq: int8 [N*Ho*Wo, O] pitch ldyq; with ldyq = O it is the
+ * NHWC input of the next convolution as it stands.  No float output is written.
+ */
+pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                    const int8_t* d_xq, const float* d_sx, const float* d_bias, int32_t relu,
+                                    const float* d_out_scale, int8_t* d_yq, int64_t ldyq, int32_t* d_partials,
+                                    void* stream);
 
 /* Which GEMM kernel the two forward calls use (process-wide, for tests and measurements):
  * 0 = automatic, 1 = CUDA-core reference kernel, 2 = tcgen05 tensor-core kernel,

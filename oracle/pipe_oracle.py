@@ -177,6 +177,17 @@ def quantize_act(x: np.ndarray, static_scale: float | None = None):
     return xq, np.float32(sx[0])
 
 
+def forward_requantized(e: "Expansion", xq: np.ndarray, sx, out_scale: float, k_begin: int = 0, k_end: int | None = None,
+                        bias: np.ndarray | None = None, relu: bool = True) -> np.ndarray:
+    """One inner layer of an ensemble branch (Sec. 3.2; Appendix B, the predictors g and h): the branch's
+    cluster of orders on its own input, the activation function, then the next layer's input quantizer Q
+    with a static scale.  Nothing new is computed here: it is `forward`, a ReLU, and `quantize_act`."""
+    y = forward(e, xq, sx, k_begin, k_end, bias).y
+    if relu:
+        y = np.maximum(y, np.float32(0))
+    return quantize_act(y, static_scale=out_scale)[0]
+
+
 @dataclass
 class Forward:
     y: np.ndarray          # float32 [T, O]

@@ -30,6 +30,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
+           "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
            "pipe_select_kernel",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string"]
 
@@ -89,6 +90,8 @@ def lib() -> C.CDLL:
         L.pipe_expanded_linear.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, p, p]
         L.pipe_expanded_conv2d.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, p, i64, p, p]
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
+        L.pipe_ensemble_forward_q8.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, i32, p, p, i64, p, p]
+        L.pipe_expanded_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
         L.pipe_select_kernel.argtypes = [i32]
         L.pipe_launch_count.restype = C.c_uint64
         L.pipe_poll_status.argtypes = [p, C.POINTER(i32)]
@@ -185,6 +188,16 @@ def pipe_expanded_conv2d(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq
                                       y.stride(0), _dp(partials), _stream_ptr(stream)), "pipe_expanded_conv2d")
 
 
+def pipe_expanded_conv2d_q8(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_nhwc: torch.Tensor, sx: torch.Tensor,
+                            out_scale: torch.Tensor, yq: torch.Tensor, bias: torch.Tensor | None = None, relu: bool = True,
+                            partials: torch.Tensor | None = None, stream=None) -> None:
+    """xq_nhwc: cuda int8 [N, H, W, C] contiguous; yq: cuda int8 [N*Ho*Wo, O]; out_scale: cuda float32, one element."""
+    assert xq_nhwc.is_contiguous() and xq_nhwc.dtype == torch.int8 and yq.dtype == torch.int8
+    _check(lib().pipe_expanded_conv2d_q8(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias),
+                                         1 if relu else 0, _dp(out_scale), _dp(yq), yq.stride(0), _dp(partials),
+                                         _stream_ptr(stream)), "pipe_expanded_conv2d_q8")
+
+
 def pipe_ensemble_forward(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,
                           sum_branches: bool = False, partials: torch.Tensor | None = None, stream=None) -> None:
     """xq_m, sx_m, y_m: sequences of M cuda tensors (xq_m entries may be the same tensor)."""
@@ -200,6 +213,26 @@ def pipe_ensemble_forward(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, y_m, 
     _check(lib().pipe_ensemble_forward(C.byref(desc), _dp(blob), xp, T, ldxq, sp, _dp(bias), yp, ldy,
                                        1 if sum_branches else 0, _dp(partials), _stream_ptr(stream)),
            "pipe_ensemble_forward")
+
+
+def pipe_ensemble_forward_q8(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, out_scale_m, yq_m,
+                             bias: torch.Tensor | None = None, relu: bool = True, partials: torch.Tensor | None = None,
+                             stream=None) -> None:
+    """Inner layer of the M predictors: yq_m[m] (cuda int8 [T, O]) receives Q(sigma(y_m)) with the static step
+    out_scale_m[m] (cuda float32, one element); xq_m, sx_m as in pipe_ensemble_forward."""
+    M = desc.num_branches
+    assert len(xq_m) == M and len(sx_m) == M and len(out_scale_m) == M and len(yq_m) == M
+    assert all(t.dtype == torch.int8 for t in yq_m)
+    T = xq_m[0].shape[0]
+    ldxq = xq_m[0].stride(0) if T > 1 else max(xq_m[0].shape[1], xq_m[0].stride(0))
+    ldyq = yq_m[0].stride(0) if T > 1 else max(yq_m[0].shape[1], yq_m[0].stride(0))
+    PA = C.c_void_p * M
+    xp = PA(*[_dp(t) for t in xq_m])
+    sp = PA(*[_dp(t) for t in sx_m])
+    op = PA(*[_dp(t) for t in out_scale_m])
+    yp = PA(*[_dp(t) for t in yq_m])
+    _check(lib().pipe_ensemble_forward_q8(C.byref(desc), _dp(blob), xp, T, ldxq, sp, _dp(bias), 1 if relu else 0, op, yp,
+                                          ldyq, _dp(partials), _stream_ptr(stream)), "pipe_ensemble_forward_q8")
 
 
 def pipe_select_kernel(which: int) -> None:

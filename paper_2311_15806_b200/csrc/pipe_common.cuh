@@ -45,6 +45,41 @@ __host__ __device__ inline T round_up(T a, T b) {
 // Raise a device-side error: first error wins.
 __device__ inline void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// clamp(rne(v / s)) as an int8 lane.  The IEEE quotient is what defines the code (Eq. 1 with true
+// division), but a division costs an order of magnitude more than a multiplication, so the quotient is
+// first estimated as t = v * r with r = rn(1 / s): t is within a relative 2^-22.9 of the real quotient,
+// as is the IEEE quotient itself (2^-24), so both round to the same integer unless the estimate lies
+// within |t| * 2^-21 of a rounding boundary (an odd multiple of one half) -- only then, a few times in a
+// hundred thousand, is the division carried out.  Beyond +-130 both clamp.
+__device__ __forceinline__ uint32_t quant_lane(float v, float s, float r) {
+  const float t = __fmul_rn(v, r);
+  float q = rintf(t);
+  const float at = fabsf(t);
+  if (at > 130.f) {
+    q = copysignf(127.f, t);
+  } else if (0.5f - fabsf(__fsub_rn(t, q)) <= at * 4.76837158203125e-07f) {
+    q = rintf(__fdiv_rn(v, s));
+  }
+  q = fminf(fmaxf(q, -127.f), 127.f);
+  return static_cast<uint32_t>(static_cast<int>(q)) & 0xffu;
+}
+
+// The same code with the division always carried out; a zero step gives the code 0 (Eq. 1 on an all-zero tensor).
+__device__ __forceinline__ uint32_t quant_lane_exact(float v, float s) {
+  float q = 0.f;
+  if (s != 0.f) q = fminf(fmaxf(rintf(__fdiv_rn(v, s)), -127.f), 127.f);
+  return static_cast<uint32_t>(static_cast<int>(q)) & 0xffu;
+}
+
+// The estimate needs a reciprocal that neither overflows nor is subnormal.
+__device__ __forceinline__ bool quant_step_is_fast(float s) { return s >= 1e-30f && s <= 1e30f; }
+
+// Four codes as the bytes of one word, lowest address first.
+__device__ __forceinline__ uint32_t quant4(const float4& f, float s, float r, bool fast) {
+  if (fast) return quant_lane(f.x, s, r) | (quant_lane(f.y, s, r) << 8) | (quant_lane(f.z, s, r) << 16) | (quant_lane(f.w, s, r) << 24);
+  return quant_lane_exact(f.x, s) | (quant_lane_exact(f.y, s) << 8) | (quant_lane_exact(f.z, s) << 16) | (quant_lane_exact(f.w, s) << 24);
+}
+
 // Per-order pointers into a blob, passed to kernels by value.
 struct OrderView {
   const uint8_t* codes;   // canonical packed codes
@@ -74,6 +109,8 @@ struct BranchArgs {
   const int8_t* xq;
   const float* sx;
   float* y;
+  int8_t* yq;              // re-quantized output (ForwardArgs::q8_out), else unused
+  const float* out_scale;  // its step: one float on the device
   int k_begin, k_end;
   int add_bias;    // bias enters this branch
   int accumulate;  // y += result (summed ensemble, branches after the first)
@@ -93,6 +130,9 @@ struct ForwardArgs {
   // implicit convolution (conv_on != 0): branch[0].xq is the NHWC input, T = N*H*W
   int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
   int cHo, cWo, csh, csw;   // output height / width and the strides
+  // fused inner-layer epilogue (q8_out != 0): yq = clamp(rne(act(y) / out_scale)) as int8, row pitch ldyq; y is not written
+  int q8_out, relu;
+  int64_t ldyq;
 };
 
 // Tensor map of a row-major byte matrix [rows, inner_bytes] with row pitch pitch_bytes (a multiple of 16) and

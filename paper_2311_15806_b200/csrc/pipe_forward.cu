@@ -6,15 +6,24 @@ namespace pipe {
 static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, const int8_t* const* xq,
                                const float* const* sx, float* const* y, const int* k_begin, const int* k_end,
                                int64_t T, int64_t ldxq, int64_t ldy, const float* d_bias, int sum_branches,
-                               int32_t* d_partials, cudaStream_t stream) {
+                               int32_t* d_partials, cudaStream_t stream, int8_t* const* yq = nullptr,
+                               const float* const* out_scale = nullptr, int64_t ldyq = 0, int relu = 0) {
+  // yq != nullptr: the fused inner-layer epilogue; y and ldy are unused then
+  const bool q8 = yq != nullptr;
   if (!d_blob) return PIPE_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) return PIPE_ERR_ALIGNMENT;
-  if (T < 0 || ldxq < L.I || ldy < L.O) return PIPE_ERR_INVALID_ARG;
+  if (T < 0 || ldxq < L.I) return PIPE_ERR_INVALID_ARG;
+  if (q8 ? (ldyq < L.O || !out_scale || sum_branches) : (ldy < L.O)) return PIPE_ERR_INVALID_ARG;
   for (int m = 0; m < M; ++m) {
     if (!sx[m]) return PIPE_ERR_INVALID_ARG;
     if (T > 0 && !xq[m]) return PIPE_ERR_INVALID_ARG;
-    if (T > 0 && (m == 0 || !sum_branches) && !y[m]) return PIPE_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(sx[m]) & 3) return PIPE_ERR_ALIGNMENT;
+    if (q8) {
+      if (!out_scale[m] || (T > 0 && !yq[m])) return PIPE_ERR_INVALID_ARG;
+      if (reinterpret_cast<uintptr_t>(out_scale[m]) & 3) return PIPE_ERR_ALIGNMENT;
+      continue;
+    }
+    if (T > 0 && (m == 0 || !sum_branches) && !y[m]) return PIPE_ERR_INVALID_ARG;
     if ((m == 0 || !sum_branches) && (reinterpret_cast<uintptr_t>(y[m]) & 3)) return PIPE_ERR_ALIGNMENT;
   }
   if ((reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3)) return PIPE_ERR_ALIGNMENT;
@@ -27,7 +36,9 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     BranchArgs& b = a.branch[m];
     b.xq = xq[m];
     b.sx = sx[m];
-    b.y = sum_branches ? y[0] : y[m];
+    b.y = q8 ? nullptr : (sum_branches ? y[0] : y[m]);
+    b.yq = q8 ? yq[m] : nullptr;
+    b.out_scale = q8 ? out_scale[m] : nullptr;
     b.k_begin = k_begin[m];
     b.k_end = k_end[m];
     b.add_bias = (m == 0);
@@ -44,6 +55,10 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   if (!a.status) return PIPE_ERR_CUDA;
   a.conv_on = 0;
   a.cN = a.cH = a.cW = a.cC = a.ckh = a.ckw = a.cph = a.cpw = 0;
+  a.cHo = a.cWo = 0; a.csh = a.csw = 1;
+  a.q8_out = q8 ? 1 : 0;
+  a.relu = relu ? 1 : 0;
+  a.ldyq = ldyq;
 
   const int choice = kernel_choice();
   if (choice == 1) return forward_reference(a, stream);
@@ -89,13 +104,32 @@ extern "C" pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const 
                      d_partials, static_cast<cudaStream_t>(stream));
 }
 
-extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
-                                            const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y,
-                                            int64_t ldy, int32_t* d_partials, void* stream) {
+extern "C" pipe_status pipe_ensemble_forward_q8(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                                int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
+                                                int32_t relu, const float* const* h_out_scale_m, int8_t* const* h_yq_m,
+                                                int64_t ldyq, int32_t* d_partials, void* stream) {
   LayerInfo L;
   pipe_status st = resolve_layer(desc, &L);
   if (st != PIPE_OK) return st;
-  if (!geom || !d_blob || !d_xq || !d_sx || !d_y) return PIPE_ERR_INVALID_ARG;
+  if (!h_xq_m || !h_sx_m || !h_out_scale_m || !h_yq_m) return PIPE_ERR_INVALID_ARG;
+  int kb[PIPE_MAX_ORDERS], ke[PIPE_MAX_ORDERS];
+  for (int m = 0; m < L.M; ++m) {
+    kb[m] = L.branch_begin[m];
+    ke[m] = L.branch_begin[m + 1];
+  }
+  return run_forward(L, d_blob, L.M, h_xq_m, h_sx_m, nullptr, kb, ke, T, ldxq, 0, d_bias, 0, d_partials,
+                     static_cast<cudaStream_t>(stream), h_yq_m, h_out_scale_m, ldyq, relu);
+}
+
+// Both convolution entries: d_yq != nullptr selects the fused inner-layer epilogue (d_y, ldy unused then).
+static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob, const int8_t* d_xq,
+                            const float* d_sx, const float* d_bias, float* d_y, int64_t ldy, int8_t* d_yq,
+                            const float* d_out_scale, int64_t ldyq, int relu, int32_t* d_partials, void* stream) {
+  const bool q8 = d_yq != nullptr;
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  if (!geom || !d_blob || !d_xq || !d_sx || (!q8 && !d_y) || (q8 && !d_out_scale)) return PIPE_ERR_INVALID_ARG;
   if (geom->batch < 1 || geom->height < 1 || geom->width < 1 || geom->channels < 1 || geom->kernel_h < 1 ||
       geom->kernel_w < 1)
     return PIPE_ERR_INVALID_ARG;
@@ -106,9 +140,10 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   const int Ho = (geom->height + 2 * geom->pad_h - geom->kernel_h) / sh + 1;
   const int Wo = (geom->width + 2 * geom->pad_w - geom->kernel_w) / sw + 1;
   if (static_cast<int64_t>(geom->kernel_h) * geom->kernel_w * geom->channels != L.I) return PIPE_ERR_SHAPE;
-  if (ldy < L.O) return PIPE_ERR_INVALID_ARG;
+  if ((q8 ? ldyq : ldy) < L.O) return PIPE_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_xq) & 15) ||
       (reinterpret_cast<uintptr_t>(d_sx) & 3) || (reinterpret_cast<uintptr_t>(d_y) & 3) ||
+      (reinterpret_cast<uintptr_t>(d_out_scale) & 3) ||
       (reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3))
     return PIPE_ERR_ALIGNMENT;
   if (geom->channels % 128 != 0 || sh > 8 || sw > 8) return PIPE_ERR_UNSUPPORTED;
@@ -119,11 +154,16 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   BranchArgs& b = a.branch[0];
   b.xq = d_xq;
   b.sx = d_sx;
-  b.y = d_y;
+  b.y = q8 ? nullptr : d_y;
   b.k_begin = 0;
   b.k_end = L.K;
   b.add_bias = 1;
   b.accumulate = 0;
+  b.yq = d_yq;
+  b.out_scale = d_out_scale;
+  a.q8_out = q8 ? 1 : 0;
+  a.relu = relu ? 1 : 0;
+  a.ldyq = ldyq;
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = static_cast<int64_t>(geom->batch) * Ho * Wo;
   a.ldxq = geom->channels;
@@ -141,4 +181,18 @@ extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const p
   a.cHo = Ho; a.cWo = Wo; a.csh = sh; a.csw = sw;
   if (kernel_choice() == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
   return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                            const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y,
+                                            int64_t ldy, int32_t* d_partials, void* stream) {
+  return run_conv(desc, geom, d_blob, d_xq, d_sx, d_bias, d_y, ldy, nullptr, nullptr, 0, 0, d_partials, stream);
+}
+
+extern "C" pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                               const int8_t* d_xq, const float* d_sx, const float* d_bias, int32_t relu,
+                                               const float* d_out_scale, int8_t* d_yq, int64_t ldyq, int32_t* d_partials,
+                                               void* stream) {
+  if (!d_yq) return PIPE_ERR_INVALID_ARG;
+  return run_conv(desc, geom, d_blob, d_xq, d_sx, d_bias, nullptr, 0, d_yq, d_out_scale, ldyq, relu, d_partials, stream);
 }

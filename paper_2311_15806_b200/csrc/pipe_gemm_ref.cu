@@ -48,6 +48,12 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
   for (int m = m_first; m < m_last; ++m) {
     const BranchArgs br = a.branch[m];
     const float sx = *br.sx;
+    float out_step = 0.f;
+    if (a.q8_out) {
+      out_step = *br.out_scale;
+      if (!(out_step >= 0.f && out_step < __uint_as_float(0x7f800000u)) && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0)
+        raise_status(a.status, PIPE_ERR_INVALID_ARG);
+    }
     float yv[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
@@ -138,6 +144,10 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
         if (sum_mode) {
           total[i][j] = (m == 0) ? v : __fadd_rn(total[i][j], v);
           if (m + 1 == m_last) a.branch[0].y[t * a.ldy + c] = total[i][j];
+        } else if (a.q8_out) {
+          // inner layer of a branch: activation, then the next layer's input quantizer (division carried out)
+          if (a.relu) v = fmaxf(v, 0.f);
+          br.yq[t * a.ldyq + c] = static_cast<int8_t>(quant_lane_exact(v, out_step));
         } else {
           br.y[t * a.ldy + c] = v;
         }
@@ -159,6 +169,7 @@ pipe_status forward_reference(const ForwardArgs& a, cudaStream_t stream) {
       for (int m = 0; m < a.num_branches; ++m) {
         part.branch[m].xq = a.branch[m].xq + t * a.ldxq;
         part.branch[m].y = a.branch[m].y ? a.branch[m].y + t * a.ldy : nullptr;
+        part.branch[m].yq = a.branch[m].yq ? a.branch[m].yq + t * a.ldyq : nullptr;
       }
       part.partials = a.partials ? a.partials + t * a.total_rows : nullptr;
       pipe_status st = forward_reference(part, stream);

@@ -403,7 +403,27 @@ struct EpiCtx {
 // through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
 // (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
 // which is what bounds the drain otherwise).
-template <int NKMAX, bool PARTIALS>
+// The code clamp(rne(v / s)) of the fused inner-layer epilogue without a conversion instruction: the estimate
+// t = v * rn(1 / s), clamped to +-127 (a t beyond 127 has a true quotient above 126.9999, whose code is 127),
+// is added to 1.5 * 2^23, where the spacing of binary32 is one, so the addition itself rounds to the nearest
+// integer, ties to even, and leaves the code in the low byte of the sum.  `edge` collects the largest
+// |t - code| + |t| * 2^-21: at 0.5 or more an estimate lies so close to a rounding boundary that the IEEE
+// quotient, which defines the code, may round the other way, and the caller divides.
+__device__ __forceinline__ float quant_magic(float v, float r, float& edge) {
+  const float t = fminf(fmaxf(__fmul_rn(v, r), -127.f), 127.f);
+  const float u = __fadd_rn(t, 12582912.f);
+  const float d = __fsub_rn(t, __fsub_rn(u, 12582912.f));
+  edge = fmaxf(edge, __fmaf_rn(fabsf(t), 4.76837158203125e-07f, fabsf(d)));
+  return u;
+}
+
+__device__ __forceinline__ uint32_t pack4_low_bytes(float a, float b, float c, float d) {
+  const uint32_t ab = __byte_perm(__float_as_uint(a), __float_as_uint(b), 0x0040);
+  const uint32_t cd = __byte_perm(__float_as_uint(c), __float_as_uint(d), 0x0040);
+  return __byte_perm(ab, cd, 0x5410);
+}
+
+template <int NKMAX, bool PARTIALS, bool Q8>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
   constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
   const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
@@ -489,10 +509,27 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int64_t tok = token_of(sr0 + 8 * i);
-      srow[i] = br.y + tok * p.f.ldy + c0 + 4 * sj;
+      srow[i] = Q8 ? nullptr : br.y + tok * p.f.ldy + c0 + 4 * sj;
       if (tile_ok && (p.f.conv_on ? inside(sr0 + 8 * i) : tok < p.f.T)) srow_ok |= 1u << i;
     }
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
+    // Fused inner-layer epilogue.  A lane's 16 channels become 16 bytes, which it stores itself: at one byte
+    // per output a row piece is half a sector however the block is turned, so the staging block is free and
+    // holds the bias of the tile's channels instead.
+    float ostep = 0.f, orcp = 0.f;
+    bool ofast = false;
+    int8_t* qrow = nullptr;      // this lane's output row at channel c0
+    int qalign = 0;              // 16, 4 or 1: widest store every piece of the row allows
+    if constexpr (Q8) {
+      ostep = __ldg(br.out_scale);
+      ofast = quant_step_is_fast(ostep);
+      orcp = ofast ? __frcp_rn(ostep) : 0.f;
+      if (!(ostep >= 0.f && ostep < __uint_as_float(0x7f800000u)) && lane == 0) raise_status(p.f.status, PIPE_ERR_INVALID_ARG);
+      qrow = br.yq + tok_own * p.f.ldyq + c0;
+      const uintptr_t bits = reinterpret_cast<uintptr_t>(br.yq) | static_cast<uintptr_t>(p.f.ldyq);
+      qalign = (bits & 15) == 0 ? 16 : ((bits & 3) == 0 ? 4 : 1);
+      for (int c = lane; c < p.BN; c += 32) x.stg[c] = (br.add_bias && p.f.bias && c0 + c < p.f.O) ? __ldg(p.f.bias + c0 + c) : 0.f;
+    }
     const bool add_bias = br.add_bias && p.f.bias;
     const float* bias_q = add_bias ? p.f.bias + c0 + 4 * sj : nullptr;
     const int ngrp = (nch + 1) >> 1;
@@ -504,11 +541,12 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
       const bool quad_ok = 2 * grp + (sj >> 1) < nch;
       float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (add_bias && quad_ok) {
+      if (!Q8 && add_bias && quad_ok) {
         const float* bp = bias_q + 16 * grp;
         bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
       }
-      // ---- this lane's row: 16 channels into the staging block
+      // ---- this lane's row: 16 channels into the staging block (as 16 codes into registers for the fused epilogue)
+      uint32_t packed[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
       for (int sub = 0; sub < 2; sub += CH) {
         int acc[CH][NKMAX][8];
@@ -564,6 +602,30 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
               for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
             }
           }
+          if constexpr (Q8) {
+            // bias last, sigma, then Q of the next layer (Sec. 3.2): eight codes of this lane's own row
+            float bv[8];
+            const uint32_t ba = smem_u32(x.stg) + static_cast<uint32_t>(chunk * 32);
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]) : "r"(ba));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7]) : "r"(ba + 16));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              if (add_bias) y[e] = __fadd_rn(y[e], bv[e]);
+              if (p.f.relu) y[e] = fmaxf(y[e], 0.f);
+            }
+            float uu[8];
+            float edge = ofast ? 0.f : 1.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) uu[e] = quant_magic(y[e], orcp, edge);
+            uint32_t w0 = pack4_low_bytes(uu[0], uu[1], uu[2], uu[3]), w1 = pack4_low_bytes(uu[4], uu[5], uu[6], uu[7]);
+            if (edge >= 0.5f) {   // some estimate sits on a rounding boundary (or the step has no usable reciprocal)
+              w0 = quant4(make_float4(y[0], y[1], y[2], y[3]), ostep, orcp, false);
+              w1 = quant4(make_float4(y[4], y[5], y[6], y[7]), ostep, orcp, false);
+            }
+            packed[2 * (sub + u)] = w0;
+            packed[2 * (sub + u) + 1] = w1;
+            continue;
+          }
           const int j0 = 2 * (sub + u);
           asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>((j0 ^ wsw) << 4)), "f"(y[0]),
                        "f"(y[1]), "f"(y[2]), "f"(y[3])
@@ -572,6 +634,27 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
                        "f"(y[5]), "f"(y[6]), "f"(y[7])
                        : "memory");
         }
+      }
+      if constexpr (Q8) {
+        if (own_ok) {
+          int8_t* dq = qrow + 16 * grp;
+          const int nw = (2 * grp + 1 < nch) ? 4 : 2;   // a tile's last group may hold eight channels only
+          if (qalign == 16 && nw == 4) {
+            *reinterpret_cast<uint4*>(dq) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          } else if (qalign >= 4) {
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+              if (w < nw) reinterpret_cast<uint32_t*>(dq)[w] = packed[w];
+          } else {
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+              if (w < nw) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) dq[4 * w + b] = static_cast<int8_t>(packed[w] >> (8 * b));
+              }
+          }
+        }
+        continue;
       }
       __syncwarp();
       // ---- 8 rows x 64 bytes per store instruction; the bias joins here, after the whole chain
@@ -603,6 +686,8 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   }
 }
 
+// Q8: the fused inner-layer epilogue (activation function and the next layer's input quantizer) replaces the fp32 store.
+template <bool Q8>
 __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[4] bt_ready[4] done[4] tmem_full[2] tmem_empty[2]
@@ -768,13 +853,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     e.cscale = epi_cscale[ew];
     e.stg = epi_stage[ew];
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
-      if (p.nkmax <= 2) epilogue_role<2, true>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, true>(p, e);
-      else epilogue_role<8, true>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, true, Q8>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true, Q8>(p, e);
+      else epilogue_role<8, true, Q8>(p, e);
     } else {
-      if (p.nkmax <= 2) epilogue_role<2, false>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, false>(p, e);
-      else epilogue_role<8, false>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, false, Q8>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false, Q8>(p, e);
+      else epilogue_role<8, false, Q8>(p, e);
     }
   }
 
@@ -923,7 +1008,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
     p.koff[k] = static_cast<uint32_t>(d >> 4);
   }
   cudaFuncAttributes fattr;
-  if (cudaFuncGetAttributes(&fattr, tc_forward_kernel) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (cudaFuncGetAttributes(&fattr, tc_forward_kernel<false>) != cudaSuccess) return PIPE_ERR_CUDA;
   p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / p.stage_bytes;  // static shared, alignment slack
   if (p.depth > kMaxRing) p.depth = kMaxRing;
   if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
@@ -937,14 +1022,17 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
                      static_cast<uint64_t>(a.ldxq), kKStep, p.tpt * kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
   }
-  static int attr_bytes = 0;
-  if (attr_bytes < dyn_smem) {
-    if (cudaFuncSetAttribute(tc_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem) != cudaSuccess)
-      return PIPE_ERR_CUDA;
-    attr_bytes = dyn_smem;
+  static int attr_bytes[2] = {0, 0};
+  const int which = a.q8_out ? 1 : 0;
+  if (attr_bytes[which] < dyn_smem) {
+    const cudaError_t e = which ? cudaFuncSetAttribute(tc_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem)
+                                : cudaFuncSetAttribute(tc_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem);
+    if (e != cudaSuccess) return PIPE_ERR_CUDA;
+    attr_bytes[which] = dyn_smem;
   }
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-  tc_forward_kernel<<<grid, kThreads, dyn_smem, stream>>>(p);
+  if (which) tc_forward_kernel<true><<<grid, kThreads, dyn_smem, stream>>>(p);
+  else tc_forward_kernel<false><<<grid, kThreads, dyn_smem, stream>>>(p);
   count_launch(1);
   return launch_status();
 }

@@ -1030,6 +1030,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
 
 pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T == 0) return PIPE_OK;
+  if (a.q8_out) return PIPE_ERR_UNSUPPORTED;   // the fused re-quantization lives in the one-SM and decode kernels
   const bool sum_mode = a.num_branches > 1 && a.branch[1].accumulate;
   if (!sum_mode) return launch_tc2(a, stream);
   // Summed ensemble: one launch per branch, in order, so that y = ((y_1 + y_2) + ...) is formed

@@ -132,38 +132,6 @@ __global__ void __launch_bounds__(kQThreads) act_absmax_flat_kernel(const float4
   }
 }
 
-// clamp(rne(v / s)) as an int8 lane.  The IEEE quotient is what defines the code (Eq. 1 with true
-// division), but a division costs an order of magnitude more than a multiplication, so the quotient is
-// first estimated as t = v * r with r = rn(1 / s): t is within a relative 2^-22.9 of the real quotient,
-// as is the IEEE quotient itself (2^-24), so both round to the same integer unless the estimate lies
-// within |t| * 2^-21 of a rounding boundary (an odd multiple of one half) -- only then, a few times in a
-// hundred thousand, is the division carried out.  Beyond +-130 both clamp.
-__device__ __forceinline__ uint32_t quant_lane(float v, float s, float r) {
-  const float t = __fmul_rn(v, r);
-  float q = rintf(t);
-  const float at = fabsf(t);
-  if (at > 130.f) {
-    q = copysignf(127.f, t);
-  } else if (0.5f - fabsf(__fsub_rn(t, q)) <= at * 4.76837158203125e-07f) {
-    q = rintf(__fdiv_rn(v, s));
-  }
-  q = fminf(fmaxf(q, -127.f), 127.f);
-  return static_cast<uint32_t>(static_cast<int>(q)) & 0xffu;
-}
-
-__device__ __forceinline__ uint32_t quant4(const float4& f, float s, float r, bool fast) {
-  if (fast) return quant_lane(f.x, s, r) | (quant_lane(f.y, s, r) << 8) | (quant_lane(f.z, s, r) << 16) | (quant_lane(f.w, s, r) << 24);
-  uint32_t w = 0;
-  const float v[4] = {f.x, f.y, f.z, f.w};
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    float q = 0.f;
-    if (s != 0.f) q = fminf(fmaxf(rintf(__fdiv_rn(v[e], s)), -127.f), 127.f);
-    w |= (static_cast<uint32_t>(static_cast<int>(q)) & 0xffu) << (8 * e);
-  }
-  return w;
-}
-
 __global__ void __launch_bounds__(kQThreads) act_quantize_flat_kernel(const float4* __restrict__ x, int64_t n4,
                                                                       uint32_t* __restrict__ xq, const uint32_t* ws,
                                                                       const float* static_scale, float* sx_out, int* status) {
@@ -176,8 +144,7 @@ __global__ void __launch_bounds__(kQThreads) act_quantize_flat_kernel(const floa
     if (mbits >= 0x7f800000u) raise_status(status, PIPE_ERR_NONFINITE);
     if (static_scale && !(s >= 0.f && s < __uint_as_float(0x7f800000u))) raise_status(status, PIPE_ERR_INVALID_ARG);
   }
-  // the estimate needs a reciprocal that neither overflows nor is subnormal
-  const bool fast = s >= 1e-30f && s <= 1e30f;
+  const bool fast = quant_step_is_fast(s);
   const float r = fast ? __frcp_rn(s) : 0.f;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
   int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;

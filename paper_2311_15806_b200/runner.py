@@ -118,6 +118,23 @@ class LayerRunner:
             sx = [self.sx[m if n > 1 else 0] for m in range(self.M)]
             B.pipe_ensemble_forward(self.desc, blob, xq, sx, self.y, None, False, partials)
 
+    def forward_q8(self, out_scale: list, relu: bool = True, blob: torch.Tensor | None = None) -> list:
+        """The layer as an inner layer of the predictors: int8 outputs Q(sigma(y_m)) with the static steps
+        ``out_scale`` (M one-element cuda float32 tensors); no fp32 output is written.  Returns the M outputs."""
+        blob = self.blob if blob is None else blob
+        if not hasattr(self, "yq"):
+            self.yq = [torch.empty(tuple(y.shape), dtype=torch.int8, device=self.device) for y in self.y]
+        if self.geom is not None:
+            N, H, W_, C = self.spec.conv[:4]
+            B.pipe_expanded_conv2d_q8(self.desc, self.geom, blob, self.xq[0].view(N, H, W_, C), self.sx[0], out_scale[0],
+                                      self.yq[0], None, relu)
+            return self.yq
+        n = len(self.xq)
+        xq = [self.xq[m if n > 1 else 0] for m in range(self.M)]
+        sx = [self.sx[m if n > 1 else 0] for m in range(self.M)]
+        B.pipe_ensemble_forward_q8(self.desc, blob, xq, sx, out_scale, self.yq, None, relu)
+        return self.yq
+
     def blob_copies(self, min_total_bytes: int) -> list:
         """The expanded blob plus enough byte copies of it that together they exceed
         ``min_total_bytes`` (for timing loops that must not re-read weights from L2)."""

@@ -113,6 +113,30 @@ def gpu_ensemble(layer, xq_m, sx_m, bias=None, sum_branches=False, want_partials
     return [y.cpu().numpy() for y in ys], (None if part is None else part.cpu().numpy())
 
 
+def gpu_ensemble_q8(layer, xq_m, sx_m, out_scales, bias=None, relu=True, want_partials=True, kernel=B.KERNEL_AUTO,
+                    pitch_extra=0):
+    """Inner layer of the M predictors through pipe_ensemble_forward_q8; out_scales: M floats.  Returns the M
+    int8 outputs (numpy) and the partials.  pitch_extra > 0 gives the outputs a row pitch of O + pitch_extra."""
+    M = layer.desc.num_branches
+    T = xq_m[0].shape[0]
+    O = layer.desc.out_features
+    bufs = [torch.full((T, O + pitch_extra), 99, dtype=torch.int8, device="cuda") for _ in range(M)]
+    yq = [b[:, :O] for b in bufs]
+    so = [torch.tensor([s], dtype=torch.float32, device="cuda") for s in out_scales]
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
+    bd = None if bias is None else torch.from_numpy(bias).cuda()
+    B.pipe_select_kernel(kernel)
+    try:
+        B.pipe_ensemble_forward_q8(layer.desc, layer.blob, xq_m, sx_m, so, yq, bd, relu, part)
+        torch.cuda.synchronize()
+    finally:
+        B.pipe_select_kernel(B.KERNEL_AUTO)
+    if pitch_extra:
+        for b in bufs:
+            assert (b[:, O:] == 99).all(), "bytes beyond the row were written"
+    return [y.cpu().numpy() for y in yq], (None if part is None else part.cpu().numpy())
+
+
 def assert_outputs_close(y_gpu: np.ndarray, f, what=""):
     """f: oracle Forward (y, y64, yabs).  The stated tolerance, element-wise, against the binary64 sum."""
     err = np.abs(y_gpu.astype(np.float64) - f.y64)

@@ -403,3 +403,31 @@ def test_accumulator_overflow_is_detected(oracle):
     with pytest.raises(oracle.OracleError) as ei:
         oracle.forward(e, xq, 1.0)
     assert ei.value.code == oracle.ERR_ACC_OVERFLOW
+
+
+def test_requantized_branch_is_the_composition_and_a_two_layer_chain_closes(oracle):
+    """Sec. 3.2 / App. B: a branch of an inner layer hands sigma(its cluster's output), quantized by the next
+    layer's Q, to the same branch of the next layer.  The helper is the composition of the pinned pieces, and
+    with every order in one branch and codes that reproduce the weights exactly the two-layer chain equals the
+    plain integer network computed with NumPy."""
+    rng = np.random.default_rng(3)
+    O1, I1, O2, T = 24, 16, 8, 9
+    # weights that one 8-bit order represents exactly: s * integers with a full-range entry per row
+    q1 = rng.integers(-127, 128, size=(O1, I1)); q1[:, 0] = 127
+    q2 = rng.integers(-127, 128, size=(O2, O1)); q2[:, 0] = -127
+    s1, s2 = np.float32(2.0 ** -9), np.float32(2.0 ** -7)
+    W1, W2 = (q1 * s1).astype(np.float32), (q2 * s2).astype(np.float32)
+    e1, e2 = oracle.expand(W1, 8, 1, 8, O1 // 8), oracle.expand(W2, 8, 1, 8, O2 // 8)
+    xq = rng.integers(-127, 128, size=(T, I1)).astype(np.int8)
+    sx, s_mid = np.float32(2.0 ** -6), np.float32(2.0 ** -3)
+    hq = oracle.forward_requantized(e1, xq, sx, float(s_mid))
+    # composition
+    y1 = oracle.forward(e1, xq, sx).y
+    want, _ = oracle.quantize_act(np.maximum(y1, 0), static_scale=float(s_mid))
+    np.testing.assert_array_equal(hq, want)
+    # plain integer network: every product below is a power-of-two multiple of an integer, exact in binary64
+    a1 = (xq.astype(np.int64) @ q1.T).astype(np.float64) * float(s1) * float(sx)
+    h_int = np.clip(np.rint(np.maximum(a1, 0) / float(s_mid)), -127, 127).astype(np.int64)
+    np.testing.assert_array_equal(hq.astype(np.int64), h_int)
+    y2 = oracle.forward(e2, hq, s_mid).y
+    np.testing.assert_array_equal(y2.astype(np.float64), (h_int @ q2.T).astype(np.float64) * float(s2) * float(s_mid))
