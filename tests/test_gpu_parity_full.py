@@ -5,7 +5,9 @@ Weight expansion is compared with the oracle in full (every code, scale and kept
 contraction is too large for the CPU at these sizes, so int32 partial sums and fp32 outputs are
 compared on sampled token rows (first/last rows, both sides of tile boundaries, seeded random rows)
 for ALL output channels and orders; between the samples the tensor-core kernel is cross-checked in
-full against the CUDA-core kernel, which shares neither its code layout nor its tiling."""
+full against the CUDA-core kernel, which shares neither its code layout nor its tiling.  The inner-layer
+form (int8 output) is checked the same way: sampled rows against the oracle, every element against the
+quantizer kernel applied to the pinned fp32 output."""
 import numpy as np
 import pytest
 import torch
@@ -74,6 +76,30 @@ def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_chec
             H.assert_outputs_close(y, f, f"{sp.name} T={run.T} branch {m}")
             np.testing.assert_array_equal(y.view(np.uint32), f.y.view(np.uint32))
             k0 += split[m]
+        # inner-layer form of the same launch (activation function and the next layer's input quantizer fused into
+        # the epilogue): the oracle on the sampled rows, and every element against ReLU + the quantizer kernel
+        # applied to the fp32 output that the lines above have just pinned
+        steps = [(y.clamp_min(0).max() * (0.5 / 127)).reshape(1).float() for y in run.y]
+        yq = run.forward_q8(steps, relu=True)
+        torch.cuda.synchronize()
+        assert B.pipe_poll_status() == B.PIPE_OK
+        k0 = 0
+        for m in range(sp.M):
+            i = m if len(xs_rows) > 1 else 0
+            step = float(steps[m].cpu())
+            xq_o, _ = oracle.quantize_act(xs_rows[i], static_scale=float(sx_full[i]))
+            want = oracle.forward_requantized(e, xq_o, sx_full[i], step, k0, k0 + split[m], relu=True)
+            np.testing.assert_array_equal(yq[m][rows_t].cpu().numpy(), want)
+            assert int(yq[m].max()) == 127 and int(yq[m].min()) == 0     # the step clamps the largest outputs; ReLU
+            a = run.y[m].clamp_min(0)
+            full, _ = H.gpu_quantize(None, static_scale=step, xd=a)
+            assert torch.equal(yq[m], full)
+            del a, full
+            k0 += split[m]
+        del yq
+        if hasattr(run, "yq"):
+            del run.yq
+        torch.cuda.empty_cache()
         if run.geom is not None:
             # implicit GEMM vs the same layer on explicitly lowered rows (and that one vs the CUDA-core kernel)
             y_conv = run.y[0].clone()
