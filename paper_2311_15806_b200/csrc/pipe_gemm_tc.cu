@@ -747,10 +747,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
     const int my_tiles = (p.num_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const uint32_t total_steps = static_cast<uint32_t>(my_tiles) * p.kblocks;
     const uint32_t P = min(static_cast<uint32_t>(kALanes), depth);
-    if (static_cast<uint32_t>(lane) < P) {
-      RingPos rp{static_cast<uint32_t>(lane), 0};
-      int tile = blockIdx.x, kb = lane;
-      for (uint32_t it = lane; it < total_steps; it += P, rp.advance(P, depth), kb += P) {
+    // The boxes of one step of the implicit convolution (2 * tpt patches) are issued by as many lanes side by
+    // side: one lane issuing them in turn would deliver the step a thousand cycles later.
+    const uint32_t nb = p.f.conv_on ? 2u * p.tpt : 1u;
+    const uint32_t sl = static_cast<uint32_t>(lane) / nb, hb = static_cast<uint32_t>(lane) % nb;
+    if (sl < P) {
+      RingPos rp{sl, 0};
+      int tile = blockIdx.x, kb = sl;
+      for (uint32_t it = sl; it < total_steps; it += P, rp.advance(P, depth), kb += P) {
         while (kb >= p.kblocks) {
           kb -= p.kblocks;
           tile += gridDim.x;
@@ -758,7 +762,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
         const int tt = tile % p.ntt;
         const int m = tile / p.ntt / p.ncb;
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
-        mbar_expect_tx(g.a_full0 + 8u * rp.slot, p.a_bytes);
+        // (a box of another lane may land before this: the transaction count may run ahead of the expectation,
+        // and the phase cannot complete before the one pending arrival, which is this instruction)
+        if (hb == 0) mbar_expect_tx(g.a_full0 + 8u * rp.slot, p.a_bytes);
         if (!p.f.conv_on) {
           // one box of tpt * 128 token rows; rows beyond T read zeros
           tma_load_2d(g.stage0 + rp.slot * p.stage_bytes, &p.tmap_a[m], kb * kKStep, tt * p.tpt * kTileM, g.a_full0 + 8u * rp.slot);
@@ -766,12 +772,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
           // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
           const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
           const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
-          for (int half = 0; half < 2 * p.tpt; ++half) {
-            int n, h0, w0;
-            patch_origin(p, 2 * p.tpt * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-            tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
-                        n, g.a_full0 + 8u * rp.slot);
-          }
+          const int half = static_cast<int>(hb);
+          int n, h0, w0;
+          patch_origin(p, 2 * p.tpt * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
+          tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
+                      n, g.a_full0 + 8u * rp.slot);
         }
       }
     }
