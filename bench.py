@@ -103,7 +103,7 @@ def workload_spec(name: str):
 
 # ------------------------------------------------------------------------------------------------
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("cfg2", "forward"): 27.795200e6 + 49.864704e6,      # profiles/ncu_tc_forward_kernel_cfg2.txt
+    ("cfg2", "forward"): 27.573504e6 + 49.119488e6,      # profiles/ncu_tc_forward_kernel_cfg2.txt
     ("cfg4a_t16", "forward"): 56.678656e6 + 0.802048e6,  # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
 }
 
