@@ -113,6 +113,39 @@ int32_t pipe_keep_groups_from_gamma(int32_t num_groups, double gamma);
  * [4,4], [3,3,2], [2,2,2,2] and [2,2].  h_out: M ints. */
 pipe_status pipe_default_branches(int32_t num_orders, int32_t num_branches, int32_t* h_out);
 
+/* Appendix H (operation head-count).  A d x d convolution with stride s on D x D x n_i feature maps
+ * and n_o outputs; a fully connected layer is d = D = s = 1.  A b-digit multiplication is counted
+ * as b*log2(b) bit operations (the appendix leaves the base of the logarithm open; every term
+ * carries one, so ratios and the order bound below do not depend on it). */
+typedef struct {
+  int32_t kernel_size;   /* d */
+  int32_t feature_size;  /* D */
+  int32_t in_channels;   /* n_i */
+  int32_t out_channels;  /* n_o */
+  int32_t stride;        /* s */
+} pipe_op_shape;
+
+/* O_original = D^2 d^2 n_i n_o / s^2 * 32 log2(32): the fp32 layer.  Returns a negative value for
+ * an invalid shape (any field < 1).  Pure host functions, no CUDA call. */
+double pipe_bit_ops_original(const pipe_op_shape* shape);
+
+/* O_R(k) = D^2 [ (n_i + n_o / s^2) * 32 log2(32) + k * d^2 n_i n_o / s^2 * b log2(b) ]: the two
+ * rescalings plus k int-b products.  `orders` is the number of full orders the layer evaluates;
+ * a group-sparse expansion (Sec. 3.1) counts as 1 + (K - 1) * gamma of them, so the argument is a
+ * double.  bits in 2..32, orders >= 0; a negative value is returned otherwise. */
+double pipe_bit_ops_expanded(const pipe_op_shape* shape, int32_t weight_bits, double orders);
+
+/* The largest whole number of orders whose operation count does not exceed the fp32 layer's
+ * ("the maximum order of expansion before which the number of operations exceeds the baseline",
+ * Appendix H); 0 when even one order does, -1 for invalid arguments. */
+int32_t pipe_max_orders_within_original(const pipe_op_shape* shape, int32_t weight_bits);
+
+/* Sec. 3.1 / 4.3, Appendix A: a budget beta ("150 %" = 1.5, "beta = 7 and order K = 8") is the
+ * number of full orders a sparse expansion of K orders costs, beta = 1 + (K - 1) * gamma.  Writes
+ * the kept fraction gamma of the orders >= 2.  PIPE_ERR_INVALID_ARG unless 1 <= beta <= K and
+ * K >= 1 (K = 1 admits beta = 1 only, gamma = 1). */
+pipe_status pipe_gamma_from_budget(double beta, int32_t num_orders, double* h_gamma);
+
 /* Validates `desc` and fills `h_out`.  Pure host function, no CUDA call. */
 pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out);
 

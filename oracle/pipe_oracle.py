@@ -236,3 +236,22 @@ def balanced_split(K: int, M: int) -> np.ndarray:
 
 def keep_groups(G: int, gamma: float) -> int:
     return int(lib().pipe_oracle_keep_groups(G, float(gamma)))
+
+
+# ---- Appendix H (operation head-count) and the budget of Sec. 3.1 / 4.3: closed forms, written out
+def bit_ops_original(d: int, D: int, n_i: int, n_o: int, s: int) -> float:
+    """O_original = D^2 * d^2 n_i n_o / s^2 * 32 log 32 (Appendix H); log to base 2."""
+    import math
+    return D ** 2 * (d ** 2 * n_i * n_o / s ** 2) * 32.0 * math.log2(32.0)
+
+
+def bit_ops_expanded(d: int, D: int, n_i: int, n_o: int, s: int, bits: int, orders: float) -> float:
+    """O_R(k) = D^2 [ (n_i + n_o / s^2) 32 log 32 + k d^2 n_i n_o / s^2 b log b ] (Appendix H)."""
+    import math
+    return D ** 2 * ((n_i + n_o / s ** 2) * 32.0 * math.log2(32.0)
+                     + orders * (d ** 2 * n_i * n_o / s ** 2) * bits * math.log2(bits))
+
+
+def budget_of(K: int, gamma: float) -> float:
+    """Full orders a group-sparse expansion costs: order 1 dense, K - 1 orders at kept fraction gamma."""
+    return 1.0 + (K - 1) * gamma

@@ -28,6 +28,7 @@ KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM, KERNEL_TCGEN05_PAI
 STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
+           "pipe_bit_ops_original", "pipe_bit_ops_expanded", "pipe_max_orders_within_original", "pipe_gamma_from_budget",
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
            "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
@@ -114,6 +115,42 @@ def _stream_ptr(stream) -> int:
 
 def _dp(t) -> int | None:
     return None if t is None else int(t.data_ptr())
+
+
+class OpShape(C.Structure):
+    _fields_ = [("kernel_size", C.c_int32), ("feature_size", C.c_int32), ("in_channels", C.c_int32),
+                ("out_channels", C.c_int32), ("stride", C.c_int32)]
+
+
+def _op_shape(d: int, D: int, n_i: int, n_o: int, s: int) -> OpShape:
+    return OpShape(int(d), int(D), int(n_i), int(n_o), int(s))
+
+
+def pipe_bit_ops_original(d: int, D: int, n_i: int, n_o: int, s: int) -> float:
+    L = lib()
+    L.pipe_bit_ops_original.restype = C.c_double
+    return float(L.pipe_bit_ops_original(C.byref(_op_shape(d, D, n_i, n_o, s))))
+
+
+def pipe_bit_ops_expanded(d: int, D: int, n_i: int, n_o: int, s: int, bits: int, orders: float) -> float:
+    L = lib()
+    L.pipe_bit_ops_expanded.restype = C.c_double
+    L.pipe_bit_ops_expanded.argtypes = [C.c_void_p, C.c_int32, C.c_double]
+    return float(L.pipe_bit_ops_expanded(C.byref(_op_shape(d, D, n_i, n_o, s)), int(bits), float(orders)))
+
+
+def pipe_max_orders_within_original(d: int, D: int, n_i: int, n_o: int, s: int, bits: int) -> int:
+    L = lib()
+    L.pipe_max_orders_within_original.restype = C.c_int32
+    return int(L.pipe_max_orders_within_original(C.byref(_op_shape(d, D, n_i, n_o, s)), int(bits)))
+
+
+def pipe_gamma_from_budget(beta: float, K: int) -> float:
+    L = lib()
+    L.pipe_gamma_from_budget.argtypes = [C.c_double, C.c_int32, C.c_void_p]
+    out = C.c_double(0.0)
+    _check(L.pipe_gamma_from_budget(float(beta), int(K), C.byref(out)), "pipe_gamma_from_budget")
+    return float(out.value)
 
 
 def pipe_keep_groups_from_gamma(num_groups: int, gamma: float) -> int:

@@ -126,6 +126,42 @@ pipe_status pipe_default_branches(int32_t K, int32_t M, int32_t* h_out) {
   return PIPE_OK;
 }
 
+static bool shape_ok(const pipe_op_shape* sh) {
+  return sh && sh->kernel_size >= 1 && sh->feature_size >= 1 && sh->in_channels >= 1 && sh->out_channels >= 1 && sh->stride >= 1;
+}
+// products per output position summed over the layer: D^2 d^2 n_i n_o / s^2
+static double products_of(const pipe_op_shape* sh) {
+  const double D = sh->feature_size, d = sh->kernel_size, s = sh->stride;
+  return D * D * d * d * static_cast<double>(sh->in_channels) * static_cast<double>(sh->out_channels) / (s * s);
+}
+static double digit_cost(int bits) { return static_cast<double>(bits) * std::log2(static_cast<double>(bits)); }
+
+double pipe_bit_ops_original(const pipe_op_shape* shape) {
+  if (!shape_ok(shape)) return -1.0;
+  return products_of(shape) * digit_cost(32);
+}
+
+double pipe_bit_ops_expanded(const pipe_op_shape* shape, int32_t weight_bits, double orders) {
+  if (!shape_ok(shape) || weight_bits < 2 || weight_bits > 32 || !(orders >= 0.0)) return -1.0;
+  const double D = shape->feature_size, s = shape->stride;
+  const double rescale = D * D * (static_cast<double>(shape->in_channels) + static_cast<double>(shape->out_channels) / (s * s)) * digit_cost(32);
+  return rescale + orders * products_of(shape) * digit_cost(weight_bits);
+}
+
+int32_t pipe_max_orders_within_original(const pipe_op_shape* shape, int32_t weight_bits) {
+  if (!shape_ok(shape) || weight_bits < 2 || weight_bits > 32) return -1;
+  const double budget = pipe_bit_ops_original(shape);
+  int32_t k = 0;
+  while (k < (1 << 20) && pipe_bit_ops_expanded(shape, weight_bits, static_cast<double>(k + 1)) <= budget) ++k;
+  return k;
+}
+
+pipe_status pipe_gamma_from_budget(double beta, int32_t K, double* h_gamma) {
+  if (!h_gamma || K < 1 || K > PIPE_MAX_ORDERS || !(beta >= 1.0) || beta > static_cast<double>(K)) return PIPE_ERR_INVALID_ARG;
+  *h_gamma = K == 1 ? 1.0 : (beta - 1.0) / static_cast<double>(K - 1);
+  return PIPE_OK;
+}
+
 pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
   if (!h_out) return PIPE_ERR_INVALID_ARG;
   LayerInfo L;
