@@ -39,7 +39,7 @@ typedef enum {
   PIPE_ERR_UNSUPPORTED = 4,  /* valid request the library has no kernel for */
   PIPE_ERR_WORKSPACE = 5,    /* blob / workspace smaller than pipe_layout says */
   PIPE_ERR_NONFINITE = 6,    /* device saw NaN or Inf in weights or activations */
-  PIPE_ERR_ACC_OVERFLOW = 7, /* in_features so large that an int32 partial sum could overflow */
+  PIPE_ERR_ACC_OVERFLOW = 7, /* in_features so large that an int32 accumulator could overflow (see pipe_expanded_linear) */
   PIPE_ERR_TIMEOUT = 8,      /* a bounded wait inside a kernel ran out */
   PIPE_ERR_CUDA = 9          /* a CUDA runtime/driver call failed (no device, launch error) */
 } pipe_status;
@@ -135,9 +135,9 @@ double pipe_bit_ops_original(const pipe_op_shape* shape);
  * double.  bits in 2..32, orders >= 0; a negative value is returned otherwise. */
 double pipe_bit_ops_expanded(const pipe_op_shape* shape, int32_t weight_bits, double orders);
 
-/* The largest whole number of orders whose operation count does not exceed the fp32 layer's
- * ("the maximum order of expansion before which the number of operations exceeds the baseline",
- * Appendix H); 0 when even one order does, -1 for invalid arguments. */
+/* The largest whole number of orders whose operation count does not exceed the fp32 layer's: the
+ * order bound Appendix H derives from its two counts; 0 when even one order does, -1 for invalid
+ * arguments. */
 int32_t pipe_max_orders_within_original(const pipe_op_shape* shape, int32_t weight_bits);
 
 /* Sec. 3.1 / 4.3, Appendix A: a budget beta ("150 %" = 1.5, "beta = 7 and order K = 8") is the
@@ -186,7 +186,10 @@ pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const float* d_W, i
  *   - Limit: the layer's expand_ws_bytes (see pipe_layout; about 4*O*I bytes) must not exceed
  *     PIPE_STATIC_SCRATCH_BYTES, otherwise PIPE_ERR_WORKSPACE is returned and nothing is queued.
  *   - The first call on each device looks up the array's device address (that device must be
- *     current, as for every call here).  Make that first call before any stream capture begins.
+ *     current, as for every call here); under lazy module loading the driver may also load the
+ *     module that holds the array at that moment.  Make that first call before any stream capture
+ *     begins and before the application freezes its memory budget; from the second call on
+ *     nothing is looked up or loaded.
  *   - All calls share the one array.  It keeps whatever the previous call left in it; this call
  *     overwrites every part before reading it, so nothing needs clearing.  Two calls whose GPU
  *     work overlaps (different streams, or different host threads) race on the array: run them
@@ -217,7 +220,9 @@ pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I, int64_t ld
  * d_xq: int8 [T, I] pitch ldxq; d_sx: 1 float; d_bias: float [O] or NULL;
  * d_y: float [T, O] pitch ldy.  d_partials (NULL, or int32 [T, total_rows]): when given,
  * receives acc_k[t, row] at column (sum_{j<k} rows[j]) + compacted row.  T = 0 is a no-op.
- * PIPE_ERR_ACC_OVERFLOW if 127 * qmax * I >= 2^31.
+ * PIPE_ERR_ACC_OVERFLOW (from every call that takes the descriptor, pipe_layout included) if
+ * 127 * qmax * 2^(8-b) * I >= 2^31, i.e. beyond I = 133144 (b = 8), 150976 (b = 4), 264208 (b = 2): the
+ * kernels hold sub-byte codes as code * 2^(8-b) in their int32 accumulators.
  */
 pipe_status pipe_expanded_linear(const pipe_layer_desc* desc, const void* d_blob, const int8_t* d_xq, int64_t T,
                                  int64_t ldxq, const float* d_sx, const float* d_bias, float* d_y, int64_t ldy,

@@ -273,8 +273,8 @@ int pipe_oracle_quantize_act(const float* x, int64_t T, int64_t I, int64_t ldx, 
 }
 
 /* ---------------------------------------------------------------------------------------
- * Appendix B, Eq. 9 restricted to one cluster of successive orders (Sec. 3.2; Appendix B,
- * "the m-th predictor corresponds to the residuals at orders sum_{l<m} K_l + i"):
+ * Appendix B, Eq. 9 restricted to one cluster of successive orders (Sec. 3.2; Appendix B:
+ * predictor m owns the K_m orders that come right after the clusters of predictors 1..m-1):
  *
  *   acc_k[t, o] = sum_i xq[t,i] * q_k[o,i]                       (exact integers)
  *   y[t, o]     = sum over k = k_begin..k_end-1 ascending, o kept at order k, of

@@ -46,8 +46,10 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
   L.qmax = (1 << (L.bits - 1)) - 1;
   if (L.n_keep < 1 || L.n_keep > L.G) return PIPE_ERR_INVALID_ARG;
   if (L.M < 1 || L.M > L.K) return PIPE_ERR_SHAPE;
-  // int32 partial sums: |acc| <= 127 * qmax * I must stay below 2^31 (Eq. 9 is exact integer work).
-  if (static_cast<int64_t>(127) * L.qmax * L.I >= (static_cast<int64_t>(1) << 31)) return PIPE_ERR_ACC_OVERFLOW;
+  // int32 partial sums (Eq. 9 is exact integer work).  The tensor-core and decode kernels accumulate sub-byte
+  // codes as code * 2^(8-b) and shift back at the end, so the bound that keeps every kernel exact is
+  // 127 * qmax * 2^(8-b) * I < 2^31: I <= 133144 (b = 8), 150976 (b = 4), 264208 (b = 2).
+  if ((static_cast<int64_t>(127) * L.qmax * L.I << (8 - L.bits)) >= (static_cast<int64_t>(1) << 31)) return PIPE_ERR_ACC_OVERFLOW;
 
   int32_t bo[PIPE_MAX_ORDERS] = {0};
   bool all_zero = true;

@@ -90,6 +90,20 @@ def test_bad_descriptors_are_rejected(lib, kwargs, status):
     assert ei.value.status == status
 
 
+@pytest.mark.parametrize("bits,last_ok", [(8, 133144), (4, 150976), (2, 264208)])
+def test_accumulator_bound_sits_where_the_scaled_codes_put_it(lib, bits, last_ok):
+    # the kernels hold sub-byte codes as code * 2^(8-b): 127 * qmax * 2^(8-b) * I must stay below 2^31
+    qmax = (1 << (bits - 1)) - 1
+    per_byte = 8 // bits
+    ok = last_ok // per_byte * per_byte
+    bad = ok + per_byte
+    assert 127 * qmax * (1 << (8 - bits)) * ok < 2 ** 31 <= 127 * qmax * (1 << (8 - bits)) * (last_ok + 1)
+    B.pipe_layout(B.make_desc(8, ok, bits, 1, 8, 1, 1))
+    with pytest.raises(B.PipeError) as ei:
+        B.pipe_layout(B.make_desc(8, bad, bits, 1, 8, 1, 1))
+    assert ei.value.status == B.PIPE_ERR_ACC_OVERFLOW
+
+
 def test_explicit_branch_orders(lib):
     lay = B.pipe_layout(B.make_desc(64, 64, 4, 4, 8, 4, 2, [3, 1]))
     assert [lay.branch_orders[m] for m in range(2)] == [3, 1]

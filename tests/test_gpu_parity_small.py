@@ -256,7 +256,7 @@ def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
     np.testing.assert_array_equal(part, f.partials)
     y_o, _ = oracle.ensemble(e, np.stack([qo[0][0]] * M), [qo[0][1]] * M, split, bias=bias, sum_branches=True)
     np.testing.assert_array_equal(ys[0].view(np.uint32), y_o.view(np.uint32))
-    assert (np.abs(ys[0] - f.y64) <= 2e-5 * f.yabs + 1e-30).all()
+    assert (np.abs(ys[0] - f.y64) <= H.REL_TOL * f.yabs + 1e-30).all()
 
 
 def test_forward_zero_tokens_and_strided_io(oracle):

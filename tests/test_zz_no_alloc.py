@@ -6,12 +6,16 @@ streams that are serving requests while a layer's weights are being swapped.  Fo
 carries a fixed internal workspace.  This test calls that entry point through the C ABI twice in a
 row (the second call finds the first call's leftovers in the shared workspace) and requires the
 blob to be byte-identical to the one the ordinary entry point writes into caller-provided
-workspace -- the expansion is integer/bit-exact work, so the tolerance is zero.  It also checks
-that a layer beyond the fixed size is refused.  Collected last on purpose."""
+workspace -- the expansion is integer/bit-exact work, so the tolerance is zero -- and to match the
+CPU oracle's expansion.  After a warm-up call (the first call on a device may make the driver load the
+module that holds the fixed array) a further call must leave the device's free memory and the
+allocator's counters exactly where they were: that is the promise the entry point exists for.  It also
+checks that a layer beyond the fixed size is refused.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import pipe_oracle as O
 from paper_2311_15806_b200 import binding as B
 from tests import gpu_harness as H
 
@@ -51,6 +55,26 @@ def test_static_workspace_expansion_matches_the_ordinary_one_twice():
         for a, b in zip(_blob_sections(desc, got), _blob_sections(desc, want)):
             np.testing.assert_array_equal(a, b)
         assert torch.equal(got, want)
+        H.assert_expansion_matches(B.ExpandedLayer(desc, lay, got), O.expand(W, bits, K, g, n_keep), O)
+
+
+def test_static_workspace_call_allocates_nothing():
+    H.ensure_built()
+    rng = np.random.default_rng(7)
+    O_, I, bits, K, g, n_keep = 128, 640, 4, 3, 8, 4
+    W = torch.from_numpy((rng.standard_normal((O_, I)) * 0.02).astype(np.float32)).cuda()
+    desc = B.make_desc(O_, I, bits, K, g, n_keep)
+    blob = B.alloc_bytes(B.pipe_layout(desc).blob_bytes)
+    B.pipe_expand_weights_static(desc, W, blob)     # warm-up: address look-up, module load
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    B.pipe_expand_weights_static(desc, W, blob)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, "device memory changed across a call that must not allocate"
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert B.pipe_poll_status() == B.PIPE_OK
 
 
 def test_static_workspace_refuses_a_layer_that_does_not_fit():
