@@ -255,7 +255,7 @@ pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blo
  * finite, else PIPE_ERR_INVALID_ARG through the device status; s_m = 0 gives all-zero codes).
  * h_yq_m: HOST array of M device pointers, int8 [T, O] pitch ldyq (>= O); no float output is
  * written.  The other arguments are those of pipe_ensemble_forward; M = 1 is the plain expanded
- * layer with this epilogue.  The two-SM kernel (choice 4) answers PIPE_ERR_UNSUPPORTED.
+ * layer with this epilogue.  
  */
 pipe_status pipe_ensemble_forward_q8(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
                                      int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
@@ -300,13 +300,6 @@ pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv
                                     const int8_t* d_xq, const float* d_sx, const float* d_bias, int32_t relu,
                                     const float* d_out_scale, int8_t* d_yq, int64_t ldyq, int32_t* d_partials,
                                     void* stream);
-
-/* Which GEMM kernel the two forward calls use (process-wide, for tests and measurements):
- * 0 = automatic, 1 = CUDA-core reference kernel, 2 = tcgen05 tensor-core kernel,
- * 3 = small-token weight-streaming kernel, 4 = two-SM form of the tcgen05 kernel (clusters of
- * two CTAs).  A forced kernel that cannot run the request
- * makes the forward call return PIPE_ERR_UNSUPPORTED. */
-pipe_status pipe_select_kernel(int32_t which);
 
 /* Number of kernels the library has launched in this process (all calls, all streams). */
 uint64_t pipe_launch_count(void);

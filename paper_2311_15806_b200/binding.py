@@ -32,8 +32,9 @@ EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout"
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
            "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
-           "pipe_select_kernel",
-           "pipe_launch_count", "pipe_poll_status", "pipe_status_string"]
+           "pipe_launch_count", "pipe_poll_status", "pipe_status_string",
+           # include/pipe_diag.h: tests and measurements only
+           "pipe_diag_select_kernel", "pipe_diag_mma_i8_rate", "pipe_diag_bounded_wait"]
 
 
 class LayerDesc(C.Structure):
@@ -93,7 +94,9 @@ def lib() -> C.CDLL:
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
         L.pipe_ensemble_forward_q8.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, i32, p, p, i64, p, p]
         L.pipe_expanded_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
-        L.pipe_select_kernel.argtypes = [i32]
+        L.pipe_diag_select_kernel.argtypes = [i32]
+        L.pipe_diag_mma_i8_rate.argtypes = [i32, i64, C.POINTER(C.c_double), p]
+        L.pipe_diag_bounded_wait.argtypes = [i64, p]
         L.pipe_launch_count.restype = C.c_uint64
         L.pipe_poll_status.argtypes = [p, C.POINTER(i32)]
         L.pipe_status_string.argtypes = [C.c_int]
@@ -272,8 +275,19 @@ def pipe_ensemble_forward_q8(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, ou
                                           ldyq, _dp(partials), _stream_ptr(stream)), "pipe_ensemble_forward_q8")
 
 
-def pipe_select_kernel(which: int) -> None:
-    _check(lib().pipe_select_kernel(which), "pipe_select_kernel")
+def pipe_diag_select_kernel(which: int) -> None:
+    _check(lib().pipe_diag_select_kernel(which), "pipe_diag_select_kernel")
+
+
+def pipe_diag_mma_i8_rate(n_cols: int, mma_per_cta: int, stream=None) -> float:
+    """Queues the issue-rate probe of the integer tensor pipe; returns the integer operations of the launch."""
+    ops = C.c_double(0.0)
+    _check(lib().pipe_diag_mma_i8_rate(int(n_cols), int(mma_per_cta), C.byref(ops), _stream_ptr(stream)), "pipe_diag_mma_i8_rate")
+    return float(ops.value)
+
+
+def pipe_diag_bounded_wait(limit_cycles: int, stream=None) -> None:
+    _check(lib().pipe_diag_bounded_wait(int(limit_cycles), _stream_ptr(stream)), "pipe_diag_bounded_wait")
 
 
 def pipe_launch_count() -> int:

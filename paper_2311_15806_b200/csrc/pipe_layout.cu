@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "pipe_common.cuh"
+#include "pipe_diag.h"
 
 namespace pipe {
 
@@ -173,7 +174,7 @@ pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
   return PIPE_OK;
 }
 
-pipe_status pipe_select_kernel(int32_t which) {
+pipe_status pipe_diag_select_kernel(int32_t which) {
   if (which < 0 || which > 4) return PIPE_ERR_INVALID_ARG;
   g_kernel_choice.store(which);
   return PIPE_OK;

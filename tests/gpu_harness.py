@@ -85,12 +85,12 @@ def gpu_linear(layer, xq, sx, bias=None, want_partials=True, kernel=B.KERNEL_AUT
     y = torch.full((T, layer.desc.out_features), float("nan"), dtype=torch.float32, device="cuda")
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
     bd = None if bias is None else torch.from_numpy(bias).cuda()
-    B.pipe_select_kernel(kernel)
+    B.pipe_diag_select_kernel(kernel)
     try:
         B.pipe_expanded_linear(layer.desc, layer.blob, xq, sx, y, bd, part)
         torch.cuda.synchronize()
     finally:
-        B.pipe_select_kernel(B.KERNEL_AUTO)
+        B.pipe_diag_select_kernel(B.KERNEL_AUTO)
     assert B.pipe_poll_status() == B.PIPE_OK
     return y.cpu().numpy(), (None if part is None else part.cpu().numpy())
 
@@ -103,12 +103,12 @@ def gpu_ensemble(layer, xq_m, sx_m, bias=None, sum_branches=False, want_partials
     ys = [torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda") for _ in range(n_out)]
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
     bd = None if bias is None else torch.from_numpy(bias).cuda()
-    B.pipe_select_kernel(kernel)
+    B.pipe_diag_select_kernel(kernel)
     try:
         B.pipe_ensemble_forward(layer.desc, layer.blob, xq_m, sx_m, ys, bd, sum_branches, part)
         torch.cuda.synchronize()
     finally:
-        B.pipe_select_kernel(B.KERNEL_AUTO)
+        B.pipe_diag_select_kernel(B.KERNEL_AUTO)
     assert B.pipe_poll_status() == B.PIPE_OK
     return [y.cpu().numpy() for y in ys], (None if part is None else part.cpu().numpy())
 
@@ -125,12 +125,12 @@ def gpu_ensemble_q8(layer, xq_m, sx_m, out_scales, bias=None, relu=True, want_pa
     so = [torch.tensor([s], dtype=torch.float32, device="cuda") for s in out_scales]
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda") if want_partials else None
     bd = None if bias is None else torch.from_numpy(bias).cuda()
-    B.pipe_select_kernel(kernel)
+    B.pipe_diag_select_kernel(kernel)
     try:
         B.pipe_ensemble_forward_q8(layer.desc, layer.blob, xq_m, sx_m, so, yq, bd, relu, part)
         torch.cuda.synchronize()
     finally:
-        B.pipe_select_kernel(B.KERNEL_AUTO)
+        B.pipe_diag_select_kernel(B.KERNEL_AUTO)
     if pitch_extra:
         for b in bufs:
             assert (b[:, O:] == 99).all(), "bytes beyond the row were written"

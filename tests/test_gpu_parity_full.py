@@ -121,12 +121,12 @@ def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_chec
             y_auto = [y.clone() for y in run.y]
             part_auto = part.clone()
             part.zero_()
-            B.pipe_select_kernel(B.KERNEL_REFERENCE)
+            B.pipe_diag_select_kernel(B.KERNEL_REFERENCE)
             try:
                 run.forward(part)
                 torch.cuda.synchronize()
             finally:
-                B.pipe_select_kernel(B.KERNEL_AUTO)
+                B.pipe_diag_select_kernel(B.KERNEL_AUTO)
             for m in range(sp.M):
                 assert torch.equal(y_auto[m].view(torch.int32), run.y[m].view(torch.int32))
             assert torch.equal(part_auto, part)

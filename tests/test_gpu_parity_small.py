@@ -327,7 +327,7 @@ def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, k
     T = N * Ho * Wo
     y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
     part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
-    B.pipe_select_kernel(kernel)
+    B.pipe_diag_select_kernel(kernel)
     try:
         B.pipe_expanded_conv2d(layer.desc, geom, layer.blob, xq4.view(N, Hh, Ww, Cc), sx, y, torch.from_numpy(bias).cuda(), part)
     except B.PipeError as ex:
@@ -335,7 +335,7 @@ def test_implicit_convolution_matches_oracle(oracle, kernel, N, Hh, Ww, Cc, O, k
             pytest.skip("the two-SM kernel needs at least two token tiles")
         raise
     finally:
-        B.pipe_select_kernel(B.KERNEL_AUTO)
+        B.pipe_diag_select_kernel(B.KERNEL_AUTO)
     torch.cuda.synchronize()
     assert B.pipe_poll_status() == B.PIPE_OK
     np.testing.assert_array_equal(part.cpu().numpy(), f.partials)

@@ -15,7 +15,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import pipe_oracle as O
+from oracle import pipe_oracle as oracle
 from paper_2311_15806_b200 import binding as B
 from tests import gpu_harness as H
 
@@ -55,7 +55,7 @@ def test_static_workspace_expansion_matches_the_ordinary_one_twice():
         for a, b in zip(_blob_sections(desc, got), _blob_sections(desc, want)):
             np.testing.assert_array_equal(a, b)
         assert torch.equal(got, want)
-        H.assert_expansion_matches(B.ExpandedLayer(desc, lay, got), O.expand(W, bits, K, g, n_keep), O)
+        H.assert_expansion_matches(B.ExpandedLayer(desc, lay, got), oracle.expand(W, bits, K, g, n_keep), oracle)
 
 
 def test_static_workspace_call_allocates_nothing():
