@@ -25,10 +25,13 @@ pipe_status pipe_diag_select_kernel(int32_t which);
 
 /* Issue-bound rate of tcgen05.mma kind::i8 on this device: one CTA per SM issues `mma_per_cta`
  * instructions of shape M = 128, N = n_cols (16..256, a multiple of 16), K = 32 on operands that stay in
- * shared memory (no loads, no epilogue), alternating between two accumulators.  The work is queued on
+ * shared memory (no loads, no epilogue), alternating between two accumulators.  cta_pairs != 0: the CTAs
+ * run as clusters of two and the first CTA of each pair issues `mma_per_cta` instructions of the two-SM
+ * form (cta_group::2, M = 256, each CTA holding half of the n_cols rows of B).  The work is queued on
  * `stream`; the caller times it (CUDA events) and divides *h_ops_per_launch -- the integer operations
  * (2 per multiply-accumulate) of the whole launch -- by the duration.  Allocates nothing. */
-pipe_status pipe_diag_mma_i8_rate(int32_t n_cols, int64_t mma_per_cta, double* h_ops_per_launch, void* stream);
+pipe_status pipe_diag_mma_i8_rate(int32_t n_cols, int64_t mma_per_cta, int32_t cta_pairs, double* h_ops_per_launch,
+                                  void* stream);
 
 /* Exercises the bounded wait of the kernels: one CTA initialises an mbarrier on which nobody ever arrives and
  * waits on it with the library's own wait routine, limited to `limit_cycles` SM cycles (1..2^31).  The wait

@@ -95,7 +95,7 @@ def lib() -> C.CDLL:
         L.pipe_ensemble_forward_q8.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, i32, p, p, i64, p, p]
         L.pipe_expanded_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
         L.pipe_diag_select_kernel.argtypes = [i32]
-        L.pipe_diag_mma_i8_rate.argtypes = [i32, i64, C.POINTER(C.c_double), p]
+        L.pipe_diag_mma_i8_rate.argtypes = [i32, i64, i32, C.POINTER(C.c_double), p]
         L.pipe_diag_bounded_wait.argtypes = [i64, p]
         L.pipe_launch_count.restype = C.c_uint64
         L.pipe_poll_status.argtypes = [p, C.POINTER(i32)]
@@ -279,10 +279,11 @@ def pipe_diag_select_kernel(which: int) -> None:
     _check(lib().pipe_diag_select_kernel(which), "pipe_diag_select_kernel")
 
 
-def pipe_diag_mma_i8_rate(n_cols: int, mma_per_cta: int, stream=None) -> float:
+def pipe_diag_mma_i8_rate(n_cols: int, mma_per_cta: int, cta_pairs: bool = False, stream=None) -> float:
     """Queues the issue-rate probe of the integer tensor pipe; returns the integer operations of the launch."""
     ops = C.c_double(0.0)
-    _check(lib().pipe_diag_mma_i8_rate(int(n_cols), int(mma_per_cta), C.byref(ops), _stream_ptr(stream)), "pipe_diag_mma_i8_rate")
+    _check(lib().pipe_diag_mma_i8_rate(int(n_cols), int(mma_per_cta), 1 if cta_pairs else 0, C.byref(ops), _stream_ptr(stream)),
+           "pipe_diag_mma_i8_rate")
     return float(ops.value)
 
 

@@ -8,59 +8,51 @@
 // the one-SM kernel this halves the unpack work and the B-tile traffic per multiply-accumulate and
 // leaves room for two accumulator buffers of up to 256 columns per SM, so the epilogue of a tile
 // always overlaps the MMAs of the next.  Roles per CTA:
-//   warp 0      activation producer (TMA, several lanes in turn); in the second CTA two more lanes
-//               forward "both operands of the stage are in place" and "accumulators drained" to the
-//               first CTA's barriers (one signal across the pair per event, not one per warp)
-//   warps 2-7   unpack half of the B tile
+//   warp 0      activation producer: one tensor load per step (two patch boxes for the implicit convolution),
+//               whose completion is counted on the FIRST CTA's stage barrier (cta_group::2 form of the copy)
+//   warps 2-7   unpack half of the B tile; every warp signals the first CTA's "B in place" barrier itself
 //   warp 1      first CTA: MMA issuer (one lane); both: owner of the tensor-memory allocation.
 //               tcgen05.commit with a two-CTA multicast returns a stage to the producers of both
 //               CTAs and hands the accumulators to the epilogue warps of both
-//   warps 8-15  epilogue of the CTA's own 128 token rows (as in the one-SM kernel)
+//   warps 8-15  epilogue of the CTA's own 128 token rows (as in the one-SM kernel); every warp signals the
+//               first CTA's "accumulators drained" barrier itself
+// Every barrier the MMA issuer waits on therefore lives in the first CTA and counts both CTAs' arrivals; no
+// thread forwards signals, and no two lanes of a warp ever spin on different barriers (lanes of one warp that
+// poll different barriers take turns, which is what made an earlier relay-lane design latency-bound).
 // Every mbarrier wait is bounded; the pair leaves through a cluster barrier so that neither CTA's
 // shared memory or barriers disappear while its peer may still signal them.
-#include <cuda.h>
-
-#include <mutex>
-
-#include "pipe_common.cuh"
+#include "pipe_tc_common.cuh"
 
 namespace pipe {
 
 namespace tc2 {
 
 constexpr int kTileM = 128;          // tokens per tile
-constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per stage
+constexpr int kKStep = 128;          // reduction bytes (int8 lanes) per block: one row of a swizzled operand tile
+constexpr int kSub = 2;              // reduction blocks per ring stage: every barrier operation, proxy fence and
+                                     // commit is paid once per stage, and each costs its thread on the order of a
+                                     // hundred cycles, so a stage carries two blocks (eight MMAs)
 constexpr int kMaxN = 256;           // stacked weight rows per tile
 constexpr int kMaxClusterOrders = 8;
 constexpr int kUnpackWarps = 6;   // 16 warps per CTA: 128 registers per thread (see the one-SM kernel)
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
 constexpr int kUnpackThreads = 32 * kUnpackWarps;
-constexpr int kABytes = kTileM * kKStep;       // 16 KiB per token tile
-constexpr int kBtBytes = (kMaxN / 2) * kKStep;   // 16 KiB: this CTA's half of the stacked rows
-constexpr int kStageBytes = kABytes + kBtBytes;
+constexpr int kABytes = kTileM * kKStep;       // 16 KiB per token tile and reduction block
+constexpr int kBtBytes = (kMaxN / 2) * kKStep;   // 16 KiB per block: this CTA's half of the stacked rows
+constexpr int kStageBytes = kSub * (kABytes + kBtBytes);   // [kSub activation tiles][kSub B tiles]
+constexpr int kStageBOff = kSub * kABytes;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
-constexpr int kMaxRing = 6;
+constexpr int kMaxRing = 3;
 constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
-constexpr long long kWaitLimitCycles = 4000000000ll;  // about 2 s per wait at the maximum SM clock
-
-// Position in a ring of `depth` slots: slot index and phase parity, advanced without divisions.
-struct RingPos {
-  uint32_t slot, phase;
-  __device__ __forceinline__ void advance(uint32_t by, uint32_t depth) {  // by <= depth
-    slot += by;
-    if (slot >= depth) {
-      slot -= depth;
-      phase ^= 1u;
-    }
-  }
-};
+using namespace tcc;
 
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
   ForwardArgs f;
-  int BN, ncb, ntt, num_tiles, kblocks;   // ntt: pairs of token tiles
+  int BN, ncb, ntt, num_tiles, kblocks;   // ntt: pairs of token tiles; kblocks: reduction blocks of 128 lanes
+  int ksteps;             // ring stages per tile: ceil(kblocks / kSub)
   int ntok_tiles;         // token tiles (128 tokens) in total
   int nkmax;              // most orders any branch has
   int depth;              // stages in the ring
@@ -80,41 +72,6 @@ struct TileMeta {
   int rowbase[kMaxClusterOrders + 1];  // row offset of order k in the stacked B tile / accumulator
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// For barriers that the peer CTA signals: the wait acquires at cluster scope.
-__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -126,78 +83,31 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
-// Arrival on a barrier of the peer CTA.  The default semantics (release at CTA scope) are enough: what
-// the peer's MMA issuer learns from the signal is that this CTA's operands are in place, and those were
-// made visible to this SM's own tensor core by the writers' proxy fences / by the copy engine; a release
-// at cluster scope costs the signalling thread several hundred cycles more.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+// Arrival on a barrier of the pair's first CTA (cluster address; the first CTA uses it for its own barriers
+// too).  The default semantics (release at CTA scope) are enough and are what is used: the signal tells the MMA
+// issuer that this warp's share of the stage is in place, and what reads that share is this SM's own tensor
+// core, for which the writers' proxy fence (before the arrival, in program order) has already made it visible.
+// A release at cluster scope makes the arriving thread wait for all of its memory operations in flight, the
+// prefetch loads of later steps included, and more than doubles the time of a reduction step.
+__device__ __forceinline__ void mbar_arrive_lead(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
-// The bound is counted in SM cycles; the abort flag and the clock are looked at only every few
-// polls so that a barrier that completes soon is seen with little delay.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (true) {
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-      if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      raise_status(status, PIPE_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-
-// The same for a barrier that the peer CTA signals.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try_cluster(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (true) {
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-      if (mbar_try_cluster(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      raise_status(status, PIPE_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-
-// After the last issue: wait (bounded) until the copies of the last `depth` ring slots have landed,
-// so that no copy is still writing into this CTA's shared memory when it exits.
-__device__ __forceinline__ void drain_ring(uint32_t full0, uint32_t issued, int depth) {
-  for (uint32_t j = (issued > static_cast<uint32_t>(depth) ? issued - depth : 0); j < issued; ++j) {
-    const int s = j % depth;
-    const uint32_t ph = (j / depth) & 1;
-    const long long t0 = clock64();
-    while (!mbar_try(full0 + 8u * s, ph) && clock64() - t0 < kWaitLimitCycles) {
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+// Tensor loads of a CTA pair: the bytes land in the issuing CTA's shared memory, the completion is counted on a
+// barrier of the pair's FIRST CTA (cluster address), where the MMA issuer waits for both CTAs' tiles.
+__device__ __forceinline__ void tma_pair_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t lead_bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(lead_bar)
       : "memory");
 }
-
-// Four-dimensional tile of an NHWC tensor (coordinates innermost first: channel, x, y, image);
-// coordinates outside the tensor read zeros, which is the convolution's padding.
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+__device__ __forceinline__ void tma_pair_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t lead_bar) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(lead_bar)
       : "memory");
 }
 
@@ -205,24 +115,7 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
 // image p / pp at patch coordinates ((p % pp) / pw, (p % pp) % pw).
 __device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n, int& h0, int& w0);
 
-// Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes, stored as
-// 8-row atoms of 1024 bytes with the 128-byte swizzle (the layout TMA writes with SWIZZLE_128B).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);  // start address
-  d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset (unused for swizzled K-major)
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset: next 8-row atom
-  d |= static_cast<uint64_t>(1) << 46;                 // descriptor version of this architecture
-  d |= static_cast<uint64_t>(2) << 61;                 // 128-byte swizzle
-  return d;
-}
-
-// Instruction descriptor: D = int32, A and B = signed int8, both K-major, M = 256 (two SMs), N = n.
-__device__ __forceinline__ uint32_t idesc_i8(int n) {
-  return (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>((2 * kTileM) >> 4) << 24);
-}
-
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+__device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.u32 p, %4, 0;\n\t"
@@ -236,13 +129,6 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
 __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
                "h"(static_cast<uint16_t>(3))
-               : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-               : "r"(taddr)
                : "memory");
 }
 
@@ -282,154 +168,147 @@ __device__ __forceinline__ void patch_origin(const Params& p, int patch, int& n,
   w0 = (rem % p.conv_pw) * 8;
 }
 
+// Rows of the MMA's B operand for a tile that stacks n_total rows: each CTA of the pair holds half of them, and a
+// half must be a whole number of unpack items (8 rows; 16 rows of 2-bit codes), so the count is rounded up to 16
+// (32); the accumulator columns of the padding rows are never read.
+__device__ __forceinline__ int pair_mma_rows(int n_total, int bits) {
+  const int q = bits == 2 ? 32 : 16;
+  const int n = (n_total + q - 1) / q * q;
+  return n < q ? q : n;
+}
+
 struct Rings {
-  uint32_t a_full0, bt_ready0, done0, tfull0, tempty0;  // barrier i of a family is 8*i bytes on
-  uint32_t bt_ready_lead0, tempty_lead0;   // the same barriers in the pair's first CTA (cluster addresses)
+  uint32_t full0, done0, tfull0, tempty0;  // barrier i of a family is 8*i bytes on
+  uint32_t full_lead0, tempty_lead0;       // the same barriers in the pair's first CTA (cluster addresses)
   int rank, pair, npairs;                  // this CTA's rank in the pair; tiles go round the pairs
   uint32_t stage0;        // shared address of stage 0 (activation tile, then B tile)
   uint8_t* stage_gen;     // generic address of stage 0
   volatile int* abort_flag;
 };
 
-// Per-tile placement of one unpack work item (stacked row r, 16-byte chunk c of its packed row):
-// offset of the chunk in the streaming layout at reduction block 0 and its step per block, both
-// in 16-byte units relative to Params::kbase; 0xffffffff marks an item beyond the tile's rows.
-// The CTA of rank q unpacks the stacked rows [q * half, (q + 1) * half), half = half of the row count
-// rounded up to the MMA's granularity of 16; r_local counts from the start of that range.
-__device__ __forceinline__ void place_item(const Params& p, int k0, int nk, const int (&start)[kMaxClusterOrders],
-                                           const int (&rowbase)[kMaxClusterOrders + 1], int rank, int r_local, int c, uint32_t& off,
-                                           uint32_t& step) {
-  const int half = ((rowbase[kMaxClusterOrders] + 15) & ~15) >> 1;
-  const int r = rank * half + r_local;
-  if (r_local >= half || r >= rowbase[kMaxClusterOrders]) {
-    off = 0xffffffffu;
-    step = 0;
-    return;
-  }
-  int rb = 0, st = start[0], ko = 0;
-#pragma unroll
-  for (int q = 1; q < kMaxClusterOrders; ++q)
-    if (q < nk && r >= rowbase[q]) {
-      rb = rowbase[q];
-      st = start[q];
-      ko = q;
-    }
-  const OrderView& ov = p.f.order[k0 + ko];
-  const uint32_t pk16 = static_cast<uint32_t>(p.pk) >> 4;
-  off = p.koff[k0 + ko] + static_cast<uint32_t>(st + r - rb) * pk16 + static_cast<uint32_t>(c);
-  step = static_cast<uint32_t>(ov.rows) * pk16;
-}
-
-// Unpack role.  Work items are (stacked row, 16-byte chunk); a thread owns the same item indices
-// in every tile.  A load cursor runs two reduction steps ahead of the step being written (also
-// across tile boundaries): the packed chunks travel global memory (L2-resident, fully coalesced)
-// -> registers -> swizzled B tile, and a step never waits for the latency of its own loads.
+// Unpack role: ONE WARP PER REDUCTION BLOCK.  The blocks of the pair's tiles form one sequence (two block
+// positions per ring stage; a tile with an odd block count ends with an empty position); unpack warp w of this CTA
+// takes the positions w, w + W, w + 2W, ... and writes this CTA's half of the stacked rows of that block
+// by itself, so that W blocks are in work at a time and the fixed costs of a block (barrier wait, proxy fence,
+// arrival, position bookkeeping: several hundred cycles of dependent instructions) are paid by one warp per block
+// instead of by every warp for every block.
+// A lane's item i is the 16-byte chunk 32 i + lane of the half tile's packed rows of the block (RPI = 32 / CPR rows
+// per item; the orders' runs start at multiples of RPI rows, so an item lies in one order and its 32 chunks are
+// contiguous in the streaming layout).  Lane l keeps, for item l, the chunk offset at block 0 and the step per block;
+// the others fetch them by shuffle.  The loads of a block are issued BEFORE the warp waits for its stage to be free.
 template <int BITS>
-__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int ut) {
-  constexpr int CPR = BITS;              // 16-byte chunks per packed row per block: 8, 4, 2
-  constexpr int CPR_LOG = (BITS == 8) ? 3 : (BITS == 4 ? 2 : 1);
-  constexpr int ITEMS = ((kMaxN / 2) * CPR + kUnpackThreads - 1) / kUnpackThreads;   // items past the last row are masked
+__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int uw, int lane) {
+  constexpr int CPR = BITS;                // 16-byte chunks per packed row per block: 8, 4, 2
+  constexpr int RPI = 32 / CPR;            // rows per item: 4, 8, 16
+  constexpr int ITEMS = (kMaxN / 2) / RPI; // items of a full half tile: 32, 16, 8
+  constexpr int PASS = ITEMS > 16 ? 16 : ITEMS;   // items held in registers at a time
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
-  constexpr int AHEAD = 2;
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
-  const uint32_t depth = p.depth;
-  const int r0 = ut >> CPR_LOG, c_item = ut & (CPR - 1);   // item i: row r0 + i * (threads / CPR), chunk c_item
-  const int sw = r0 & 7;                                   // the row step between items is a multiple of 8
   const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
   if (my_tiles <= 0) return;
-  const uint32_t total_steps = static_cast<uint32_t>(my_tiles) * p.kblocks;
+  const int slots_per_tile = kSub * p.ksteps;
+  const uint32_t total_slots = static_cast<uint32_t>(my_tiles) * slots_per_tile;
+  // this lane's place inside an item: row (lane / CPR) of the item's RPI rows, chunk (lane % CPR) of that row
+  const int lr = lane / CPR, lc = lane % CPR;
+  const int sw = lr & 7;                   // RPI is 4, 8 or 16 and items start at multiples of RPI rows:
+                                           // for RPI = 4 the swizzle also depends on the item (added below)
+  const uint32_t out_lane = static_cast<uint32_t>((lr >> 3) * 1024 + (lr & 7) * 128);
 
-  // ---- load cursor
-  uint32_t off[ITEMS], stp[ITEMS];
-  int cur_tile = g.pair, cur_kb = 0;
-  uint32_t issued = 0;
-  TileMeta tn;   // metadata of the tile after the cursor's tile, fetched when the cursor enters a tile
-  {
-    TileMeta t;
-    decode_tile(p, cur_tile, t);
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-      const int idx = ut + i * kUnpackThreads;
-      place_item(p, t.k0, t.nk, t.start, t.rowbase, g.rank, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
-    }
-    const int nt = cur_tile + g.npairs;
-    decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
+  int tile_i = -1;                         // index (0, 1, ...) of the tile whose placement the lanes hold
+  uint32_t my_off[ITEMS / 16 > 0 ? ITEMS / 16 : 1], my_stp[ITEMS / 16 > 0 ? ITEMS / 16 : 1];   // lane l: items l, l + 16
+  int n_items = 0;                         // items of this CTA's half tile that hold rows
+  int kbs = uw, ti = 0;                    // block position inside the tile, tile index
+  while (kbs >= slots_per_tile) {
+    kbs -= slots_per_tile;
+    ++ti;
   }
-  auto fetch = [&](uint4 (&w)[ITEMS], uint32_t& mask) {
-    mask = 0;
-    if (issued >= total_steps) return;
+  for (uint32_t pos = uw; pos < total_slots; pos += kUnpackWarps) {
+    if (ti != tile_i) {
+      tile_i = ti;
+      TileMeta t;
+      decode_tile(p, g.pair + ti * g.npairs, t);
+      const int n_total = t.rowbase[kMaxClusterOrders];
+      const int half = pair_mma_rows(n_total, BITS) >> 1;
+      const int mine = max(0, min(half, n_total - g.rank * half));   // rows of this CTA's half that exist
+      n_items = (mine + RPI - 1) / RPI;
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i)
-      if (off[i] != 0xffffffffu) {
-        w[i] = __ldg(kb16 + off[i]);
-        mask |= 1u << i;
+      for (int h = 0; h < (ITEMS / 16 > 0 ? ITEMS / 16 : 1); ++h) {
+        const int item = lane + 16 * h;
+        const int r = g.rank * half + item * RPI;                     // first stacked row of the item
+        uint32_t off = 0, stp = 0;
+        if (lane < 16 && item < n_items) {
+          int rb = 0, st = t.start[0], ko = 0;
+#pragma unroll
+          for (int q = 1; q < kMaxClusterOrders; ++q)
+            if (q < t.nk && r >= t.rowbase[q]) {
+              rb = t.rowbase[q];
+              st = t.start[q];
+              ko = q;
+            }
+          const uint32_t pk16 = static_cast<uint32_t>(p.pk) >> 4;
+          off = p.koff[t.k0 + ko] + static_cast<uint32_t>(st + r - rb) * pk16;
+          stp = static_cast<uint32_t>(p.f.order[t.k0 + ko].rows) * pk16;
+        }
+        my_off[h] = off;
+        my_stp[h] = stp;
       }
-    ++issued;
-    if (++cur_kb < p.kblocks) {
+    }
+    const uint32_t gs = static_cast<uint32_t>(ti) * p.ksteps + static_cast<uint32_t>(kbs / kSub);   // stage number
+    const uint32_t slot = gs % p.depth, use = gs / p.depth;
+    const int sub = kbs % kSub;
+    const bool real = kbs < p.kblocks;     // false: the empty position behind an odd block count
+    uint8_t* bt = g.stage_gen + static_cast<size_t>(slot) * kStageBytes + kStageBOff + sub * kBtBytes;
 #pragma unroll
-      for (int i = 0; i < ITEMS; ++i)
-        if (off[i] != 0xffffffffu) off[i] += stp[i];
-    } else if (issued < total_steps) {
-      cur_kb = 0;
-      cur_tile += g.npairs;
+    for (int pass = 0; pass < ITEMS / PASS; ++pass) {
+      uint4 w[PASS];
+      if (real) {
+        const uint32_t here = my_off[pass] + static_cast<uint32_t>(kbs) * my_stp[pass];
 #pragma unroll
-      for (int i = 0; i < ITEMS; ++i) {
-        const int idx = ut + i * kUnpackThreads;
-        place_item(p, tn.k0, tn.nk, tn.start, tn.rowbase, g.rank, idx >> CPR_LOG, idx & (CPR - 1), off[i], stp[i]);
+        for (int i = 0; i < PASS; ++i) {
+          const uint32_t a = __shfl_sync(0xffffffffu, here, i);
+          if (i + PASS * pass < n_items) w[i] = __ldg(kb16 + a + lane);
+        }
       }
-      const int nt = cur_tile + g.npairs;
-      decode_tile(p, nt < p.num_tiles ? nt : cur_tile, tn);
-    }
-  };
-
-  uint4 q1[ITEMS], q2[ITEMS];
-  uint32_t m1 = 0, m2 = 0;
-  fetch(q1, m1);
-  if (AHEAD == 2) fetch(q2, m2);
-
-  RingPos rp{0, 0};
-  for (uint32_t it = 0; it < total_steps; ++it, rp.advance(1, depth)) {
-    uint4 w[ITEMS];
-    const uint32_t mask = m1;
+      // the stage is free once the MMAs of its previous use have completed (first pass of the block only)
+      if (pass == 0 && !mbar_wait(g.done0 + 8u * slot, (use & 1) ^ 1, g.abort_flag, p.f.status)) return;
+      if (real) {
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) w[i] = q1[i];
-    if (AHEAD == 2) {
+        for (int i = 0; i < PASS; ++i) {
+          const int item = i + PASS * pass;
+          if (item >= n_items) continue;
+          // rows item * RPI + lr; for RPI = 4 the item's parity moves the row inside its 8-row atom
+          const int row0 = item * RPI;
+          uint8_t* row = bt + (row0 >> 3) * 1024 + (row0 & 7) * 128 + out_lane;
+          const int swz = (RPI == 4) ? ((row0 + lr) & 7) : sw;
+          const int c0 = lc * OUT_PER_CHUNK;
+          if (BITS == 8) {
+            *reinterpret_cast<uint4*>(row + ((c0 ^ swz) << 4)) = w[i];
+          } else if (BITS == 4) {
+            const uint32_t m4 = 0xF0F0F0F0u;
+            const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
+            const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
+            *reinterpret_cast<uint4*>(row + ((c0 ^ swz) << 4)) = v0;
+            *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ swz) << 4)) = v1;
+          } else {
+            const uint32_t m2c = 0xC0C0C0C0u;
+            const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
-      for (int i = 0; i < ITEMS; ++i) q1[i] = q2[i];
-      m1 = m2;
-      fetch(q2, m2);
-    } else {
-      fetch(q1, m1);
-    }
-    if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) return;
-    uint8_t* bt = g.stage_gen + static_cast<size_t>(rp.slot) * kStageBytes + kABytes;
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-      if (!((mask >> i) & 1u)) continue;
-      const int r = r0 + i * (kUnpackThreads >> CPR_LOG);
-      uint8_t* row = bt + (r >> 3) * 1024 + (r & 7) * 128;
-      const int c0 = c_item * OUT_PER_CHUNK;
-      if (BITS == 8) {
-        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = w[i];
-      } else if (BITS == 4) {
-        const uint32_t m4 = 0xF0F0F0F0u;
-        const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
-        const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
-        *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = v0;
-        *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ sw) << 4)) = v1;
-      } else {
-        const uint32_t m2c = 0xC0C0C0C0u;
-        const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
-#pragma unroll
-        for (int h = 0; h < 4; ++h) {
-          const uint4 v = make_uint4((ww[h] << 6) & m2c, (ww[h] << 4) & m2c, (ww[h] << 2) & m2c, ww[h] & m2c);
-          *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
+            for (int h = 0; h < 4; ++h) {
+              const uint4 v = make_uint4((ww[h] << 6) & m2c, (ww[h] << 4) & m2c, (ww[h] << 2) & m2c, ww[h] & m2c);
+              *reinterpret_cast<uint4*>(row + (((c0 + h) ^ swz) << 4)) = v;
+            }
+          }
         }
       }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
     __syncwarp();
-    if ((ut & 31) == 0) mbar_arrive(g.bt_ready0 + 8u * rp.slot);   // one arrival per warp, on this CTA's barrier
+    if (lane == 0) mbar_arrive_lead(g.full_lead0 + 8u * slot);   // one arrival per block position, on the first CTA's barrier
+    kbs += kUnpackWarps;
+    while (kbs >= slots_per_tile) {
+      kbs -= slots_per_tile;
+      ++ti;
+    }
   }
 }
 
@@ -652,13 +531,13 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncwarp();
-    if (lane == 0) mbar_arrive(x.tempty0 + 8u * buf);   // one arrival per warp, on this CTA's barrier
+    if (lane == 0) mbar_arrive_lead(x.tempty_lead0 + 8u * buf);   // one arrival per warp, on the first CTA's barrier
   }
 }
 
 __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t bars[3 * kMaxRing + 4];  // a_full[6] bt_ready[6] done[6] tmem_full[2] tmem_empty[2]
+  __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
@@ -669,15 +548,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar0 = smem_u32(bars);
   Rings g;
-  g.a_full0 = bar0;
-  g.bt_ready0 = bar0 + 8u * kMaxRing;
-  g.done0 = bar0 + 8u * 2 * kMaxRing;
-  g.tfull0 = bar0 + 8u * 3 * kMaxRing;
+  g.full0 = bar0;
+  g.done0 = bar0 + 8u * kMaxRing;
+  g.tfull0 = bar0 + 8u * 2 * kMaxRing;
   g.tempty0 = g.tfull0 + 8u * 2;
   g.rank = static_cast<int>(cluster_rank());
   g.pair = static_cast<int>(blockIdx.x >> 1);
   g.npairs = static_cast<int>(gridDim.x >> 1);
-  g.bt_ready_lead0 = map_to_cta(g.bt_ready0, 0);
+  g.full_lead0 = map_to_cta(g.full0, 0);
   g.tempty_lead0 = map_to_cta(g.tempty0, 0);
   g.stage0 = smem_base;
   g.stage_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -685,16 +563,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    // The MMA issuer sits in the pair's first CTA, so the barriers it waits on live there and count the
+    // arrivals of BOTH CTAs: "stage full" = the first CTA's producer (which posts the bytes of both CTAs'
+    // activation tiles) + one unpack warp per block position and CTA; "accumulators drained" = every epilogue warp of the
+    // pair.  The same barriers of the second CTA are initialised but never used.
     for (int s = 0; s < kMaxRing; ++s) {
-      mbar_init(g.a_full0 + 8u * s, 1);
-      // own unpack warps; in the first CTA also the peer's "both of my operands are in place"
-      mbar_init(g.bt_ready0 + 8u * s, kUnpackWarps + (g.rank == 0 ? 1 : 0));
+      mbar_init(g.full0 + 8u * s, 1 + 2 * kSub);
       mbar_init(g.done0 + 8u * s, 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
-      // own epilogue warps; in the first CTA also the peer's "my accumulators are drained"
-      mbar_init(g.tempty0 + 8u * b, kEpiWarps + (g.rank == 0 ? 1 : 0));
+      mbar_init(g.tempty0 + 8u * b, 2 * kEpiWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -711,67 +590,57 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   const uint32_t tmem_base = tmem_base_slot;
   const uint32_t depth = p.depth;
   const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
-  const uint32_t total_steps = static_cast<uint32_t>(my_tiles > 0 ? my_tiles : 0) * p.kblocks;
+  const uint32_t total_steps = static_cast<uint32_t>(my_tiles > 0 ? my_tiles : 0) * p.ksteps;   // ring stages
 
   if (warp == 0) {
     // ------------------------------------------------------------------ activation producer
-    // Lane j < P owns the steps j, j + P, ... (P <= ring depth, see the one-SM kernel for why).  In
-    // the second CTA lane P forwards every "tile landed" to the first CTA's stage barrier, where
-    // the MMA issuer waits for both CTAs' operands.
-    const uint32_t P = min(static_cast<uint32_t>(kALanes), depth);
-    if (static_cast<uint32_t>(lane) < P) {
-      RingPos rp{static_cast<uint32_t>(lane), 0};
-      int tile = g.pair, kb = lane;
-      for (uint32_t it = lane; it < total_steps; it += P, rp.advance(P, depth), kb += P) {
-        while (kb >= p.kblocks) {
-          kb -= p.kblocks;
+    // One lane per copy of a stage (per reduction block one box for a matrix of tokens, two patch boxes for the
+    // implicit convolution); the lanes run the same loop on the same barriers, so the warp stays converged.  The
+    // completion of both CTAs' copies is counted on the FIRST CTA's stage barrier, whose expected byte count
+    // (both tiles) that CTA's lane 0 posts; a copy of the second CTA may land before that, which only lets the
+    // transaction count run ahead of the expectation while the barrier's one arrival is still pending.
+    const int per_block = p.f.conv_on ? 2 : 1;        // copies per reduction block
+    const int sub = lane / per_block, half = lane % per_block;
+    if (lane < kSub * per_block) {
+      RingPos rp{0, 0};
+      int tile = g.pair, ks = 0;
+      for (uint32_t it = 0; it < total_steps; ++it, rp.advance(1, depth), ++ks) {
+        if (ks == p.ksteps) {
+          ks = 0;
           tile += g.npairs;
         }
         const int ttile = 2 * (tile % p.ntt) + g.rank;   // this CTA's 128 token rows of the pair's tile
         const int m = tile / p.ntt / p.ncb;
+        const int nsub = min(kSub, p.kblocks - ks * kSub);   // the last stage of a tile may hold one block only
+        const int kb = ks * kSub + sub;
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
-        mbar_expect_tx(g.a_full0 + 8u * rp.slot, kABytes);
+        if (g.rank == 0 && lane == 0) mbar_expect_tx(g.full0 + 8u * rp.slot, 2 * nsub * kABytes);
+        if (sub >= nsub) continue;
+        const uint32_t bar = g.full_lead0 + 8u * rp.slot;
+        const uint32_t dst = g.stage0 + rp.slot * kStageBytes + sub * kABytes;
         if (!p.f.conv_on) {
           // rows beyond T read zeros
-          tma_load_2d(g.stage0 + rp.slot * kStageBytes, &p.tmap_a[m], kb * kKStep, ttile * kTileM, g.a_full0 + 8u * rp.slot);
+          tma_pair_load_2d(dst, &p.tmap_a[m], kb * kKStep, ttile * kTileM, bar);
         } else {
           // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
           const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
           const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            int n, h0, w0;
-            patch_origin(p, 2 * ttile + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-            tma_load_4d(g.stage0 + rp.slot * kStageBytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
-                        n, g.a_full0 + 8u * rp.slot);
-          }
+          int n, h0, w0;
+          patch_origin(p, 2 * ttile + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
+          tma_pair_load_4d(dst + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh, n, bar);
         }
-      }
-    } else if (static_cast<uint32_t>(lane) < P + depth && g.rank == 1) {
-      // stage relays: one signal per step across the pair instead of one per warp.  A signal to the
-      // peer keeps its thread busy for a couple of thousand cycles, so every ring slot has its own
-      // relay lane (slot s <-> lane P + s; the steps of one slot stay in order).
-      const uint32_t slot = static_cast<uint32_t>(lane) - P;
-      uint32_t phase = 0;
-      for (uint32_t it = slot; it < total_steps; it += depth, phase ^= 1u) {
-        if (!mbar_wait(g.a_full0 + 8u * slot, phase, g.abort_flag, p.f.status)) break;
-        if (!mbar_wait(g.bt_ready0 + 8u * slot, phase, g.abort_flag, p.f.status)) break;
-        mbar_arrive_cluster(g.bt_ready_lead0 + 8u * slot);
-      }
-    } else if (static_cast<uint32_t>(lane) == P + depth && g.rank == 1) {
-      // accumulator relay: this CTA's epilogue warps have drained a buffer
-      for (int n = 0; n < my_tiles; ++n) {
-        if (!mbar_wait(g.tempty0 + 8u * (n & 1), (n >> 1) & 1, g.abort_flag, p.f.status)) break;
-        mbar_arrive_cluster(g.tempty_lead0 + 8u * (n & 1));
       }
     }
     __syncwarp();
-    if (lane == 0) drain_ring(g.a_full0, total_steps, p.depth);
+    // (Every issued copy is consumed by an MMA before the accumulators of its tile are handed over, so on the
+    // normal path nothing is in flight here.  After an abort the first CTA gives the copies of both CTAs a
+    // bounded time to land before the pair leaves through the cluster barrier below.)
+    if (lane == 0 && g.rank == 0 && *g.abort_flag) drain_ring(g.full0, total_steps, p.depth, 20000000ll);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (first CTA of the pair)
     if (lane == 0 && g.rank == 0) {
       RingPos rp{0, 0};
-      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kABytes);
+      const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kStageBOff);
       uint32_t tcount = 0;
       bool ok = true;
       // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
@@ -793,23 +662,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
         if (tile + g.npairs < p.num_tiles) n_next = stacked_rows(tile + g.npairs);
         const int buf = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
-        if (!mbar_wait(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
-        int n = (n_total + 15) & ~15;
-        if (n < 16) n = 16;
-        const uint32_t idesc = idesc_i8(n);
+        if (!mbar_wait<true>(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
+        const int n = pair_mma_rows(n_total, p.f.bits);
+        const uint32_t idesc = idesc_i8(2 * kTileM, n);
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
-        for (int kb = 0; kb < p.kblocks; ++kb, rp.advance(1, depth)) {
-          // both barriers are polled before either result is tested so that the two polls overlap
-          const bool r1 = mbar_try(g.a_full0 + 8u * rp.slot, rp.phase);
-          const bool r2 = mbar_try(g.bt_ready0 + 8u * rp.slot, rp.phase);
-          if (!r1 && !mbar_wait(g.a_full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
-          if (!r2 && !mbar_wait(g.bt_ready0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
+        for (int ks = 0; ks < p.ksteps; ++ks, rp.advance(1, depth)) {
+          if (!mbar_wait<true>(g.full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
-          const uint64_t adesc = adesc0 + so, bdesc = bdesc0 + so;
+          const int nsub = min(kSub, p.kblocks - ks * kSub);
+          for (int sub = 0; sub < nsub; ++sub) {
+            const uint64_t adesc = adesc0 + so + static_cast<uint64_t>(sub * (kABytes >> 4));
+            const uint64_t bdesc = bdesc0 + so + static_cast<uint64_t>(sub * (kBtBytes >> 4));
 #pragma unroll
-          for (int k = 0; k < kKStep / 32; ++k)
-            mma_i8(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (kb | k) != 0);
+            for (int k = 0; k < kKStep / 32; ++k)
+              mma_i8_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (ks | sub | k) != 0);
+          }
           mma_commit_pair(g.done0 + 8u * rp.slot);   // frees the stage for the producers of both CTAs
         }
         if (ok) mma_commit_pair(g.tfull0 + 8u * buf);
@@ -817,10 +685,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     }
   } else if (warp < 2 + kUnpackWarps) {
     // ------------------------------------------------------------------ unpack warps
-    const int ut = threadIdx.x - 64;
-    if (p.f.bits == 8) unpack_role<8>(p, g, ut);
-    else if (p.f.bits == 4) unpack_role<4>(p, g, ut);
-    else unpack_role<2>(p, g, ut);
+    if (p.f.bits == 8) unpack_role<8>(p, g, warp - 2, lane);
+    else if (p.f.bits == 4) unpack_role<4>(p, g, warp - 2, lane);
+    else unpack_role<2>(p, g, warp - 2, lane);
   } else {
     // ------------------------------------------------------------------ epilogue warps
     EpiCtx e;
@@ -836,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.lane = lane;
     const int ew = warp - 2 - kUnpackWarps;
     e.part = ew >> 2;
-    e.nparts = 2;
+    e.nparts = kEpiWarps / 4;
     e.colmap = epi_colmap[ew];
     e.cscale = epi_cscale[ew];
     e.stg = epi_stage[ew];
@@ -864,53 +731,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
 }
 
 // ---------------------------------------------------------------------------------------------
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeFn encode_fn() {
-  static std::once_flag once;
-  static EncodeFn fn = nullptr;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeFn>(p);
-  });
-  return fn;
-}
-
-static bool make_map_2d(CUtensorMap* map, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
-                        uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
-  EncodeFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {inner_bytes, rows};
-  const cuuint64_t strides[1] = {pitch_bytes};
-  const cuuint32_t box[2] = {box_inner, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// NHWC int8 tensor as a 4-D map; one box = 128 channels x 8 x 8 pixels of one image (64 rows of 128 bytes).
-static bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int W, int C, int sh, int sw) {
-  EncodeFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
-                              static_cast<cuuint64_t>(N)};
-  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W) * C,
-                                 static_cast<cuuint64_t>(H) * W * C};
-  // 8 x 8 pixels at the convolution's stride: the box spans 8 * stride positions and the copy takes every
-  // stride-th of them
-  const cuuint32_t box[4] = {128, static_cast<cuuint32_t>(8 * sw), static_cast<cuuint32_t>(8 * sh), 1};
-  const cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(sw), static_cast<cuuint32_t>(sh), 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace tc2
 
 static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
@@ -935,6 +755,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
     if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand;
   }
   if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
+  if (a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.conv_on && (a.cC % kKStep != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
@@ -961,6 +782,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
   p.num_tiles = static_cast<int>(tiles);
   p.kblocks = ceil_div(a.I, kKStep);
+  p.ksteps = ceil_div(p.kblocks, kSub);
   p.pk = kKStep * a.bits / 8;
   p.shift = 8 - a.bits;
   int k_lo = PIPE_MAX_ORDERS, k_hi = 0;

@@ -67,15 +67,19 @@ __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
 // The bound is counted in SM cycles; the abort flag and the clock are looked at only every few
 // polls so that a barrier that completes soon is seen with little delay.
-template <bool CLUSTER = false>
+// SLEEP_NS > 0: a wait that is expected to last long (an epilogue warp waiting for a whole tile's MMAs) backs off
+// between polls, so that its polling does not take shared-memory and issue slots from the warps that feed the MMAs.
+template <bool CLUSTER = false, int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           long long limit = kWaitLimitCycles) {
   if (CLUSTER ? mbar_try_cluster(bar, parity) : mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
 #pragma unroll 1
-    for (int i = 0; i < 16; ++i)
+    for (int i = 0; i < 16; ++i) {
       if (CLUSTER ? mbar_try_cluster(bar, parity) : mbar_try(bar, parity)) return true;
+      if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+    }
     if (*abort_flag) return false;
     if (clock64() - t0 > limit) {
       *abort_flag = 1;
