@@ -188,21 +188,27 @@ struct Rings {
 
 // Unpack role: ONE WARP PER REDUCTION BLOCK.  The blocks of the pair's tiles form one sequence (two block
 // positions per ring stage; a tile with an odd block count ends with an empty position); unpack warp w of this CTA
-// takes the positions w, w + W, w + 2W, ... and writes this CTA's half of the stacked rows of that block
-// by itself, so that W blocks are in work at a time and the fixed costs of a block (barrier wait, proxy fence,
-// arrival, position bookkeeping: several hundred cycles of dependent instructions) are paid by one warp per block
-// instead of by every warp for every block.
-// A lane's item i is the 16-byte chunk 32 i + lane of the half tile's packed rows of the block (RPI = 32 / CPR rows
-// per item; the orders' runs start at multiples of RPI rows, so an item lies in one order and its 32 chunks are
-// contiguous in the streaming layout).  Lane l keeps, for item l, the chunk offset at block 0 and the step per block;
-// the others fetch them by shuffle.  The loads of a block are issued BEFORE the warp waits for its stage to be free.
+// takes the positions w, w + W, w + 2W, ... -- with W = 6 = stages x positions per stage that is always the same
+// block slot of the ring -- and writes this CTA's half of the stacked rows of that block by itself, so that W blocks
+// are in work at a time and the fixed costs of a block (barrier waits, proxy fence, arrival, position bookkeeping:
+// several hundred cycles of dependent instructions) are paid by one warp per block instead of by every warp for
+// every block.
+// Sub-byte codes: as soon as the slot is free the warp brings the packed rows of its half tile -- at most one
+// contiguous run per order, because the streaming layout is reduction-block-major -- into the END of the slot with
+// bulk copies (the copy engine sustains far more bytes in flight than a warp's own loads, which stalled at issue
+// when six warps each had 8 KiB outstanding), reads them into registers, and only then overwrites the slot with the
+// widened rows; nothing else is staged.  A lane's item i is the 16-byte chunk 32 i + lane of those packed rows
+// (RPI = 32 / CPR rows per item).
+// int8 codes need no widening and fill the slot exactly; they are loaded through registers.
 template <int BITS>
-__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int uw, int lane) {
+__device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int uw, int lane, uint32_t pkbar) {
   constexpr int CPR = BITS;                // 16-byte chunks per packed row per block: 8, 4, 2
   constexpr int RPI = 32 / CPR;            // rows per item: 4, 8, 16
   constexpr int ITEMS = (kMaxN / 2) / RPI; // items of a full half tile: 32, 16, 8
   constexpr int PASS = ITEMS > 16 ? 16 : ITEMS;   // items held in registers at a time
   constexpr int OUT_PER_CHUNK = 8 / BITS;  // 16-byte vectors written per chunk read
+  constexpr int PK = kKStep * BITS / 8;    // packed bytes of a row of a block
+  constexpr int kPackedOff = kBtBytes - (kMaxN / 2) * PK;   // sub-byte codes: where the packed rows land in the slot
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
   const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
   if (my_tiles <= 0) return;
@@ -210,13 +216,17 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
   const uint32_t total_slots = static_cast<uint32_t>(my_tiles) * slots_per_tile;
   // this lane's place inside an item: row (lane / CPR) of the item's RPI rows, chunk (lane % CPR) of that row
   const int lr = lane / CPR, lc = lane % CPR;
-  const int sw = lr & 7;                   // RPI is 4, 8 or 16 and items start at multiples of RPI rows:
-                                           // for RPI = 4 the swizzle also depends on the item (added below)
+  const int sw = lr & 7;
   const uint32_t out_lane = static_cast<uint32_t>((lr >> 3) * 1024 + (lr & 7) * 128);
 
+  // With W = stages x positions per stage the warp always works on the same block slot, so the barrier of that
+  // slot's packed rows is this warp's alone and its phase is simply the parity of the warp's uses so far.
+  uint32_t pk_phase = 0;
   int tile_i = -1;                         // index (0, 1, ...) of the tile whose placement the lanes hold
-  uint32_t my_off[ITEMS / 16 > 0 ? ITEMS / 16 : 1], my_stp[ITEMS / 16 > 0 ? ITEMS / 16 : 1];   // lane l: items l, l + 16
-  int n_items = 0;                         // items of this CTA's half tile that hold rows
+  // lane q < 8: the run of order q inside this CTA's half tile -- offset of its first chunk at block 0 and step per
+  // block (16-byte units relative to kbase), bytes, and byte offset inside the packed rows of the half tile
+  uint32_t run_off = 0, run_stp = 0, run_bytes = 0, run_dst = 0;
+  int n_items = 0, mine = 0;               // items / rows of this CTA's half tile that exist
   int kbs = uw, ti = 0;                    // block position inside the tile, tile index
   while (kbs >= slots_per_tile) {
     kbs -= slots_per_tile;
@@ -229,73 +239,115 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
       decode_tile(p, g.pair + ti * g.npairs, t);
       const int n_total = t.rowbase[kMaxClusterOrders];
       const int half = pair_mma_rows(n_total, BITS) >> 1;
-      const int mine = max(0, min(half, n_total - g.rank * half));   // rows of this CTA's half that exist
+      const int h0 = g.rank * half;
+      mine = max(0, min(half, n_total - h0));   // rows of this CTA's half that exist
       n_items = (mine + RPI - 1) / RPI;
+      run_bytes = 0;
+      int lo = 0, hi = 0, st = 0, ko = 0;
 #pragma unroll
-      for (int h = 0; h < (ITEMS / 16 > 0 ? ITEMS / 16 : 1); ++h) {
-        const int item = lane + 16 * h;
-        const int r = g.rank * half + item * RPI;                     // first stacked row of the item
-        uint32_t off = 0, stp = 0;
-        if (lane < 16 && item < n_items) {
-          int rb = 0, st = t.start[0], ko = 0;
-#pragma unroll
-          for (int q = 1; q < kMaxClusterOrders; ++q)
-            if (q < t.nk && r >= t.rowbase[q]) {
-              rb = t.rowbase[q];
-              st = t.start[q];
-              ko = q;
-            }
-          const uint32_t pk16 = static_cast<uint32_t>(p.pk) >> 4;
-          off = p.koff[t.k0 + ko] + static_cast<uint32_t>(st + r - rb) * pk16;
-          stp = static_cast<uint32_t>(p.f.order[t.k0 + ko].rows) * pk16;
+      for (int q = 0; q < kMaxClusterOrders; ++q)
+        if (q == lane) {
+          lo = t.rowbase[q];
+          hi = t.rowbase[q + 1];
+          st = t.start[q];
+          ko = q;
         }
-        my_off[h] = off;
-        my_stp[h] = stp;
+      if (lane < t.nk) {
+        const int a = max(lo, h0), b = min(hi, h0 + mine);
+        if (a < b) {
+          const uint32_t pk16 = PK >> 4;
+          run_off = p.koff[t.k0 + ko] + static_cast<uint32_t>(st + a - lo) * pk16;
+          run_stp = static_cast<uint32_t>(p.f.order[t.k0 + ko].rows) * pk16;
+          run_bytes = static_cast<uint32_t>(b - a) * PK;
+          run_dst = static_cast<uint32_t>(a - h0) * PK;
+        }
       }
     }
     const uint32_t gs = static_cast<uint32_t>(ti) * p.ksteps + static_cast<uint32_t>(kbs / kSub);   // stage number
     const uint32_t slot = gs % p.depth, use = gs / p.depth;
     const int sub = kbs % kSub;
-    const bool real = kbs < p.kblocks;     // false: the empty position behind an odd block count
-    uint8_t* bt = g.stage_gen + static_cast<size_t>(slot) * kStageBytes + kStageBOff + sub * kBtBytes;
+    const bool real = kbs < p.kblocks && mine > 0;     // false: the empty position behind an odd block count
+    const uint32_t bt_off = slot * kStageBytes + kStageBOff + sub * kBtBytes;
+    uint8_t* bt = g.stage_gen + bt_off;
+    if constexpr (BITS == 8) {
 #pragma unroll
-    for (int pass = 0; pass < ITEMS / PASS; ++pass) {
-      uint4 w[PASS];
-      if (real) {
-        const uint32_t here = my_off[pass] + static_cast<uint32_t>(kbs) * my_stp[pass];
+      for (int pass = 0; pass < ITEMS / PASS; ++pass) {
+        uint4 w[PASS];
+        if (real) {
 #pragma unroll
-        for (int i = 0; i < PASS; ++i) {
-          const uint32_t a = __shfl_sync(0xffffffffu, here, i);
-          if (i + PASS * pass < n_items) w[i] = __ldg(kb16 + a + lane);
+          for (int i = 0; i < PASS; ++i) {
+            const int item = i + PASS * pass;
+            // the run that holds the item's first row
+            const int byte0 = item * RPI * PK;
+            uint32_t src = 0;
+#pragma unroll
+            for (int q = 0; q < kMaxClusterOrders; ++q) {
+              const uint32_t ro = __shfl_sync(0xffffffffu, run_off + static_cast<uint32_t>(kbs) * run_stp, q);
+              const uint32_t rd = __shfl_sync(0xffffffffu, run_dst, q), rbts = __shfl_sync(0xffffffffu, run_bytes, q);
+              if (static_cast<uint32_t>(byte0) >= rd && static_cast<uint32_t>(byte0) < rd + rbts) src = ro + ((byte0 - rd) >> 4);
+            }
+            if (item < n_items) w[i] = __ldg(kb16 + src + lane);
+          }
+        }
+        // the stage is free once the MMAs of its previous use have completed (first pass of the block only)
+        if (pass == 0 && !mbar_wait(g.done0 + 8u * slot, (use & 1) ^ 1, g.abort_flag, p.f.status)) return;
+        if (real) {
+#pragma unroll
+          for (int i = 0; i < PASS; ++i) {
+            const int item = i + PASS * pass;
+            if (item >= n_items) continue;
+            const int row0 = item * RPI;   // rows row0 + lr; the item's parity moves the row inside its 8-row atom
+            uint8_t* row = bt + (row0 >> 3) * 1024 + (row0 & 7) * 128 + out_lane;
+            *reinterpret_cast<uint4*>(row + ((lc ^ ((row0 + lr) & 7)) << 4)) = w[i];
+          }
         }
       }
-      // the stage is free once the MMAs of its previous use have completed (first pass of the block only)
-      if (pass == 0 && !mbar_wait(g.done0 + 8u * slot, (use & 1) ^ 1, g.abort_flag, p.f.status)) return;
+    } else {
+      if (!mbar_wait(g.done0 + 8u * slot, (use & 1) ^ 1, g.abort_flag, p.f.status)) return;
       if (real) {
+        const uint32_t bar = pkbar + 8u * (slot * kSub + sub);
+        if (lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(mine) * PK);
+        __syncwarp();
+        if (run_bytes != 0) {
+          const uint8_t* src = p.kbase + (static_cast<size_t>(run_off + static_cast<uint32_t>(kbs) * run_stp) << 4);
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                           g.stage0 + bt_off + kPackedOff + run_dst),
+                       "l"(src), "r"(run_bytes), "r"(bar)
+                       : "memory");
+        }
+        __syncwarp();
+        if (!mbar_wait(bar, pk_phase, g.abort_flag, p.f.status)) {
+          // leaving with a copy possibly in flight: give it a bounded time to land in this CTA's shared memory
+          const long long t0 = clock64();
+          while (!mbar_try(bar, pk_phase) && clock64() - t0 < 20000000ll) {
+          }
+          return;
+        }
+        pk_phase ^= 1u;
+        uint4 w[ITEMS];
+        const uint4* pk_in = reinterpret_cast<const uint4*>(bt + kPackedOff) + lane;
 #pragma unroll
-        for (int i = 0; i < PASS; ++i) {
-          const int item = i + PASS * pass;
-          if (item >= n_items) continue;
-          // rows item * RPI + lr; for RPI = 4 the item's parity moves the row inside its 8-row atom
-          const int row0 = item * RPI;
-          uint8_t* row = bt + (row0 >> 3) * 1024 + (row0 & 7) * 128 + out_lane;
-          const int swz = (RPI == 4) ? ((row0 + lr) & 7) : sw;
+        for (int i = 0; i < ITEMS; ++i)
+          if (i < n_items) w[i] = pk_in[i * 32];
+        __syncwarp();   // every lane holds its packed chunks before any lane overwrites them
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+          if (i >= n_items) continue;
+          uint8_t* row = bt + i * (RPI >> 3) * 1024 + out_lane;   // rows i * RPI + lr (RPI is 8 or 16)
           const int c0 = lc * OUT_PER_CHUNK;
-          if (BITS == 8) {
-            *reinterpret_cast<uint4*>(row + ((c0 ^ swz) << 4)) = w[i];
-          } else if (BITS == 4) {
+          if (BITS == 4) {
             const uint32_t m4 = 0xF0F0F0F0u;
             const uint4 v0 = make_uint4((w[i].x << 4) & m4, w[i].x & m4, (w[i].y << 4) & m4, w[i].y & m4);
             const uint4 v1 = make_uint4((w[i].z << 4) & m4, w[i].z & m4, (w[i].w << 4) & m4, w[i].w & m4);
-            *reinterpret_cast<uint4*>(row + ((c0 ^ swz) << 4)) = v0;
-            *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ swz) << 4)) = v1;
+            *reinterpret_cast<uint4*>(row + ((c0 ^ sw) << 4)) = v0;
+            *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ sw) << 4)) = v1;
           } else {
             const uint32_t m2c = 0xC0C0C0C0u;
             const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
               const uint4 v = make_uint4((ww[h] << 6) & m2c, (ww[h] << 4) & m2c, (ww[h] << 2) & m2c, ww[h] & m2c);
-              *reinterpret_cast<uint4*>(row + (((c0 + h) ^ swz) << 4)) = v;
+              *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
             }
           }
         }
@@ -538,6 +590,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
+  __shared__ uint64_t pk_bars[kMaxRing * kSub];   // "packed rows have landed", one per block slot of the ring
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
@@ -571,6 +624,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       mbar_init(g.full0 + 8u * s, 1 + 2 * kSub);
       mbar_init(g.done0 + 8u * s, 1);
     }
+    for (int s = 0; s < kMaxRing * kSub; ++s) mbar_init(smem_u32(&pk_bars[s]), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
       mbar_init(g.tempty0 + 8u * b, 2 * kEpiWarps);
@@ -685,9 +739,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     }
   } else if (warp < 2 + kUnpackWarps) {
     // ------------------------------------------------------------------ unpack warps
-    if (p.f.bits == 8) unpack_role<8>(p, g, warp - 2, lane);
-    else if (p.f.bits == 4) unpack_role<4>(p, g, warp - 2, lane);
-    else unpack_role<2>(p, g, warp - 2, lane);
+    if (p.f.bits == 8) unpack_role<8>(p, g, warp - 2, lane, smem_u32(pk_bars));
+    else if (p.f.bits == 4) unpack_role<4>(p, g, warp - 2, lane, smem_u32(pk_bars));
+    else unpack_role<2>(p, g, warp - 2, lane, smem_u32(pk_bars));
   } else {
     // ------------------------------------------------------------------ epilogue warps
     EpiCtx e;
@@ -807,7 +861,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (cudaFuncGetAttributes(&fattr, tc2_forward_kernel) != cudaSuccess) return PIPE_ERR_CUDA;
   p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / kStageBytes;  // static shared, alignment slack
   if (p.depth > kMaxRing) p.depth = kMaxRing;
-  if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
+  if (p.depth * kSub != kUnpackWarps) return PIPE_ERR_UNSUPPORTED;   // every unpack warp owns one block slot of the ring
   const int dyn_smem = p.depth * kStageBytes + 1024;
 
   if (a.conv_on) {
