@@ -85,7 +85,17 @@ typedef struct pipe_layer_desc {
  *                 reduction order: int4 -> code 4h+j of the word's 8 codes sits in nibble 2j+h;
  *                 ternary -> code 4h+j of the word's 16 codes sits in bits 8j+2h..8j+2h+1;
  *                 int8 -> unchanged.
+ * Channel-block tables, one per cluster of orders that a forward call can evaluate on one input: entry m < M
+ * for predictor m (Sec. 3.2), entry M for all K orders (pipe_expanded_linear, pipe_expanded_conv2d).
+ *   blk_off[m]    int32 [2 + blk_cap[m]]: n, then b_0 = 0 < b_1 < ... < b_n = G.  Block i is the channel groups
+ *                 b_i .. b_{i+1} - 1; the blocks are cut greedily from group 0 so that the rows a block stacks over
+ *                 the cluster's orders (kept groups only) stay within PIPE_BLOCK_ROWS and its channels within
+ *                 PIPE_BLOCK_CHANNELS -- the unit of work of the SM-pair tensor-core kernel, whose MMAs then always
+ *                 run close to their widest shape however sparse the orders are.  A cluster of more than 8 orders,
+ *                 or whose single group can exceed the row limit (orders * g > PIPE_BLOCK_ROWS), has no table.
  */
+#define PIPE_BLOCK_ROWS 256
+#define PIPE_BLOCK_CHANNELS 512
 typedef struct pipe_layer_layout {
   int32_t num_groups;        /* G = O / g */
   int32_t total_rows;        /* R_total = sum_k rows[k] = O + (K-1) * keep_groups * g */
@@ -99,6 +109,9 @@ typedef struct pipe_layer_layout {
   uint64_t scales_off[PIPE_MAX_ORDERS];
   uint64_t kept_off[PIPE_MAX_ORDERS];
   uint64_t cum_off[PIPE_MAX_ORDERS];
+  uint64_t blk_off[PIPE_MAX_ORDERS + 1]; /* channel-block tables (see above); 0 = the cluster has none */
+  int32_t blk_cap[PIPE_MAX_ORDERS + 1];  /* blocks each table has room for */
+  int32_t reserved_;
   uint64_t blob_bytes;        /* size d_blob must have */
   uint64_t expand_ws_bytes;   /* size d_ws must have for pipe_expand_weights */
   uint64_t quantize_ws_bytes; /* size d_ws must have for pipe_quantize_act */

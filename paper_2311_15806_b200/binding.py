@@ -55,7 +55,9 @@ class LayerLayout(C.Structure):
                 ("kept_groups", C.c_int32 * MAX_ORDERS), ("branch_orders", C.c_int32 * MAX_ORDERS),
                 ("codes_off", C.c_uint64 * MAX_ORDERS), ("kcodes_off", C.c_uint64 * MAX_ORDERS),
                 ("scales_off", C.c_uint64 * MAX_ORDERS), ("kept_off", C.c_uint64 * MAX_ORDERS),
-                ("cum_off", C.c_uint64 * MAX_ORDERS), ("blob_bytes", C.c_uint64), ("expand_ws_bytes", C.c_uint64),
+                ("cum_off", C.c_uint64 * MAX_ORDERS), ("blk_off", C.c_uint64 * (MAX_ORDERS + 1)),
+                ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("reserved_", C.c_int32),
+                ("blob_bytes", C.c_uint64), ("expand_ws_bytes", C.c_uint64),
                 ("quantize_ws_bytes", C.c_uint64)]
 
 
@@ -332,6 +334,12 @@ class ExpandedLayer:
 
     def cum(self, k: int) -> torch.Tensor:
         return self.section(self.layout.cum_off[k], (self.layout.num_groups + 1) * 4).view(torch.int32)
+
+    def block_table(self, m: int) -> torch.Tensor | None:
+        """Channel-block table m (int32: n, b_0 .. b_n), or None when the cluster has none."""
+        if self.layout.blk_off[m] == 0:
+            return None
+        return self.section(self.layout.blk_off[m], (self.layout.blk_cap[m] + 2) * 4).view(torch.int32)
 
 
 def alloc_bytes(nbytes: int, device="cuda") -> torch.Tensor:

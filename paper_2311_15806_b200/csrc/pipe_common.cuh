@@ -112,6 +112,7 @@ struct BranchArgs {
   int8_t* yq;              // re-quantized output (ForwardArgs::q8_out), else unused
   const float* out_scale;  // its step: one float on the device
   int k_begin, k_end;
+  const int32_t* blk;      // channel-block table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
   int add_bias;    // bias enters this branch
   int accumulate;  // y += result (summed ensemble, branches after the first)
 };

@@ -5,6 +5,7 @@
 // row maximum,) divides, rounds, packs both code layouts, updates the residual with one FMA per
 // element and leaves the next order's row absmax behind.  All kernels are
 // HBM-bound streaming passes: 128-bit loads, warp-shuffle reductions, one block per row.
+#include <cstring>
 #include <mutex>
 
 #include "pipe_common.cuh"
@@ -355,6 +356,58 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
   }
 }
 
+// Channel-block table of one cluster of orders (see pipe.h): the groups are walked from 0 and a block is closed
+// when the next group would take its stacked rows beyond PIPE_BLOCK_ROWS or its channels beyond PIPE_BLOCK_CHANNELS.
+// One thread block per cluster: all threads gather the rows every group stacks (kept orders of the cluster only),
+// thread 0 then cuts the blocks.
+struct BlockTableArgs {
+  const int32_t* cum[PIPE_MAX_ORDERS + 1][8];   // prefix counts of the cluster's orders
+  int nk[PIPE_MAX_ORDERS + 1];
+  int32_t* out[PIPE_MAX_ORDERS + 1];
+  int cap[PIPE_MAX_ORDERS + 1];
+  int G, g;
+};
+
+constexpr int kTableChunk = 2048;
+
+__global__ void block_table_kernel(const __grid_constant__ BlockTableArgs a) {
+  __shared__ int rows_s[kTableChunk];
+  const int m = blockIdx.x;
+  int32_t* out = a.out[m];
+  if (!out) return;
+  int cur_rows = 0, cur_groups = 0, n = 0;
+  const int max_groups = PIPE_BLOCK_CHANNELS / a.g > 0 ? PIPE_BLOCK_CHANNELS / a.g : 1;
+  for (int base = 0; base < a.G; base += kTableChunk) {
+    const int cnt = min(kTableChunk, a.G - base);
+    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
+      int r = 0;
+      for (int q = 0; q < a.nk[m]; ++q) r += (a.cum[m][q][base + j + 1] - a.cum[m][q][base + j]) * a.g;
+      rows_s[j] = r;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      if (base == 0) out[1] = 0;
+      for (int j = 0; j < cnt; ++j) {
+        const int r = rows_s[j];
+        if (cur_groups > 0 && (cur_rows + r > PIPE_BLOCK_ROWS || cur_groups + 1 > max_groups)) {
+          if (n < a.cap[m]) out[2 + n] = base + j;   // (the capacity bound holds by construction; never write past it)
+          ++n;
+          cur_rows = 0;
+          cur_groups = 0;
+        }
+        cur_rows += r;
+        ++cur_groups;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    if (n < a.cap[m]) out[2 + n] = a.G;
+    ++n;
+    out[0] = n <= a.cap[m] ? n : 0;
+  }
+}
+
 __global__ void write_header_kernel(uint32_t* hdr, pipe_layer_desc d) {
   if (threadIdx.x == 0) {
     hdr[0] = kBlobMagic;
@@ -435,6 +488,26 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     else if (L.bits == 4) quantize_rows_kernel<4><<<rows, kRowThreads, 0, s>>>(q);
     else quantize_rows_kernel<2><<<rows, kRowThreads, 0, s>>>(q);
     count_launch(1);
+  }
+  {
+    BlockTableArgs t;
+    std::memset(&t, 0, sizeof(t));
+    t.G = L.G;
+    t.g = L.g;
+    bool any = false;
+    for (int m = 0; m <= L.M; ++m) {
+      if (L.lay.blk_off[m] == 0) continue;
+      const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
+      t.nk[m] = k1 - k0;
+      for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
+      t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.blk_off[m]);
+      t.cap[m] = L.lay.blk_cap[m];
+      any = true;
+    }
+    if (any) {
+      block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
+      count_launch(1);
+    }
   }
   return launch_status();
 }

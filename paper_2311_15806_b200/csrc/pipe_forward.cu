@@ -3,6 +3,11 @@
 
 namespace pipe {
 
+// Channel-block table m of the blob (m < L.M: predictor m; m = L.M: all K orders), or nullptr.
+static const int32_t* block_table(const LayerInfo& L, const void* d_blob, int m) {
+  return L.lay.blk_off[m] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.blk_off[m]) : nullptr;
+}
+
 static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, const int8_t* const* xq,
                                const float* const* sx, float* const* y, const int* k_begin, const int* k_end,
                                int64_t T, int64_t ldxq, int64_t ldy, const float* d_bias, int sum_branches,
@@ -43,6 +48,8 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     b.k_end = k_end[m];
     b.add_bias = (m == 0);
     b.accumulate = (sum_branches && m > 0);
+    // one branch running all K orders is the "all orders" cluster (entry L.M), otherwise predictor m's own
+    b.blk = block_table(L, d_blob, (k_end[m] - k_begin[m] == L.K) ? L.M : m);
   }
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = T; a.ldxq = ldxq; a.ldy = ldy;
@@ -65,8 +72,11 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   if (choice == 2) return forward_tcgen05(a, stream);
   if (choice == 3) return forward_stream(a, stream);
   if (choice == 4) return forward_tcgen05_pair(a, stream);
+  // T <= 16: weight streaming; from two token tiles on the SM-pair kernel; the one-SM kernel for what lies between
+  // and for layers without channel-block tables; the CUDA-core kernel for every other shape
   pipe_status st = PIPE_ERR_UNSUPPORTED;
   if (T <= 16) st = forward_stream(a, stream);
+  if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05_pair(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_reference(a, stream);
   return st;
@@ -159,6 +169,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   b.k_end = L.K;
   b.add_bias = 1;
   b.accumulate = 0;
+  b.blk = block_table(L, d_blob, L.M);
   b.yq = d_yq;
   b.out_scale = d_out_scale;
   a.q8_out = q8 ? 1 : 0;
@@ -179,8 +190,12 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   a.cN = geom->batch; a.cH = geom->height; a.cW = geom->width; a.cC = geom->channels;
   a.ckh = geom->kernel_h; a.ckw = geom->kernel_w; a.cph = geom->pad_h; a.cpw = geom->pad_w;
   a.cHo = Ho; a.cWo = Wo; a.csh = sh; a.csw = sw;
-  if (kernel_choice() == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
-  return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  const int choice = kernel_choice();
+  if (choice == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
+  if (choice == 2) return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  pipe_status cst = forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
+  if (cst == PIPE_ERR_UNSUPPORTED) cst = forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  return cst;
 }
 
 extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,

@@ -51,7 +51,7 @@ using namespace tcc;
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
   ForwardArgs f;
-  int BN, ncb, ntt, num_tiles, kblocks;   // ntt: pairs of token tiles; kblocks: reduction blocks of 128 lanes
+  int ntt, kblocks;       // ntt: pairs of token tiles; kblocks: reduction blocks of 128 lanes
   int ksteps;             // ring stages per tile: ceil(kblocks / kSub)
   int ntok_tiles;         // token tiles (128 tokens) in total
   int nkmax;              // most orders any branch has
@@ -64,7 +64,8 @@ struct Params {
 };
 
 struct TileMeta {
-  int m, cb, tt;                       // branch, channel block, token-tile group
+  int m, cb, tt;                       // branch, channel block of the branch's table, token-tile group
+  int c0, c1;                          // the block's output channels [c0, c1)
   int nk;                              // orders in this branch
   int k0;                              // first order
   int start[kMaxClusterOrders];        // first compacted row of the channel block in order k
@@ -132,17 +133,26 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
                : "memory");
 }
 
-__device__ __forceinline__ void decode_tile(const Params& p, int tile, TileMeta& t) {
-  t.tt = tile % p.ntt;
-  const int rest = tile / p.ntt;
-  t.cb = rest % p.ncb;
-  t.m = rest / p.ncb;
+// Tiles are numbered branch by branch, inside a branch channel block by channel block, the token-tile pairs of a
+// block next to each other (so that the pairs working at the same time read the same weight rows).  tile_base[m] is
+// the number of tiles of the branches before m; the block counts come from the blob's channel-block tables and are
+// known on the device only.
+__device__ __forceinline__ void locate_tile(const Params& p, const int* tile_base, int tile, int& m, int& cb, int& tt) {
+  m = 0;
+  while (m + 1 < p.f.num_branches && tile >= tile_base[m + 1]) ++m;
+  const int rest = tile - tile_base[m];
+  cb = rest / p.ntt;
+  tt = rest - cb * p.ntt;
+}
+
+__device__ __forceinline__ void decode_tile(const Params& p, const int* tile_base, int tile, TileMeta& t) {
+  locate_tile(p, tile_base, tile, t.m, t.cb, t.tt);
   const BranchArgs& br = p.f.branch[t.m];
   t.k0 = br.k_begin;
   t.nk = br.k_end - br.k_begin;
-  const int c0 = t.cb * p.BN;
-  const int c1 = min(c0 + p.BN, p.f.O);
-  const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
+  const int j0 = __ldg(br.blk + 1 + t.cb), j1 = __ldg(br.blk + 2 + t.cb);
+  t.c0 = j0 * p.f.g;
+  t.c1 = j1 * p.f.g;
   int rb = 0;
 #pragma unroll
   for (int ko = 0; ko < kMaxClusterOrders; ++ko) {
@@ -181,6 +191,8 @@ struct Rings {
   uint32_t full0, done0, tfull0, tempty0;  // barrier i of a family is 8*i bytes on
   uint32_t full_lead0, tempty_lead0;       // the same barriers in the pair's first CTA (cluster addresses)
   int rank, pair, npairs;                  // this CTA's rank in the pair; tiles go round the pairs
+  const int* tile_base;                    // shared memory: tiles before each branch, then the total
+  int num_tiles;
   uint32_t stage0;        // shared address of stage 0 (activation tile, then B tile)
   uint8_t* stage_gen;     // generic address of stage 0
   volatile int* abort_flag;
@@ -210,7 +222,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
   constexpr int PK = kKStep * BITS / 8;    // packed bytes of a row of a block
   constexpr int kPackedOff = kBtBytes - (kMaxN / 2) * PK;   // sub-byte codes: where the packed rows land in the slot
   const uint4* kb16 = reinterpret_cast<const uint4*>(p.kbase);
-  const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
+  const int my_tiles = (g.num_tiles - g.pair + g.npairs - 1) / g.npairs;
   if (my_tiles <= 0) return;
   const int slots_per_tile = kSub * p.ksteps;
   const uint32_t total_slots = static_cast<uint32_t>(my_tiles) * slots_per_tile;
@@ -236,7 +248,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
     if (ti != tile_i) {
       tile_i = ti;
       TileMeta t;
-      decode_tile(p, g.pair + ti * g.npairs, t);
+      decode_tile(p, g.tile_base, g.pair + ti * g.npairs, t);
       const int n_total = t.rowbase[kMaxClusterOrders];
       const int half = pair_mma_rows(n_total, BITS) >> 1;
       const int h0 = g.rank * half;
@@ -369,6 +381,8 @@ struct EpiCtx {
   volatile int* abort_flag;
   int warp, lane;
   int rank, pair, npairs;
+  const int* tile_base;
+  int num_tiles;
   uint32_t tempty_lead0;   // the accumulator-released barriers of the pair's first CTA (cluster address)
   int part, nparts;  // share of the 16-channel groups this warp drains (two warps per lane quarter)
   int16_t* colmap;
@@ -387,7 +401,10 @@ struct EpiCtx {
 // through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
 // (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
 // which is what bounds the drain otherwise).
-template <int NKMAX, bool PARTIALS>
+// Q8: the fused inner-layer epilogue (activation function and the next layer's input quantizer, see the one-SM
+// kernel) replaces the fp32 store; a lane then stores the 16 codes of its own row itself and the staging block holds
+// the bias of the tile's channels.
+template <int NKMAX, bool PARTIALS, bool Q8>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
   constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
   const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
@@ -401,21 +418,22 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   const uint32_t stg_w = smem_u32(x.stg) + static_cast<uint32_t>(lane * 64);
   const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
   const uint32_t colmap_s = smem_u32(x.colmap), cscale_s = smem_u32(x.cscale);
-  for (int tile = x.pair; tile < p.num_tiles; tile += x.npairs, ++tcount) {
+  for (int tile = x.pair; tile < x.num_tiles; tile += x.npairs, ++tcount) {
     TileMeta t;
-    decode_tile(p, tile, t);
+    decode_tile(p, x.tile_base, tile, t);
     const BranchArgs& br = p.f.branch[t.m];
     const int buf = tcount & 1;
     const uint32_t aph = (tcount >> 1) & 1;
     const float sx = __ldg(br.sx);
-    const int c0 = t.cb * p.BN;
-    const int c1 = min(c0 + p.BN, p.f.O);
-    const int nch = (c1 - c0) >> 3;
+    const int c0 = t.c0, c1 = t.c1;
+    const int nch = (c1 - c0) >> 3;       // at most PIPE_BLOCK_CHANNELS / 8
     const int n_total = t.rowbase[kMaxClusterOrders];
     __syncwarp();
     {
       // accumulator column of (8-channel chunk, order), or -1: entry [chunk][order]
-      for (int e = lane; e < NKMAX * 16; e += 32) {
+      // (entries up to an even chunk count: the drain loads the columns of two chunks at a time, so the chunk
+      // behind an odd count must read as absent)
+      for (int e = lane; e < NKMAX * ((nch + 1) & ~1); e += 32) {
         const int cc = e / NKMAX, ko = e % NKMAX;
         int col = -1;
         if (ko < t.nk && cc < nch) {
@@ -473,10 +491,25 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int64_t tok = token_of(sr0 + 8 * i);
-      srow[i] = br.y + tok * p.f.ldy + c0 + 4 * sj;
+      srow[i] = Q8 ? nullptr : br.y + tok * p.f.ldy + c0 + 4 * sj;
       if (tile_ok && (p.f.conv_on ? inside(sr0 + 8 * i) : tok < p.f.T)) srow_ok |= 1u << i;
     }
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
+    float ostep = 0.f, orcp = 0.f;
+    bool ofast = false;
+    int8_t* qrow = nullptr;      // this lane's output row at channel c0
+    int qalign = 0;              // 16, 4 or 1: widest store every piece of the row allows
+    if constexpr (Q8) {
+      ostep = __ldg(br.out_scale);
+      ofast = quant_step_is_fast(ostep);
+      orcp = ofast ? __frcp_rn(ostep) : 0.f;
+      if (!(ostep >= 0.f && ostep < __uint_as_float(0x7f800000u)) && lane == 0) raise_status(p.f.status, PIPE_ERR_INVALID_ARG);
+      qrow = br.yq + tok_own * p.f.ldyq + c0;
+      // the block starts at a multiple of 8 channels; 16-byte stores need the row piece aligned as well
+      const uintptr_t bits = reinterpret_cast<uintptr_t>(br.yq) | static_cast<uintptr_t>(p.f.ldyq) | static_cast<uintptr_t>(c0);
+      qalign = (bits & 15) == 0 ? 16 : ((bits & 3) == 0 ? 4 : 1);
+      for (int c = lane; c < c1 - c0; c += 32) x.stg[c] = (br.add_bias && p.f.bias) ? __ldg(p.f.bias + c0 + c) : 0.f;
+    }
     const bool add_bias = br.add_bias && p.f.bias;
     const float* bias_q = add_bias ? p.f.bias + c0 + 4 * sj : nullptr;
     const int ngrp = (nch + 1) >> 1;
@@ -488,11 +521,12 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
       const bool quad_ok = 2 * grp + (sj >> 1) < nch;
       float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (add_bias && quad_ok) {
+      if (!Q8 && add_bias && quad_ok) {
         const float* bp = bias_q + 16 * grp;
         bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
       }
-      // ---- this lane's row: 16 channels into the staging block
+      // ---- this lane's row: 16 channels into the staging block (as 16 codes into registers for the fused epilogue)
+      uint32_t packed[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
       for (int sub = 0; sub < 2; sub += CH) {
         int acc[CH][NKMAX][8];
@@ -548,6 +582,30 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
               for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
             }
           }
+          if constexpr (Q8) {
+            // bias last, sigma, then Q of the next layer (Sec. 3.2): eight codes of this lane's own row
+            float bv[8];
+            const uint32_t ba = smem_u32(x.stg) + static_cast<uint32_t>(chunk * 32);
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(bv[0]), "=f"(bv[1]), "=f"(bv[2]), "=f"(bv[3]) : "r"(ba));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(bv[4]), "=f"(bv[5]), "=f"(bv[6]), "=f"(bv[7]) : "r"(ba + 16));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              if (add_bias) y[e] = __fadd_rn(y[e], bv[e]);
+              if (p.f.relu) y[e] = fmaxf(y[e], 0.f);
+            }
+            float uu[8];
+            float edge = ofast ? 0.f : 1.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) uu[e] = quant_magic(y[e], orcp, edge);
+            uint32_t w0 = pack4_low_bytes(uu[0], uu[1], uu[2], uu[3]), w1 = pack4_low_bytes(uu[4], uu[5], uu[6], uu[7]);
+            if (edge >= 0.5f) {   // some estimate sits on a rounding boundary (or the step has no usable reciprocal)
+              w0 = quant4(make_float4(y[0], y[1], y[2], y[3]), ostep, orcp, false);
+              w1 = quant4(make_float4(y[4], y[5], y[6], y[7]), ostep, orcp, false);
+            }
+            packed[2 * (sub + u)] = w0;
+            packed[2 * (sub + u) + 1] = w1;
+            continue;
+          }
           const int j0 = 2 * (sub + u);
           asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>((j0 ^ wsw) << 4)), "f"(y[0]),
                        "f"(y[1]), "f"(y[2]), "f"(y[3])
@@ -556,6 +614,27 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
                        "f"(y[5]), "f"(y[6]), "f"(y[7])
                        : "memory");
         }
+      }
+      if constexpr (Q8) {
+        if (own_ok) {
+          int8_t* dq = qrow + 16 * grp;
+          const int nw = (2 * grp + 1 < nch) ? 4 : 2;   // a tile's last group may hold eight channels only
+          if (qalign == 16 && nw == 4) {
+            *reinterpret_cast<uint4*>(dq) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          } else if (qalign >= 4) {
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+              if (w < nw) reinterpret_cast<uint32_t*>(dq)[w] = packed[w];
+          } else {
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+              if (w < nw) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) dq[4 * w + b] = static_cast<int8_t>(packed[w] >> (8 * b));
+              }
+          }
+        }
+        continue;
       }
       __syncwarp();
       // ---- 8 rows x 64 bytes per store instruction; the bias joins here, after the whole chain
@@ -587,13 +666,15 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   }
 }
 
+template <bool Q8>
 __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
   __shared__ uint64_t pk_bars[kMaxRing * kSub];   // "packed rows have landed", one per block slot of the ring
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][128];    // per epilogue warp: accumulator column of (order, 8-channel chunk) or -1
+  __shared__ int tile_base_s[PIPE_MAX_ORDERS + 1];   // tiles before each branch, then the total
+  __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][kMaxClusterOrders * (PIPE_BLOCK_CHANNELS / 8)];   // per epilogue warp: accumulator column of (8-channel chunk, order) or -1
   __shared__ __align__(16) float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
   __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
 
@@ -616,6 +697,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    int acc = 0;
+    for (int m = 0; m < p.f.num_branches; ++m) {
+      tile_base_s[m] = acc;
+      acc += __ldg(p.f.branch[m].blk) * p.ntt;   // blocks of the branch's table x token-tile pairs
+    }
+    tile_base_s[p.f.num_branches] = acc;
     // The MMA issuer sits in the pair's first CTA, so the barriers it waits on live there and count the
     // arrivals of BOTH CTAs: "stage full" = the first CTA's producer (which posts the bytes of both CTAs'
     // activation tiles) + one unpack warp per block position and CTA; "accumulators drained" = every epilogue warp of the
@@ -643,7 +730,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_slot;
   const uint32_t depth = p.depth;
-  const int my_tiles = (p.num_tiles - g.pair + g.npairs - 1) / g.npairs;
+  g.tile_base = tile_base_s;
+  g.num_tiles = tile_base_s[p.f.num_branches];
+  const int my_tiles = (g.num_tiles - g.pair + g.npairs - 1) / g.npairs;
   const uint32_t total_steps = static_cast<uint32_t>(my_tiles > 0 ? my_tiles : 0) * p.ksteps;   // ring stages
 
   if (warp == 0) {
@@ -663,8 +752,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
           ks = 0;
           tile += g.npairs;
         }
-        const int ttile = 2 * (tile % p.ntt) + g.rank;   // this CTA's 128 token rows of the pair's tile
-        const int m = tile / p.ntt / p.ncb;
+        int m, cb, tt;
+        locate_tile(p, g.tile_base, tile, m, cb, tt);
+        const int ttile = 2 * tt + g.rank;   // this CTA's 128 token rows of the pair's tile
         const int nsub = min(kSub, p.kblocks - ks * kSub);   // the last stage of a tile may hold one block only
         const int kb = ks * kSub + sub;
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
@@ -699,10 +789,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       bool ok = true;
       // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
       auto stacked_rows = [&](int tile) {
-        const int cb = (tile / p.ntt) % p.ncb, m = tile / p.ntt / p.ncb;
+        int m, cb, tt;
+        locate_tile(p, g.tile_base, tile, m, cb, tt);
         const BranchArgs& br = p.f.branch[m];
-        const int c0 = cb * p.BN, c1 = min(c0 + p.BN, p.f.O);
-        const int j0 = c0 / p.f.g, j1 = c1 / p.f.g;
+        const int j0 = __ldg(br.blk + 1 + cb), j1 = __ldg(br.blk + 2 + cb);
         int n = 0;
         for (int k = br.k_begin; k < br.k_end; ++k) {
           const int32_t* cum = p.f.order[k].cum;
@@ -710,10 +800,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
         }
         return n;
       };
-      int n_next = g.pair < p.num_tiles ? stacked_rows(g.pair) : 0;
-      for (int tile = g.pair; ok && tile < p.num_tiles; tile += g.npairs, ++tcount) {
+      int n_next = g.pair < g.num_tiles ? stacked_rows(g.pair) : 0;
+      for (int tile = g.pair; ok && tile < g.num_tiles; tile += g.npairs, ++tcount) {
         const int n_total = n_next;
-        if (tile + g.npairs < p.num_tiles) n_next = stacked_rows(tile + g.npairs);
+        if (tile + g.npairs < g.num_tiles) n_next = stacked_rows(tile + g.npairs);
         const int buf = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
         if (!mbar_wait<true>(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
@@ -752,6 +842,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.rank = g.rank;
     e.pair = g.pair;
     e.npairs = g.npairs;
+    e.tile_base = g.tile_base;
+    e.num_tiles = g.num_tiles;
     e.abort_flag = g.abort_flag;
     e.warp = warp;
     e.lane = lane;
@@ -762,13 +854,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.cscale = epi_cscale[ew];
     e.stg = epi_stage[ew];
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
-      if (p.nkmax <= 2) epilogue_role<2, true>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, true>(p, e);
-      else epilogue_role<8, true>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, true, Q8>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true, Q8>(p, e);
+      else epilogue_role<8, true, Q8>(p, e);
     } else {
-      if (p.nkmax <= 2) epilogue_role<2, false>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, false>(p, e);
-      else epilogue_role<8, false>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, false, Q8>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false, Q8>(p, e);
+      else epilogue_role<8, false, Q8>(p, e);
     }
   }
 
@@ -787,28 +879,75 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
 // ---------------------------------------------------------------------------------------------
 }  // namespace tc2
 
+namespace tc2 {
+
+// What a launch needs to know about the current device, asked once per device: the ring depth that fits its
+// shared memory, the dynamic shared memory to request (the attribute is set on both instantiations then) and how
+// many CTA pairs can be resident.
+struct DeviceSetup {
+  int depth = 0, dyn_smem = 0, max_pairs = 0;
+  pipe_status status = PIPE_ERR_CUDA;
+};
+
+static const DeviceSetup& device_setup() {
+  constexpr int kMaxDevices = 64;
+  static DeviceSetup setups[kMaxDevices];
+  static std::once_flag once[kMaxDevices];
+  static const DeviceSetup bad;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return bad;
+  std::call_once(once[dev], [dev] {
+    DeviceSetup& d = setups[dev];
+    int smem_max = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
+    cudaFuncAttributes f0, f1;
+    if (cudaFuncGetAttributes(&f0, tc2_forward_kernel<false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f1, tc2_forward_kernel<true>) != cudaSuccess) return;
+    const int fixed = static_cast<int>(f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes);
+    d.depth = (smem_max - fixed - 1024) / kStageBytes;   // static shared memory, alignment slack
+    if (d.depth > kMaxRing) d.depth = kMaxRing;
+    d.status = PIPE_ERR_UNSUPPORTED;
+    if (d.depth * kSub != kUnpackWarps) return;   // every unpack warp owns one block slot of the ring
+    d.dyn_smem = d.depth * kStageBytes + 1024;
+    d.status = PIPE_ERR_CUDA;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(sms & ~1, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = d.dyn_smem;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    d.status = PIPE_ERR_UNSUPPORTED;
+    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel<false>, &cfg) != cudaSuccess || n < 1) return;
+    d.max_pairs = n < sms / 2 ? n : sms / 2;
+    d.status = PIPE_OK;
+  });
+  return setups[dev];
+}
+
+}  // namespace tc2
+
 static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   using namespace tc2;
-  static Params p;  // large; filled per call under the lock
-  static std::mutex mu;
-  std::lock_guard<std::mutex> lock(mu);
+  const DeviceSetup& ds = device_setup();
+  if (ds.status != PIPE_OK) return ds.status;
+  Params p;
 
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
   if (max_cluster > kMaxClusterOrders) return PIPE_ERR_UNSUPPORTED;
-  // Widest channel block whose stacked rows fit the 256 accumulator columns in the worst case:
-  // order 1 contributes BN rows, a sparse order at most min(BN, rows it keeps in the whole layer).
-  int BN = 0;
-  for (int cand = 128; cand >= 32 && BN == 0; cand >>= 1) {
-    int worst = 0;
-    for (int m = 0; m < a.num_branches; ++m) {
-      int w = 0;
-      for (int k = a.branch[m].k_begin; k < a.branch[m].k_end; ++k) w += min(cand, a.order[k].rows);
-      worst = max(worst, w);
-    }
-    if (worst <= kMaxN && a.g <= cand && cand % a.g == 0) BN = cand;
-  }
-  if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
+  // every branch needs the channel-block table of its cluster of orders (written by the expansion)
+  for (int m = 0; m < a.num_branches; ++m)
+    if (!a.branch[m].blk) return PIPE_ERR_UNSUPPORTED;
+  if (a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.conv_on && (a.cC % kKStep != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
@@ -818,9 +957,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T > (1ll << 30)) return PIPE_ERR_UNSUPPORTED;
 
   p.f = a;
-  p.BN = BN;
   p.nkmax = max_cluster;
-  p.ncb = ceil_div(a.O, BN);
   p.ntok_tiles = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
   p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
   if (a.conv_on) {
@@ -832,9 +969,8 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   }
   if (p.ntok_tiles < 2) return PIPE_ERR_UNSUPPORTED;   // a pair needs two token tiles; the one-SM kernel takes these
   p.ntt = ceil_div(p.ntok_tiles, 2);
-  const int64_t tiles = static_cast<int64_t>(p.ncb) * p.ntt * a.num_branches;
-  if (tiles > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
-  p.num_tiles = static_cast<int>(tiles);
+  // the tile count is known on the device only (block counts of the tables); a table never has more blocks than groups
+  if (static_cast<int64_t>(a.G) * p.ntt * a.num_branches > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
   p.kblocks = ceil_div(a.I, kKStep);
   p.ksteps = ceil_div(p.kblocks, kSub);
   p.pk = kKStep * a.bits / 8;
@@ -853,16 +989,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
     if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
     p.koff[k] = static_cast<uint32_t>(d >> 4);
   }
-  int dev = 0, smem_max = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
-  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaFuncAttributes fattr;
-  if (cudaFuncGetAttributes(&fattr, tc2_forward_kernel) != cudaSuccess) return PIPE_ERR_CUDA;
-  p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / kStageBytes;  // static shared, alignment slack
-  if (p.depth > kMaxRing) p.depth = kMaxRing;
-  if (p.depth * kSub != kUnpackWarps) return PIPE_ERR_UNSUPPORTED;   // every unpack warp owns one block slot of the ring
-  const int dyn_smem = p.depth * kStageBytes + 1024;
+  p.depth = ds.depth;
 
   if (a.conv_on) {
     if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
@@ -872,41 +999,27 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
                      static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
   }
-  static int attr_bytes = 0;
-  if (attr_bytes < dyn_smem) {
-    if (cudaFuncSetAttribute(tc2_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem) != cudaSuccess)
-      return PIPE_ERR_CUDA;
-    attr_bytes = dyn_smem;
-  }
-  // one cluster of two CTAs per SM pair; how many pairs can be resident is asked of the runtime once
+  // one cluster of two CTAs per SM pair; the tiles (counted on the device) go round all resident pairs
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(2 * ds.max_pairs, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = dyn_smem;
+  cfg.dynamicSmemBytes = ds.dyn_smem;
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  static int max_pairs = 0;
-  if (max_pairs == 0) {
-    cfg.gridDim = dim3(sms & ~1, 1, 1);
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel, &cfg) != cudaSuccess || n < 1) return PIPE_ERR_UNSUPPORTED;
-    max_pairs = n;
-  }
-  const int pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
-  cfg.gridDim = dim3(2 * pairs, 1, 1);
-  if (cudaLaunchKernelEx(&cfg, tc2_forward_kernel, p) != cudaSuccess) return PIPE_ERR_CUDA;
+  const cudaError_t e = a.q8_out ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true>, p) : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false>, p);
+  if (e != cudaSuccess) return PIPE_ERR_CUDA;
   count_launch(1);
   return launch_status();
 }
 
 pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T == 0) return PIPE_OK;
-  if (a.q8_out) return PIPE_ERR_UNSUPPORTED;   // the fused re-quantization lives in the one-SM and decode kernels
   const bool sum_mode = a.num_branches > 1 && a.branch[1].accumulate;
   if (!sum_mode) return launch_tc2(a, stream);
   // Summed ensemble: one launch per branch, in order, so that y = ((y_1 + y_2) + ...) is formed

@@ -96,6 +96,18 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     y.kcodes_off[k] = off;
     off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * y.kernel_row_bytes, 1024);
   }
+  // channel-block tables: predictors 0..M-1, then the cluster of all K orders
+  for (int m = 0; m <= L.M; ++m) {
+    const int nk = (m < L.M) ? bo[m] : L.K;
+    y.blk_off[m] = 0;
+    y.blk_cap[m] = 0;
+    if (nk > 8 || static_cast<int64_t>(nk) * L.g > PIPE_BLOCK_ROWS) continue;
+    // a block that was closed holds at least floor(PIPE_BLOCK_ROWS / (nk * g)) groups
+    const int min_groups = PIPE_BLOCK_ROWS / (nk * L.g);
+    y.blk_cap[m] = ceil_div(L.G, min_groups);
+    y.blk_off[m] = off;
+    off = align_up64(off + static_cast<uint64_t>(y.blk_cap[m] + 2) * 4, 256);
+  }
   if (total > INT32_MAX) return PIPE_ERR_SHAPE;
   y.total_rows = static_cast<int32_t>(total);
   y.blob_bytes = off;

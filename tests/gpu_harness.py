@@ -67,6 +67,44 @@ def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_lay
         if check_kernel_layout:
             np.testing.assert_array_equal(layer.kcodes(k).cpu().numpy(), kernel_layout_from_codes(e.order_codes(k), e.bits),
                                           err_msg=f"streaming layout, order {k}")
+    assert_block_tables_match(layer, e)
+
+
+def expected_block_table(kept_lists, G: int, g: int, row_limit: int = 256, channel_limit: int = 512):
+    """The channel-block table of a cluster of orders as include/pipe.h defines it, from the kept-group lists: walk
+    the groups from 0, close a block when the next group would take its stacked rows past row_limit or its channels
+    past channel_limit."""
+    rows = np.zeros(G, np.int64)
+    for kept in kept_lists:
+        rows[np.asarray(kept)] += g
+    bounds = [0]
+    cur_rows, cur_groups = 0, 0
+    for j in range(G):
+        if cur_groups > 0 and (cur_rows + rows[j] > row_limit or (cur_groups + 1) * g > channel_limit):
+            bounds.append(j)
+            cur_rows, cur_groups = 0, 0
+        cur_rows += int(rows[j])
+        cur_groups += 1
+    bounds.append(G)
+    return np.array([len(bounds) - 1] + bounds, np.int32)
+
+
+def assert_block_tables_match(layer: B.ExpandedLayer, e):
+    """Every channel-block table of the blob against the definition evaluated on the ORACLE's kept lists."""
+    lay = layer.layout
+    M = layer.desc.num_branches
+    split = [lay.branch_orders[m] for m in range(M)]
+    begin = np.concatenate([[0], np.cumsum(split)])
+    for m in range(M + 1):
+        k0, k1 = (int(begin[m]), int(begin[m + 1])) if m < M else (0, e.K)
+        table = layer.block_table(m)
+        if (k1 - k0) > 8 or (k1 - k0) * e.g > 256:
+            assert table is None
+            continue
+        want = expected_block_table([e.order_kept(k) for k in range(k0, k1)], e.G, e.g)
+        got = table.cpu().numpy()
+        assert want[0] <= lay.blk_cap[m]
+        np.testing.assert_array_equal(got[:len(want)], want, err_msg=f"channel-block table {m}")
 
 
 def gpu_quantize(x: np.ndarray, static_scale=None, xd=None):

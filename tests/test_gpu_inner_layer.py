@@ -10,7 +10,7 @@ from tests import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_STREAM, B.KERNEL_AUTO]
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_AUTO]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -197,7 +197,7 @@ def test_inner_layer_argument_errors(oracle):
     for kernel in (B.KERNEL_REFERENCE, B.KERNEL_TCGEN05):
         H.gpu_ensemble_q8(layer, [xq], [sx], [-1.0], kernel=kernel)
         assert B.pipe_poll_status() == B.PIPE_ERR_INVALID_ARG
-    # the two-SM kernel has no such epilogue
+    # the SM-pair kernel needs two token tiles: forced onto 40 tokens it declines
     with pytest.raises(B.PipeError) as ei:
         H.gpu_ensemble_q8(layer, [xq], [sx], [1.0], kernel=B.KERNEL_TCGEN05_PAIR)
     assert ei.value.status == B.PIPE_ERR_UNSUPPORTED

@@ -67,13 +67,17 @@ def test_static_workspace_call_allocates_nothing():
     blob = B.alloc_bytes(B.pipe_layout(desc).blob_bytes)
     B.pipe_expand_weights_static(desc, W, blob)     # warm-up: address look-up, module load
     torch.cuda.synchronize()
+    # (counters of allocation EVENTS, which a tensor freed by the garbage collector in between does not move)
+    def allocation_events():
+        st = torch.cuda.memory_stats()
+        return st["allocation.all.allocated"], st["segment.all.allocated"]
     free0, _ = torch.cuda.mem_get_info()
-    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    events0, reserved0 = allocation_events(), torch.cuda.memory_reserved()
     B.pipe_expand_weights_static(desc, W, blob)
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
     assert free1 == free0, "device memory changed across a call that must not allocate"
-    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert allocation_events() == events0 and torch.cuda.memory_reserved() == reserved0
     assert B.pipe_poll_status() == B.PIPE_OK
 
 
