@@ -88,11 +88,15 @@ typedef struct pipe_layer_desc {
  * Channel-block tables, one per cluster of orders that a forward call can evaluate on one input: entry m < M
  * for predictor m (Sec. 3.2), entry M for all K orders (pipe_expanded_linear, pipe_expanded_conv2d).
  *   blk_off[m]    int32 [2 + blk_cap[m]]: n, then b_0 = 0 < b_1 < ... < b_n = G.  Block i is the channel groups
- *                 b_i .. b_{i+1} - 1; the blocks are cut greedily from group 0 so that the rows a block stacks over
- *                 the cluster's orders (kept groups only) stay within PIPE_BLOCK_ROWS and its channels within
- *                 PIPE_BLOCK_CHANNELS -- the unit of work of the SM-pair tensor-core kernel, whose MMAs then always
- *                 run close to their widest shape however sparse the orders are.  A cluster of more than 8 orders,
- *                 or whose single group can exceed the row limit (orders * g > PIPE_BLOCK_ROWS), has no table.
+ *                 b_i .. b_{i+1} - 1.  With R the rows the cluster's orders keep in the whole layer and
+ *                 n0 = max(ceil(R / PIPE_BLOCK_ROWS), ceil(O / PIPE_BLOCK_CHANNELS)) the fewest blocks that could
+ *                 hold them, the limit of a block is L = min(PIPE_BLOCK_ROWS, roundup(ceil(R / n0), 16) + orders * g):
+ *                 the groups are walked from 0 and a block is closed when the next group would take the rows it
+ *                 stacks over the cluster's orders (kept groups only) beyond L or its channels beyond
+ *                 PIPE_BLOCK_CHANNELS.  Blocks are the unit of work of the SM-pair tensor-core kernel, whose MMAs then
+ *                 run close to their widest shape, and evenly, however sparse the orders are.  A cluster of more
+ *                 than 8 orders, or whose single group can exceed the row limit (orders * g > PIPE_BLOCK_ROWS), has
+ *                 no table.
  */
 #define PIPE_BLOCK_ROWS 256
 #define PIPE_BLOCK_CHANNELS 512

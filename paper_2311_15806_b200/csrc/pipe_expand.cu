@@ -365,6 +365,7 @@ struct BlockTableArgs {
   int nk[PIPE_MAX_ORDERS + 1];
   int32_t* out[PIPE_MAX_ORDERS + 1];
   int cap[PIPE_MAX_ORDERS + 1];
+  int limit[PIPE_MAX_ORDERS + 1];   // rows a block of the cluster may stack
   int G, g;
 };
 
@@ -389,7 +390,7 @@ __global__ void block_table_kernel(const __grid_constant__ BlockTableArgs a) {
       if (base == 0) out[1] = 0;
       for (int j = 0; j < cnt; ++j) {
         const int r = rows_s[j];
-        if (cur_groups > 0 && (cur_rows + r > PIPE_BLOCK_ROWS || cur_groups + 1 > max_groups)) {
+        if (cur_groups > 0 && (cur_rows + r > a.limit[m] || cur_groups + 1 > max_groups)) {
           if (n < a.cap[m]) out[2 + n] = base + j;   // (the capacity bound holds by construction; never write past it)
           ++n;
           cur_rows = 0;
@@ -502,6 +503,13 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
       for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
       t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.blk_off[m]);
       t.cap[m] = L.lay.blk_cap[m];
+      // even blocks: the fewest blocks that could hold the cluster's rows, their mean size plus one group of slack
+      int64_t R = 0;
+      for (int k = k0; k < k1; ++k) R += L.lay.rows[k];
+      const int64_t n0r = ceil_div<int64_t>(R, PIPE_BLOCK_ROWS), n0c = ceil_div<int64_t>(L.O, PIPE_BLOCK_CHANNELS);
+      const int64_t n0 = n0r > n0c ? n0r : n0c;
+      const int64_t even = round_up<int64_t>(ceil_div<int64_t>(R, n0), 16) + static_cast<int64_t>(k1 - k0) * L.g;
+      t.limit[m] = static_cast<int>(even < PIPE_BLOCK_ROWS ? even : PIPE_BLOCK_ROWS);
       any = true;
     }
     if (any) {

@@ -43,6 +43,7 @@ constexpr int kBtBytes = (kMaxN / 2) * kKStep;   // 16 KiB per block: this CTA's
 constexpr int kStageBytes = kSub * (kABytes + kBtBytes);   // [kSub activation tiles][kSub B tiles]
 constexpr int kStageBOff = kSub * kABytes;
 constexpr int kTmemCols = 512;
+constexpr int kColmapEntries = kMaxClusterOrders * (PIPE_BLOCK_CHANNELS / 8);
 constexpr int kAccCols = 256;
 constexpr int kMaxRing = 3;
 constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
@@ -378,6 +379,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
 
 struct EpiCtx {
   uint32_t tmem_base, tfull0, tempty0;
+  uint32_t tables0;   // two barriers: the tile tables of an even / odd tile are complete
   volatile int* abort_flag;
   int warp, lane;
   int rank, pair, npairs;
@@ -385,7 +387,7 @@ struct EpiCtx {
   int num_tiles;
   uint32_t tempty_lead0;   // the accumulator-released barriers of the pair's first CTA (cluster address)
   int part, nparts;  // share of the 16-channel groups this warp drains (two warps per lane quarter)
-  int16_t* colmap;
+  int16_t* colmap;   // two copies of the tile tables (even / odd tiles), shared by the CTA's epilogue warps
   float* cscale;
   float* stg;        // 32 rows x 16 floats, swizzled
 };
@@ -417,7 +419,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   const int sj = spp ^ ((sr0 >> 1) & 3);     // the same for all four rows (they differ by multiples of 8)
   const uint32_t stg_w = smem_u32(x.stg) + static_cast<uint32_t>(lane * 64);
   const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
-  const uint32_t colmap_s = smem_u32(x.colmap), cscale_s = smem_u32(x.cscale);
+  const int et = (x.warp - 2 - kUnpackWarps) * 32 + lane;   // this thread among the epilogue threads
   for (int tile = x.pair; tile < x.num_tiles; tile += x.npairs, ++tcount) {
     TileMeta t;
     decode_tile(p, x.tile_base, tile, t);
@@ -428,12 +430,17 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     const int c0 = t.c0, c1 = t.c1;
     const int nch = (c1 - c0) >> 3;       // at most PIPE_BLOCK_CHANNELS / 8
     const int n_total = t.rowbase[kMaxClusterOrders];
-    __syncwarp();
+    // The tables of the tile are built ONCE per CTA, by all epilogue threads together, in the copy of the tile's
+    // parity: a warp that runs ahead into the next tile writes the other copy, and nobody reaches the tile after
+    // that before every warp has passed this tile's barrier, i.e. has finished reading the copy of the tile before.
+    int16_t* colmap = x.colmap + buf * kColmapEntries;
+    float* cscale = x.cscale + buf * kMaxN;
+    const uint32_t colmap_s = smem_u32(colmap), cscale_s = smem_u32(cscale);
     {
       // accumulator column of (8-channel chunk, order), or -1: entry [chunk][order]
       // (entries up to an even chunk count: the drain loads the columns of two chunks at a time, so the chunk
       // behind an odd count must read as absent)
-      for (int e = lane; e < NKMAX * ((nch + 1) & ~1); e += 32) {
+      for (int e = et; e < NKMAX * ((nch + 1) & ~1); e += 32 * kEpiWarps) {
         const int cc = e / NKMAX, ko = e % NKMAX;
         int col = -1;
         if (ko < t.nk && cc < nch) {
@@ -451,9 +458,9 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
           const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
           if (hi > lo) col = rb + lo * p.f.g + c % p.f.g - st;
         }
-        x.colmap[e] = static_cast<int16_t>(col);
+        colmap[e] = static_cast<int16_t>(col);
       }
-      for (int r = lane; r < n_total; r += 32) {
+      for (int r = et; r < n_total; r += 32 * kEpiWarps) {
         int rb = 0, st = t.start[0];
         const float* sc = p.f.order[t.k0].scales;
 #pragma unroll
@@ -463,8 +470,13 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
             st = t.start[u];
             sc = p.f.order[t.k0 + u].scales;
           }
-        x.cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
+        cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
       }
+      // every epilogue warp has written its share (a bounded wait, like all others: a warp that leaves on an abort
+      // must not leave the rest stuck in a barrier that cannot time out)
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x.tables0 + 8u * buf);
+      if (!mbar_wait(x.tables0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
     }
     // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
     // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
@@ -671,11 +683,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
   __shared__ uint64_t pk_bars[kMaxRing * kSub];   // "packed rows have landed", one per block slot of the ring
+  __shared__ uint64_t tbl_bars[2];                // "tile tables complete", even / odd tile
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_base_s[PIPE_MAX_ORDERS + 1];   // tiles before each branch, then the total
-  __shared__ __align__(16) int16_t epi_colmap[kEpiWarps][kMaxClusterOrders * (PIPE_BLOCK_CHANNELS / 8)];   // per epilogue warp: accumulator column of (8-channel chunk, order) or -1
-  __shared__ __align__(16) float epi_cscale[kEpiWarps][kMaxN];    // per epilogue warp: s_k * lambda_x of every stacked row
+  __shared__ __align__(16) int16_t epi_colmap[2][kColmapEntries];   // even / odd tile: accumulator column of (8-channel chunk, order) or -1
+  __shared__ __align__(16) float epi_cscale[2][kMaxN];             // even / odd tile: s_k * lambda_x of every stacked row
   __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -712,6 +725,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       mbar_init(g.done0 + 8u * s, 1);
     }
     for (int s = 0; s < kMaxRing * kSub; ++s) mbar_init(smem_u32(&pk_bars[s]), 1);
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&tbl_bars[b]), kEpiWarps);
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
       mbar_init(g.tempty0 + 8u * b, 2 * kEpiWarps);
@@ -838,6 +852,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.tmem_base = tmem_base;
     e.tfull0 = g.tfull0;
     e.tempty0 = g.tempty0;
+    e.tables0 = smem_u32(tbl_bars);
     e.tempty_lead0 = g.tempty_lead0;
     e.rank = g.rank;
     e.pair = g.pair;
@@ -850,8 +865,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     const int ew = warp - 2 - kUnpackWarps;
     e.part = ew >> 2;
     e.nparts = kEpiWarps / 4;
-    e.colmap = epi_colmap[ew];
-    e.cscale = epi_cscale[ew];
+    e.colmap = &epi_colmap[0][0];
+    e.cscale = &epi_cscale[0][0];
     e.stg = epi_stage[ew];
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
       if (p.nkmax <= 2) epilogue_role<2, true, Q8>(p, e);

@@ -102,9 +102,7 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     y.blk_off[m] = 0;
     y.blk_cap[m] = 0;
     if (nk > 8 || static_cast<int64_t>(nk) * L.g > PIPE_BLOCK_ROWS) continue;
-    // a block that was closed holds at least floor(PIPE_BLOCK_ROWS / (nk * g)) groups
-    const int min_groups = PIPE_BLOCK_ROWS / (nk * L.g);
-    y.blk_cap[m] = ceil_div(L.G, min_groups);
+    y.blk_cap[m] = L.G;   // a block holds at least one group
     y.blk_off[m] = off;
     off = align_up64(off + static_cast<uint64_t>(y.blk_cap[m] + 2) * 4, 256);
   }

@@ -70,13 +70,17 @@ def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_lay
     assert_block_tables_match(layer, e)
 
 
-def expected_block_table(kept_lists, G: int, g: int, row_limit: int = 256, channel_limit: int = 512):
-    """The channel-block table of a cluster of orders as include/pipe.h defines it, from the kept-group lists: walk
-    the groups from 0, close a block when the next group would take its stacked rows past row_limit or its channels
-    past channel_limit."""
+def expected_block_table(kept_lists, G: int, g: int, row_max: int = 256, channel_limit: int = 512):
+    """The channel-block table of a cluster of orders as include/pipe.h defines it, from the kept-group lists: the
+    row limit is the mean block size for the fewest possible blocks plus one group of every order (at most row_max);
+    walk the groups from 0, close a block when the next group would take its stacked rows past the limit or its
+    channels past channel_limit."""
     rows = np.zeros(G, np.int64)
     for kept in kept_lists:
         rows[np.asarray(kept)] += g
+    R = int(rows.sum())
+    n0 = max(-(-R // row_max), -(-(G * g) // channel_limit))
+    row_limit = min(row_max, (-(-(-(-R // n0)) // 16)) * 16 + len(kept_lists) * g)
     bounds = [0]
     cur_rows, cur_groups = 0, 0
     for j in range(G):
