@@ -15,6 +15,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "pipe_oracle.c")
+_SRC_EXT = os.path.join(_HERE, "pipe_oracle_ext.c")
 _LIB = os.path.join(_HERE, "libpipe_oracle.so")
 
 OK, ERR_ARG, ERR_NONFINITE, ERR_ACC_OVERFLOW = 0, 1, 2, 3
@@ -22,9 +23,9 @@ OK, ERR_ARG, ERR_NONFINITE, ERR_ACC_OVERFLOW = 0, 1, 2, 3
 
 def build(force: bool = False) -> str:
     """Compile the oracle (plain C, -O2, OpenMP over rows, no contraction of a*b+c)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_EXT)):
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
-               "-fno-fast-math", "-Wall", "-o", _LIB, _SRC, "-lm"]
+               "-fno-fast-math", "-Wall", "-o", _LIB, _SRC, _SRC_EXT, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -51,6 +52,15 @@ def lib() -> C.CDLL:
         _lib.pipe_oracle_balanced_split.argtypes = [C.c_int, C.c_int, p]
         _lib.pipe_oracle_keep_groups.argtypes = [i32, C.c_double]
         _lib.pipe_oracle_keep_groups.restype = i32
+        # pipe_oracle_ext.c
+        _lib.pipe_oracle_select_groups_ex.argtypes = [p, i64, i64, i32, i32, C.c_int, p, p]
+        _lib.pipe_oracle_expand_ex.argtypes = [p, i64, i64, i64, C.c_int, C.c_int, i32, i32, C.c_int, i64, p, p, p, p, p]
+        _lib.pipe_oracle_container_bits.argtypes = [C.c_int]
+        _lib.pipe_oracle_pack_ex.argtypes = [p, i64, i64, C.c_int, p]
+        _lib.pipe_oracle_quantize_act_ex.argtypes = [p, i64, i64, i64, C.c_int, C.c_int, p, p, p, i64, p, p]
+        _lib.pipe_oracle_forward_zp.argtypes = [p, i64, i64, i64, i64, C.c_int, i32, p, p, p, p, C.c_int, C.c_int,
+                                                C.c_float, i32, p, p, i64, p, p, p, p]
+        _lib.pipe_oracle_activation.argtypes = [p, i64, C.c_int, p]
     return _lib
 
 
@@ -123,6 +133,8 @@ class Expansion:
         return (kg[:, None] * self.g + np.arange(self.g)[None, :]).reshape(-1)
 
     def packed(self, k: int) -> np.ndarray:
+        if self.bits in (3, 6):
+            return pack_ex(self.order_codes(k), self.bits)
         return pack(self.order_codes(k), self.bits)
 
 
@@ -175,6 +187,91 @@ def quantize_act(x: np.ndarray, static_scale: float | None = None):
     ss = None if static_scale is None else np.array([static_scale], np.float32)
     _check(lib().pipe_oracle_quantize_act(_ptr(x), T, I, I, _ptr(ss), _ptr(xq), I, _ptr(sx)))
     return xq, np.float32(sx[0])
+
+
+# ---- variants beside the main setting (pipe_oracle_ext.c) --------------------------------------------------
+SCORE_MAXABS, SCORE_L2 = 0, 1
+ACT_IDENTITY, ACT_RELU, ACT_SILU, ACT_GELU, ACT_SIGMOID = 0, 1, 2, 3, 4
+
+
+def container_bits(bits: int) -> int:
+    return int(lib().pipe_oracle_container_bits(bits))
+
+
+def select_groups_ex(r: np.ndarray, g: int, n_keep: int, score_mode: int):
+    """Kept groups (ascending) and the scores [G] (binary64) of the residual r [O, I]."""
+    r = _c(r, np.float32)
+    O, I = r.shape
+    out = np.empty(n_keep, np.int32)
+    score = np.empty(O // g, np.float64)
+    _check(lib().pipe_oracle_select_groups_ex(_ptr(r), O, I, g, n_keep, score_mode, _ptr(out), _ptr(score)))
+    return out, score
+
+
+def expand_ex(W: np.ndarray, bits: int, K: int, g: int, n_keep: int, score_mode: int = 0, elem_keep: int = 0) -> Expansion:
+    """The expansion for b in {2, 3, 4, 6, 8}, either group score, optionally the unstructured mask."""
+    W = _c(W, np.float32)
+    O, I = W.shape
+    G = O // g
+    R_max = O + (K - 1) * n_keep * g
+    codes = np.zeros((R_max, I), np.int8)
+    scales = np.zeros(R_max, np.float32)
+    kept = np.full((K, G), -1, np.int32)
+    kept_count = np.zeros(K, np.int32)
+    residual = np.empty((O, I), np.float32)
+    _check(lib().pipe_oracle_expand_ex(_ptr(W), O, I, I, bits, K, g, n_keep, score_mode, elem_keep, _ptr(codes), _ptr(scales),
+                                       _ptr(kept), _ptr(kept_count), _ptr(residual)))
+    R = int(kept_count.astype(np.int64).sum()) * g
+    return Expansion(O, I, bits, K, g, n_keep, codes[:R], scales[:R], kept, kept_count, residual, np.zeros((K, O), np.float32))
+
+
+def pack_ex(codes: np.ndarray, bits: int) -> np.ndarray:
+    codes = _c(codes, np.int8)
+    rows, I = codes.shape
+    per = 8 // container_bits(bits)
+    out = np.empty((rows, (I + per - 1) // per), np.uint8)
+    _check(lib().pipe_oracle_pack_ex(_ptr(codes), rows, I, bits, _ptr(out)))
+    return out
+
+
+def quantize_act_ex(x: np.ndarray, act_bits: int = 8, asymmetric: bool = False, static_scale: float | None = None,
+                    static_range=None):
+    """Returns (codes int8 [T, I], lambda_x, zero point)."""
+    x = _c(x, np.float32)
+    T, I = x.shape
+    xq = np.empty((T, I), np.int8)
+    sx = np.zeros(1, np.float32)
+    zp = np.zeros(1, np.int32)
+    ss = None if static_scale is None else np.array([static_scale], np.float32)
+    sr = None if static_range is None else np.array(static_range, np.float32)
+    _check(lib().pipe_oracle_quantize_act_ex(_ptr(x), T, I, I, act_bits, int(bool(asymmetric)), _ptr(ss), _ptr(sr), _ptr(xq), I,
+                                             _ptr(sx), _ptr(zp)))
+    return xq, np.float32(sx[0]), int(zp[0])
+
+
+def forward_zp(e: Expansion, xq: np.ndarray, sx, zero_point: int, k_begin: int = 0, k_end: int | None = None,
+               bias: np.ndarray | None = None):
+    """`forward` on asymmetric codes: the contraction runs on (c - zero_point).  Returns (Forward, rowsum int64 [R_total])."""
+    xq = _c(xq, np.int8)
+    T, I = xq.shape
+    k_end = e.K if k_end is None else k_end
+    y = np.empty((T, e.O), np.float32)
+    y64 = np.empty((T, e.O), np.float64)
+    yabs = np.empty((T, e.O), np.float64)
+    partials = np.zeros((T, e.R_total), np.int32)
+    rowsum = np.zeros(e.R_total, np.int64)
+    b = None if bias is None else _c(bias, np.float32)
+    _check(lib().pipe_oracle_forward_zp(_ptr(xq), T, I, I, e.O, e.K, e.g, _ptr(e.codes), _ptr(e.scales), _ptr(e.kept),
+                                        _ptr(e.kept_count), k_begin, k_end, C.c_float(float(sx)), int(zero_point), _ptr(b),
+                                        _ptr(y), e.O, _ptr(y64), _ptr(yabs), _ptr(partials), _ptr(rowsum)))
+    return Forward(y, y64, yabs, partials), rowsum
+
+
+def activation(v: np.ndarray, kind: int) -> np.ndarray:
+    v = _c(v, np.float32)
+    out = np.empty_like(v)
+    _check(lib().pipe_oracle_activation(_ptr(v), v.size, kind, _ptr(out)))
+    return out
 
 
 def forward_requantized(e: "Expansion", xq: np.ndarray, sx, out_scale: float, k_begin: int = 0, k_end: int | None = None,
