@@ -53,13 +53,25 @@ typedef enum {
 typedef struct pipe_layer_desc {
   int32_t out_features;  /* O: rows of W = output channels */
   int32_t in_features;   /* I: reduction length; a multiple of the codes per byte (1, 2, 4) */
-  int32_t weight_bits;   /* b: 8, 4, or 2 (2 = ternary {-1,0,+1}); activations are int8 */
+  int32_t weight_bits;   /* b: 8, 6, 4, 3 or 2 (2 = ternary {-1,0,+1}; Sec. 4.2 runs int3, int4, int6 and ternary).
+                            Codes lie in [-(2^(b-1) - 1), 2^(b-1) - 1]; 3-bit codes are stored in the 4-bit format and
+                            6-bit codes in the 8-bit format (every layout below then reads b = 4 resp. b = 8) */
   int32_t num_orders;    /* K, 1..PIPE_MAX_ORDERS */
   int32_t group_size;    /* g: consecutive output channels per sparsity group; divides O */
   int32_t keep_groups;   /* groups kept by every order >= 2, 1..O/g (order 1 is dense) */
   int32_t num_branches;  /* M, 1..K */
   int32_t branch_orders[PIPE_MAX_ORDERS]; /* K_m, sum = K; all zero = balanced default */
+  int32_t score_mode;    /* score of the structured mask (Sec. 3.1 names no criterion): PIPE_SCORE_MAXABS = largest
+                            magnitude of the current residual over the group's rows; PIPE_SCORE_L2 = its squared
+                            Euclidean norm, summed in binary64 in the fixed order given at pipe_expand_weights */
+  int32_t keep_elems;    /* 0, or the unstructured mask of Sec. 3.1 for the orders >= 2: in every row only the
+                            keep_elems entries of the current residual with the largest magnitude are quantized (ties
+                            to the lower index), the others get the code 0 and keep their residual.  Needs
+                            keep_groups = G: an unstructured R^k keeps every row */
 } pipe_layer_desc;
+
+#define PIPE_SCORE_MAXABS 0
+#define PIPE_SCORE_L2 1
 
 /*
  * Byte layout of the expanded-layer blob and the workspace sizes, as computed by
@@ -178,6 +190,11 @@ pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out);
  *              a zero scale gives zero codes and an unchanged residual
  *     rows of pruned groups keep their residual (R^k has a zero row there).
  * d_W: float [O, I], pitch ldw, 4-byte aligned (16-byte aligned rows take the fast path).
+ * PIPE_SCORE_L2: the score of group j is sum over its rows o (ascending) of S[o], binary64, where
+ *     S[o] = tree(P_0..P_31), P_l = sum over i = l, l+32, ... (ascending) of (double) r[o,i]^2, and the tree adds
+ *     P_l += P_{l+off} for off = 16, 8, 4, 2, 1 (a sum of squares depends on the order of its additions in the last
+ *     bits, and the kept lists are compared bit for bit, so the order is part of the definition).
+ * keep_elems > 0: see pipe_layer_desc.
  * d_blob: blob_bytes bytes aligned to PIPE_BLOB_ALIGN; fully overwritten.
  * d_ws: expand_ws_bytes bytes, 256-byte aligned; contents undefined afterwards.
  * Non-finite weights set PIPE_ERR_NONFINITE in the device status word.
@@ -229,6 +246,22 @@ pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I, int64_t ld
                               int8_t* d_xq, int64_t ldxq, float* d_sx, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
+ * The activation quantizers of Sec. 4.3 beside the int8 symmetric one: A6 and A4 ("150 % x W4/A6", W4/A4) and
+ * asymmetric quantization (the parallelized comparison).  Codes are int8 values in every case, so the GEMM calls
+ * take them unchanged.
+ *   symmetric (asymmetric = 0), act_bits in {8, 6, 4}: qx = 2^(b-1) - 1, lambda_x = max|x| / qx or the static
+ *       scale, c = clamp(rne(x / lambda_x), -qx, qx); *d_zp = 0.
+ *   asymmetric: lo = min(x, 0), hi = max(x, 0) over the tensor, or d_static_range = {lo, hi} (lo <= 0 <= hi);
+ *       lambda_x = (hi - lo) / (2^b - 1); z = clamp(rne(-2^(b-1) - lo / lambda_x)), c = clamp(rne(x / lambda_x) + z),
+ *       both clamped to [-2^(b-1), 2^(b-1) - 1]; x ~ lambda_x * (c - z).  *d_zp = z is what
+ *       pipe_ensemble_forward_zp takes.  d_static_scale must be NULL.
+ * d_zp: one int32 (written).  Everything else as in pipe_quantize_act (binary32, IEEE division, ties to even).
+ */
+pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t I, int64_t ldx, int32_t act_bits, int32_t asymmetric,
+                                 const float* d_static_scale, const float* d_static_range, int8_t* d_xq, int64_t ldxq,
+                                 float* d_sx, int32_t* d_zp, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
  * Appendix B, Eq. 9 without the activation function: all K orders on one input,
  *     acc_k[t,o] = sum_i xq[t,i] * q_k[o,i]                    (exact int32)
  *     y[t,o]     = sum_{k ascending, o kept at k} fma(float(acc_k[t,o]), s_k[o] * lambda_x, .) (+ b[o])
@@ -259,6 +292,19 @@ pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blo
                                   int64_t T, int64_t ldxq, const float* const* h_sx_m, const float* d_bias,
                                   float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials,
                                   void* stream);
+
+/*
+ * pipe_ensemble_forward on asymmetric activation codes (Sec. 4.3): with x_m ~ lambda_{x_m} (c_m - z_m) the
+ * contraction is acc_k[t,o] = sum_i (c_m[t,i] - z_m) * q_k[o,i], an exact integer that the kernel forms as
+ * sum_i c q - z_m * sum_i q; everything after it is unchanged.  h_zp_m: HOST array of M device pointers to one int32
+ * each (NULL entries mean 0).  d_partials receives acc_k with the zero point taken out.  PIPE_ERR_ACC_OVERFLOW
+ * cannot be excluded by the descriptor alone here: |c - z| reaches 255, so the layer must satisfy
+ * 255 * qmax * I < 2^31 (checked).  Runs on the CUDA-core kernel.
+ */
+pipe_status pipe_ensemble_forward_zp(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                     int64_t T, int64_t ldxq, const float* const* h_sx_m, const int32_t* const* h_zp_m,
+                                     const float* d_bias, float* const* h_y_m, int64_t ldy, int32_t sum_branches,
+                                     int32_t* d_partials, void* stream);
 
 /*
  * An INNER layer of the M predictors (Sec. 3.2, Fig. 2; Appendix B, Eq. 9 with its activation

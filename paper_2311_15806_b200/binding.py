@@ -30,7 +30,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
            "pipe_bit_ops_original", "pipe_bit_ops_expanded", "pipe_max_orders_within_original", "pipe_gamma_from_budget",
            "pipe_expand_weights_static",
-           "pipe_quantize_act", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
+           "pipe_quantize_act", "pipe_quantize_act_ex", "pipe_ensemble_forward_zp", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
            "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string",
            # include/pipe_diag.h: tests and measurements only
@@ -40,7 +40,8 @@ EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout"
 class LayerDesc(C.Structure):
     _fields_ = [("out_features", C.c_int32), ("in_features", C.c_int32), ("weight_bits", C.c_int32),
                 ("num_orders", C.c_int32), ("group_size", C.c_int32), ("keep_groups", C.c_int32),
-                ("num_branches", C.c_int32), ("branch_orders", C.c_int32 * MAX_ORDERS)]
+                ("num_branches", C.c_int32), ("branch_orders", C.c_int32 * MAX_ORDERS),
+                ("score_mode", C.c_int32), ("keep_elems", C.c_int32)]
 
 
 class ConvGeom(C.Structure):
@@ -91,6 +92,8 @@ def lib() -> C.CDLL:
         L.pipe_expand_weights.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p, sz, p]
         L.pipe_expand_weights_static.argtypes = [C.POINTER(LayerDesc), p, i64, p, sz, p]
         L.pipe_quantize_act.argtypes = [p, i64, i32, i64, p, p, i64, p, p, sz, p]
+        L.pipe_quantize_act_ex.argtypes = [p, i64, i32, i64, i32, i32, p, p, p, i64, p, p, p, sz, p]
+        L.pipe_ensemble_forward_zp.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, p, i64, i32, p, p]
         L.pipe_expanded_linear.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, p, p]
         L.pipe_expanded_conv2d.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, p, i64, p, p]
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
@@ -168,11 +171,15 @@ def pipe_default_branches(K: int, M: int) -> list[int]:
     return [int(out[m]) for m in range(M)]
 
 
+SCORE_MAXABS, SCORE_L2 = 0, 1
+
+
 def make_desc(O: int, I: int, bits: int, K: int, g: int, keep_groups: int, M: int = 1,
-              branch_orders=None) -> LayerDesc:
+              branch_orders=None, score_mode: int = 0, keep_elems: int = 0) -> LayerDesc:
     d = LayerDesc()
     d.out_features, d.in_features, d.weight_bits, d.num_orders = O, I, bits, K
     d.group_size, d.keep_groups, d.num_branches = g, keep_groups, M
+    d.score_mode, d.keep_elems = score_mode, keep_elems
     if branch_orders is not None:
         for m, v in enumerate(branch_orders):
             d.branch_orders[m] = int(v)
@@ -210,6 +217,36 @@ def pipe_quantize_act(x: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, ws: t
     ldxq = xq.stride(0) if T > 1 else max(I, xq.stride(0))
     _check(lib().pipe_quantize_act(_dp(x), T, I, ldx, _dp(static_scale), _dp(xq), ldxq, _dp(sx), _dp(ws), ws.numel(),
                                    _stream_ptr(stream)), "pipe_quantize_act")
+
+
+def pipe_quantize_act_ex(x: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, zp: torch.Tensor, ws: torch.Tensor, act_bits: int = 8,
+                         asymmetric: bool = False, static_scale: torch.Tensor | None = None,
+                         static_range: torch.Tensor | None = None, stream=None) -> None:
+    """x: cuda float32 [T, I]; xq: cuda int8 [T, I]; sx: cuda float32 [1]; zp: cuda int32 [1]; ws: cuda uint8 >= 256 bytes."""
+    assert x.is_cuda and x.dtype == torch.float32 and xq.dtype == torch.int8 and zp.dtype == torch.int32
+    T, I = x.shape
+    ldx = x.stride(0) if T > 1 else max(I, x.stride(0))
+    ldxq = xq.stride(0) if T > 1 else max(I, xq.stride(0))
+    _check(lib().pipe_quantize_act_ex(_dp(x), T, I, ldx, int(act_bits), 1 if asymmetric else 0, _dp(static_scale), _dp(static_range),
+                                      _dp(xq), ldxq, _dp(sx), _dp(zp), _dp(ws), ws.numel(), _stream_ptr(stream)), "pipe_quantize_act_ex")
+
+
+def pipe_ensemble_forward_zp(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, zp_m, y_m, bias: torch.Tensor | None = None,
+                             sum_branches: bool = False, partials: torch.Tensor | None = None, stream=None) -> None:
+    """pipe_ensemble_forward on asymmetric codes; zp_m: sequence of M cuda int32 one-element tensors (or None entries)."""
+    M = desc.num_branches
+    assert len(xq_m) == M and len(sx_m) == M and len(zp_m) == M and len(y_m) >= (1 if sum_branches else M)
+    T = xq_m[0].shape[0]
+    ldxq = xq_m[0].stride(0) if T > 1 else max(xq_m[0].shape[1], xq_m[0].stride(0))
+    ldy = y_m[0].stride(0) if T > 1 else max(y_m[0].shape[1], y_m[0].stride(0))
+    PA = C.c_void_p * M
+    xp = PA(*[_dp(t) for t in xq_m])
+    sp = PA(*[_dp(t) for t in sx_m])
+    zp = PA(*[_dp(t) for t in zp_m])
+    yp = PA(*[(_dp(y_m[m]) if m < len(y_m) else None) for m in range(M)])
+    _check(lib().pipe_ensemble_forward_zp(C.byref(desc), _dp(blob), xp, T, ldxq, sp, zp, _dp(bias), yp, ldy,
+                                          1 if sum_branches else 0, _dp(partials), _stream_ptr(stream)),
+           "pipe_ensemble_forward_zp")
 
 
 def pipe_expanded_linear(desc: LayerDesc, blob: torch.Tensor, xq: torch.Tensor, sx: torch.Tensor, y: torch.Tensor,

@@ -15,7 +15,9 @@ constexpr int kKernelKAlign = 128;  // kernel-layout rows are padded to this man
 
 // Resolved, validated view of a pipe_layer_desc.
 struct LayerInfo {
-  int O, I, bits, K, g, G, n_keep, M;
+  int O, I, bits, K, g, G, n_keep, M;   // bits: the storage format of the codes (8, 4 or 2)
+  int wbits;             // b of the quantizer (8, 6, 4, 3 or 2): qmax = 2^(b-1) - 1
+  int score_mode, keep_elems;
   int qmax;
   int branch_begin[PIPE_MAX_ORDERS + 1];  // first order (0-based) of every branch, then K
   pipe_layer_layout lay;
@@ -112,6 +114,7 @@ struct BranchArgs {
   int8_t* yq;              // re-quantized output (ForwardArgs::q8_out), else unused
   const float* out_scale;  // its step: one float on the device
   int k_begin, k_end;
+  const int32_t* zp;       // zero point of asymmetric activation codes (one int on the device), or nullptr for 0
   const int32_t* blk;      // channel-block table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
   int add_bias;    // bias enters this branch
   int accumulate;  // y += result (summed ensemble, branches after the first)

@@ -55,10 +55,11 @@ __global__ void group_score_kernel(const float* __restrict__ a, int G, int g, fl
 // keep[j] = 1 iff fewer than n_keep groups precede j in the order (score descending, index
 // ascending).  Scores are non-negative finite floats, so the comparison is exact and the
 // result does not depend on any reduction order.
-__global__ void group_rank_kernel(const float* __restrict__ score, int G, int n_keep, int32_t* __restrict__ keep) {
-  __shared__ float tile[1024];
+template <typename S>
+__global__ void group_rank_kernel(const S* __restrict__ score, int G, int n_keep, int32_t* __restrict__ keep) {
+  __shared__ S tile[1024];
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  const float sj = j < G ? score[j] : 0.f;
+  const S sj = j < G ? score[j] : S(0);
   int rank = 0;
   for (int base = 0; base < G; base += 1024) {
     const int n = min(1024, G - base);
@@ -67,12 +68,92 @@ __global__ void group_rank_kernel(const float* __restrict__ score, int G, int n_
     __syncthreads();
     if (j < G) {
       for (int t = 0; t < n; ++t) {
-        const float si = tile[t];
+        const S si = tile[t];
         rank += (si > sj) || (si == sj && base + t < j);
       }
     }
   }
   if (j < G) keep[j] = rank < n_keep ? 1 : 0;
+}
+
+// Second score of the structured mask (PIPE_SCORE_L2): the squared Euclidean norm of the group's residual rows in
+// binary64, with the order of the additions fixed as include/pipe.h states it so that the kept lists can be compared
+// bit for bit: one warp per row, lane l sums the squares of the elements l, l + 32, ... in ascending order (a square
+// of a binary32 value is exact in binary64), then the 32 partial sums are added as a tree with offsets 16, 8, 4, 2, 1.
+__global__ void __launch_bounds__(256) row_sumsq_kernel(const float* __restrict__ r, int64_t ld, int O, int I, double* __restrict__ rowsq) {
+  const int o = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (o >= O) return;
+  const float* row = r + static_cast<int64_t>(o) * ld;
+  double s = 0.0;
+  for (int i = lane; i < I; i += 32) {
+    const double v = static_cast<double>(row[i]);
+    s = __dadd_rn(s, __dmul_rn(v, v));
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) s = __dadd_rn(s, __shfl_down_sync(0xffffffffu, s, off));
+  if (lane == 0) rowsq[o] = s;
+}
+
+// score[j] = sum over the group's rows, ascending, of rowsq; one thread per group.
+__global__ void group_score_l2_kernel(const double* __restrict__ rowsq, int G, int g, double* __restrict__ score) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= G) return;
+  double s = 0.0;
+  for (int u = 0; u < g; ++u) s = __dadd_rn(s, rowsq[static_cast<int64_t>(j) * g + u]);
+  score[j] = s;
+}
+
+// Unstructured mask (pipe_layer_desc::keep_elems): per row, the magnitude key of the n-th largest entry of the
+// residual and the index up to which entries EQUAL to it are kept (ties go to the lower index).  One block per row:
+// a radix select over the four bytes of the key, then a bisection on the index among the ties.  An entry i of the
+// row is kept iff key_i > thr, or key_i == thr and i <= tie_cut.
+__global__ void __launch_bounds__(256) row_topn_kernel(const float* __restrict__ r, int64_t ld, int I, int n,
+                                                       uint32_t* __restrict__ thr_out, int32_t* __restrict__ cut_out) {
+  __shared__ int hist[256];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_remaining, sh_count;
+  const float* row = r + static_cast<int64_t>(blockIdx.x) * ld;
+  uint32_t prefix = 0, mask = 0;
+  int remaining = n;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < I; i += blockDim.x) {
+      const uint32_t k = abs_key(row[i]);
+      if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 0xffu], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int b = 255, rem = remaining;
+      while (b > 0 && hist[b] < rem) rem -= hist[b--];   // the bin that holds the rem-th largest of the candidates
+      sh_prefix = prefix | (static_cast<uint32_t>(b) << shift);
+      sh_remaining = rem;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    remaining = sh_remaining;
+    mask |= 0xffu << shift;
+    __syncthreads();
+  }
+  // `remaining` of the entries equal to prefix are kept: the smallest index c such that #{i <= c : key_i == prefix} = remaining
+  int lo = 0, hi = I - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (threadIdx.x == 0) sh_count = 0;
+    __syncthreads();
+    int c = 0;
+    for (int i = threadIdx.x; i <= mid; i += blockDim.x) c += abs_key(row[i]) == prefix;
+    if (c) atomicAdd(&sh_count, c);
+    __syncthreads();
+    const int total = sh_count;
+    __syncthreads();
+    if (total >= remaining) hi = mid;
+    else lo = mid + 1;
+  }
+  if (threadIdx.x == 0) {
+    thr_out[blockIdx.x] = prefix;
+    cut_out[blockIdx.x] = lo;
+  }
 }
 
 // Exclusive prefix sum of keep[] -> cum[0..G], and the ascending list of kept groups.
@@ -202,6 +283,8 @@ struct QuantizeRowsArgs {
   float* scales;         // [rows]
   int I, g, qmax;
   int canon_row_bytes, kernel_row_bytes;
+  const uint32_t* mask_thr;   // unstructured mask of this order, per ORIGINAL row (nullptr: every entry is kept):
+  const int32_t* mask_cut;    // an entry is kept iff its magnitude key > thr, or == thr and its index <= cut
 };
 
 // One block per compacted row: Eq. 1 on the residual, then the residual update of Eq. 3.
@@ -234,6 +317,9 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
     amax = p.a[o];
   }
   const float s = __fdiv_rn(amax, fq);
+  const bool masked = p.mask_thr != nullptr;
+  const uint32_t mthr = masked ? p.mask_thr[o] : 0u;
+  const int mcut = masked ? p.mask_cut[o] : 0;
   __syncthreads();  // every thread has read a[o] before thread 0 overwrites it at the end
   if (threadIdx.x == 0) p.scales[n] = s;
   uint8_t* crow = p.codes + static_cast<int64_t>(n) * p.canon_row_bytes;
@@ -273,7 +359,8 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           float c = 0.f;
-          if (s != 0.f) {
+          const uint32_t key = abs_key(x[j]);
+          if (s != 0.f && (!masked || key > mthr || (key == mthr && e0 + j <= mcut))) {
             c = rintf(__fdiv_rn(x[j], s));         // round half to even
             c = fminf(fmaxf(c, -fq), fq);
             x[j] = __fmaf_rn(-s, c, x[j]);         // exact new residual, rounded once
@@ -314,7 +401,8 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
       float c = 0.f;
-      if (s != 0.f) {
+      const uint32_t key = abs_key(v[e]);
+      if (s != 0.f && (!masked || key > mthr || (key == mthr && i0 + e <= mcut))) {
         c = rintf(__fdiv_rn(v[e], s));           // round half to even
         c = fminf(fmaxf(c, -fq), fq);
         v[e] = __fmaf_rn(-s, c, v[e]);           // exact new residual, rounded once
@@ -445,9 +533,24 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
   uint64_t off = round_up<uint64_t>(static_cast<uint64_t>(L.O) * I4 * 4, 256);
   float* a = reinterpret_cast<float*>(ws + off);
   off += round_up<uint64_t>(static_cast<uint64_t>(L.O) * 4, 256);
-  float* score = reinterpret_cast<float*>(ws + off);
-  off += round_up<uint64_t>(static_cast<uint64_t>(L.G) * 4, 256);
+  float* score = reinterpret_cast<float*>(ws + off);          // G doubles for the L2 score, G floats otherwise
+  double* score64 = reinterpret_cast<double*>(ws + off);
+  off += round_up<uint64_t>(static_cast<uint64_t>(L.G) * 8, 256);
   int32_t* keep = reinterpret_cast<int32_t*>(ws + off);
+  off += round_up<uint64_t>(static_cast<uint64_t>(L.G) * 4, 256);
+  double* rowsq = nullptr;
+  if (L.score_mode == PIPE_SCORE_L2) {
+    rowsq = reinterpret_cast<double*>(ws + off);
+    off += round_up<uint64_t>(static_cast<uint64_t>(L.O) * 8, 256);
+  }
+  uint32_t* mask_thr = nullptr;
+  int32_t* mask_cut = nullptr;
+  if (L.keep_elems > 0) {
+    mask_thr = reinterpret_cast<uint32_t*>(ws + off);
+    off += round_up<uint64_t>(static_cast<uint64_t>(L.O) * 4, 256);
+    mask_cut = reinterpret_cast<int32_t*>(ws + off);
+    off += round_up<uint64_t>(static_cast<uint64_t>(L.O) * 4, 256);
+  }
   uint8_t* blob = static_cast<uint8_t*>(d_blob);
 
   write_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<uint32_t*>(blob), *desc);
@@ -456,13 +559,19 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     int32_t* kept = reinterpret_cast<int32_t*>(blob + L.lay.kept_off[k]);
     int32_t* cum = reinterpret_cast<int32_t*>(blob + L.lay.cum_off[k]);
     const bool dense = (k == 0) || (L.n_keep == L.G);
-    if (!dense && L.G <= kFusedGroups) {
+    if (!dense && L.G <= kFusedGroups && L.score_mode == PIPE_SCORE_MAXABS) {
       group_select_kernel<<<1, kFusedGroups, 0, s>>>(a, L.G, L.g, L.n_keep, cum, kept);
       count_launch(1);
     } else {
-      if (!dense) {
+      if (!dense && L.score_mode == PIPE_SCORE_L2) {
+        // (a sparse order is never the first, so the current residual is in the workspace)
+        row_sumsq_kernel<<<ceil_div(L.O, 8), 256, 0, s>>>(resid, I4, L.O, L.I, rowsq);
+        group_score_l2_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(rowsq, L.G, L.g, score64);
+        group_rank_kernel<double><<<ceil_div(L.G, 256), 256, 0, s>>>(score64, L.G, L.n_keep, keep);
+        count_launch(3);
+      } else if (!dense) {
         group_score_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(a, L.G, L.g, score);
-        group_rank_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
+        group_rank_kernel<float><<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
         count_launch(2);
       }
       group_compact_kernel<<<1, 1024, 0, s>>>(dense ? nullptr : keep, L.G, cum, kept);
@@ -484,6 +593,14 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     q.canon_row_bytes = L.lay.canon_row_bytes;
     q.kernel_row_bytes = L.lay.kernel_row_bytes;
     q.rows = L.lay.rows[k];
+    q.mask_thr = nullptr;
+    q.mask_cut = nullptr;
+    if (L.keep_elems > 0 && k > 0) {
+      row_topn_kernel<<<L.O, 256, 0, s>>>(resid, I4, L.I, L.keep_elems, mask_thr, mask_cut);
+      count_launch(1);
+      q.mask_thr = mask_thr;
+      q.mask_cut = mask_cut;
+    }
     const int rows = L.lay.rows[k];
     if (L.bits == 8) quantize_rows_kernel<8><<<rows, kRowThreads, 0, s>>>(q);
     else if (L.bits == 4) quantize_rows_kernel<4><<<rows, kRowThreads, 0, s>>>(q);

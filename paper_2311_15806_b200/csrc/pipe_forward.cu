@@ -12,7 +12,8 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
                                const float* const* sx, float* const* y, const int* k_begin, const int* k_end,
                                int64_t T, int64_t ldxq, int64_t ldy, const float* d_bias, int sum_branches,
                                int32_t* d_partials, cudaStream_t stream, int8_t* const* yq = nullptr,
-                               const float* const* out_scale = nullptr, int64_t ldyq = 0, int relu = 0) {
+                               const float* const* out_scale = nullptr, int64_t ldyq = 0, int relu = 0,
+                               const int32_t* const* zp = nullptr) {
   // yq != nullptr: the fused inner-layer epilogue; y and ldy are unused then
   const bool q8 = yq != nullptr;
   if (!d_blob) return PIPE_ERR_INVALID_ARG;
@@ -41,6 +42,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     BranchArgs& b = a.branch[m];
     b.xq = xq[m];
     b.sx = sx[m];
+    b.zp = zp ? zp[m] : nullptr;
     b.y = q8 ? nullptr : (sum_branches ? y[0] : y[m]);
     b.yq = q8 ? yq[m] : nullptr;
     b.out_scale = q8 ? out_scale[m] : nullptr;
@@ -68,6 +70,12 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   a.ldyq = ldyq;
 
   const int choice = kernel_choice();
+  if (zp) {   // asymmetric codes: the CUDA-core kernel folds the zero point in (the others decline)
+    if (static_cast<int64_t>(255) * L.qmax * L.I >= (static_cast<int64_t>(1) << 31)) return PIPE_ERR_ACC_OVERFLOW;
+    for (int m = 0; m < M; ++m)
+      if (reinterpret_cast<uintptr_t>(zp[m]) & 3) return PIPE_ERR_ALIGNMENT;
+    return (choice == 0 || choice == 1) ? forward_reference(a, stream) : PIPE_ERR_UNSUPPORTED;
+  }
   if (choice == 1) return forward_reference(a, stream);
   if (choice == 2) return forward_tcgen05(a, stream);
   if (choice == 3) return forward_stream(a, stream);
@@ -112,6 +120,23 @@ extern "C" pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const 
   }
   return run_forward(L, d_blob, L.M, h_xq_m, h_sx_m, h_y_m, kb, ke, T, ldxq, ldy, d_bias, sum_branches ? 1 : 0,
                      d_partials, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pipe_status pipe_ensemble_forward_zp(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
+                                                int64_t T, int64_t ldxq, const float* const* h_sx_m,
+                                                const int32_t* const* h_zp_m, const float* d_bias, float* const* h_y_m,
+                                                int64_t ldy, int32_t sum_branches, int32_t* d_partials, void* stream) {
+  LayerInfo L;
+  pipe_status st = resolve_layer(desc, &L);
+  if (st != PIPE_OK) return st;
+  if (!h_xq_m || !h_sx_m || !h_zp_m || !h_y_m) return PIPE_ERR_INVALID_ARG;
+  int kb[PIPE_MAX_ORDERS], ke[PIPE_MAX_ORDERS];
+  for (int m = 0; m < L.M; ++m) {
+    kb[m] = L.branch_begin[m];
+    ke[m] = L.branch_begin[m + 1];
+  }
+  return run_forward(L, d_blob, L.M, h_xq_m, h_sx_m, h_y_m, kb, ke, T, ldxq, ldy, d_bias, sum_branches ? 1 : 0,
+                     d_partials, static_cast<cudaStream_t>(stream), nullptr, nullptr, 0, 0, h_zp_m);
 }
 
 extern "C" pipe_status pipe_ensemble_forward_q8(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
@@ -164,6 +189,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   BranchArgs& b = a.branch[0];
   b.xq = d_xq;
   b.sx = d_sx;
+  b.zp = nullptr;
   b.y = q8 ? nullptr : d_y;
   b.k_begin = 0;
   b.k_end = L.K;

@@ -48,6 +48,9 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
   for (int m = m_first; m < m_last; ++m) {
     const BranchArgs br = a.branch[m];
     const float sx = *br.sx;
+    // asymmetric activation codes (Sec. 4.3): sum_i (c - z) q = sum_i c q - z * sum_i q; the row sum of the weight
+    // codes comes out of the same loop (dp4a against four ones)
+    const int zp = br.zp ? *br.zp : 0;
     float out_step = 0.f;
     if (a.q8_out) {
       out_step = *br.out_scale;
@@ -75,6 +78,7 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
       }
       __syncthreads();
       int acc[4][4];
+      int rsum[4] = {0, 0, 0, 0};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -112,6 +116,10 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
           for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = __dp4a(xa[i], wb[j], acc[i][j]);
+          if (zp != 0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) rsum[j] = __dp4a(0x01010101, wb[j], rsum[j]);
+          }
         }
         __syncthreads();
       }
@@ -125,8 +133,9 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
         for (int i = 0; i < 4; ++i) {
           const int64_t t = t0 + 4 * ty + i;
           if (t >= a.T) continue;
-          yv[i][j] = __fmaf_rn(__int2float_rn(acc[i][j]), cs, yv[i][j]);
-          if (a.partials) a.partials[t * a.total_rows + ov.row_off + cr] = acc[i][j];
+          const int av = acc[i][j] - zp * rsum[j];
+          yv[i][j] = __fmaf_rn(__int2float_rn(av), cs, yv[i][j]);
+          if (a.partials) a.partials[t * a.total_rows + ov.row_off + cr] = av;
         }
       }
     }

@@ -28,24 +28,32 @@ static uint64_t align_up64(uint64_t v, uint64_t a) { return (v + a - 1) / a * a;
 pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
   if (!d || !out) return PIPE_ERR_INVALID_ARG;
   if (d->out_features <= 0 || d->in_features <= 0) return PIPE_ERR_INVALID_ARG;
-  if (!(d->weight_bits == 8 || d->weight_bits == 4 || d->weight_bits == 2)) return PIPE_ERR_INVALID_ARG;
+  if (!(d->weight_bits == 8 || d->weight_bits == 6 || d->weight_bits == 4 || d->weight_bits == 3 || d->weight_bits == 2))
+    return PIPE_ERR_INVALID_ARG;
+  if (d->score_mode != PIPE_SCORE_MAXABS && d->score_mode != PIPE_SCORE_L2) return PIPE_ERR_INVALID_ARG;
+  if (d->keep_elems < 0 || d->keep_elems > d->in_features) return PIPE_ERR_INVALID_ARG;
   if (d->num_orders < 1 || d->num_orders > PIPE_MAX_ORDERS) return PIPE_ERR_INVALID_ARG;
   if (d->group_size < 1) return PIPE_ERR_INVALID_ARG;
   if (d->out_features % d->group_size != 0) return PIPE_ERR_SHAPE;
-  const int per_byte = 8 / d->weight_bits;
+  const int container = d->weight_bits == 2 ? 2 : (d->weight_bits <= 4 ? 4 : 8);   // storage format of the codes
+  const int per_byte = 8 / container;
   if (d->in_features % per_byte != 0) return PIPE_ERR_SHAPE;
   LayerInfo L;
   std::memset(&L, 0, sizeof(L));
   L.O = d->out_features;
   L.I = d->in_features;
-  L.bits = d->weight_bits;
+  L.bits = container;
+  L.wbits = d->weight_bits;
+  L.score_mode = d->score_mode;
+  L.keep_elems = d->keep_elems;
   L.K = d->num_orders;
   L.g = d->group_size;
   L.G = L.O / L.g;
   L.n_keep = d->keep_groups;
   L.M = d->num_branches;
-  L.qmax = (1 << (L.bits - 1)) - 1;
+  L.qmax = (1 << (L.wbits - 1)) - 1;
   if (L.n_keep < 1 || L.n_keep > L.G) return PIPE_ERR_INVALID_ARG;
+  if (L.keep_elems > 0 && L.n_keep != L.G) return PIPE_ERR_SHAPE;
   if (L.M < 1 || L.M > L.K) return PIPE_ERR_SHAPE;
   // int32 partial sums (Eq. 9 is exact integer work).  The tensor-core and decode kernels accumulate sub-byte
   // codes as code * 2^(8-b) and shift back at the end, so the bound that keeps every kernel exact is
@@ -109,10 +117,13 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
   if (total > INT32_MAX) return PIPE_ERR_SHAPE;
   y.total_rows = static_cast<int32_t>(total);
   y.blob_bytes = off;
-  // expansion workspace: residual [O, I4] float + absmax [O] + group score [G] + keep flag [G]
+  // expansion workspace: residual [O, I4] float + absmax [O] + group score [G] (double) + keep flag [G]
+  // (+ the rows' sums of squares [O] double for the L2 score)
   const uint64_t I4 = round_up(L.I, 4);
   y.expand_ws_bytes = align_up64(static_cast<uint64_t>(L.O) * I4 * 4, 256) + align_up64(static_cast<uint64_t>(L.O) * 4, 256) +
-                      2 * align_up64(static_cast<uint64_t>(L.G) * 4, 256);
+                      align_up64(static_cast<uint64_t>(L.G) * 8, 256) + align_up64(static_cast<uint64_t>(L.G) * 4, 256) +
+                      (L.score_mode == PIPE_SCORE_L2 ? align_up64(static_cast<uint64_t>(L.O) * 8, 256) : 0) +
+                      (L.keep_elems > 0 ? 2 * align_up64(static_cast<uint64_t>(L.O) * 4, 256) : 0);
   y.quantize_ws_bytes = 256;
   *out = L;
   return PIPE_OK;

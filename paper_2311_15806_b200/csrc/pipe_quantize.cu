@@ -207,6 +207,100 @@ pipe_status quantize_act_impl(const float* d_x, int64_t T, int32_t I, int64_t ld
   return launch_status();
 }
 
+// ---- the other activation quantizers of Sec. 4.3 (A6 / A4, asymmetric): same two passes, division always carried
+// out.  ws[0] = largest magnitude key (non-finite check, symmetric scale), ws[1] = bits of max(x, 0),
+// ws[2] = bits of max(-x, 0); all three are non-negative floats, whose order is the order of their bit patterns.
+__global__ void __launch_bounds__(kQThreads) act_range_kernel(const QuantArgs p, uint32_t* ws) {
+  uint32_t m = 0, hi = 0, nlo = 0;
+  for (int64_t c = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; c < p.total_chunks;
+       c += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    float v[16];
+    int64_t t;
+    int i0;
+    load16(p, c, v, t, i0);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      m = max(m, q_abs_key(v[e]));
+      hi = max(hi, __float_as_uint(fmaxf(v[e], 0.f)) & 0x7fffffffu);   // (the mask turns a -0 into +0)
+      nlo = max(nlo, __float_as_uint(fmaxf(-v[e], 0.f)) & 0x7fffffffu);
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    m = max(m, __shfl_xor_sync(0xffffffffu, m, d));
+    hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+    nlo = max(nlo, __shfl_xor_sync(0xffffffffu, nlo, d));
+  }
+  if ((threadIdx.x & 31) == 0) {
+    if (m) atomicMax(ws, m);
+    if (hi) atomicMax(ws + 1, hi);
+    if (nlo) atomicMax(ws + 2, nlo);
+  }
+}
+
+__global__ void __launch_bounds__(kQThreads) act_quantize_ex_kernel(const QuantArgs p, const uint32_t* ws, int act_bits, int asym,
+                                                                    const float* static_scale, const float* static_range,
+                                                                    float* sx_out, int32_t* zp_out, int* status) {
+  const uint32_t mbits = ws[0];
+  const float half = static_cast<float>(1 << (act_bits - 1));
+  float s, z = 0.f, cmin, cmax;
+  bool bad_arg = false;
+  if (!asym) {
+    const float qx = half - 1.f;
+    s = static_scale ? *static_scale : __fdiv_rn(__uint_as_float(mbits), qx);
+    bad_arg = static_scale && !(s >= 0.f && s < __uint_as_float(0x7f800000u));
+    cmin = -qx;
+    cmax = qx;
+  } else {
+    float lo = -__uint_as_float(ws[2]), hi = __uint_as_float(ws[1]);
+    if (static_range) {
+      lo = static_range[0];
+      hi = static_range[1];
+      bad_arg = !(lo <= 0.f && hi >= 0.f && lo > -__uint_as_float(0x7f800000u) && hi < __uint_as_float(0x7f800000u));
+    }
+    s = __fdiv_rn(__fsub_rn(hi, lo), 2.f * half - 1.f);
+    cmin = -half;
+    cmax = half - 1.f;
+    if (s != 0.f) z = fminf(fmaxf(rintf(__fsub_rn(-half, __fdiv_rn(lo, s))), cmin), cmax);
+  }
+  if (bad_arg) s = 0.f, z = 0.f;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *sx_out = s;
+    *zp_out = static_cast<int32_t>(z);
+    if (mbits >= 0x7f800000u) raise_status(status, PIPE_ERR_NONFINITE);
+    if (bad_arg) raise_status(status, PIPE_ERR_INVALID_ARG);
+  }
+  for (int64_t c = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; c < p.total_chunks;
+       c += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    float v[16];
+    int64_t t;
+    int i0;
+    load16(p, c, v, t, i0);
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      float q = z;
+      if (s != 0.f) q = fminf(fmaxf(__fadd_rn(rintf(__fdiv_rn(v[e], s)), z), cmin), cmax);
+      w[e >> 2] |= (static_cast<uint32_t>(static_cast<int>(q)) & 0xffu) << (8 * (e & 3));
+    }
+    int8_t* orow = p.xq + t * p.ldxq;
+    if (p.vec_out && i0 + 16 <= p.I) {
+      *reinterpret_cast<uint4*>(orow + i0) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (i0 + e < p.I) orow[i0 + e] = static_cast<int8_t>(w[e >> 2] >> (8 * (e & 3)));
+    }
+  }
+}
+
+__global__ void act_empty_ex_kernel(const float* static_scale, float* sx_out, int32_t* zp_out) {
+  if (threadIdx.x == 0) {
+    *sx_out = static_scale ? *static_scale : 0.f;
+    *zp_out = 0;
+  }
+}
+
 }  // namespace pipe
 
 using namespace pipe;
@@ -224,4 +318,46 @@ extern "C" pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I,
   if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
   return quantize_act_impl(d_x, T, I, ldx, d_static_scale, d_xq, ldxq, d_sx, static_cast<uint32_t*>(d_ws),
                            static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t I, int64_t ldx, int32_t act_bits,
+                                            int32_t asymmetric, const float* d_static_scale, const float* d_static_range,
+                                            int8_t* d_xq, int64_t ldxq, float* d_sx, int32_t* d_zp, void* d_ws,
+                                            size_t ws_bytes, void* stream) {
+  if (T < 0 || I <= 0) return PIPE_ERR_INVALID_ARG;
+  if (!(act_bits == 8 || act_bits == 6 || act_bits == 4)) return PIPE_ERR_INVALID_ARG;
+  if (!d_sx || !d_zp || !d_ws) return PIPE_ERR_INVALID_ARG;
+  if (T > 0 && (!d_x || !d_xq)) return PIPE_ERR_INVALID_ARG;
+  if (ldx < I || ldxq < I) return PIPE_ERR_INVALID_ARG;
+  if (asymmetric ? d_static_scale != nullptr : d_static_range != nullptr) return PIPE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_x) & 3) || (reinterpret_cast<uintptr_t>(d_ws) & 255) || (reinterpret_cast<uintptr_t>(d_sx) & 3) ||
+      (reinterpret_cast<uintptr_t>(d_zp) & 3) || (reinterpret_cast<uintptr_t>(d_static_scale) & 3) ||
+      (reinterpret_cast<uintptr_t>(d_static_range) & 3))
+    return PIPE_ERR_ALIGNMENT;
+  if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int* status = device_status_word();
+  if (!status) return PIPE_ERR_CUDA;
+  if (T == 0) {
+    act_empty_ex_kernel<<<1, 32, 0, s>>>(d_static_scale, d_sx, d_zp);
+    count_launch(1);
+    return launch_status();
+  }
+  QuantArgs p;
+  p.x = d_x; p.xq = d_xq; p.T = T; p.ldx = ldx; p.ldxq = ldxq; p.I = I;
+  p.chunks_per_row = ceil_div(I, 16);
+  p.total_chunks = T * p.chunks_per_row;
+  p.vec_in = ((reinterpret_cast<uintptr_t>(d_x) & 15) == 0) && (ldx % 4 == 0);
+  p.vec_out = ((reinterpret_cast<uintptr_t>(d_xq) & 15) == 0) && (ldxq % 16 == 0);
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t want = ceil_div<int64_t>(p.total_chunks, kQThreads);
+  const int grid = static_cast<int>(want < static_cast<int64_t>(sms) * 8 ? want : static_cast<int64_t>(sms) * 8);
+  uint32_t* scratch = static_cast<uint32_t*>(d_ws);
+  if (cudaMemsetAsync(scratch, 0, 16, s) != cudaSuccess) return PIPE_ERR_CUDA;
+  act_range_kernel<<<grid, kQThreads, 0, s>>>(p, scratch);
+  act_quantize_ex_kernel<<<grid, kQThreads, 0, s>>>(p, scratch, act_bits, asymmetric ? 1 : 0, d_static_scale, d_static_range, d_sx,
+                                                    d_zp, status);
+  count_launch(2);
+  return launch_status();
 }

@@ -65,7 +65,8 @@ def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_lay
                                       err_msg=f"scales, order {k}")
         np.testing.assert_array_equal(layer.codes(k).cpu().numpy(), e.packed(k), err_msg=f"codes, order {k}")
         if check_kernel_layout:
-            np.testing.assert_array_equal(layer.kcodes(k).cpu().numpy(), kernel_layout_from_codes(e.order_codes(k), e.bits),
+            np.testing.assert_array_equal(layer.kcodes(k).cpu().numpy(),
+                                          kernel_layout_from_codes(e.order_codes(k), 2 if e.bits == 2 else (4 if e.bits <= 4 else 8)),
                                           err_msg=f"streaming layout, order {k}")
     assert_block_tables_match(layer, e)
 

@@ -81,7 +81,7 @@ def test_layout_sections_are_disjoint_and_aligned(lib):
 
 
 @pytest.mark.parametrize("kwargs,status", [
-    (dict(O=0), B.PIPE_ERR_INVALID_ARG), (dict(bits=3), B.PIPE_ERR_INVALID_ARG), (dict(K=17), B.PIPE_ERR_INVALID_ARG),
+    (dict(O=0), B.PIPE_ERR_INVALID_ARG), (dict(bits=5), B.PIPE_ERR_INVALID_ARG), (dict(K=17), B.PIPE_ERR_INVALID_ARG),
     (dict(g=7), B.PIPE_ERR_SHAPE), (dict(keep=0), B.PIPE_ERR_INVALID_ARG), (dict(keep=9), B.PIPE_ERR_INVALID_ARG),
     (dict(M=5), B.PIPE_ERR_SHAPE), (dict(I=63, bits=4), B.PIPE_ERR_SHAPE), (dict(I=133200, bits=8), B.PIPE_ERR_ACC_OVERFLOW),
     (dict(branch=[3, 2]), B.PIPE_ERR_SHAPE), (dict(branch=[4, 0]), B.PIPE_ERR_SHAPE),
