@@ -175,6 +175,41 @@ int32_t pipe_max_orders_within_original(const pipe_op_shape* shape, int32_t weig
  * K >= 1 (K = 1 admits beta = 1 only, gamma = 1). */
 pipe_status pipe_gamma_from_budget(double beta, int32_t num_orders, double* h_gamma);
 
+/* Appendix C (upper bound of the error, first theorem): for an L-layer ReLU network with spectral norms s_l and
+ * per-layer quantization steps u_l, U = prod_{l=1..L} ( sum_{i=1..l} s_i u_i + 1 ) - 1 bounds
+ * max_{|X| = 1} |F(X) - F^(K)(X)|.  h_s, h_u: L doubles each (all >= 0).  Returns a negative value for invalid
+ * arguments.  The same expression is U_sparse of the second theorem when u_l are the steps of the sparse expansion. */
+double pipe_bound_network(const double* h_s, const double* h_u, int32_t L);
+
+/* u_l^(K) of the first theorem / Lemma B.1 for a dense expansion: (1 / (2^(b-1) - 1))^(K-1) * lambda / 2, lambda the
+ * largest first-order scale of the layer's rows (the reading of the lemma's lambda under which it holds).
+ * Negative for invalid arguments. */
+double pipe_bound_step_dense(int32_t weight_bits, int32_t num_orders, double first_scale_max);
+
+/* u_l of a SPARSE expansion (second theorem; its printed factor refers to a quantity this paper does not define).
+ * Reading: round-to-nearest leaves a row within half the step of the LAST order that quantized it, whichever orders
+ * pruned it in between, so u_l = max over rows of that step / 2.  h_last_scale: float [O], the scale each output
+ * channel had at the last order that kept it (the binding gathers it from a blob). */
+double pipe_bound_step_rows(const float* h_last_scale, int32_t O);
+
+/* Largest singular value of a host matrix W [O, I] (pitch ldw) by power iteration on W^T W in binary64, started
+ * from the all-ones vector; stops after max_iters rounds or when the estimate changes by less than tol (relative).
+ * The s_l of Appendix C.  Pure host function. */
+pipe_status pipe_spectral_norm(const float* h_W, int32_t O, int32_t I, int64_t ldw, int32_t max_iters, double tol,
+                               double* h_sigma);
+
+/* Sec. 3.1 ("to match a total budget of operations"), Sec. 4.2 and Appendix A ("budget 7 and order 8") with the
+ * head-count of Appendix H: picks (K, gamma, [K_m]) for a layer shape, a weight bit-width and a budget of bit
+ * operations.  beta = the number of full orders the budget pays for, (budget - rescaling) / (one order's products),
+ * capped at max_orders; the paper's best trade-offs use high orders with sparse residuals, so K is the largest
+ * order count <= max_orders whose kept fraction gamma = (beta - 1) / (K - 1) stays >= min_gamma (K = 1, gamma = 1
+ * when the budget pays for one order only); [K_m] is the balanced split of pipe_default_branches for
+ * min(num_branches, K) predictors.  h_branch_orders: PIPE_MAX_ORDERS ints (unused entries zeroed).
+ * PIPE_ERR_INVALID_ARG when the budget does not pay for one order or an argument is out of range. */
+pipe_status pipe_choose_expansion(const pipe_op_shape* shape, int32_t weight_bits, double bit_ops_budget, int32_t max_orders,
+                                  double min_gamma, int32_t num_branches, int32_t* h_num_orders, double* h_gamma,
+                                  int32_t* h_num_branches, int32_t* h_branch_orders);
+
 /* Validates `desc` and fills `h_out`.  Pure host function, no CUDA call. */
 pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out);
 

@@ -349,6 +349,33 @@ def bit_ops_expanded(d: int, D: int, n_i: int, n_o: int, s: int, bits: int, orde
                      + orders * (d ** 2 * n_i * n_o / s ** 2) * bits * math.log2(bits))
 
 
+def bound_network(s, u) -> float:
+    """Appendix C, first theorem: U = prod_{l=1..L} (sum_{i<=l} s_i u_i + 1) - 1, written out."""
+    U, acc = 1.0, 0.0
+    for sl, ul in zip(s, u):
+        acc += sl * ul
+        U *= acc + 1.0
+    return U - 1.0
+
+
+def bound_step_dense(bits: int, K: int, first_scale_max: float) -> float:
+    """u^(K) of Lemma B.1 / Appendix C: (1 / (2^(b-1) - 1))^(K-1) * lambda / 2."""
+    return (1.0 / (2 ** (bits - 1) - 1)) ** (K - 1) * first_scale_max / 2.0
+
+
+def choose_expansion(d, D, n_i, n_o, s, bits, budget, max_orders, min_gamma, num_branches):
+    """Sec. 3.1 / App. A / App. H: the number of full orders the budget pays for, then the largest K whose kept
+    fraction stays >= min_gamma; balanced predictors.  Returns (K, gamma, [K_m])."""
+    import math
+    rescale = bit_ops_expanded(d, D, n_i, n_o, s, bits, 0.0)
+    one = bit_ops_expanded(d, D, n_i, n_o, s, bits, 1.0) - rescale
+    beta = min((budget - rescale) / one, float(max_orders))
+    K = max(1, min(max_orders, 1 + int(math.floor((beta - 1.0) / min_gamma + 1e-9))))
+    gamma = 1.0 if K == 1 else min(1.0, (beta - 1.0) / (K - 1))
+    M = min(num_branches, K)
+    return K, gamma, [int(v) for v in balanced_split(K, M)]
+
+
 def budget_of(K: int, gamma: float) -> float:
     """Full orders a group-sparse expansion costs: order 1 dense, K - 1 orders at kept fraction gamma."""
     return 1.0 + (K - 1) * gamma

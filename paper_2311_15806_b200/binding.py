@@ -29,6 +29,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 
 EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout", "pipe_expand_weights",
            "pipe_bit_ops_original", "pipe_bit_ops_expanded", "pipe_max_orders_within_original", "pipe_gamma_from_budget",
+           "pipe_bound_network", "pipe_bound_step_dense", "pipe_bound_step_rows", "pipe_spectral_norm", "pipe_choose_expansion",
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_quantize_act_ex", "pipe_ensemble_forward_zp", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
            "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
@@ -159,6 +160,59 @@ def pipe_gamma_from_budget(beta: float, K: int) -> float:
     out = C.c_double(0.0)
     _check(L.pipe_gamma_from_budget(float(beta), int(K), C.byref(out)), "pipe_gamma_from_budget")
     return float(out.value)
+
+
+def pipe_bound_network(s, u) -> float:
+    """U of Appendix C for spectral norms s and steps u (sequences of equal length)."""
+    L = lib()
+    L.pipe_bound_network.restype = C.c_double
+    L.pipe_bound_network.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+    n = len(s)
+    sa, ua = (C.c_double * n)(*[float(v) for v in s]), (C.c_double * n)(*[float(v) for v in u])
+    return float(L.pipe_bound_network(sa, ua, n))
+
+
+def pipe_bound_step_dense(bits: int, K: int, first_scale_max: float) -> float:
+    L = lib()
+    L.pipe_bound_step_dense.restype = C.c_double
+    L.pipe_bound_step_dense.argtypes = [C.c_int32, C.c_int32, C.c_double]
+    return float(L.pipe_bound_step_dense(int(bits), int(K), float(first_scale_max)))
+
+
+def pipe_bound_step_rows(last_scale) -> float:
+    """last_scale: host float32 array [O] (see last_kept_scales)."""
+    import numpy as np
+    L = lib()
+    L.pipe_bound_step_rows.restype = C.c_double
+    L.pipe_bound_step_rows.argtypes = [C.c_void_p, C.c_int32]
+    a = np.ascontiguousarray(last_scale, dtype=np.float32)
+    return float(L.pipe_bound_step_rows(a.ctypes.data_as(C.c_void_p), a.shape[0]))
+
+
+def pipe_spectral_norm(W, max_iters: int = 200, tol: float = 1e-9) -> float:
+    """W: host float32 array [O, I]."""
+    import numpy as np
+    L = lib()
+    L.pipe_spectral_norm.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_int32, C.c_double, C.c_void_p]
+    a = np.ascontiguousarray(W, dtype=np.float32)
+    out = C.c_double(0.0)
+    _check(L.pipe_spectral_norm(a.ctypes.data_as(C.c_void_p), a.shape[0], a.shape[1], a.shape[1], int(max_iters), float(tol),
+                                C.byref(out)), "pipe_spectral_norm")
+    return float(out.value)
+
+
+def pipe_choose_expansion(d: int, D: int, n_i: int, n_o: int, s: int, bits: int, bit_ops_budget: float, max_orders: int,
+                          min_gamma: float, num_branches: int):
+    """Returns (K, gamma, [K_m])."""
+    L = lib()
+    L.pipe_choose_expansion.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_double, C.c_int32, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_void_p]
+    K, M, g = C.c_int32(0), C.c_int32(0), C.c_double(0.0)
+    bo = (C.c_int32 * MAX_ORDERS)()
+    _check(L.pipe_choose_expansion(C.byref(_op_shape(d, D, n_i, n_o, s)), int(bits), float(bit_ops_budget), int(max_orders),
+                                   float(min_gamma), int(num_branches), C.byref(K), C.byref(g), C.byref(M), bo),
+           "pipe_choose_expansion")
+    return int(K.value), float(g.value), [int(bo[m]) for m in range(M.value)]
 
 
 def pipe_keep_groups_from_gamma(num_groups: int, gamma: float) -> int:
@@ -377,6 +431,19 @@ class ExpandedLayer:
         if self.layout.blk_off[m] == 0:
             return None
         return self.section(self.layout.blk_off[m], (self.layout.blk_cap[m] + 2) * 4).view(torch.int32)
+
+
+def last_kept_scales(layer: "ExpandedLayer"):
+    """float32 host array [O]: the scale every output channel had at the last order that kept it (a device -> host
+    read of the blob's scale sections and kept lists; no arithmetic)."""
+    import numpy as np
+    O, g = layer.desc.out_features, layer.desc.group_size
+    out = np.zeros(O, np.float32)
+    for k in range(layer.desc.num_orders):
+        kept = layer.kept(k).cpu().numpy().astype(np.int64)
+        ch = (kept[:, None] * g + np.arange(g)[None, :]).reshape(-1)
+        out[ch] = layer.scales(k).cpu().numpy()
+    return out
 
 
 def alloc_bytes(nbytes: int, device="cuda") -> torch.Tensor:

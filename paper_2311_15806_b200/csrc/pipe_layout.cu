@@ -186,6 +186,94 @@ pipe_status pipe_gamma_from_budget(double beta, int32_t K, double* h_gamma) {
   return PIPE_OK;
 }
 
+double pipe_bound_network(const double* h_s, const double* h_u, int32_t L) {
+  if (!h_s || !h_u || L < 1) return -1.0;
+  double prod = 1.0, sum = 0.0;
+  for (int l = 0; l < L; ++l) {
+    if (!(h_s[l] >= 0.0) || !(h_u[l] >= 0.0)) return -1.0;
+    sum += h_s[l] * h_u[l];
+    prod *= sum + 1.0;
+  }
+  return prod - 1.0;
+}
+
+double pipe_bound_step_dense(int32_t weight_bits, int32_t K, double first_scale_max) {
+  if (weight_bits < 2 || weight_bits > 8 || K < 1 || K > PIPE_MAX_ORDERS || !(first_scale_max >= 0.0)) return -1.0;
+  const double qmax = static_cast<double>((1 << (weight_bits - 1)) - 1);
+  return std::pow(1.0 / qmax, K - 1) * first_scale_max / 2.0;
+}
+
+double pipe_bound_step_rows(const float* h_last_scale, int32_t O) {
+  if (!h_last_scale || O < 1) return -1.0;
+  double m = 0.0;
+  for (int o = 0; o < O; ++o) {
+    const double v = static_cast<double>(h_last_scale[o]);
+    if (!(v >= 0.0)) return -1.0;
+    if (v > m) m = v;
+  }
+  return m / 2.0;
+}
+
+pipe_status pipe_spectral_norm(const float* h_W, int32_t O, int32_t I, int64_t ldw, int32_t max_iters, double tol, double* h_sigma) {
+  if (!h_W || !h_sigma || O < 1 || I < 1 || ldw < I || max_iters < 1 || !(tol >= 0.0)) return PIPE_ERR_INVALID_ARG;
+  double* v = new double[I];
+  double* w = new double[O];
+  for (int i = 0; i < I; ++i) v[i] = 1.0 / std::sqrt(static_cast<double>(I));
+  double sigma = 0.0;
+  for (int it = 0; it < max_iters; ++it) {
+    double nw = 0.0;
+    for (int o = 0; o < O; ++o) {   // w = W v
+      const float* row = h_W + static_cast<int64_t>(o) * ldw;
+      double s = 0.0;
+      for (int i = 0; i < I; ++i) s += static_cast<double>(row[i]) * v[i];
+      w[o] = s;
+      nw += s * s;
+    }
+    const double est = std::sqrt(nw);   // |W v| with |v| = 1
+    for (int i = 0; i < I; ++i) v[i] = 0.0;
+    for (int o = 0; o < O; ++o) {   // v = W^T w
+      const float* row = h_W + static_cast<int64_t>(o) * ldw;
+      for (int i = 0; i < I; ++i) v[i] += static_cast<double>(row[i]) * w[o];
+    }
+    double nv = 0.0;
+    for (int i = 0; i < I; ++i) nv += v[i] * v[i];
+    nv = std::sqrt(nv);
+    const bool done = nv == 0.0 || std::fabs(est - sigma) <= tol * est;
+    sigma = est;
+    if (nv == 0.0) break;
+    for (int i = 0; i < I; ++i) v[i] /= nv;
+    if (done && it > 0) break;
+  }
+  *h_sigma = sigma;
+  delete[] v;
+  delete[] w;
+  return PIPE_OK;
+}
+
+pipe_status pipe_choose_expansion(const pipe_op_shape* shape, int32_t weight_bits, double bit_ops_budget, int32_t max_orders,
+                                  double min_gamma, int32_t num_branches, int32_t* h_K, double* h_gamma, int32_t* h_M,
+                                  int32_t* h_branch_orders) {
+  if (!shape_ok(shape) || !h_K || !h_gamma || !h_M || !h_branch_orders) return PIPE_ERR_INVALID_ARG;
+  if (weight_bits < 2 || weight_bits > 8 || max_orders < 1 || max_orders > PIPE_MAX_ORDERS || num_branches < 1) return PIPE_ERR_INVALID_ARG;
+  if (!(min_gamma > 0.0) || min_gamma > 1.0 || !(bit_ops_budget > 0.0)) return PIPE_ERR_INVALID_ARG;
+  const double rescale = pipe_bit_ops_expanded(shape, weight_bits, 0.0);
+  const double one_order = pipe_bit_ops_expanded(shape, weight_bits, 1.0) - rescale;
+  double beta = (bit_ops_budget - rescale) / one_order;
+  if (!(beta >= 1.0)) return PIPE_ERR_INVALID_ARG;
+  if (beta > static_cast<double>(max_orders)) beta = static_cast<double>(max_orders);
+  int K = 1 + static_cast<int>(std::floor((beta - 1.0) / min_gamma + 1e-9));
+  if (K > max_orders) K = max_orders;
+  if (K < 1) K = 1;
+  double gamma = K == 1 ? 1.0 : (beta - 1.0) / static_cast<double>(K - 1);
+  if (gamma > 1.0) gamma = 1.0;
+  *h_K = K;
+  *h_gamma = gamma;
+  const int M = num_branches < K ? num_branches : K;
+  *h_M = M;
+  for (int m = 0; m < PIPE_MAX_ORDERS; ++m) h_branch_orders[m] = 0;
+  return pipe_default_branches(K, M, h_branch_orders);
+}
+
 pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
   if (!h_out) return PIPE_ERR_INVALID_ARG;
   LayerInfo L;
