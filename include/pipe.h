@@ -70,6 +70,11 @@ typedef struct pipe_layer_desc {
                             keep_groups = G: an unstructured R^k keeps every row */
 } pipe_layer_desc;
 
+#define PIPE_ACT_IDENTITY 0
+#define PIPE_ACT_RELU 1
+#define PIPE_ACT_SILU 2
+#define PIPE_ACT_GELU 3
+#define PIPE_ACT_SIGMOID 4
 #define PIPE_SCORE_MAXABS 0
 #define PIPE_SCORE_L2 1
 
@@ -345,7 +350,12 @@ pipe_status pipe_ensemble_forward_zp(const pipe_layer_desc* desc, const void* d_
  * An INNER layer of the M predictors (Sec. 3.2, Fig. 2; Appendix B, Eq. 9 with its activation
  * function): predictor m's output never leaves the integer pipeline as floats.  Per predictor
  *     y_m            as in pipe_ensemble_forward (same order of operations, bias with predictor 1),
- *     a_m[t,o]       = relu != 0 ? max(y_m[t,o], 0) : y_m[t,o]           (sigma of Eq. 9)
+ *     a_m[t,o]       = sigma(y_m[t,o]), sigma chosen by `relu` (the argument keeps its first name): PIPE_ACT_IDENTITY,
+ *                      PIPE_ACT_RELU, PIPE_ACT_SILU v / (1 + exp(-v)), PIPE_ACT_GELU v (1 + erf(v / sqrt 2)) / 2,
+ *                      PIPE_ACT_SIGMOID 1 / (1 + exp(-v)) -- the functions Sec. 3.2 names for Eq. 9.  Identity and
+ *                      ReLU are exact; the other three are evaluated in binary32 with the device's exp and erf, so
+ *                      a_m can differ from a correctly rounded evaluation in its last bits and a code that lies on a
+ *                      rounding boundary can come out one step off
  *     yq_m[t,o]      = clamp(rne(a_m[t,o] / s_m), -127, 127)             (Eq. 1 as the next layer's Q,
  *                                                                         IEEE binary32 quotient, ties to even)
  * so that yq_m and s_m are the next layer's xq_m and lambda_{x_m}.  s_m is a static step the caller

@@ -226,6 +226,7 @@ def pipe_default_branches(K: int, M: int) -> list[int]:
 
 
 SCORE_MAXABS, SCORE_L2 = 0, 1
+ACT_IDENTITY, ACT_RELU, ACT_SILU, ACT_GELU, ACT_SIGMOID = 0, 1, 2, 3, 4
 
 
 def make_desc(O: int, I: int, bits: int, K: int, g: int, keep_groups: int, M: int = 1,
@@ -327,7 +328,7 @@ def pipe_expanded_conv2d_q8(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor,
     """xq_nhwc: cuda int8 [N, H, W, C] contiguous; yq: cuda int8 [N*Ho*Wo, O]; out_scale: cuda float32, one element."""
     assert xq_nhwc.is_contiguous() and xq_nhwc.dtype == torch.int8 and yq.dtype == torch.int8
     _check(lib().pipe_expanded_conv2d_q8(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias),
-                                         1 if relu else 0, _dp(out_scale), _dp(yq), yq.stride(0), _dp(partials),
+                                         int(relu), _dp(out_scale), _dp(yq), yq.stride(0), _dp(partials),
                                          _stream_ptr(stream)), "pipe_expanded_conv2d_q8")
 
 
@@ -364,7 +365,7 @@ def pipe_ensemble_forward_q8(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, ou
     sp = PA(*[_dp(t) for t in sx_m])
     op = PA(*[_dp(t) for t in out_scale_m])
     yp = PA(*[_dp(t) for t in yq_m])
-    _check(lib().pipe_ensemble_forward_q8(C.byref(desc), _dp(blob), xp, T, ldxq, sp, _dp(bias), 1 if relu else 0, op, yp,
+    _check(lib().pipe_ensemble_forward_q8(C.byref(desc), _dp(blob), xp, T, ldxq, sp, _dp(bias), int(relu), op, yp,
                                           ldyq, _dp(partials), _stream_ptr(stream)), "pipe_ensemble_forward_q8")
 
 

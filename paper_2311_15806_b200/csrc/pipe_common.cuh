@@ -82,6 +82,18 @@ __device__ __forceinline__ uint32_t quant4(const float4& f, float s, float r, bo
   return quant_lane_exact(f.x, s) | (quant_lane_exact(f.y, s) << 8) | (quant_lane_exact(f.z, s) << 16) | (quant_lane_exact(f.w, s) << 24);
 }
 
+// sigma of Eq. 9 for an inner layer (Sec. 3.2 names ReLU, SiLU, GeLU and sigmoid), in binary32: kind 0 identity,
+// 1 ReLU, 2 SiLU v / (1 + exp(-v)), 3 GeLU v (1 + erf(v / sqrt 2)) / 2, 4 sigmoid 1 / (1 + exp(-v)).
+__device__ __forceinline__ float apply_activation(float v, int kind) {
+  switch (kind) {
+    case 1: return fmaxf(v, 0.f);
+    case 2: return __fdiv_rn(v, __fadd_rn(1.f, expf(-v)));
+    case 3: return __fmul_rn(__fmul_rn(0.5f, v), __fadd_rn(1.f, erff(__fmul_rn(v, 0.70710678118654752f))));
+    case 4: return __fdiv_rn(1.f, __fadd_rn(1.f, expf(-v)));
+    default: return v;
+  }
+}
+
 // Per-order pointers into a blob, passed to kernels by value.
 struct OrderView {
   const uint8_t* codes;   // canonical packed codes
@@ -135,7 +147,7 @@ struct ForwardArgs {
   int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
   int cHo, cWo, csh, csw;   // output height / width and the strides
   // fused inner-layer epilogue (q8_out != 0): yq = clamp(rne(act(y) / out_scale)) as int8, row pitch ldyq; y is not written
-  int q8_out, relu;
+  int q8_out, relu;   // relu: the activation kind (see apply_activation; the name is from the first version)
   int64_t ldyq;
 };
 

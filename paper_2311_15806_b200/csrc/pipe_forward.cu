@@ -16,7 +16,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
                                const int32_t* const* zp = nullptr) {
   // yq != nullptr: the fused inner-layer epilogue; y and ldy are unused then
   const bool q8 = yq != nullptr;
-  if (!d_blob) return PIPE_ERR_INVALID_ARG;
+  if (!d_blob || relu < 0 || relu > 4) return PIPE_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) return PIPE_ERR_ALIGNMENT;
   if (T < 0 || ldxq < L.I) return PIPE_ERR_INVALID_ARG;
   if (q8 ? (ldyq < L.O || !out_scale || sum_branches) : (ldy < L.O)) return PIPE_ERR_INVALID_ARG;
@@ -66,7 +66,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   a.cN = a.cH = a.cW = a.cC = a.ckh = a.ckw = a.cph = a.cpw = 0;
   a.cHo = a.cWo = 0; a.csh = a.csw = 1;
   a.q8_out = q8 ? 1 : 0;
-  a.relu = relu ? 1 : 0;
+  a.relu = relu;
   a.ldyq = ldyq;
 
   const int choice = kernel_choice();
@@ -161,6 +161,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
                             const float* d_sx, const float* d_bias, float* d_y, int64_t ldy, int8_t* d_yq,
                             const float* d_out_scale, int64_t ldyq, int relu, int32_t* d_partials, void* stream) {
   const bool q8 = d_yq != nullptr;
+  if (relu < 0 || relu > 4) return PIPE_ERR_INVALID_ARG;
   LayerInfo L;
   pipe_status st = resolve_layer(desc, &L);
   if (st != PIPE_OK) return st;
@@ -199,7 +200,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   b.yq = d_yq;
   b.out_scale = d_out_scale;
   a.q8_out = q8 ? 1 : 0;
-  a.relu = relu ? 1 : 0;
+  a.relu = relu;
   a.ldyq = ldyq;
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = static_cast<int64_t>(geom->batch) * Ho * Wo;

@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(256) ref_forward_kernel(const ForwardArgs a, c
           if (m + 1 == m_last) a.branch[0].y[t * a.ldy + c] = total[i][j];
         } else if (a.q8_out) {
           // inner layer of a branch: activation, then the next layer's input quantizer (division carried out)
-          if (a.relu) v = fmaxf(v, 0.f);
+          v = apply_activation(v, a.relu);
           br.yq[t * a.ldyq + c] = static_cast<int8_t>(quant_lane_exact(v, out_step));
         } else {
           br.y[t * a.ldy + c] = v;

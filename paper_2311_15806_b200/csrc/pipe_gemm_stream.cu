@@ -523,7 +523,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
             if (bias) v = __fadd_rn(v, bv);
             if (p.f.q8_out) {
               // inner layer of a branch: sigma, then the next layer's input quantizer (Sec. 3.2)
-              if (p.f.relu) v = fmaxf(v, 0.f);
+              v = apply_activation(v, p.f.relu);
               const float os = __ldg(br.out_scale);
               if (!(os >= 0.f && os < __uint_as_float(0x7f800000u))) raise_status(p.f.status, PIPE_ERR_INVALID_ARG);
               br.yq[static_cast<int64_t>(tok) * p.f.ldyq + c] = static_cast<int8_t>(quant_lane_exact(v, os));

@@ -603,7 +603,8 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               if (add_bias) y[e] = __fadd_rn(y[e], bv[e]);
-              if (p.f.relu) y[e] = fmaxf(y[e], 0.f);
+              if (p.f.relu == 1) y[e] = fmaxf(y[e], 0.f);
+              else if (p.f.relu) y[e] = apply_activation(y[e], p.f.relu);
             }
             float uu[8];
             float edge = ofast ? 0.f : 1.f;
