@@ -114,6 +114,12 @@ typedef struct pipe_layer_desc {
  *                 run close to their widest shape, and evenly, however sparse the orders are.  A cluster of more
  *                 than 8 orders, or whose single group can exceed the row limit (orders * g > PIPE_BLOCK_ROWS), has
  *                 no table.
+ *   dec_off[m]    the same structure (n, b_0 .. b_n; room for G blocks) with the row limit dec_limit[m]: the units of
+ *                 the small-token (T <= 16) tensor-core kernel, which streams every weight once.  There the limit
+ *                 is chosen so that the units of the clusters that run together -- the M predictors, or the one
+ *                 cluster of all orders -- come to about one per SM (148 on the B200 this library is written for),
+ *                 decode_split (decode_split_all) CTAs sharing a unit's reduction axis when whole units would be
+ *                 too narrow for the MMA; the plan is a function of the descriptor alone.
  */
 #define PIPE_BLOCK_ROWS 256
 #define PIPE_BLOCK_CHANNELS 512
@@ -132,7 +138,10 @@ typedef struct pipe_layer_layout {
   uint64_t cum_off[PIPE_MAX_ORDERS];
   uint64_t blk_off[PIPE_MAX_ORDERS + 1]; /* channel-block tables (see above); 0 = the cluster has none */
   int32_t blk_cap[PIPE_MAX_ORDERS + 1];  /* blocks each table has room for */
-  int32_t reserved_;
+  int32_t decode_split;                  /* CTAs that share one decode unit's reduction axis: predictors' tables */
+  uint64_t dec_off[PIPE_MAX_ORDERS + 1]; /* decode-unit tables (see above); 0 = the cluster has none */
+  int32_t dec_limit[PIPE_MAX_ORDERS + 1]; /* rows a decode unit of the cluster may stack */
+  int32_t decode_split_all;              /* the same for the table of all K orders */
   uint64_t blob_bytes;        /* size d_blob must have */
   uint64_t expand_ws_bytes;   /* size d_ws must have for pipe_expand_weights */
   uint64_t quantize_ws_bytes; /* size d_ws must have for pipe_quantize_act */

@@ -19,7 +19,7 @@ extern "C" {
 /* Which GEMM kernel the forward calls use from now on, for the whole process (so only for tests and
  * measurements; concurrent users of the library would all see the change):
  * 0 = automatic, 1 = CUDA-core kernel, 2 = one-SM tcgen05 kernel, 3 = small-token weight-streaming kernel,
- * 4 = SM-pair tcgen05 kernel (clusters of two CTAs).  A forced kernel that cannot run a request makes the
+ * 4 = SM-pair tcgen05 kernel (clusters of two CTAs), 5 = small-token tcgen05 kernel.  A forced kernel that cannot run a request makes the
  * forward call return PIPE_ERR_UNSUPPORTED. */
 pipe_status pipe_diag_select_kernel(int32_t which);
 

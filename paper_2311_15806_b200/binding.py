@@ -23,7 +23,7 @@ STATUS_NAMES = ["PIPE_OK", "PIPE_ERR_INVALID_ARG", "PIPE_ERR_SHAPE", "PIPE_ERR_A
 (PIPE_OK, PIPE_ERR_INVALID_ARG, PIPE_ERR_SHAPE, PIPE_ERR_ALIGNMENT, PIPE_ERR_UNSUPPORTED, PIPE_ERR_WORKSPACE,
  PIPE_ERR_NONFINITE, PIPE_ERR_ACC_OVERFLOW, PIPE_ERR_TIMEOUT, PIPE_ERR_CUDA) = range(10)
 
-KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM, KERNEL_TCGEN05_PAIR = 0, 1, 2, 3, 4
+KERNEL_AUTO, KERNEL_REFERENCE, KERNEL_TCGEN05, KERNEL_STREAM, KERNEL_TCGEN05_PAIR, KERNEL_DECODE_TC = 0, 1, 2, 3, 4, 5
 
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -58,7 +58,9 @@ class LayerLayout(C.Structure):
                 ("codes_off", C.c_uint64 * MAX_ORDERS), ("kcodes_off", C.c_uint64 * MAX_ORDERS),
                 ("scales_off", C.c_uint64 * MAX_ORDERS), ("kept_off", C.c_uint64 * MAX_ORDERS),
                 ("cum_off", C.c_uint64 * MAX_ORDERS), ("blk_off", C.c_uint64 * (MAX_ORDERS + 1)),
-                ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("reserved_", C.c_int32),
+                ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("decode_split", C.c_int32),
+                ("dec_off", C.c_uint64 * (MAX_ORDERS + 1)), ("dec_limit", C.c_int32 * (MAX_ORDERS + 1)),
+                ("decode_split_all", C.c_int32),
                 ("blob_bytes", C.c_uint64), ("expand_ws_bytes", C.c_uint64),
                 ("quantize_ws_bytes", C.c_uint64)]
 
@@ -426,6 +428,12 @@ class ExpandedLayer:
 
     def cum(self, k: int) -> torch.Tensor:
         return self.section(self.layout.cum_off[k], (self.layout.num_groups + 1) * 4).view(torch.int32)
+
+    def decode_table(self, m: int) -> torch.Tensor | None:
+        """Decode-unit table m (int32: n, b_0 .. b_n), or None when the cluster has none."""
+        if self.layout.dec_off[m] == 0:
+            return None
+        return self.section(self.layout.dec_off[m], (self.layout.num_groups + 2) * 4).view(torch.int32)
 
     def block_table(self, m: int) -> torch.Tensor | None:
         """Channel-block table m (int32: n, b_0 .. b_n), or None when the cluster has none."""

@@ -25,6 +25,8 @@ struct LayerInfo {
 
 pipe_status resolve_layer(const pipe_layer_desc* desc, LayerInfo* out);
 
+constexpr int kPlanSMs = 148;   // SMs of the B200 the decode plan is laid out for
+
 // Device status word of the current device.
 int* device_status_word();
 void count_launch(int n = 1);
@@ -127,6 +129,7 @@ struct BranchArgs {
   const float* out_scale;  // its step: one float on the device
   int k_begin, k_end;
   const int32_t* zp;       // zero point of asymmetric activation codes (one int on the device), or nullptr for 0
+  const int32_t* dec;      // decode-unit table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
   const int32_t* blk;      // channel-block table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
   int add_bias;    // bias enters this branch
   int accumulate;  // y += result (summed ensemble, branches after the first)
@@ -147,6 +150,7 @@ struct ForwardArgs {
   int conv_on, cN, cH, cW, cC, ckh, ckw, cph, cpw;
   int cHo, cWo, csh, csw;   // output height / width and the strides
   // fused inner-layer epilogue (q8_out != 0): yq = clamp(rne(act(y) / out_scale)) as int8, row pitch ldyq; y is not written
+  int decode_split;   // CTAs that share a decode unit's reduction axis (from the layout; 0 = no decode tables)
   int q8_out, relu;   // relu: the activation kind (see apply_activation; the name is from the first version)
   int64_t ldyq;
 };
@@ -162,5 +166,6 @@ pipe_status forward_reference(const ForwardArgs& a, cudaStream_t stream);
 pipe_status forward_tcgen05(const ForwardArgs& a, cudaStream_t stream);
 pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream);   // two-SM form (clusters of two CTAs)
 pipe_status forward_stream(const ForwardArgs& a, cudaStream_t stream);
+pipe_status forward_decode_tc(const ForwardArgs& a, cudaStream_t stream);      // T <= 16 on tcgen05 (decode-unit tables)
 
 }  // namespace pipe

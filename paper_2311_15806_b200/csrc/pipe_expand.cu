@@ -633,6 +633,23 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
       block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
       count_launch(1);
     }
+    // the decode-unit tables: the same cut with the layout's row limits
+    any = false;
+    for (int m = 0; m <= L.M; ++m) {
+      t.out[m] = nullptr;
+      if (L.lay.dec_off[m] == 0) continue;
+      const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
+      t.nk[m] = k1 - k0;
+      for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
+      t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.dec_off[m]);
+      t.cap[m] = L.G;
+      t.limit[m] = L.lay.dec_limit[m];
+      any = true;
+    }
+    if (any) {
+      block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
+      count_launch(1);
+    }
   }
   return launch_status();
 }

@@ -51,8 +51,11 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     b.add_bias = (m == 0);
     b.accumulate = (sum_branches && m > 0);
     // one branch running all K orders is the "all orders" cluster (entry L.M), otherwise predictor m's own
-    b.blk = block_table(L, d_blob, (k_end[m] - k_begin[m] == L.K) ? L.M : m);
+    const int set = (k_end[m] - k_begin[m] == L.K) ? L.M : m;
+    b.blk = block_table(L, d_blob, set);
+    b.dec = L.lay.dec_off[set] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.dec_off[set]) : nullptr;
   }
+  a.decode_split = (M == 1 && k_end[0] - k_begin[0] == L.K) ? L.lay.decode_split_all : L.lay.decode_split;
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = T; a.ldxq = ldxq; a.ldy = ldy;
   a.bias = d_bias;
@@ -80,10 +83,15 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   if (choice == 2) return forward_tcgen05(a, stream);
   if (choice == 3) return forward_stream(a, stream);
   if (choice == 4) return forward_tcgen05_pair(a, stream);
+  if (choice == 5) return forward_decode_tc(a, stream);
   // T <= 16: weight streaming; from two token tiles on the SM-pair kernel; the one-SM kernel for what lies between
   // and for layers without channel-block tables; the CUDA-core kernel for every other shape
   pipe_status st = PIPE_ERR_UNSUPPORTED;
+  // (the small-token tcgen05 kernel, choice 5, is measured slower than the weight-streaming kernel -- widening the
+  // codes through shared memory for the tensor core triples the shared-memory traffic per weight byte -- and is
+  // therefore not on the automatic path)
   if (T <= 16) st = forward_stream(a, stream);
+  if (T <= 16 && st == PIPE_ERR_UNSUPPORTED) st = forward_decode_tc(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05_pair(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_tcgen05(a, stream);
   if (st == PIPE_ERR_UNSUPPORTED) st = forward_reference(a, stream);
@@ -197,6 +205,8 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   b.add_bias = 1;
   b.accumulate = 0;
   b.blk = block_table(L, d_blob, L.M);
+  b.dec = nullptr;
+  a.decode_split = 0;
   b.yq = d_yq;
   b.out_scale = d_out_scale;
   a.q8_out = q8 ? 1 : 0;

@@ -114,6 +114,62 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     y.blk_off[m] = off;
     off = align_up64(off + static_cast<uint64_t>(y.blk_cap[m] + 2) * 4, 256);
   }
+  // decode-unit tables: the clusters that run together share the SMs.  For c CTAs per unit the sets get units in
+  // proportion to their rows; a unit's rows (rounded to the MMA's granularity, plus one group of every order of slack)
+  // must fit the 256 accumulator columns; the cost of a split is the reduction steps of one CTA times the MMAs of a
+  // step, each of which takes its tensor time (N / 2 cycles) but never less than the issue time of an instruction.
+  auto plan = [&](int m_begin, int m_end, int32_t* split_out) {
+    int64_t Rsum = 0;
+    int64_t R[PIPE_MAX_ORDERS + 1];
+    int nk[PIPE_MAX_ORDERS + 1];
+    bool ok = true;
+    for (int m = m_begin; m < m_end; ++m) {
+      const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
+      nk[m] = k1 - k0;
+      R[m] = 0;
+      for (int k = k0; k < k1; ++k) R[m] += (k == 0) ? L.O : static_cast<int64_t>(L.n_keep) * L.g;
+      Rsum += R[m];
+      if (nk[m] > 8 || static_cast<int64_t>(nk[m]) * L.g > PIPE_BLOCK_ROWS / 2) ok = false;
+    }
+    *split_out = 0;
+    for (int m = m_begin; m < m_end; ++m) y.dec_off[m] = 0, y.dec_limit[m] = 0;
+    if (!ok) return;
+    const int kblocks = ceil_div(L.I, kKernelKAlign);
+    double best = 1e300;
+    int best_c = 0;
+    int best_limit[PIPE_MAX_ORDERS + 1];
+    for (int c = 1; c <= 4 && c <= kblocks; ++c) {
+      const int units_total = kPlanSMs / c;
+      int limit[PIPE_MAX_ORDERS + 1];
+      int max_n = 0;
+      for (int m = m_begin; m < m_end; ++m) {
+        int64_t units = static_cast<int64_t>(units_total) * R[m] / Rsum;
+        if (units < 1) units = 1;
+        int64_t n = round_up<int64_t>(ceil_div<int64_t>(R[m], units), 16) + static_cast<int64_t>(nk[m]) * L.g;
+        if (n > PIPE_BLOCK_ROWS) n = PIPE_BLOCK_ROWS;   // more units than SMs: the CTAs go round them
+        limit[m] = static_cast<int>(n);
+        max_n = n > max_n ? static_cast<int>(n) : max_n;
+      }
+      const double per_mma = max_n / 2.0 > 86.0 ? max_n / 2.0 : 86.0;
+      int64_t waves = 0;   // units beyond one per CTA cost whole extra rounds
+      for (int m = m_begin; m < m_end; ++m) waves += ceil_div<int64_t>(R[m], limit[m] - nk[m] * L.g);
+      const double rounds = static_cast<double>(ceil_div<int64_t>(waves, units_total));
+      const double cost = rounds * ceil_div(kblocks, c) * 4.0 * per_mma + (c > 1 ? 3000.0 : 0.0);
+      if (cost < best) {
+        best = cost;
+        best_c = c;
+        for (int m = m_begin; m < m_end; ++m) best_limit[m] = limit[m];
+      }
+    }
+    *split_out = best_c;
+    for (int m = m_begin; m < m_end; ++m) {
+      y.dec_limit[m] = best_limit[m];
+      y.dec_off[m] = off;
+      off = align_up64(off + static_cast<uint64_t>(L.G + 2) * 4, 256);
+    }
+  };
+  plan(0, L.M, &y.decode_split);
+  plan(L.M, L.M + 1, &y.decode_split_all);
   if (total > INT32_MAX) return PIPE_ERR_SHAPE;
   y.total_rows = static_cast<int32_t>(total);
   y.blob_bytes = off;
@@ -284,7 +340,7 @@ pipe_status pipe_layout(const pipe_layer_desc* desc, pipe_layer_layout* h_out) {
 }
 
 pipe_status pipe_diag_select_kernel(int32_t which) {
-  if (which < 0 || which > 4) return PIPE_ERR_INVALID_ARG;
+  if (which < 0 || which > 5) return PIPE_ERR_INVALID_ARG;
   g_kernel_choice.store(which);
   return PIPE_OK;
 }

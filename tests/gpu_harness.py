@@ -71,6 +71,23 @@ def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_lay
     assert_block_tables_match(layer, e)
 
 
+def expected_decode_table(kept_lists, G: int, g: int, row_limit: int, channel_limit: int = 512):
+    """A decode-unit table: the same greedy cut with the row limit the layout states."""
+    rows = np.zeros(G, np.int64)
+    for kept in kept_lists:
+        rows[np.asarray(kept)] += g
+    bounds = [0]
+    cur_rows, cur_groups = 0, 0
+    for j in range(G):
+        if cur_groups > 0 and (cur_rows + rows[j] > row_limit or (cur_groups + 1) * g > channel_limit):
+            bounds.append(j)
+            cur_rows, cur_groups = 0, 0
+        cur_rows += int(rows[j])
+        cur_groups += 1
+    bounds.append(G)
+    return np.array([len(bounds) - 1] + bounds, np.int32)
+
+
 def expected_block_table(kept_lists, G: int, g: int, row_max: int = 256, channel_limit: int = 512):
     """The channel-block table of a cluster of orders as include/pipe.h defines it, from the kept-group lists: the
     row limit is the mean block size for the fewest possible blocks plus one group of every order (at most row_max);
@@ -110,6 +127,11 @@ def assert_block_tables_match(layer: B.ExpandedLayer, e):
         got = table.cpu().numpy()
         assert want[0] <= lay.blk_cap[m]
         np.testing.assert_array_equal(got[:len(want)], want, err_msg=f"channel-block table {m}")
+        dtable = layer.decode_table(m)
+        if dtable is not None:
+            assert 16 <= lay.dec_limit[m] <= 256
+            want = expected_decode_table([e.order_kept(k) for k in range(k0, k1)], e.G, e.g, lay.dec_limit[m])
+            np.testing.assert_array_equal(dtable.cpu().numpy()[:len(want)], want, err_msg=f"decode-unit table {m}")
 
 
 def gpu_quantize(x: np.ndarray, static_scale=None, xd=None):

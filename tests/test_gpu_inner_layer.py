@@ -10,7 +10,7 @@ from tests import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_AUTO]
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_DECODE_TC, B.KERNEL_AUTO]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -87,7 +87,7 @@ def test_requantization_at_rounding_boundaries(oracle, kernel):
     """Weights, steps and inputs are powers of two times integers, so every fp32 output is exact and many
     quotients y / s fall exactly half way between two codes: ties must go to the even code on both sides."""
     rng = np.random.default_rng(5)
-    O, I, T = 128, 256, 96 if kernel != B.KERNEL_STREAM else 16
+    O, I, T = 128, 256, 96 if kernel not in (B.KERNEL_STREAM, B.KERNEL_DECODE_TC) else 16
     qw = rng.integers(-7, 8, size=(O, I))
     qw[:, 0] = 7                                   # every row spans the full 4-bit range: its scale is 2^-6 exactly
     W = (qw * 2.0 ** -6).astype(np.float32)

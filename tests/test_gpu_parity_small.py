@@ -11,7 +11,7 @@ from tests import gpu_harness as H
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_AUTO]
+KERNELS = [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_DECODE_TC, B.KERNEL_AUTO]
 
 
 @pytest.fixture(scope="module", autouse=True)

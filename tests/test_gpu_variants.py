@@ -17,7 +17,7 @@ def _w(rng, O, I, heavy=False):
     return W.astype(np.float32)
 
 
-@pytest.mark.parametrize("kernel", [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_AUTO])
+@pytest.mark.parametrize("kernel", [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_DECODE_TC, B.KERNEL_AUTO])
 @pytest.mark.parametrize("bits,O,I,T,K,g,n_keep,M", [(3, 256, 384, 300, 3, 8, 12, 1), (6, 192, 200, 270, 2, 8, 10, 2),
                                                       (3, 128, 640, 9, 4, 8, 5, 2), (6, 64, 128, 16, 2, 8, 8, 1)])
 def test_int3_and_int6_layers_match_the_oracle(oracle, kernel, bits, O, I, T, K, g, n_keep, M):
@@ -188,7 +188,7 @@ def test_unstructured_mask_matches_the_oracle(oracle, O, I, bits, K, g, keep_ele
     np.testing.assert_array_equal(y.view(np.uint32), f.y.view(np.uint32))
 
 
-@pytest.mark.parametrize("kernel", [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_AUTO])
+@pytest.mark.parametrize("kernel", [B.KERNEL_REFERENCE, B.KERNEL_TCGEN05, B.KERNEL_TCGEN05_PAIR, B.KERNEL_STREAM, B.KERNEL_DECODE_TC, B.KERNEL_AUTO])
 @pytest.mark.parametrize("act", [B.ACT_SILU, B.ACT_GELU, B.ACT_SIGMOID])
 def test_smooth_activations_in_the_fused_epilogue(oracle, kernel, act):
     """Inner layer with SiLU / GeLU / sigmoid (Sec. 3.2): the oracle evaluates sigma in binary64 and rounds once, the
@@ -196,7 +196,7 @@ def test_smooth_activations_in_the_fused_epilogue(oracle, kernel, act):
     step off -- the tolerance is one code, on at most half a percent of the outputs; the integer sums stay exact."""
     H.ensure_built()
     rng = np.random.default_rng(act)
-    O, I, T, bits, K, g, n_keep, M = 192, 256, 300 if kernel != B.KERNEL_STREAM else 16, 4, 4, 8, 12, 2
+    O, I, T, bits, K, g, n_keep, M = 192, 256, 300 if kernel not in (B.KERNEL_STREAM, B.KERNEL_DECODE_TC) else 16, 4, 4, 8, 12, 2
     W = _w(rng, O, I)
     bias = rng.standard_normal(O).astype(np.float32) * 0.1
     e = oracle.expand(W, bits, K, g, n_keep)
