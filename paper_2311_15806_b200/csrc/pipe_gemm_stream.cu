@@ -542,6 +542,57 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
 
 }  // namespace st
 
+namespace st {
+
+// What a launch has to ask the runtime, asked once per device (and once per kernel instantiation): the device's
+// shared memory and SM count, an instantiation's static shared memory, and the largest dynamic shared memory its
+// attribute has been raised to.
+struct KernelInfo {
+  const void* fn = nullptr;
+  int fixed = 0, dyn_set = 0;
+};
+struct DeviceCache {
+  std::mutex mu;
+  bool ready = false;
+  int smem_max = 0, sms = 0, n = 0;
+  KernelInfo k[24];
+};
+
+static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* smem_max, int* sms, int* fixed) {
+  constexpr int kMaxDevices = 64;
+  static DeviceCache cache[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+  DeviceCache& c = cache[dev];
+  std::lock_guard<std::mutex> lock(c.mu);
+  if (!c.ready) {
+    if (cudaDeviceGetAttribute(&c.smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&c.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    c.ready = true;
+  }
+  KernelInfo* ki = nullptr;
+  for (int i = 0; i < c.n; ++i)
+    if (c.k[i].fn == reinterpret_cast<const void*>(kern)) ki = &c.k[i];
+  if (!ki) {
+    if (c.n >= 24) return false;
+    cudaFuncAttributes fattr;
+    if (cudaFuncGetAttributes(&fattr, kern) != cudaSuccess) return false;
+    ki = &c.k[c.n++];
+    ki->fn = reinterpret_cast<const void*>(kern);
+    ki->fixed = static_cast<int>(fattr.sharedSizeBytes);
+  }
+  if (dyn_wanted_or_0 > ki->dyn_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_wanted_or_0) != cudaSuccess) return false;
+    ki->dyn_set = dyn_wanted_or_0;
+  }
+  *smem_max = c.smem_max;
+  *sms = c.sms;
+  *fixed = ki->fixed;
+  return true;
+}
+
+}  // namespace st
+
 static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   using namespace st;
   if (a.T > 16 || a.g % 8 != 0 || a.O % 8 != 0) return PIPE_ERR_UNSUPPORTED;
@@ -551,9 +602,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
   if (max_cluster > kMaxOrd) return PIPE_ERR_UNSUPPORTED;
-  static Params p;   // large; filled per call under the lock
-  static std::mutex mu;
-  std::lock_guard<std::mutex> lock(mu);
+  Params p;
   p.f = a;
   const int nt = a.T <= 8 ? 1 : 2;
   const int np = max_cluster <= 2 ? 1 : (max_cluster <= 4 ? 2 : 4);
@@ -567,10 +616,15 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   p.slabs_per_branch = a.O / 8;
   p.total_slabs = p.slabs_per_branch * a.num_branches;
   p.pass_slabs = kGroupWarps * spw;
-  int dev = 0, smem_max = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
-  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  // (the kernel instantiation depends only on bits, tokens and orders, all known here)
+  void (*kern)(const Params) = nullptr;
+#define PIPE_ST_PICK(B)                                                                     \
+  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1> : (np == 2 ? stream_forward_kernel<B, 1, 2> : stream_forward_kernel<B, 1, 4>); \
+  else kern = np == 1 ? stream_forward_kernel<B, 2, 1> : (np == 2 ? stream_forward_kernel<B, 2, 2> : stream_forward_kernel<B, 2, 4>);
+  if (a.bits == 8) { PIPE_ST_PICK(8) } else if (a.bits == 4) { PIPE_ST_PICK(4) } else { PIPE_ST_PICK(2) }
+#undef PIPE_ST_PICK
+  int smem_max = 0, sms = 0, fixed = 0;
+  if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
   p.ctas_per_branch = sms / a.num_branches;
   if (p.ctas_per_branch < 1) return PIPE_ERR_UNSUPPORTED;
   if (p.ctas_per_branch > p.slabs_per_branch) p.ctas_per_branch = p.slabs_per_branch;
@@ -583,15 +637,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   p.stage_bytes = round_up(p.kbps * (kXTile + pass_cap * 8 * max_cluster * p.pk), 1024);
   const int table_bytes = p.own_max * (max_cluster * 4 + max_cluster * 32 + 32) + kConsWarps * spw * (1 + 3 * max_cluster) * 4 +
                           p.pass_slabs * np * nt * 4 * 32 * 4;
-  void (*kern)(const Params) = nullptr;
-#define PIPE_ST_PICK(B)                                                                     \
-  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1> : (np == 2 ? stream_forward_kernel<B, 1, 2> : stream_forward_kernel<B, 1, 4>); \
-  else kern = np == 1 ? stream_forward_kernel<B, 2, 1> : (np == 2 ? stream_forward_kernel<B, 2, 2> : stream_forward_kernel<B, 2, 4>);
-  if (a.bits == 8) { PIPE_ST_PICK(8) } else if (a.bits == 4) { PIPE_ST_PICK(4) } else { PIPE_ST_PICK(2) }
-#undef PIPE_ST_PICK
-  cudaFuncAttributes fattr;
-  if (cudaFuncGetAttributes(&fattr, kern) != cudaSuccess) return PIPE_ERR_CUDA;
-  const int avail = smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024 - round_up(table_bytes, 16);
+  const int avail = smem_max - fixed - 1024 - round_up(table_bytes, 16);
   p.depth = avail / p.stage_bytes;
   if (p.depth > kMaxDepth) p.depth = kMaxDepth;
   // no more ring than the stages a CTA will ever fill
@@ -604,7 +650,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
     if (!make_tensor_map_2d_u8(&p.tmap_x[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
                                static_cast<uint64_t>(a.ldxq), 128, 16, true))
       return PIPE_ERR_CUDA;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess) return PIPE_ERR_CUDA;
+  if (!kernel_info(kern, dyn, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
   kern<<<grid, kThreads, dyn, stream>>>(p);
   count_launch(1);
   return launch_status();

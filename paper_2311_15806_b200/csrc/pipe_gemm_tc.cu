@@ -744,11 +744,46 @@ bool make_tensor_map_2d_u8(CUtensorMap* map, const void* base, uint64_t inner_by
                          swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
+namespace tc {
+
+// Asked of the runtime once per device: shared memory, SM count, the kernels' static shared memory; the dynamic
+// shared-memory attribute of both instantiations is raised to everything the device allows then.
+struct DeviceSetup {
+  int smem_max = 0, sms = 0, fixed = 0;
+  pipe_status status = PIPE_ERR_CUDA;
+};
+
+static const DeviceSetup& device_setup() {
+  constexpr int kMaxDevices = 64;
+  static DeviceSetup setups[kMaxDevices];
+  static std::once_flag once[kMaxDevices];
+  static const DeviceSetup bad;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return bad;
+  std::call_once(once[dev], [dev] {
+    DeviceSetup& d = setups[dev];
+    if (cudaDeviceGetAttribute(&d.smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return;
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
+    cudaFuncAttributes f0, f1;
+    if (cudaFuncGetAttributes(&f0, tc_forward_kernel<false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f1, tc_forward_kernel<true>) != cudaSuccess) return;
+    d.fixed = static_cast<int>(f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes);
+    const int dyn = d.smem_max - d.fixed;
+    if (cudaFuncSetAttribute(tc_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess) return;
+    d.status = PIPE_OK;
+  });
+  return setups[dev];
+}
+
+}  // namespace tc
+
 static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   using namespace tc;
-  static Params p;  // large; filled per call under the lock
-  static std::mutex mu;
-  std::lock_guard<std::mutex> lock(mu);
+  const DeviceSetup& ds = device_setup();
+  if (ds.status != PIPE_OK) return ds.status;
+  const int smem_max = ds.smem_max, sms = ds.sms;
+  Params p;
 
   int max_cluster = 0;
   for (int m = 0; m < a.num_branches; ++m) max_cluster = max(max_cluster, a.branch[m].k_end - a.branch[m].k_begin);
@@ -786,10 +821,6 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
     p.conv_chunks = a.cC / kKStep;
     p.ntok_tiles = ceil_div(p.conv_np, 2);
   }
-  int dev = 0, smem_max = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return PIPE_ERR_CUDA;
-  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   // Two token tiles per CTA tile halve the unpack work per multiply-accumulate; worth it once the
   // paired tiles still give every SM a tile.
   p.tpt = (static_cast<int64_t>(p.ncb) * ceil_div(p.ntok_tiles, 2) * a.num_branches >= sms) ? 2 : 1;
@@ -823,9 +854,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
     if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
     p.koff[k] = static_cast<uint32_t>(d >> 4);
   }
-  cudaFuncAttributes fattr;
-  if (cudaFuncGetAttributes(&fattr, tc_forward_kernel<false>) != cudaSuccess) return PIPE_ERR_CUDA;
-  p.depth = (smem_max - static_cast<int>(fattr.sharedSizeBytes) - 1024) / p.stage_bytes;  // static shared, alignment slack
+  p.depth = (smem_max - ds.fixed - 1024) / p.stage_bytes;  // static shared, alignment slack
   if (p.depth > kMaxRing) p.depth = kMaxRing;
   if (p.depth < 2) return PIPE_ERR_UNSUPPORTED;
   const int dyn_smem = p.depth * p.stage_bytes + 1024;
@@ -838,14 +867,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
                      static_cast<uint64_t>(a.ldxq), kKStep, p.tpt * kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
   }
-  static int attr_bytes[2] = {0, 0};
   const int which = a.q8_out ? 1 : 0;
-  if (attr_bytes[which] < dyn_smem) {
-    const cudaError_t e = which ? cudaFuncSetAttribute(tc_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem)
-                                : cudaFuncSetAttribute(tc_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_smem);
-    if (e != cudaSuccess) return PIPE_ERR_CUDA;
-    attr_bytes[which] = dyn_smem;
-  }
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;
   if (which) tc_forward_kernel<true><<<grid, kThreads, dyn_smem, stream>>>(p);
   else tc_forward_kernel<false><<<grid, kThreads, dyn_smem, stream>>>(p);

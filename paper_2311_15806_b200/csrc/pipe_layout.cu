@@ -17,9 +17,15 @@ void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::m
 int kernel_choice() { return g_kernel_choice.load(); }
 
 int* device_status_word() {
-  // The symbol is per device; look the address up for whichever device is current.
-  int* p = nullptr;
+  // The symbol is per device; its address is looked up once for whichever device is current and kept.
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int*> cached[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  int* p = cached[dev].load(std::memory_order_acquire);
+  if (p) return p;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
+  cached[dev].store(p, std::memory_order_release);
   return p;
 }
 

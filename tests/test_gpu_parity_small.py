@@ -366,3 +366,34 @@ def test_launch_counter_moves():
     before = B.pipe_launch_count()
     H.gpu_quantize(np.ones((4, 16), np.float32))
     assert B.pipe_launch_count() >= before + 2
+
+
+def test_forward_is_deterministic_across_repeated_runs(oracle):
+    """The same call three times over gives the same bits: integer sums, fp32 outputs, and a re-expansion of the same
+    weights (no atomics or race decides anything in the path)."""
+    rng = np.random.default_rng(2024)
+    O, I, T, bits, K, g, n_keep, M = 256, 640, 700, 4, 4, 8, 16, 2
+    W = _w(rng, O, I)
+    d = H.desc_of(O, I, bits, K, g, n_keep, M)
+    xs = [rng.standard_normal((T, I)).astype(np.float32) for _ in range(M)]
+    ref = None
+    for rep in range(3):
+        layer = H.gpu_expand(d, W)
+        q = [H.gpu_quantize(x) for x in xs]
+        ys, part = H.gpu_ensemble(layer, [a for a, _ in q], [b for _, b in q], None)
+        sections = np.concatenate([t.cpu().numpy().view(np.uint8).reshape(-1) for k in range(K)
+                                   for t in (layer.codes(k), layer.kcodes(k), layer.scales(k), layer.kept(k), layer.cum(k))])
+        got = (sections, [y.view(np.uint32).copy() for y in ys], part.copy())
+        if ref is None:
+            ref = got
+            continue
+        np.testing.assert_array_equal(got[0], ref[0])
+        for a, b in zip(got[1], ref[1]):
+            np.testing.assert_array_equal(a, b)
+        np.testing.assert_array_equal(got[2], ref[2])
+    for T_small in (1, 16):      # the small-token path too
+        q = [H.gpu_quantize(x[:T_small]) for x in xs]
+        outs = [H.gpu_ensemble(layer, [a for a, _ in q], [b for _, b in q], None)[0] for _ in range(3)]
+        for o in outs[1:]:
+            for a, b in zip(o, outs[0]):
+                np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
