@@ -54,6 +54,7 @@ struct Params {
   ForwardArgs f;
   int ntt, kblocks;       // ntt: pairs of token tiles; kblocks: reduction blocks of 128 lanes
   int ksteps;             // ring stages per tile: ceil(kblocks / kSub)
+  int blocks_fastest;     // tile order inside a branch, see locate_tile
   int ntok_tiles;         // token tiles (128 tokens) in total
   int nkmax;              // most orders any branch has
   int depth;              // stages in the ring
@@ -134,16 +135,24 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
                : "memory");
 }
 
-// Tiles are numbered branch by branch, inside a branch channel block by channel block, the token-tile pairs of a
-// block next to each other (so that the pairs working at the same time read the same weight rows).  tile_base[m] is
-// the number of tiles of the branches before m; the block counts come from the blob's channel-block tables and are
-// known on the device only.
+// Tiles are numbered branch by branch.  Inside a branch either the token-tile pairs of a channel block lie next to
+// each other (the pairs working at the same time then read the same weight rows and sweep the activations once per
+// block) or the channel blocks of a token-tile pair do (they share the activation tiles and sweep the weights once per
+// pair): Params::blocks_fastest picks the second order when the activations are too large to stay in L2.
+// tile_base[m] is the number of tiles of the branches before m; the block counts come from the blob's channel-block
+// tables and are known on the device only.
 __device__ __forceinline__ void locate_tile(const Params& p, const int* tile_base, int tile, int& m, int& cb, int& tt) {
   m = 0;
   while (m + 1 < p.f.num_branches && tile >= tile_base[m + 1]) ++m;
   const int rest = tile - tile_base[m];
-  cb = rest / p.ntt;
-  tt = rest - cb * p.ntt;
+  if (p.blocks_fastest) {
+    const int nblk = (tile_base[m + 1] - tile_base[m]) / p.ntt;
+    tt = rest / nblk;
+    cb = rest - tt * nblk;
+  } else {
+    cb = rest / p.ntt;
+    tt = rest - cb * p.ntt;
+  }
 }
 
 __device__ __forceinline__ void decode_tile(const Params& p, const int* tile_base, int tile, TileMeta& t) {
@@ -989,6 +998,16 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (static_cast<int64_t>(a.G) * p.ntt * a.num_branches > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
   p.kblocks = ceil_div(a.I, kKStep);
   p.ksteps = ceil_div(p.kblocks, kSub);
+  {
+    // bytes one branch sweeps in either order: its activations, or the packed rows of its orders
+    const int64_t x_bytes = a.conv_on ? static_cast<int64_t>(a.cN) * a.cH * a.cW * a.cC : a.T * static_cast<int64_t>(a.I);
+    int64_t w_bytes = 0;
+    for (int k = a.branch[0].k_begin; k < a.branch[0].k_end; ++k) w_bytes += static_cast<int64_t>(a.order[k].rows) * a.kernel_row_bytes;
+    // (sweeping the activations once per channel block is the better order while they stay in L2 beside the outputs
+    // streaming through it -- the pairs working together then share one weight block -- so the other order is taken
+    // only for activations of tens of megabytes)
+    p.blocks_fastest = (x_bytes > w_bytes && x_bytes > (48ll << 20)) ? 1 : 0;
+  }
   p.pk = kKStep * a.bits / 8;
   p.shift = 8 - a.bits;
   int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
