@@ -113,6 +113,12 @@ def workload_spec(name: str):
 # program (summaries under profiles/, named in the comment).  A workload without a capture of the present
 # kernel has no entry and reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
+    "cfg2": 32994816 + 53515264,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
+    "cfg3a": 9401344 + 47268608,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
+    "cfg4a_t4096": 90932480 + 308943872,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
+    "cfg5": 403271168 + 1026669312,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
+    "cfg4a_t1": 56556288 + 42240,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
+    "cfg4a_t16": 56684288 + 76288,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
 }
 
 
@@ -304,7 +310,7 @@ def time_forward_alone(run, torch, device_index, flush_needed: bool, min_seconds
     return statistics.median(launch_ms), min(launch_ms), how, clocks
 
 
-def forward_row(run, spec, fwd_ms, fwd_best_ms, how, clocks, peaks, int8):
+def forward_row(run, spec, fwd_ms, fwd_best_ms, how, clocks, peaks, int8, sms: int = 148):
     """One row of the workloads table: the GEMM of one configuration against its roofline."""
     macs = run.macs_per_token() * run.T
     ops = 2.0 * macs
@@ -321,6 +327,10 @@ def forward_row(run, spec, fwd_ms, fwd_best_ms, how, clocks, peaks, int8):
            "frac_int8_int_mm": (tops / int8["int_mm_8192"]) if int8.get("int_mm_8192") else None,
            "frac_int8_2x_bf16_burst": tops / (2.0 * peaks["bf16_tflops"]),
            "frac_int8_nominal_4500": tops / 4500.0,
+           # per clock and SM against the tensor pipe's issue rate (8192 MAC), at the SM clock sampled during this loop:
+           # a seconds-long loop of a dense kernel runs into the power cap, so its clock is below the probe's burst clock
+           "mac_per_clk_per_sm": (macs / (fwd_ms * 1e-3) / (clocks["sm_mhz"] * 1e6) / sms) if clocks.get("sm_mhz") else None,
+           "frac_issue_rate_at_sampled_clock": (macs / (fwd_ms * 1e-3) / (clocks["sm_mhz"] * 1e6) / sms / 8192.0) if clocks.get("sm_mhz") else None,
            "frac_hbm_copy": gbs / peaks["hbm_gbs"], "frac_hbm_nominal_8000": gbs / 8000.0,
            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(spec.name),
            "clocks": clocks}
@@ -498,7 +508,8 @@ def run_ours(args):
     st = B.pipe_poll_status()
     if st != B.PIPE_OK:
         raise SystemExit(f"device status after the kernel timing loop: {B.pipe_status_string(st)}")
-    head_row = forward_row(run, spec, fwd_ms, fwd_best, how, fclocks, peaks, int8)
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    head_row = forward_row(run, spec, fwd_ms, fwd_best, how, fclocks, peaks, int8, sms)
     phases = {"expand": statistics.mean(t_expand), "quantize": statistics.mean(t_quant), "forward": statistics.mean(t_fwd)}
     expand_gbs = run.expand_bytes() / (phases["expand"] * 1e-3) / 1e9
     quant_gbs = run.quantize_bytes() / (phases["quantize"] * 1e-3) / 1e9 if phases["quantize"] > 0 else None
@@ -530,7 +541,7 @@ def run_ours(args):
             except B.PipeError as exc:   # only with --kernel: the forced back end does not take this shape
                 table.append({"workload": name, "tokens": run.T, "error": str(exc)})
                 continue
-            row = forward_row(run, s2, ms, best, how2, ck, peaks, int8)
+            row = forward_row(run, s2, ms, best, how2, ck, peaks, int8, sms)
             row["quantize_ms"] = q0.elapsed_time(q1)
             if name == "cfg4a_t1":
                 host_us = host_time_per_forward_call(run, B, torch)
