@@ -46,11 +46,14 @@ constexpr int kTmemCols = 512;
 constexpr int kColmapEntries = kMaxClusterOrders * (PIPE_BLOCK_CHANNELS / 8);
 constexpr int kAccCols = 256;
 constexpr int kMaxRing = 3;
-constexpr int kALanes = 4;   // lanes of the activation producer warp that issue copies
+constexpr int kTileRing = 8;   // tiles whose stacked-row count the unpack warps keep for the MMA issuer (they are at
+                               // most a ring of stages, i.e. three tiles, ahead of it)
 using namespace tcc;
 
 struct Params {
   CUtensorMap tmap_a[PIPE_MAX_ORDERS];  // one per branch input
+  CUtensorMap tmap_y[PIPE_MAX_ORDERS];  // one per branch output (fp32), valid where y_tma has the branch's bit
+  uint32_t y_tma;                       // branches whose fp32 output the epilogue may write with tensor stores
   ForwardArgs f;
   int ntt, kblocks;       // ntt: pairs of token tiles; kblocks: reduction blocks of 128 lanes
   int ksteps;             // ring stages per tile: ceil(kblocks / kSub)
@@ -112,6 +115,19 @@ __device__ __forceinline__ void tma_pair_load_4d(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(lead_bar)
       : "memory");
+}
+
+// Tensor stores of the epilogue (shared memory -> global, one bulk group per store).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(reinterpret_cast<uint64_t>(map)),
+               "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
 }
 
 // Implicit convolution: a token tile is two 8 x 8 pixel patches (64 rows each); patch p lies in
@@ -203,6 +219,7 @@ struct Rings {
   int rank, pair, npairs;                  // this CTA's rank in the pair; tiles go round the pairs
   const int* tile_base;                    // shared memory: tiles before each branch, then the total
   int num_tiles;
+  volatile int* ntot;                      // shared memory: stacked rows of this pair's tile i at [i % kTileRing]
   uint32_t stage0;        // shared address of stage 0 (activation tile, then B tile)
   uint8_t* stage_gen;     // generic address of stage 0
   volatile int* abort_flag;
@@ -260,6 +277,8 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
       TileMeta t;
       decode_tile(p, g.tile_base, g.pair + ti * g.npairs, t);
       const int n_total = t.rowbase[kMaxClusterOrders];
+      // for the MMA issuer, which learns of it through the stage barrier this warp arrives on below
+      if (lane == 0) g.ntot[ti % kTileRing] = n_total;
       const int half = pair_mma_rows(n_total, BITS) >> 1;
       const int h0 = g.rank * half;
       mine = max(0, min(half, n_total - h0));   // rows of this CTA's half that exist
@@ -428,6 +447,8 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   const int sj = spp ^ ((sr0 >> 1) & 3);     // the same for all four rows (they differ by multiples of 8)
   const uint32_t stg_w = smem_u32(x.stg) + static_cast<uint32_t>(lane * 64);
   const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
+  const bool bias_vec = (reinterpret_cast<uintptr_t>(p.f.bias) & 15) == 0;
+  bool stg_busy = false;   // a tensor store of this warp may still be reading the staging block
   const int et = (x.warp - 2 - kUnpackWarps) * 32 + lane;   // this thread among the epilogue threads
   for (int tile = x.pair; tile < x.num_tiles; tile += x.npairs, ++tcount) {
     TileMeta t;
@@ -516,6 +537,17 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       if (tile_ok && (p.f.conv_on ? inside(sr0 + 8 * i) : tok < p.f.T)) srow_ok |= 1u << i;
     }
     const bool vec_ok = y_vec && ((reinterpret_cast<uintptr_t>(br.y) & 15) == 0);
+    // Tensor stores (one per full 16-channel group, issued by one lane, straight from the staging block) where the
+    // host found the output eligible: they leave the warp with neither the second pass over the staging block nor
+    // the store instructions, and rows beyond T -- for a convolution, pixels beyond the image -- are clipped by
+    // the copy engine.  A sum into y keeps the path through registers, which alone adds in binary32 round-to-nearest.
+    const bool tma_out = !Q8 && ((p.y_tma >> t.m) & 1u) && !br.accumulate && tile_ok;
+    int ty1 = static_cast<int>(tok_base), ty2 = 0, ty3 = 0;   // coordinates behind the channel: token, or (x, y, image)
+    if (p.f.conv_on) {
+      const int patch = 2 * ttile + (q >> 1);
+      patch_origin(p, patch, ty3, ty2, ty1);
+      ty2 += (q & 1) * 4;
+    }
     float ostep = 0.f, orcp = 0.f;
     bool ofast = false;
     int8_t* qrow = nullptr;      // this lane's output row at channel c0
@@ -547,6 +579,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
         bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
       }
       // ---- this lane's row: 16 channels into the staging block (as 16 codes into registers for the fused epilogue)
+      const bool use_tma = tma_out && 2 * grp + 1 < nch;
       uint32_t packed[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
       for (int sub = 0; sub < 2; sub += CH) {
@@ -629,6 +662,27 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
             continue;
           }
           const int j0 = 2 * (sub + u);
+          if (use_tma && add_bias) {
+            // tensor stores: the bias of this lane's own channels joins before the staging block (the same addition,
+            // after the whole chain, as on the other path)
+            const float* bp = p.f.bias + c0 + 8 * chunk;
+            float bo[8];
+            if (bias_vec) {
+              const float4 b0 = __ldg(reinterpret_cast<const float4*>(bp)), b1 = __ldg(reinterpret_cast<const float4*>(bp) + 1);
+              bo[0] = b0.x, bo[1] = b0.y, bo[2] = b0.z, bo[3] = b0.w, bo[4] = b1.x, bo[5] = b1.y, bo[6] = b1.z, bo[7] = b1.w;
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) bo[e] = __ldg(bp + e);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], bo[e]);
+          }
+          if (sub + u == 0 && stg_busy) {
+            // the tensor store of the group before must have read the staging block
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncwarp();
+            stg_busy = false;
+          }
           asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg_w + static_cast<uint32_t>((j0 ^ wsw) << 4)), "f"(y[0]),
                        "f"(y[1]), "f"(y[2]), "f"(y[3])
                        : "memory");
@@ -656,6 +710,18 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
               }
           }
         }
+        continue;
+      }
+      if (use_tma) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the staging block, for the copy engine
+        __syncwarp();
+        if (lane == 0) {
+          const int cch = c0 + 16 * grp;
+          if (p.f.conv_on) tma_store_4d(&p.tmap_y[t.m], smem_u32(x.stg), cch, ty1, ty2, ty3);
+          else tma_store_2d(&p.tmap_y[t.m], smem_u32(x.stg), cch, ty1);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        stg_busy = true;
         continue;
       }
       __syncwarp();
@@ -686,6 +752,9 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     __syncwarp();
     if (lane == 0) mbar_arrive_lead(x.tempty_lead0 + 8u * buf);   // one arrival per warp, on the first CTA's barrier
   }
+  // the warp's tensor stores are complete before it leaves (the staging block is read, the rows are written)
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  __syncwarp();
 }
 
 template <bool Q8>
@@ -697,9 +766,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_base_s[PIPE_MAX_ORDERS + 1];   // tiles before each branch, then the total
+  __shared__ int ntot_s[kTileRing];
   __shared__ __align__(16) int16_t epi_colmap[2][kColmapEntries];   // even / odd tile: accumulator column of (8-channel chunk, order) or -1
   __shared__ __align__(16) float epi_cscale[2][kMaxN];             // even / odd tile: s_k * lambda_x of every stacked row
-  __shared__ __align__(16) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels
+  __shared__ __align__(1024) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels (the
+                                                                    // source of tensor stores with the 64-byte swizzle)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -717,6 +788,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   g.stage0 = smem_base;
   g.stage_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   g.abort_flag = &abort_flag_s;
+  g.ntot = ntot_s;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -811,32 +883,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kStageBOff);
       uint32_t tcount = 0;
       bool ok = true;
-      // stacked rows of a tile (the only tile metadata this role needs); fetched one tile ahead
-      auto stacked_rows = [&](int tile) {
-        int m, cb, tt;
-        locate_tile(p, g.tile_base, tile, m, cb, tt);
-        const BranchArgs& br = p.f.branch[m];
-        const int j0 = __ldg(br.blk + 1 + cb), j1 = __ldg(br.blk + 2 + cb);
-        int n = 0;
-        for (int k = br.k_begin; k < br.k_end; ++k) {
-          const int32_t* cum = p.f.order[k].cum;
-          n += (__ldg(cum + j1) - __ldg(cum + j0)) * p.f.g;
-        }
-        return n;
-      };
-      int n_next = g.pair < g.num_tiles ? stacked_rows(g.pair) : 0;
+      // The stacked rows of a tile (the only tile metadata this role needs) come from the unpack warps, which decode
+      // every tile anyway: a global load here, two dependent levels of them, would stall the one thread that feeds
+      // the tensor core for thousands of cycles per tile.
       for (int tile = g.pair; ok && tile < g.num_tiles; tile += g.npairs, ++tcount) {
-        const int n_total = n_next;
-        if (tile + g.npairs < g.num_tiles) n_next = stacked_rows(tile + g.npairs);
         const int buf = tcount & 1;
         const uint32_t aph = (tcount >> 1) & 1;
         if (!mbar_wait<true>(g.tempty0 + 8u * buf, aph ^ 1, g.abort_flag, p.f.status)) { ok = false; break; }
-        const int n = pair_mma_rows(n_total, p.f.bits);
-        const uint32_t idesc = idesc_i8(2 * kTileM, n);
+        uint32_t idesc = 0;
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
         for (int ks = 0; ks < p.ksteps; ++ks, rp.advance(1, depth)) {
           if (!mbar_wait<true>(g.full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // (written by an unpack warp of this CTA before its arrival on the barrier just waited for)
+          if (ks == 0) idesc = idesc_i8(2 * kTileM, pair_mma_rows(g.ntot[tcount % kTileRing], p.f.bits));
           const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
           const int nsub = min(kSub, p.kblocks - ks * kSub);
           for (int sub = 0; sub < nsub; ++sub) {
@@ -1033,6 +1093,17 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),
                      static_cast<uint64_t>(a.ldxq), kKStep, kTileM, CU_TENSOR_MAP_SWIZZLE_128B))
       return PIPE_ERR_CUDA;
+  }
+  // fp32 outputs that tensor stores can write: 16-byte aligned rows of at least one box
+  p.y_tma = 0;
+  if (!a.q8_out && a.ldy % 4 == 0 && a.O >= 16) {
+    for (int m = 0; m < a.num_branches; ++m) {
+      const float* y = a.branch[m].y;
+      if (!y || (reinterpret_cast<uintptr_t>(y) & 15) || a.branch[m].accumulate) continue;
+      const bool ok = a.conv_on ? make_map_out_nhwc(&p.tmap_y[m], y, a.cN, a.cHo, a.cWo, static_cast<uint64_t>(a.O), static_cast<uint64_t>(a.ldy))
+                                : make_map_out_2d(&p.tmap_y[m], y, static_cast<uint64_t>(a.O), static_cast<uint64_t>(a.T), static_cast<uint64_t>(a.ldy));
+      if (ok) p.y_tma |= 1u << m;
+    }
   }
   // one cluster of two CTAs per SM pair; the tiles (counted on the device) go round all resident pairs
   cudaLaunchConfig_t cfg = {};

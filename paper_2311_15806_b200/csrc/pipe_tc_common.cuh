@@ -222,5 +222,32 @@ inline bool make_map_nhwc(CUtensorMap* map, const void* base, int N, int H, int 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 output [rows, channels] with a row pitch: one box = 16 channels x 32 rows (64-byte rows, 64-byte swizzle).
+inline bool make_map_out_2d(CUtensorMap* map, const float* base, uint64_t channels, uint64_t rows, uint64_t pitch_elems) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {channels, rows};
+  const cuuint64_t strides[1] = {pitch_elems * 4};
+  const cuuint32_t box[2] = {16, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 output of a convolution, pixels in NHW order with a pixel pitch: one box = 16 channels x 8 pixels x 4 image
+// rows of one image (half of an 8 x 8 patch); what hangs over the right or lower edge of the image is not written.
+inline bool make_map_out_nhwc(CUtensorMap* map, const float* base, int N, int Ho, int Wo, uint64_t channels, uint64_t pitch_elems) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {channels, static_cast<cuuint64_t>(Wo), static_cast<cuuint64_t>(Ho), static_cast<cuuint64_t>(N)};
+  const cuuint64_t strides[3] = {pitch_elems * 4, pitch_elems * 4 * Wo, pitch_elems * 4 * Wo * Ho};
+  const cuuint32_t box[4] = {16, 8, 4, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tcc
 }  // namespace pipe
