@@ -114,6 +114,15 @@ typedef struct pipe_layer_desc {
  *                 run close to their widest shape, and evenly, however sparse the orders are.  A cluster of more
  *                 than 8 orders, or whose single group can exceed the row limit (orders * g > PIPE_BLOCK_ROWS), has
  *                 no table.
+ *   rec_off[m]    one record of PIPE_BLOCK_RECORD_BYTES per block of table m (room for rec_cap[m] records, a bound on
+ *                 the block count that follows from the cut), everything the epilogue of a tile of that block needs,
+ *                 so that a kernel fetches it with one bulk copy instead of walking the prefix counts:
+ *                   int32 [32]   c0, c1 (the block's channels [c0, c1)), orders of the cluster, stacked rows n, 4 x 0,
+ *                                rowbase[0..7] (row of order i's first kept row in the stacked block; n beyond the
+ *                                cluster's orders), start[0..7] (that row's index in order i's compacted rows), 8 x 0
+ *                   int16 [512]  entry 8 c + i: the stacked row of channel c0 + 8 c in order i, or -1 when the
+ *                                order has pruned that channel's group (or c, i lie beyond the block / the cluster)
+ *                   float [256]  the scale of every stacked row (0 beyond n)
  *   dec_off[m]    the same structure (n, b_0 .. b_n; room for G blocks) with the row limit dec_limit[m]: the units of
  *                 the small-token (T <= 16) tensor-core kernel, which streams every weight once.  There the limit
  *                 is chosen so that the units of the clusters that run together -- the M predictors, or the one
@@ -123,6 +132,7 @@ typedef struct pipe_layer_desc {
  */
 #define PIPE_BLOCK_ROWS 256
 #define PIPE_BLOCK_CHANNELS 512
+#define PIPE_BLOCK_RECORD_BYTES (32 * 4 + 8 * (PIPE_BLOCK_CHANNELS / 8) * 2 + PIPE_BLOCK_ROWS * 4)
 typedef struct pipe_layer_layout {
   int32_t num_groups;        /* G = O / g */
   int32_t total_rows;        /* R_total = sum_k rows[k] = O + (K-1) * keep_groups * g */
@@ -138,6 +148,8 @@ typedef struct pipe_layer_layout {
   uint64_t cum_off[PIPE_MAX_ORDERS];
   uint64_t blk_off[PIPE_MAX_ORDERS + 1]; /* channel-block tables (see above); 0 = the cluster has none */
   int32_t blk_cap[PIPE_MAX_ORDERS + 1];  /* blocks each table has room for */
+  uint64_t rec_off[PIPE_MAX_ORDERS + 1]; /* block records of table m (see above); 0 = the cluster has no table */
+  int32_t rec_cap[PIPE_MAX_ORDERS + 1];  /* records there is room for */
   int32_t decode_split;                  /* CTAs that share one decode unit's reduction axis: predictors' tables */
   uint64_t dec_off[PIPE_MAX_ORDERS + 1]; /* decode-unit tables (see above); 0 = the cluster has none */
   int32_t dec_limit[PIPE_MAX_ORDERS + 1]; /* rows a decode unit of the cluster may stack */

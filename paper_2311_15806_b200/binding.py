@@ -15,6 +15,9 @@ import torch
 from . import build as _build
 
 MAX_ORDERS = 16
+BLOCK_ROWS = 256
+BLOCK_CHANNELS = 512
+BLOCK_RECORD_BYTES = 32 * 4 + 8 * (BLOCK_CHANNELS // 8) * 2 + BLOCK_ROWS * 4
 BLOB_ALIGN = 1024
 
 STATUS_NAMES = ["PIPE_OK", "PIPE_ERR_INVALID_ARG", "PIPE_ERR_SHAPE", "PIPE_ERR_ALIGNMENT", "PIPE_ERR_UNSUPPORTED",
@@ -58,7 +61,8 @@ class LayerLayout(C.Structure):
                 ("codes_off", C.c_uint64 * MAX_ORDERS), ("kcodes_off", C.c_uint64 * MAX_ORDERS),
                 ("scales_off", C.c_uint64 * MAX_ORDERS), ("kept_off", C.c_uint64 * MAX_ORDERS),
                 ("cum_off", C.c_uint64 * MAX_ORDERS), ("blk_off", C.c_uint64 * (MAX_ORDERS + 1)),
-                ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("decode_split", C.c_int32),
+                ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("rec_off", C.c_uint64 * (MAX_ORDERS + 1)),
+                ("rec_cap", C.c_int32 * (MAX_ORDERS + 1)), ("decode_split", C.c_int32),
                 ("dec_off", C.c_uint64 * (MAX_ORDERS + 1)), ("dec_limit", C.c_int32 * (MAX_ORDERS + 1)),
                 ("decode_split_all", C.c_int32),
                 ("blob_bytes", C.c_uint64), ("expand_ws_bytes", C.c_uint64),
@@ -434,6 +438,12 @@ class ExpandedLayer:
         if self.layout.dec_off[m] == 0:
             return None
         return self.section(self.layout.dec_off[m], (self.layout.num_groups + 2) * 4).view(torch.int32)
+
+    def block_records(self, m: int) -> torch.Tensor | None:
+        """Block records of table m as bytes [rec_cap, BLOCK_RECORD_BYTES] (the first n of them are written), or None."""
+        if self.layout.rec_off[m] == 0:
+            return None
+        return self.section(self.layout.rec_off[m], self.layout.rec_cap[m] * BLOCK_RECORD_BYTES).view(-1, BLOCK_RECORD_BYTES)
 
     def block_table(self, m: int) -> torch.Tensor | None:
         """Channel-block table m (int32: n, b_0 .. b_n), or None when the cluster has none."""

@@ -46,6 +46,32 @@ __host__ __device__ inline T round_up(T a, T b) {
   return ceil_div(a, b) * b;
 }
 
+// Block records of a channel-block table (layout in pipe.h).
+constexpr int kRecHeaderInts = 32;
+constexpr int kRecRowbase = 8, kRecStart = 16;              // header words of rowbase[0..7], start[0..7]
+constexpr int kRecColmapOff = kRecHeaderInts * 4;           // bytes
+constexpr int kRecColmapEntries = 8 * (PIPE_BLOCK_CHANNELS / 8);
+constexpr int kRecScaleOff = kRecColmapOff + kRecColmapEntries * 2;
+constexpr int kRecBytes = kRecScaleOff + PIPE_BLOCK_ROWS * 4;
+static_assert(kRecBytes == PIPE_BLOCK_RECORD_BYTES && kRecBytes % 16 == 0, "record layout");
+
+// Row limit of the blocks of a channel-block table (the definition in pipe.h): R rows kept by the cluster's nk orders.
+inline int block_row_limit(int64_t R, int O, int nk, int g) {
+  const int64_t n0r = ceil_div<int64_t>(R, PIPE_BLOCK_ROWS), n0c = ceil_div<int64_t>(O, PIPE_BLOCK_CHANNELS);
+  const int64_t n0 = n0r > n0c ? n0r : n0c;
+  const int64_t even = round_up<int64_t>(ceil_div<int64_t>(R, n0 > 0 ? n0 : 1), 16) + static_cast<int64_t>(nk) * g;
+  return static_cast<int>(even < PIPE_BLOCK_ROWS ? even : PIPE_BLOCK_ROWS);
+}
+// A bound on the blocks the cut can make: a block closed by its rows stacks more than limit - nk * g of them (the
+// next group would have added nk * g at most), a block closed by its channels holds PIPE_BLOCK_CHANNELS / g groups,
+// and one block is left open at the end.
+inline int block_count_bound(int64_t R, int O, int G, int nk, int g) {
+  const int64_t per = block_row_limit(R, O, nk, g) - static_cast<int64_t>(nk) * g;
+  const int64_t maxg = PIPE_BLOCK_CHANNELS / g > 0 ? PIPE_BLOCK_CHANNELS / g : 1;
+  const int64_t n = R / (per > 0 ? per + 1 : 1) + G / maxg + 2;
+  return static_cast<int>(n < G ? n : G);
+}
+
 // Raise a device-side error: first error wins.
 __device__ inline void raise_status(int* status, int code) { atomicCAS(status, 0, code); }
 
@@ -131,6 +157,7 @@ struct BranchArgs {
   const int32_t* zp;       // zero point of asymmetric activation codes (one int on the device), or nullptr for 0
   const int32_t* dec;      // decode-unit table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
   const int32_t* blk;      // channel-block table of this branch's cluster of orders (n, b_0 .. b_n), or nullptr
+  const uint8_t* rec;      // the table's block records (PIPE_BLOCK_RECORD_BYTES each), or nullptr
   int add_bias;    // bias enters this branch
   int accumulate;  // y += result (summed ensemble, branches after the first)
 };

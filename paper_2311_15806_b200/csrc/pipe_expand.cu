@@ -497,6 +497,82 @@ __global__ void block_table_kernel(const __grid_constant__ BlockTableArgs a) {
   }
 }
 
+// Block records (layout in pipe.h): one thread block per (block of a table, table).
+struct BlockRecordArgs {
+  const int32_t* cum[PIPE_MAX_ORDERS + 1][8];   // prefix counts of the cluster's orders
+  const float* scales[PIPE_MAX_ORDERS + 1][8];  // their row scales
+  int nk[PIPE_MAX_ORDERS + 1];
+  const int32_t* tbl[PIPE_MAX_ORDERS + 1];      // the channel-block table (n, b_0 .. b_n)
+  uint8_t* out[PIPE_MAX_ORDERS + 1];
+  int cap[PIPE_MAX_ORDERS + 1];
+  int g;
+  int* status;
+};
+
+__global__ void block_record_kernel(const __grid_constant__ BlockRecordArgs a) {
+  const int m = blockIdx.y, cb = blockIdx.x;
+  if (!a.out[m]) return;
+  const int n_blocks = a.tbl[m][0];
+  if (n_blocks > a.cap[m]) {   // cannot happen (the capacity is a bound on the cut); never write past it
+    if (cb == 0 && threadIdx.x == 0) raise_status(a.status, PIPE_ERR_WORKSPACE);
+    return;
+  }
+  if (cb >= n_blocks) return;
+  __shared__ int rowbase_s[9], start_s[8];
+  const int j0 = a.tbl[m][1 + cb], j1 = a.tbl[m][2 + cb];
+  const int nk = a.nk[m];
+  if (threadIdx.x == 0) {
+    int rb = 0;
+    for (int q = 0; q < 8; ++q) {
+      rowbase_s[q] = rb;
+      start_s[q] = 0;
+      if (q < nk) {
+        const int lo = a.cum[m][q][j0], hi = a.cum[m][q][j1];
+        start_s[q] = lo * a.g;
+        rb += (hi - lo) * a.g;
+      }
+    }
+    rowbase_s[8] = rb;
+  }
+  __syncthreads();
+  uint8_t* rec = a.out[m] + static_cast<size_t>(cb) * kRecBytes;
+  int32_t* hdr = reinterpret_cast<int32_t*>(rec);
+  int16_t* colmap = reinterpret_cast<int16_t*>(rec + kRecColmapOff);
+  float* scale = reinterpret_cast<float*>(rec + kRecScaleOff);
+  const int c0 = j0 * a.g, c1 = j1 * a.g, n_total = rowbase_s[8];
+  for (int i = threadIdx.x; i < kRecHeaderInts; i += blockDim.x) {
+    int v = 0;
+    if (i == 0) v = c0;
+    else if (i == 1) v = c1;
+    else if (i == 2) v = nk;
+    else if (i == 3) v = n_total;
+    else if (i >= kRecRowbase && i < kRecRowbase + 8) v = rowbase_s[i - kRecRowbase];
+    else if (i >= kRecStart && i < kRecStart + 8) v = start_s[i - kRecStart];
+    hdr[i] = v;
+  }
+  const int nch = (c1 - c0) >> 3;
+  for (int e = threadIdx.x; e < kRecColmapEntries; e += blockDim.x) {
+    const int cc = e >> 3, q = e & 7;
+    int col = -1;
+    if (q < nk && cc < nch) {
+      const int c = c0 + 8 * cc;
+      const int j = c / a.g;
+      const int lo = a.cum[m][q][j], hi = a.cum[m][q][j + 1];
+      if (hi > lo) col = rowbase_s[q] + lo * a.g + c % a.g - start_s[q];
+    }
+    colmap[e] = static_cast<int16_t>(col);
+  }
+  for (int r = threadIdx.x; r < PIPE_BLOCK_ROWS; r += blockDim.x) {
+    float v = 0.f;
+    if (r < n_total) {
+      int q = 0;
+      while (q + 1 < nk && r >= rowbase_s[q + 1]) ++q;
+      v = a.scales[m][q][start_s[q] + (r - rowbase_s[q])];
+    }
+    scale[r] = v;
+  }
+}
+
 __global__ void write_header_kernel(uint32_t* hdr, pipe_layer_desc d) {
   if (threadIdx.x == 0) {
     hdr[0] = kBlobMagic;
@@ -623,15 +699,35 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
       // even blocks: the fewest blocks that could hold the cluster's rows, their mean size plus one group of slack
       int64_t R = 0;
       for (int k = k0; k < k1; ++k) R += L.lay.rows[k];
-      const int64_t n0r = ceil_div<int64_t>(R, PIPE_BLOCK_ROWS), n0c = ceil_div<int64_t>(L.O, PIPE_BLOCK_CHANNELS);
-      const int64_t n0 = n0r > n0c ? n0r : n0c;
-      const int64_t even = round_up<int64_t>(ceil_div<int64_t>(R, n0), 16) + static_cast<int64_t>(k1 - k0) * L.g;
-      t.limit[m] = static_cast<int>(even < PIPE_BLOCK_ROWS ? even : PIPE_BLOCK_ROWS);
+      t.limit[m] = block_row_limit(R, L.O, k1 - k0, L.g);
       any = true;
     }
     if (any) {
       block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
       count_launch(1);
+      // the records of the blocks just cut
+      BlockRecordArgs r;
+      std::memset(&r, 0, sizeof(r));
+      r.g = L.g;
+      r.status = status;
+      int max_cap = 0;
+      for (int m = 0; m <= L.M; ++m) {
+        if (L.lay.rec_off[m] == 0) continue;
+        const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
+        r.nk[m] = k1 - k0;
+        for (int q = 0; q < k1 - k0; ++q) {
+          r.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
+          r.scales[m][q] = reinterpret_cast<const float*>(blob + L.lay.scales_off[k0 + q]);
+        }
+        r.tbl[m] = reinterpret_cast<const int32_t*>(blob + L.lay.blk_off[m]);
+        r.out[m] = blob + L.lay.rec_off[m];
+        r.cap[m] = L.lay.rec_cap[m];
+        max_cap = max_cap > r.cap[m] ? max_cap : r.cap[m];
+      }
+      if (max_cap > 0) {
+        block_record_kernel<<<dim3(max_cap, L.M + 1), 256, 0, s>>>(r);
+        count_launch(1);
+      }
     }
     // the decode-unit tables: the same cut with the layout's row limits
     any = false;

@@ -53,6 +53,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     // one branch running all K orders is the "all orders" cluster (entry L.M), otherwise predictor m's own
     const int set = (k_end[m] - k_begin[m] == L.K) ? L.M : m;
     b.blk = block_table(L, d_blob, set);
+    b.rec = L.lay.rec_off[set] ? static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[set] : nullptr;
     b.dec = L.lay.dec_off[set] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.dec_off[set]) : nullptr;
   }
   a.decode_split = (M == 1 && k_end[0] - k_begin[0] == L.K) ? L.lay.decode_split_all : L.lay.decode_split;
@@ -205,6 +206,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   b.add_bias = 1;
   b.accumulate = 0;
   b.blk = block_table(L, d_blob, L.M);
+  b.rec = L.lay.rec_off[L.M] ? static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[L.M] : nullptr;
   b.dec = nullptr;
   a.decode_split = 0;
   b.yq = d_yq;

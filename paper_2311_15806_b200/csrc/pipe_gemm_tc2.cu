@@ -37,15 +37,14 @@ constexpr int kMaxClusterOrders = 8;
 constexpr int kUnpackWarps = 6;   // 16 warps per CTA: 128 registers per thread (see the one-SM kernel)
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kUnpackWarps + kEpiWarps);
-constexpr int kUnpackThreads = 32 * kUnpackWarps;
 constexpr int kABytes = kTileM * kKStep;       // 16 KiB per token tile and reduction block
 constexpr int kBtBytes = (kMaxN / 2) * kKStep;   // 16 KiB per block: this CTA's half of the stacked rows
 constexpr int kStageBytes = kSub * (kABytes + kBtBytes);   // [kSub activation tiles][kSub B tiles]
 constexpr int kStageBOff = kSub * kABytes;
 constexpr int kTmemCols = 512;
-constexpr int kColmapEntries = kMaxClusterOrders * (PIPE_BLOCK_CHANNELS / 8);
 constexpr int kAccCols = 256;
 constexpr int kMaxRing = 3;
+constexpr int kRecBufs = 3;    // copies of block records in shared memory (this tile, the next, the one before)
 constexpr int kTileRing = 8;   // tiles whose stacked-row count the unpack warps keep for the MMA issuer (they are at
                                // most a ring of stages, i.e. three tiles, ahead of it)
 using namespace tcc;
@@ -407,7 +406,9 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
 
 struct EpiCtx {
   uint32_t tmem_base, tfull0, tempty0;
-  uint32_t tables0;   // two barriers: the tile tables of an even / odd tile are complete
+  uint32_t recbar0;   // kRecBufs barriers: the block record of the tile has landed
+  uint32_t rec0;      // shared address of the first record copy
+  const float* sx_s;  // shared memory: lambda_x of every branch (and, behind them, the output steps of the fused epilogue)
   volatile int* abort_flag;
   int warp, lane;
   int rank, pair, npairs;
@@ -415,8 +416,6 @@ struct EpiCtx {
   int num_tiles;
   uint32_t tempty_lead0;   // the accumulator-released barriers of the pair's first CTA (cluster address)
   int part, nparts;  // share of the 16-channel groups this warp drains (two warps per lane quarter)
-  int16_t* colmap;   // two copies of the tile tables (even / odd tiles), shared by the CTA's epilogue warps
-  float* cscale;
   float* stg;        // 32 rows x 16 floats, swizzled
 };
 
@@ -424,9 +423,9 @@ struct EpiCtx {
 // The CTA drains the 128 token rows held by its own tensor memory; the channel groups are split
 // between the two warps of a lane quarter.
 // NKMAX bounds the orders of a branch (2, 4 or 8); the channel block is BN = 8 * nch_max channels.
-// Before the accumulators are ready the warp prepares, from the prefix counts, where each
-// (order, 8-channel chunk) sits in the accumulator and the products s_k * lambda_x of all stacked
-// rows, so that the drain loop has no dependent global loads.
+// Where each (order, 8-channel chunk) sits in the accumulator and the scale of every stacked row come from the
+// block's record in the blob (written by the expansion), which one lane of the CTA fetches with a bulk copy one
+// tile ahead into one of three copies; the epilogue itself does no dependent global load.
 // A lane computes 16 channels of its own token row at a time; the 32 x 16 block is then turned
 // through shared memory so that each store instruction writes 64 contiguous bytes of 8 rows
 // (a lane writing its own row directly would emit 32 separate 16-byte pieces per instruction,
@@ -449,65 +448,37 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   const uint32_t stg_r = smem_u32(x.stg) + static_cast<uint32_t>(sr0 * 64 + spp * 16);
   const bool bias_vec = (reinterpret_cast<uintptr_t>(p.f.bias) & 15) == 0;
   bool stg_busy = false;   // a tensor store of this warp may still be reading the staging block
-  const int et = (x.warp - 2 - kUnpackWarps) * 32 + lane;   // this thread among the epilogue threads
+  const bool rec_issuer = (x.warp == 2 + kUnpackWarps) && lane == 0;   // the lane that fetches the block records
+  // Record of the pair's tile number tc (tile index `tile`) into copy tc % kRecBufs.
+  auto fetch_record = [&](uint32_t tc, int tile) {
+    int m, cb, tt;
+    locate_tile(p, x.tile_base, tile, m, cb, tt);
+    const uint8_t* src = p.f.branch[m].rec + static_cast<size_t>(cb) * kRecBytes;
+    const uint32_t bar = x.recbar0 + 8u * (tc % kRecBufs);
+    mbar_expect_tx(bar, kRecBytes);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     x.rec0 + (tc % kRecBufs) * kRecBytes),
+                 "l"(src), "r"(kRecBytes), "r"(bar)
+                 : "memory");
+  };
+  if (rec_issuer) {
+    if (x.pair < x.num_tiles) fetch_record(0, x.pair);
+    if (x.pair + x.npairs < x.num_tiles) fetch_record(1, x.pair + x.npairs);
+  }
   for (int tile = x.pair; tile < x.num_tiles; tile += x.npairs, ++tcount) {
-    TileMeta t;
-    decode_tile(p, x.tile_base, tile, t);
+    struct { int m, cb, tt, k0; } t;
+    locate_tile(p, x.tile_base, tile, t.m, t.cb, t.tt);
     const BranchArgs& br = p.f.branch[t.m];
+    t.k0 = br.k_begin;
     const int buf = tcount & 1;
     const uint32_t aph = (tcount >> 1) & 1;
-    const float sx = __ldg(br.sx);
-    const int c0 = t.c0, c1 = t.c1;
+    const float sx = x.sx_s[t.m];
+    const uint32_t rec_s = x.rec0 + (tcount % kRecBufs) * kRecBytes;
+    if (!mbar_wait(x.recbar0 + 8u * (tcount % kRecBufs), (tcount / kRecBufs) & 1, x.abort_flag, p.f.status)) break;
+    int c0, c1;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(rec_s));
     const int nch = (c1 - c0) >> 3;       // at most PIPE_BLOCK_CHANNELS / 8
-    const int n_total = t.rowbase[kMaxClusterOrders];
-    // The tables of the tile are built ONCE per CTA, by all epilogue threads together, in the copy of the tile's
-    // parity: a warp that runs ahead into the next tile writes the other copy, and nobody reaches the tile after
-    // that before every warp has passed this tile's barrier, i.e. has finished reading the copy of the tile before.
-    int16_t* colmap = x.colmap + buf * kColmapEntries;
-    float* cscale = x.cscale + buf * kMaxN;
-    const uint32_t colmap_s = smem_u32(colmap), cscale_s = smem_u32(cscale);
-    {
-      // accumulator column of (8-channel chunk, order), or -1: entry [chunk][order]
-      // (entries up to an even chunk count: the drain loads the columns of two chunks at a time, so the chunk
-      // behind an odd count must read as absent)
-      for (int e = et; e < NKMAX * ((nch + 1) & ~1); e += 32 * kEpiWarps) {
-        const int cc = e / NKMAX, ko = e % NKMAX;
-        int col = -1;
-        if (ko < t.nk && cc < nch) {
-          int rb = 0, st = 0;
-          const int32_t* cum = nullptr;
-#pragma unroll
-          for (int u = 0; u < NKMAX; ++u)
-            if (u == ko) {
-              rb = t.rowbase[u];
-              st = t.start[u];
-              cum = p.f.order[t.k0 + u].cum;
-            }
-          const int c = c0 + 8 * cc;
-          const int j = c / p.f.g;
-          const int lo = __ldg(cum + j), hi = __ldg(cum + j + 1);
-          if (hi > lo) col = rb + lo * p.f.g + c % p.f.g - st;
-        }
-        colmap[e] = static_cast<int16_t>(col);
-      }
-      for (int r = et; r < n_total; r += 32 * kEpiWarps) {
-        int rb = 0, st = t.start[0];
-        const float* sc = p.f.order[t.k0].scales;
-#pragma unroll
-        for (int u = 1; u < NKMAX; ++u)
-          if (u < t.nk && r >= t.rowbase[u]) {
-            rb = t.rowbase[u];
-            st = t.start[u];
-            sc = p.f.order[t.k0 + u].scales;
-          }
-        cscale[r] = __fmul_rn(__ldg(sc + st + (r - rb)), sx);
-      }
-      // every epilogue warp has written its share (a bounded wait, like all others: a warp that leaves on an abort
-      // must not leave the rest stuck in a barrier that cannot time out)
-      __syncwarp();
-      if (lane == 0) mbar_arrive(x.tables0 + 8u * buf);
-      if (!mbar_wait(x.tables0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
-    }
+    const uint32_t colmap_s = rec_s + kRecColmapOff, cscale_s = rec_s + kRecScaleOff;
     // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
     // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
     const int ttile = 2 * t.tt + x.rank;
@@ -553,7 +524,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     int8_t* qrow = nullptr;      // this lane's output row at channel c0
     int qalign = 0;              // 16, 4 or 1: widest store every piece of the row allows
     if constexpr (Q8) {
-      ostep = __ldg(br.out_scale);
+      ostep = x.sx_s[PIPE_MAX_ORDERS + t.m];
       ofast = quant_step_is_fast(ostep);
       orcp = ofast ? __frcp_rn(ostep) : 0.f;
       if (!(ostep >= 0.f && ostep < __uint_as_float(0x7f800000u)) && lane == 0) raise_status(p.f.status, PIPE_ERR_INVALID_ARG);
@@ -569,6 +540,9 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     __syncwarp();
     if (!mbar_wait(x.tfull0 + 8u * buf, aph, x.abort_flag, p.f.status)) break;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // The record of the NEXT tile goes into the copy the tile before the last one used: the accumulators just handed
+    // over were computed after every epilogue warp of the pair had finished that tile.
+    if (rec_issuer && tcount >= 1 && tile + x.npairs < x.num_tiles) fetch_record(tcount + 1, tile + x.npairs);
     const uint32_t tbase = x.tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * kAccCols;
     for (int grp = x.part; grp < ngrp && tile_ok; grp += x.nparts) {
       // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
@@ -585,23 +559,21 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       for (int sub = 0; sub < 2; sub += CH) {
         int acc[CH][NKMAX][8];
         int cols[CH][NKMAX];
-        {
-          // CH * NKMAX int16 entries, contiguous
-          constexpr int W = CH * NKMAX / 2;   // 32-bit words: 2, 2 or 4
+#pragma unroll
+        for (int u = 0; u < CH; ++u) {
+          // the chunk's eight int16 entries (one per order of a cluster), of which the first NKMAX can be present
+          constexpr int W = NKMAX / 2;   // 32-bit words: 1, 2 or 4
           uint32_t cw[W];
-          const uint32_t addr = colmap_s + static_cast<uint32_t>((2 * grp + sub) * NKMAX * 2);
-          if constexpr (W == 2) {
+          const uint32_t addr = colmap_s + static_cast<uint32_t>((2 * grp + sub + u) * 16);
+          if constexpr (W == 1) {
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(cw[0]) : "r"(addr));
+          } else if constexpr (W == 2) {
             asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(cw[0]), "=r"(cw[1]) : "r"(addr));
           } else {
             asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(cw[0]), "=r"(cw[1]), "=r"(cw[2]), "=r"(cw[3]) : "r"(addr));
           }
 #pragma unroll
-          for (int u = 0; u < CH; ++u)
-#pragma unroll
-            for (int ko = 0; ko < NKMAX; ++ko) {
-              const int idx = u * NKMAX + ko;
-              cols[u][ko] = static_cast<int16_t>((cw[idx >> 1] >> (16 * (idx & 1))) & 0xffffu);
-            }
+          for (int ko = 0; ko < NKMAX; ++ko) cols[u][ko] = static_cast<int16_t>((cw[ko >> 1] >> (16 * (ko & 1))) & 0xffffu);
         }
 #pragma unroll
         for (int u = 0; u < CH; ++u)
@@ -627,10 +599,13 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
             for (int e = 0; e < 8; ++e) {
               const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
               acc[u][ko][e] = a;
-              y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+              y[e] = __fmaf_rn(__int2float_rn(a), __fmul_rn(cs[e], sx), y[e]);   // c = s_k * lambda_x first
             }
             if (PARTIALS && own_ok) {
-              const int crow = cols[u][ko] - t.rowbase[ko] + t.start[ko];   // compacted row of the chunk's first channel
+              int rb_ko, st_ko;   // the order's first row in the stacked block and in its own compacted rows
+              asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rb_ko) : "r"(rec_s + 4u * (kRecRowbase + ko)));
+              asm volatile("ld.shared.u32 %0, [%1];" : "=r"(st_ko) : "r"(rec_s + 4u * (kRecStart + ko)));
+              const int crow = cols[u][ko] - rb_ko + st_ko;   // compacted row of the chunk's first channel
               int32_t* prow = p.f.partials + tok_own * p.f.total_rows + p.f.order[t.k0 + ko].row_off + crow;
 #pragma unroll
               for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
@@ -762,13 +737,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
   __shared__ uint64_t pk_bars[kMaxRing * kSub];   // "packed rows have landed", one per block slot of the ring
-  __shared__ uint64_t tbl_bars[2];                // "tile tables complete", even / odd tile
+  __shared__ uint64_t rec_bars[kRecBufs];         // "block record landed", one per copy
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_base_s[PIPE_MAX_ORDERS + 1];   // tiles before each branch, then the total
   __shared__ int ntot_s[kTileRing];
-  __shared__ __align__(16) int16_t epi_colmap[2][kColmapEntries];   // even / odd tile: accumulator column of (8-channel chunk, order) or -1
-  __shared__ __align__(16) float epi_cscale[2][kMaxN];             // even / odd tile: s_k * lambda_x of every stacked row
+  __shared__ __align__(16) uint8_t tile_recs[kRecBufs][kRecBytes];   // block records of the tiles in the epilogue's hands
+  __shared__ float sx_s[2 * PIPE_MAX_ORDERS];                        // lambda_x of every branch, then the fused epilogue's output steps
   __shared__ __align__(1024) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels (the
                                                                     // source of tensor stores with the 64-byte swizzle)
 
@@ -790,6 +765,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   g.abort_flag = &abort_flag_s;
   g.ntot = ntot_s;
 
+  if (threadIdx.x >= 32 && threadIdx.x < 32 + 2 * PIPE_MAX_ORDERS) {
+    // (inputs of this launch: written before it started)
+    const int i = threadIdx.x - 32, m = i % PIPE_MAX_ORDERS;
+    float v = 0.f;
+    if (m < p.f.num_branches) {
+      if (i < PIPE_MAX_ORDERS) v = __ldg(p.f.branch[m].sx);
+      else if (Q8) v = __ldg(p.f.branch[m].out_scale);
+    }
+    sx_s[i] = v;
+  }
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     int acc = 0;
@@ -807,7 +792,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       mbar_init(g.done0 + 8u * s, 1);
     }
     for (int s = 0; s < kMaxRing * kSub; ++s) mbar_init(smem_u32(&pk_bars[s]), 1);
-    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&tbl_bars[b]), kEpiWarps);
+    for (int b = 0; b < kRecBufs; ++b) mbar_init(smem_u32(&rec_bars[b]), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
       mbar_init(g.tempty0 + 8u * b, 2 * kEpiWarps);
@@ -922,7 +907,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.tmem_base = tmem_base;
     e.tfull0 = g.tfull0;
     e.tempty0 = g.tempty0;
-    e.tables0 = smem_u32(tbl_bars);
+    e.recbar0 = smem_u32(rec_bars);
+    e.rec0 = smem_u32(tile_recs);
+    e.sx_s = sx_s;
     e.tempty_lead0 = g.tempty_lead0;
     e.rank = g.rank;
     e.pair = g.pair;
@@ -935,8 +922,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     const int ew = warp - 2 - kUnpackWarps;
     e.part = ew >> 2;
     e.nparts = kEpiWarps / 4;
-    e.colmap = &epi_colmap[0][0];
-    e.cscale = &epi_cscale[0][0];
     e.stg = epi_stage[ew];
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
       if (p.nkmax <= 2) epilogue_role<2, true, Q8>(p, e);
@@ -1031,7 +1016,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (max_cluster > kMaxClusterOrders) return PIPE_ERR_UNSUPPORTED;
   // every branch needs the channel-block table of its cluster of orders (written by the expansion)
   for (int m = 0; m < a.num_branches; ++m)
-    if (!a.branch[m].blk) return PIPE_ERR_UNSUPPORTED;
+    if (!a.branch[m].blk || !a.branch[m].rec) return PIPE_ERR_UNSUPPORTED;
   if (a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;

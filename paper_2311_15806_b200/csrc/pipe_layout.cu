@@ -115,10 +115,17 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     const int nk = (m < L.M) ? bo[m] : L.K;
     y.blk_off[m] = 0;
     y.blk_cap[m] = 0;
+    y.rec_off[m] = 0;
+    y.rec_cap[m] = 0;
     if (nk > 8 || static_cast<int64_t>(nk) * L.g > PIPE_BLOCK_ROWS) continue;
     y.blk_cap[m] = L.G;   // a block holds at least one group
     y.blk_off[m] = off;
     off = align_up64(off + static_cast<uint64_t>(y.blk_cap[m] + 2) * 4, 256);
+    int64_t R = 0;
+    for (int k = (m < L.M ? L.branch_begin[m] : 0); k < (m < L.M ? L.branch_begin[m + 1] : L.K); ++k) R += y.rows[k];
+    y.rec_cap[m] = block_count_bound(R, L.O, L.G, nk, L.g);
+    y.rec_off[m] = off;
+    off = align_up64(off + static_cast<uint64_t>(y.rec_cap[m]) * kRecBytes, 256);
   }
   // decode-unit tables: the clusters that run together share the SMs.  For c CTAs per unit the sets get units in
   // proportion to their rows; a unit's rows (rounded to the MMA's granularity, plus one group of every order of slack)

@@ -111,6 +111,44 @@ def expected_block_table(kept_lists, G: int, g: int, row_max: int = 256, channel
     return np.array([len(bounds) - 1] + bounds, np.int32)
 
 
+def expected_block_records(kept_lists, scale_lists, table, g):
+    """The block records (pipe.h) of a channel-block table, from the definition: kept groups and scales of the cluster's
+    orders (the ORACLE's), the table's boundaries."""
+    n = int(table[0])
+    nk = len(kept_lists)
+    G = int(table[1 + n])
+    # compacted row of every channel in every order, or -1
+    crow = np.full((nk, G * g), -1, np.int64)
+    for q, kept in enumerate(kept_lists):
+        for i, j in enumerate(np.asarray(kept)):
+            crow[q, j * g:(j + 1) * g] = i * g + np.arange(g)
+    recs = np.zeros((n, B.BLOCK_RECORD_BYTES), np.uint8)
+    for cb in range(n):
+        j0, j1 = int(table[1 + cb]), int(table[2 + cb])
+        c0, c1 = j0 * g, j1 * g
+        hdr = np.zeros(32, np.int32)
+        colmap = np.full(512, -1, np.int16)
+        scale = np.zeros(256, np.float32)
+        rb = 0
+        for q in range(8):
+            hdr[8 + q] = rb
+            if q < nk:
+                rows = crow[q, c0:c1]
+                rows = rows[rows >= 0]
+                hdr[16 + q] = int(np.sum(np.asarray(kept_lists[q]) < j0)) * g
+                scale[rb:rb + len(rows)] = np.asarray(scale_lists[q])[rows]
+                for cc in range((c1 - c0) // 8):
+                    r = crow[q, c0 + 8 * cc]
+                    if r >= 0:
+                        colmap[8 * cc + q] = rb + r - hdr[16 + q]
+                rb += len(rows)
+        hdr[0], hdr[1], hdr[2], hdr[3] = c0, c1, nk, rb
+        recs[cb, :128] = hdr.view(np.uint8)
+        recs[cb, 128:128 + 1024] = colmap.view(np.uint8)
+        recs[cb, 128 + 1024:] = scale.view(np.uint8)
+    return recs
+
+
 def assert_block_tables_match(layer: B.ExpandedLayer, e):
     """Every channel-block table of the blob against the definition evaluated on the ORACLE's kept lists."""
     lay = layer.layout
@@ -127,6 +165,10 @@ def assert_block_tables_match(layer: B.ExpandedLayer, e):
         got = table.cpu().numpy()
         assert want[0] <= lay.blk_cap[m]
         np.testing.assert_array_equal(got[:len(want)], want, err_msg=f"channel-block table {m}")
+        assert want[0] <= lay.rec_cap[m]
+        recs = layer.block_records(m).cpu().numpy()
+        want_recs = expected_block_records([e.order_kept(k) for k in range(k0, k1)], [e.order_scales(k) for k in range(k0, k1)], want, e.g)
+        np.testing.assert_array_equal(recs[:len(want_recs)], want_recs, err_msg=f"block records of table {m}")
         dtable = layer.decode_table(m)
         if dtable is not None:
             assert 16 <= lay.dec_limit[m] <= 256
