@@ -184,6 +184,11 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   const int s0 = my_branch * p.slabs_per_branch + cib * base + min(cib, rem);
   const int cnt = base + (cib < rem ? 1 : 0);
 
+  // A launch of this kernel that follows in the stream may be brought onto the SMs as they become free: its CTAs
+  // then exist, with their barriers set up, when this launch's last CTA ends, instead of being launched only then
+  // (a chain of small-token layers otherwise pays a launch gap per layer).  They wait below, before their first
+  // access to global memory, until this launch is complete.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < depth; ++s) {
@@ -197,6 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   // passes: pieces of at most pass_slabs slabs of the CTA's range (which lies in one branch)
   const int npass = min((cnt + p.pass_slabs - 1) / p.pass_slabs, kMaxPasses);
   for (int e = threadIdx.x; e < p.pass_slabs * NP * NT * 4 * 32; e += kThreads) sums[e] = 0;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // ---- which orders keep each own slab, and where its 8 rows start
   for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
     const int li = e / p.nkmax, ko = e % p.nkmax;
@@ -651,7 +657,18 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
                                static_cast<uint64_t>(a.ldxq), 128, 16, true))
       return PIPE_ERR_CUDA;
   if (!kernel_info(kern, dyn, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
-  kern<<<grid, kThreads, dyn, stream>>>(p);
+  // (programmatic stream serialization: see the kernel's first lines)
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = dyn;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return PIPE_ERR_CUDA;
   count_launch(1);
   return launch_status();
 }

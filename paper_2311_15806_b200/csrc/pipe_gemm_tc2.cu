@@ -408,6 +408,8 @@ struct EpiCtx {
   uint32_t tmem_base, tfull0, tempty0;
   uint32_t recbar0;   // kRecBufs barriers: the block record of the tile has landed
   uint32_t rec0;      // shared address of the first record copy
+  uint32_t prebar0;   // kRecBufs barriers: the scale products of the tile are complete
+  float* cfold;       // [kRecBufs][kMaxN]: s_k * lambda_x of every stacked row of the tile
   const float* sx_s;  // shared memory: lambda_x of every branch (and, behind them, the output steps of the fused epilogue)
   volatile int* abort_flag;
   int warp, lane;
@@ -478,7 +480,25 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
     int c0, c1;
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(rec_s));
     const int nch = (c1 - c0) >> 3;       // at most PIPE_BLOCK_CHANNELS / 8
-    const uint32_t colmap_s = rec_s + kRecColmapOff, cscale_s = rec_s + kRecScaleOff;
+    const uint32_t colmap_s = rec_s + kRecColmapOff;
+    // The products c = s_k * lambda_x of the tile's stacked rows, once per CTA instead of once per token row.
+    float* cf = x.cfold + (tcount % kRecBufs) * kMaxN;
+    {
+      const int et = (x.warp - 2 - kUnpackWarps) * 32 + lane;   // this thread among the epilogue threads
+      for (int r = et; r < kMaxN; r += 32 * kEpiWarps) {
+        float sc;
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(sc) : "r"(rec_s + kRecScaleOff + 4u * r));
+        cf[r] = __fmul_rn(sc, sx);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(x.prebar0 + 8u * (tcount % kRecBufs));
+      if (!mbar_wait(x.prebar0 + 8u * (tcount % kRecBufs), (tcount / kRecBufs) & 1, x.abort_flag, p.f.status)) break;
+    }
+    const uint32_t cscale_s = smem_u32(cf);
+    // The accumulators hold 2^(8-b) times the sums; float(2^(8-b) a) = 2^(8-b) float(a) exactly, so the shift is
+    // taken as a multiplication by 2^-(8-b) after the conversion (exact for every int32, and on the pipe with the
+    // most issue slots); only the verification output needs the shifted integers themselves.
+    const float unshift = __int_as_float((127 - p.shift) << 23);
     // Token of row r (0..31) of this warp: tok_base + r for a matrix of tokens; for the implicit
     // convolution the warp holds half of an 8 x 8 pixel patch (4 image rows of 8 pixels).
     const int ttile = 2 * t.tt + x.rank;
@@ -548,7 +568,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       // bias of this lane's channel quad: needed in the store phase only, so its latency is hidden
       const bool quad_ok = 2 * grp + (sj >> 1) < nch;
       float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (!Q8 && add_bias && quad_ok) {
+      if (!Q8 && add_bias && quad_ok && !(tma_out && 2 * grp + 1 < nch)) {
         const float* bp = bias_q + 16 * grp;
         bq = make_float4(__ldg(bp), __ldg(bp + 1), __ldg(bp + 2), __ldg(bp + 3));
       }
@@ -595,11 +615,16 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
             const uint32_t ca = cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[0]), "=f"(cs[1]), "=f"(cs[2]), "=f"(cs[3]) : "r"(ca));
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[4]), "=f"(cs[5]), "=f"(cs[6]), "=f"(cs[7]) : "r"(ca + 16));
+            if constexpr (PARTIALS) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
-              acc[u][ko][e] = a;
-              y[e] = __fmaf_rn(__int2float_rn(a), __fmul_rn(cs[e], sx), y[e]);   // c = s_k * lambda_x first
+              for (int e = 0; e < 8; ++e) {
+                const int a = acc[u][ko][e] >> p.shift;  // exact: the accumulator holds 2^shift times the sum
+                acc[u][ko][e] = a;
+                y[e] = __fmaf_rn(__int2float_rn(a), cs[e], y[e]);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) y[e] = __fmaf_rn(__fmul_rn(__int2float_rn(acc[u][ko][e]), unshift), cs[e], y[e]);
             }
             if (PARTIALS && own_ok) {
               int rb_ko, st_ko;   // the order's first row in the stacked block and in its own compacted rows
@@ -743,6 +768,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   __shared__ int tile_base_s[PIPE_MAX_ORDERS + 1];   // tiles before each branch, then the total
   __shared__ int ntot_s[kTileRing];
   __shared__ __align__(16) uint8_t tile_recs[kRecBufs][kRecBytes];   // block records of the tiles in the epilogue's hands
+  __shared__ __align__(16) float cfold_s[kRecBufs][kMaxN];            // s_k * lambda_x of the stacked rows of those tiles
+  __shared__ uint64_t pre_bars[kRecBufs];
   __shared__ float sx_s[2 * PIPE_MAX_ORDERS];                        // lambda_x of every branch, then the fused epilogue's output steps
   __shared__ __align__(1024) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels (the
                                                                     // source of tensor stores with the 64-byte swizzle)
@@ -765,6 +792,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   g.abort_flag = &abort_flag_s;
   g.ntot = ntot_s;
 
+  // A launch of this kernel that follows in the stream may be brought onto the SMs as they become free (its CTAs then
+  // exist when this launch's last pair ends); it waits here, before its first access to global memory, until the
+  // launch before it is complete.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x >= 32 && threadIdx.x < 32 + 2 * PIPE_MAX_ORDERS) {
     // (inputs of this launch: written before it started)
     const int i = threadIdx.x - 32, m = i % PIPE_MAX_ORDERS;
@@ -792,7 +824,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
       mbar_init(g.done0 + 8u * s, 1);
     }
     for (int s = 0; s < kMaxRing * kSub; ++s) mbar_init(smem_u32(&pk_bars[s]), 1);
-    for (int b = 0; b < kRecBufs; ++b) mbar_init(smem_u32(&rec_bars[b]), 1);
+    for (int b = 0; b < kRecBufs; ++b) {
+      mbar_init(smem_u32(&rec_bars[b]), 1);
+      mbar_init(smem_u32(&pre_bars[b]), kEpiWarps);
+    }
     for (int b = 0; b < 2; ++b) {
       mbar_init(g.tfull0 + 8u * b, 1);
       mbar_init(g.tempty0 + 8u * b, 2 * kEpiWarps);
@@ -909,6 +944,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.tempty0 = g.tempty0;
     e.recbar0 = smem_u32(rec_bars);
     e.rec0 = smem_u32(tile_recs);
+    e.prebar0 = smem_u32(pre_bars);
+    e.cfold = &cfold_s[0][0];
     e.sx_s = sx_s;
     e.tempty_lead0 = g.tempty_lead0;
     e.rank = g.rank;
@@ -1055,6 +1092,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   }
   p.pk = kKStep * a.bits / 8;
   p.shift = 8 - a.bits;
+
   int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
   for (int m = 0; m < a.num_branches; ++m) {
     k_lo = min(k_lo, a.branch[m].k_begin);
@@ -1092,17 +1130,19 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   }
   // one cluster of two CTAs per SM pair; the tiles (counted on the device) go round all resident pairs
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see the kernel's first lines
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.gridDim = dim3(2 * ds.max_pairs, 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = ds.dyn_smem;
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t e = a.q8_out ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true>, p) : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false>, p);
   if (e != cudaSuccess) return PIPE_ERR_CUDA;
   count_launch(1);
