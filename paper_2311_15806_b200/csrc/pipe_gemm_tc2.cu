@@ -364,16 +364,25 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
           return;
         }
         pk_phase ^= 1u;
-        uint4 w[ITEMS];
+        // Two passes over half of the items each, as a loop (half the registers and half the code of one pass over
+        // all of them: the instruction footprint of the warps that share an SM partition is what the inner loops
+        // of this kernel are most sensitive to).  The widened rows of the first half lie in the part of the slot
+        // that holds no packed bytes; those of the second half cover the packed rows of both, all of which are in
+        // registers (or used up) once every lane has loaded its share of the second half.
         const uint4* pk_in = reinterpret_cast<const uint4*>(bt + kPackedOff) + lane;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+        constexpr int HI = ITEMS / 2;
+        const int ibase = half * HI;
+        uint4 w[HI];
 #pragma unroll
-        for (int i = 0; i < ITEMS; ++i)
-          if (i < n_items) w[i] = pk_in[i * 32];
+        for (int i = 0; i < HI; ++i)
+          if (ibase + i < n_items) w[i] = pk_in[(ibase + i) * 32];
         __syncwarp();   // every lane holds its packed chunks before any lane overwrites them
 #pragma unroll
-        for (int i = 0; i < ITEMS; ++i) {
-          if (i >= n_items) continue;
-          uint8_t* row = bt + i * (RPI >> 3) * 1024 + out_lane;   // rows i * RPI + lr (RPI is 8 or 16)
+        for (int i = 0; i < HI; ++i) {
+          if (ibase + i >= n_items) continue;
+          uint8_t* row = bt + (ibase + i) * (RPI >> 3) * 1024 + out_lane;   // rows (ibase + i) * RPI + lr (RPI is 8 or 16)
           const int c0 = lc * OUT_PER_CHUNK;
           if (BITS == 4) {
             const uint32_t m4 = 0xF0F0F0F0u;
@@ -390,6 +399,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
               *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
             }
           }
+        }
         }
       }
     }
