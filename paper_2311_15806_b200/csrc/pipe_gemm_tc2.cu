@@ -1084,7 +1084,8 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
     p.conv_chunks = a.cC / kKStep;
     p.ntok_tiles = ceil_div(p.conv_np, 2);
   }
-  if (p.ntok_tiles < 2) return PIPE_ERR_UNSUPPORTED;   // a pair needs two token tiles; the one-SM kernel takes these
+  // (a single token tile: the second CTA of a pair then stages zeros and stores nothing, but still unpacks its half of
+  // every block, which is what such a launch spends its time on)
   p.ntt = ceil_div(p.ntok_tiles, 2);
   // the tile count is known on the device only (block counts of the tables); a table never has more blocks than groups
   if (static_cast<int64_t>(a.G) * p.ntt * a.num_branches > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
