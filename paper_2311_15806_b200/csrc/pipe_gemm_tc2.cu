@@ -343,16 +343,18 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
         }
       }
     } else {
+      // everything the copies need is prepared before the wait for the slot: what follows the wait is on the
+      // critical path of the ring (the barrier of the packed rows belongs to this warp alone, so its byte count can
+      // be posted while the slot is still being read)
+      const uint32_t bar = pkbar + 8u * (slot * kSub + sub);
+      const uint8_t* src = p.kbase + (static_cast<size_t>(run_off + static_cast<uint32_t>(kbs) * run_stp) << 4);
+      const uint32_t dst = g.stage0 + bt_off + kPackedOff + run_dst;
+      if (real && lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(mine) * PK);
       if (!mbar_wait(g.done0 + 8u * slot, (use & 1) ^ 1, g.abort_flag, p.f.status)) return;
       if (real) {
-        const uint32_t bar = pkbar + 8u * (slot * kSub + sub);
-        if (lane == 0) mbar_expect_tx(bar, static_cast<uint32_t>(mine) * PK);
-        __syncwarp();
         if (run_bytes != 0) {
-          const uint8_t* src = p.kbase + (static_cast<size_t>(run_off + static_cast<uint32_t>(kbs) * run_stp) << 4);
-          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                           g.stage0 + bt_off + kPackedOff + run_dst),
-                       "l"(src), "r"(run_bytes), "r"(bar)
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                       "r"(run_bytes), "r"(bar)
                        : "memory");
         }
         __syncwarp();
@@ -883,6 +885,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
         const int ttile = 2 * tt + g.rank;   // this CTA's 128 token rows of the pair's tile
         const int nsub = min(kSub, p.kblocks - ks * kSub);   // the last stage of a tile may hold one block only
         const int kb = ks * kSub + sub;
+        // (the byte count of the stage barrier must NOT be posted ahead of this wait: the producer runs up to a ring
+        // ahead of the MMAs, so the barrier's phase of the slot's use before may still be collecting its arrivals,
+        // and an early arrival would be counted into that phase)
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
         if (g.rank == 0 && lane == 0) mbar_expect_tx(g.full0 + 8u * rp.slot, 2 * nsub * kABytes);
         if (sub >= nsub) continue;
