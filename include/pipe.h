@@ -430,6 +430,28 @@ pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv
                                     const float* d_out_scale, int8_t* d_yq, int64_t ldyq, int32_t* d_partials,
                                     void* stream);
 
+/*
+ * Sec. 3.2 (Fig. 2) for a convolution: predictor m applies its own cluster of orders (pipe_default_branches, or
+ * desc->branch_orders) to its own NHWC input h_xq_m[m] with step *h_sx_m[m]; everything else as in
+ * pipe_expanded_conv2d (geometry, layouts, alignment) and pipe_ensemble_forward (bias with predictor 0 only;
+ * sum_branches != 0: the predictors' outputs are added in ascending m into h_y_m[0], each by the thread that wrote it;
+ * otherwise predictor m writes h_y_m[m]; d_partials covers all K orders, each from its own predictor's input).
+ * h_* are host arrays of num_branches device pointers.  One grouped launch unless sum_branches is set.
+ */
+pipe_status pipe_ensemble_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                 const int8_t* const* h_xq_m, const float* const* h_sx_m, const float* d_bias,
+                                 float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials, void* stream);
+
+/*
+ * The same as an inner layer of the M predictors (pipe_ensemble_forward_q8 on convolutions): predictor m hands
+ * Q(sigma(y_m)) with the static step *h_out_scale_m[m] to h_yq_m[m], int8 [N*Ho*Wo, O] pitch ldyq -- with ldyq = O the
+ * NHWC input of predictor m's next convolution.  `relu` is the activation kind (PIPE_ACT_*).
+ */
+pipe_status pipe_ensemble_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                    const int8_t* const* h_xq_m, const float* const* h_sx_m, const float* d_bias,
+                                    int32_t relu, const float* const* h_out_scale_m, int8_t* const* h_yq_m, int64_t ldyq,
+                                    int32_t* d_partials, void* stream);
+
 /* Number of kernels the library has launched in this process (all calls, all streams). */
 uint64_t pipe_launch_count(void);
 

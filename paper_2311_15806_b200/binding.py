@@ -35,7 +35,7 @@ EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout"
            "pipe_bound_network", "pipe_bound_step_dense", "pipe_bound_step_rows", "pipe_spectral_norm", "pipe_choose_expansion",
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_quantize_act_ex", "pipe_ensemble_forward_zp", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
-           "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8",
+           "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8", "pipe_ensemble_conv2d", "pipe_ensemble_conv2d_q8",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string",
            # include/pipe_diag.h: tests and measurements only
            "pipe_diag_select_kernel", "pipe_diag_mma_i8_rate", "pipe_diag_bounded_wait"]
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.pipe_ensemble_forward.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, p, i64, i32, p, p]
         L.pipe_ensemble_forward_q8.argtypes = [C.POINTER(LayerDesc), p, p, i64, i64, p, p, i32, p, p, i64, p, p]
         L.pipe_expanded_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
+        L.pipe_ensemble_conv2d.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, p, i64, i32, p, p]
+        L.pipe_ensemble_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
         L.pipe_diag_select_kernel.argtypes = [i32]
         L.pipe_diag_mma_i8_rate.argtypes = [i32, i64, i32, C.POINTER(C.c_double), p]
         L.pipe_diag_bounded_wait.argtypes = [i64, p]
@@ -336,6 +338,36 @@ def pipe_expanded_conv2d_q8(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor,
     _check(lib().pipe_expanded_conv2d_q8(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias),
                                          int(relu), _dp(out_scale), _dp(yq), yq.stride(0), _dp(partials),
                                          _stream_ptr(stream)), "pipe_expanded_conv2d_q8")
+
+
+def pipe_ensemble_conv2d(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,
+                         sum_branches: bool = False, partials: torch.Tensor | None = None, stream=None) -> None:
+    """xq_m: M cuda int8 [N, H, W, C] contiguous tensors; y_m: M (or, summed, one) cuda float32 [N*Ho*Wo, O] tensors."""
+    M = desc.num_branches
+    assert len(xq_m) == M and len(sx_m) == M and len(y_m) >= (1 if sum_branches else M)
+    assert all(t.is_contiguous() and t.dtype == torch.int8 for t in xq_m)
+    PA = C.c_void_p * M
+    xp = PA(*[_dp(t) for t in xq_m])
+    sp = PA(*[_dp(t) for t in sx_m])
+    yp = PA(*[(_dp(y_m[m]) if m < len(y_m) else None) for m in range(M)])
+    _check(lib().pipe_ensemble_conv2d(C.byref(desc), C.byref(geom), _dp(blob), xp, sp, _dp(bias), yp, y_m[0].stride(0),
+                                      1 if sum_branches else 0, _dp(partials), _stream_ptr(stream)), "pipe_ensemble_conv2d")
+
+
+def pipe_ensemble_conv2d_q8(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_m, sx_m, out_scale_m, yq_m,
+                            bias: torch.Tensor | None = None, relu: bool = True, partials: torch.Tensor | None = None,
+                            stream=None) -> None:
+    """Inner convolution of the M predictors: yq_m[m] (cuda int8 [N*Ho*Wo, O]) receives Q(sigma(y_m))."""
+    M = desc.num_branches
+    assert len(xq_m) == M and len(sx_m) == M and len(out_scale_m) == M and len(yq_m) == M
+    assert all(t.is_contiguous() and t.dtype == torch.int8 for t in xq_m) and all(t.dtype == torch.int8 for t in yq_m)
+    PA = C.c_void_p * M
+    xp = PA(*[_dp(t) for t in xq_m])
+    sp = PA(*[_dp(t) for t in sx_m])
+    op = PA(*[_dp(t) for t in out_scale_m])
+    yp = PA(*[_dp(t) for t in yq_m])
+    _check(lib().pipe_ensemble_conv2d_q8(C.byref(desc), C.byref(geom), _dp(blob), xp, sp, _dp(bias), int(relu), op, yp,
+                                         yq_m[0].stride(0), _dp(partials), _stream_ptr(stream)), "pipe_ensemble_conv2d_q8")
 
 
 def pipe_ensemble_forward(desc: LayerDesc, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,

@@ -165,16 +165,19 @@ extern "C" pipe_status pipe_ensemble_forward_q8(const pipe_layer_desc* desc, con
                      static_cast<cudaStream_t>(stream), h_yq_m, h_out_scale_m, ldyq, relu);
 }
 
-// Both convolution entries: d_yq != nullptr selects the fused inner-layer epilogue (d_y, ldy unused then).
-static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob, const int8_t* d_xq,
-                            const float* d_sx, const float* d_bias, float* d_y, int64_t ldy, int8_t* d_yq,
-                            const float* d_out_scale, int64_t ldyq, int relu, int32_t* d_partials, void* stream) {
-  const bool q8 = d_yq != nullptr;
+// All convolution entries.  M inputs with their clusters of orders [k_begin[m], k_end[m]) (one input with all K orders
+// for pipe_expanded_conv2d); yq != nullptr selects the fused inner-layer epilogue (y, ldy unused then).
+static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob, int M, bool all_orders,
+                            const int8_t* const* xq, const float* const* sx, const float* d_bias, float* const* y,
+                            int64_t ldy, int sum_branches, int8_t* const* yq, const float* const* out_scale, int64_t ldyq,
+                            int relu, int32_t* d_partials, void* stream) {
+  const bool q8 = yq != nullptr;
   if (relu < 0 || relu > 4) return PIPE_ERR_INVALID_ARG;
   LayerInfo L;
   pipe_status st = resolve_layer(desc, &L);
   if (st != PIPE_OK) return st;
-  if (!geom || !d_blob || !d_xq || !d_sx || (!q8 && !d_y) || (q8 && !d_out_scale)) return PIPE_ERR_INVALID_ARG;
+  if (!all_orders) M = L.M;
+  if (!geom || !d_blob || !xq || !sx || (!q8 && !y) || (q8 && (!out_scale || sum_branches))) return PIPE_ERR_INVALID_ARG;
   if (geom->batch < 1 || geom->height < 1 || geom->width < 1 || geom->channels < 1 || geom->kernel_h < 1 ||
       geom->kernel_w < 1)
     return PIPE_ERR_INVALID_ARG;
@@ -186,31 +189,44 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   const int Wo = (geom->width + 2 * geom->pad_w - geom->kernel_w) / sw + 1;
   if (static_cast<int64_t>(geom->kernel_h) * geom->kernel_w * geom->channels != L.I) return PIPE_ERR_SHAPE;
   if ((q8 ? ldyq : ldy) < L.O) return PIPE_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_xq) & 15) ||
-      (reinterpret_cast<uintptr_t>(d_sx) & 3) || (reinterpret_cast<uintptr_t>(d_y) & 3) ||
-      (reinterpret_cast<uintptr_t>(d_out_scale) & 3) ||
-      (reinterpret_cast<uintptr_t>(d_bias) & 3) || (reinterpret_cast<uintptr_t>(d_partials) & 3))
+  if ((reinterpret_cast<uintptr_t>(d_blob) & (PIPE_BLOB_ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_bias) & 3) ||
+      (reinterpret_cast<uintptr_t>(d_partials) & 3))
     return PIPE_ERR_ALIGNMENT;
+  for (int m = 0; m < M; ++m) {
+    if (!xq[m] || !sx[m]) return PIPE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(xq[m]) & 15) || (reinterpret_cast<uintptr_t>(sx[m]) & 3)) return PIPE_ERR_ALIGNMENT;
+    if (q8) {
+      if (!yq[m] || !out_scale[m]) return PIPE_ERR_INVALID_ARG;
+      if (reinterpret_cast<uintptr_t>(out_scale[m]) & 3) return PIPE_ERR_ALIGNMENT;
+    } else if (m == 0 || !sum_branches) {
+      if (!y[m]) return PIPE_ERR_INVALID_ARG;
+      if (reinterpret_cast<uintptr_t>(y[m]) & 3) return PIPE_ERR_ALIGNMENT;
+    }
+  }
   if (geom->channels % 128 != 0 || sh > 8 || sw > 8) return PIPE_ERR_UNSUPPORTED;
 
   ForwardArgs a;
   for (int k = 0; k < L.K; ++k) a.order[k] = order_view(L, d_blob, k);
-  a.num_branches = 1;
-  BranchArgs& b = a.branch[0];
-  b.xq = d_xq;
-  b.sx = d_sx;
-  b.zp = nullptr;
-  b.y = q8 ? nullptr : d_y;
-  b.k_begin = 0;
-  b.k_end = L.K;
-  b.add_bias = 1;
-  b.accumulate = 0;
-  b.blk = block_table(L, d_blob, L.M);
-  b.rec = L.lay.rec_off[L.M] ? static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[L.M] : nullptr;
-  b.dec = nullptr;
+  a.num_branches = M;
+  for (int m = 0; m < M; ++m) {
+    BranchArgs& b = a.branch[m];
+    b.xq = xq[m];
+    b.sx = sx[m];
+    b.zp = nullptr;
+    b.y = q8 ? nullptr : (sum_branches ? y[0] : y[m]);
+    b.k_begin = all_orders ? 0 : L.branch_begin[m];
+    b.k_end = all_orders ? L.K : L.branch_begin[m + 1];
+    b.add_bias = (m == 0);
+    b.accumulate = (sum_branches && m > 0);
+    // one input running all K orders is the "all orders" cluster (entry L.M), otherwise predictor m's own
+    const int set = (b.k_end - b.k_begin == L.K) ? L.M : m;
+    b.blk = block_table(L, d_blob, set);
+    b.rec = L.lay.rec_off[set] ? static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[set] : nullptr;
+    b.dec = nullptr;
+    b.yq = q8 ? yq[m] : nullptr;
+    b.out_scale = q8 ? out_scale[m] : nullptr;
+  }
   a.decode_split = 0;
-  b.yq = d_yq;
-  b.out_scale = d_out_scale;
   a.q8_out = q8 ? 1 : 0;
   a.relu = relu;
   a.ldyq = ldyq;
@@ -240,13 +256,32 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
 extern "C" pipe_status pipe_expanded_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
                                             const int8_t* d_xq, const float* d_sx, const float* d_bias, float* d_y,
                                             int64_t ldy, int32_t* d_partials, void* stream) {
-  return run_conv(desc, geom, d_blob, d_xq, d_sx, d_bias, d_y, ldy, nullptr, nullptr, 0, 0, d_partials, stream);
+  if (!d_xq || !d_sx || !d_y) return PIPE_ERR_INVALID_ARG;
+  return run_conv(desc, geom, d_blob, 1, true, &d_xq, &d_sx, d_bias, &d_y, ldy, 0, nullptr, nullptr, 0, 0, d_partials, stream);
 }
 
 extern "C" pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
                                                const int8_t* d_xq, const float* d_sx, const float* d_bias, int32_t relu,
                                                const float* d_out_scale, int8_t* d_yq, int64_t ldyq, int32_t* d_partials,
                                                void* stream) {
-  if (!d_yq) return PIPE_ERR_INVALID_ARG;
-  return run_conv(desc, geom, d_blob, d_xq, d_sx, d_bias, nullptr, 0, d_yq, d_out_scale, ldyq, relu, d_partials, stream);
+  if (!d_xq || !d_sx || !d_yq || !d_out_scale) return PIPE_ERR_INVALID_ARG;
+  return run_conv(desc, geom, d_blob, 1, true, &d_xq, &d_sx, d_bias, nullptr, 0, 0, &d_yq, &d_out_scale, ldyq, relu, d_partials, stream);
+}
+
+extern "C" pipe_status pipe_ensemble_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                            const int8_t* const* h_xq_m, const float* const* h_sx_m, const float* d_bias,
+                                            float* const* h_y_m, int64_t ldy, int32_t sum_branches, int32_t* d_partials,
+                                            void* stream) {
+  if (!h_xq_m || !h_sx_m || !h_y_m) return PIPE_ERR_INVALID_ARG;
+  return run_conv(desc, geom, d_blob, 0, false, h_xq_m, h_sx_m, d_bias, h_y_m, ldy, sum_branches ? 1 : 0, nullptr, nullptr, 0, 0,
+                  d_partials, stream);
+}
+
+extern "C" pipe_status pipe_ensemble_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
+                                               const int8_t* const* h_xq_m, const float* const* h_sx_m, const float* d_bias,
+                                               int32_t relu, const float* const* h_out_scale_m, int8_t* const* h_yq_m,
+                                               int64_t ldyq, int32_t* d_partials, void* stream) {
+  if (!h_xq_m || !h_sx_m || !h_out_scale_m || !h_yq_m) return PIPE_ERR_INVALID_ARG;
+  return run_conv(desc, geom, d_blob, 0, false, h_xq_m, h_sx_m, d_bias, nullptr, 0, 0, h_yq_m, h_out_scale_m, ldyq, relu, d_partials,
+                  stream);
 }

@@ -902,7 +902,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
           const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
           int n, h0, w0;
           patch_origin(p, 2 * ttile + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-          tma_pair_load_4d(dst + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh, n, bar);
+          tma_pair_load_4d(dst + half * (kABytes / 2), &p.tmap_a[m], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh, n, bar);
         }
       }
     }
@@ -1072,7 +1072,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
-  if (a.conv_on && (a.cC % kKStep != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
+  if (a.conv_on && a.cC % kKStep != 0) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
     if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   }
@@ -1126,7 +1126,8 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   p.depth = ds.depth;
 
   if (a.conv_on) {
-    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
+    for (int m = 0; m < a.num_branches; ++m)
+      if (!make_map_nhwc(&p.tmap_a[m], a.branch[m].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
   } else
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),

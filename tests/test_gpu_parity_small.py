@@ -397,3 +397,103 @@ def test_forward_is_deterministic_across_repeated_runs(oracle):
         for o in outs[1:]:
             for a, b in zip(o, outs[0]):
                 np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def _lower_im2col(xq_nhwc, kh, kw, ph, pw, stride):
+    """Explicit lowering of an int8 NHWC tensor to the rows of the convolution's GEMM (reduction index (tap, channel))."""
+    N, Hh, Ww, Cc = xq_nhwc.shape
+    Ho, Wo = (Hh + 2 * ph - kh) // stride + 1, (Ww + 2 * pw - kw) // stride + 1
+    xp = np.zeros((N, Hh + 2 * ph, Ww + 2 * pw, Cc), np.int8)
+    xp[:, ph:ph + Hh, pw:pw + Ww] = xq_nhwc
+    rows = np.zeros((N, Ho, Wo, kh * kw * Cc), np.int8)
+    for dh in range(kh):
+        for dw in range(kw):
+            tap = dh * kw + dw
+            rows[..., tap * Cc:(tap + 1) * Cc] = xp[:, dh:dh + stride * (Ho - 1) + 1:stride, dw:dw + stride * (Wo - 1) + 1:stride]
+    return rows.reshape(N * Ho * Wo, kh * kw * Cc), Ho, Wo
+
+
+ENSEMBLE_CONV_CASES = [
+    # N, H,  W,  C,   O,  kh, kw, bits, K, g, n_keep, M, stride, sum
+    (2, 16, 16, 128, 64, 3, 3, 4, 4, 8, 4, 2, 1, False),
+    (1, 14, 14, 128, 72, 3, 3, 4, 3, 8, 3, 3, 1, False),    # edge patches hang over; three predictors of one order each
+    (2, 16, 16, 256, 80, 1, 1, 2, 4, 16, 2, 2, 2, False),   # strided 1x1, ternary
+    (1, 15, 17, 128, 64, 3, 3, 4, 4, 8, 4, 2, 2, True),     # summed: one launch per predictor, in order
+    (2, 12, 12, 128, 48, 3, 3, 8, 2, 8, 3, 2, 1, True),
+]
+
+
+@pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep,M,stride,summed", ENSEMBLE_CONV_CASES)
+def test_ensemble_convolution_matches_oracle(oracle, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep, M, stride, summed):
+    """pipe_ensemble_conv2d (Sec. 3.2 on a convolution: predictor m applies its cluster of orders to its own NHWC
+    input) == the oracle's ensemble on explicitly lowered im2col rows of every predictor's input."""
+    rng = np.random.default_rng(N * 1000 + Hh * 10 + Cc + M)
+    I = kh * kw * Cc
+    W = _w(rng, O, I, heavy=(bits == 2))
+    bias = rng.standard_normal(O).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep, M), W)
+    split = oracle.balanced_split(K, M)
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    xq_gpu, sx_gpu, rows_m, sx_o = [], [], [], []
+    for m in range(M):
+        x4 = (np.maximum(rng.standard_normal((N, Hh, Ww, Cc)), 0) * (1.0 + m)).astype(np.float32)
+        xq4, sx = H.gpu_quantize(x4.reshape(-1, Cc))
+        xq_o, s_o = oracle.quantize_act(x4.reshape(-1, Cc))
+        np.testing.assert_array_equal(xq4.cpu().numpy(), xq_o)
+        rows, Ho, Wo = _lower_im2col(xq_o.reshape(N, Hh, Ww, Cc), kh, kw, ph, pw, stride)
+        xq_gpu.append(xq4.view(N, Hh, Ww, Cc))
+        sx_gpu.append(sx)
+        rows_m.append(rows)
+        sx_o.append(s_o)
+    want_y, want_part = oracle.ensemble(e, np.stack(rows_m), sx_o, split, bias=bias, sum_branches=summed)
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, ph, pw
+    geom.stride_h = geom.stride_w = stride
+    T = N * Ho * Wo
+    ys = [torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda") for _ in range(1 if summed else M)]
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
+    B.pipe_ensemble_conv2d(layer.desc, geom, layer.blob, xq_gpu, sx_gpu, ys, torch.from_numpy(bias).cuda(), summed, part)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    np.testing.assert_array_equal(part.cpu().numpy(), want_part)
+    got = ys[0].cpu().numpy() if summed else np.stack([y.cpu().numpy() for y in ys])
+    np.testing.assert_array_equal(got.view(np.uint32), want_y.view(np.uint32))
+
+
+def test_ensemble_convolution_inner_layer_matches_oracle(oracle):
+    """pipe_ensemble_conv2d_q8: every predictor's int8 output equals forward -> ReLU -> quantize(static step) of the
+    oracle on the lowered rows of that predictor's input."""
+    rng = np.random.default_rng(77)
+    N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep, M = 2, 16, 16, 128, 64, 3, 3, 4, 4, 8, 4, 2
+    I = kh * kw * Cc
+    W = _w(rng, O, I)
+    bias = rng.standard_normal(O).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep, M), W)
+    split = oracle.balanced_split(K, M)
+    begin = np.concatenate([[0], np.cumsum(split)]).astype(int)
+    steps = [0.05, 0.11]
+    xq_gpu, sx_gpu, want = [], [], []
+    for m in range(M):
+        x4 = np.maximum(rng.standard_normal((N, Hh, Ww, Cc)), 0).astype(np.float32)
+        xq4, sx = H.gpu_quantize(x4.reshape(-1, Cc))
+        xq_o, s_o = oracle.quantize_act(x4.reshape(-1, Cc))
+        rows, Ho, Wo = _lower_im2col(xq_o.reshape(N, Hh, Ww, Cc), kh, kw, 1, 1, 1)
+        xq_gpu.append(xq4.view(N, Hh, Ww, Cc))
+        sx_gpu.append(sx)
+        want.append(oracle.forward_requantized(e, rows, s_o, steps[m], int(begin[m]), int(begin[m + 1]),
+                                               bias=bias if m == 0 else None, relu=True))
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, 1, 1
+    geom.stride_h = geom.stride_w = 1
+    T = N * Ho * Wo
+    yq = [torch.full((T, O), 99, dtype=torch.int8, device="cuda") for _ in range(M)]
+    so = [torch.tensor([s], dtype=torch.float32, device="cuda") for s in steps]
+    B.pipe_ensemble_conv2d_q8(layer.desc, geom, layer.blob, xq_gpu, sx_gpu, so, yq, torch.from_numpy(bias).cuda(), True)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    for m in range(M):
+        np.testing.assert_array_equal(yq[m].cpu().numpy(), want[m])
