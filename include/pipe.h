@@ -452,6 +452,18 @@ pipe_status pipe_ensemble_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv
                                     int32_t relu, const float* const* h_out_scale_m, int8_t* const* h_yq_m, int64_t ldyq,
                                     int32_t* d_partials, void* stream);
 
+/*
+ * The explicit form of the same contraction (Appendix H: reduction index (tap, input channel)), for the geometries
+ * pipe_expanded_conv2d does not take -- a channel count that is not a multiple of 128, as in a network's first
+ * layer: lowers the quantized NHWC tensor d_xq [N, H, W, C] to the rows
+ *     d_rows[t, (dh*kernel_w + dw)*C + c] = d_xq[n, stride_h*ho + dh - pad_h, stride_w*wo + dw - pad_w, c]   (0 outside the image),
+ * t = (n*Ho + ho)*Wo + wo, int8 [N*Ho*Wo, kernel_h*kernel_w*C] with row pitch ld_rows, which pipe_expanded_linear /
+ * pipe_ensemble_forward then take as their [T, I] input with the tensor's own step.  Bytes of a row beyond
+ * kernel_h*kernel_w*C are not written.  Caller-owned buffers; any alignment (16-byte aligned pointers, pitch and C give
+ * the fast path).
+ */
+pipe_status pipe_lower_conv_input(const pipe_conv_geom* geom, const int8_t* d_xq, int8_t* d_rows, int64_t ld_rows, void* stream);
+
 /* Number of kernels the library has launched in this process (all calls, all streams). */
 uint64_t pipe_launch_count(void);
 

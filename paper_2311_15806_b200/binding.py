@@ -36,6 +36,7 @@ EXPORTS = ["pipe_keep_groups_from_gamma", "pipe_default_branches", "pipe_layout"
            "pipe_expand_weights_static",
            "pipe_quantize_act", "pipe_quantize_act_ex", "pipe_ensemble_forward_zp", "pipe_expanded_linear", "pipe_expanded_conv2d", "pipe_ensemble_forward",
            "pipe_ensemble_forward_q8", "pipe_expanded_conv2d_q8", "pipe_ensemble_conv2d", "pipe_ensemble_conv2d_q8",
+           "pipe_lower_conv_input",
            "pipe_launch_count", "pipe_poll_status", "pipe_status_string",
            # include/pipe_diag.h: tests and measurements only
            "pipe_diag_select_kernel", "pipe_diag_mma_i8_rate", "pipe_diag_bounded_wait"]
@@ -108,6 +109,7 @@ def lib() -> C.CDLL:
         L.pipe_expanded_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
         L.pipe_ensemble_conv2d.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, p, i64, i32, p, p]
         L.pipe_ensemble_conv2d_q8.argtypes = [C.POINTER(LayerDesc), C.POINTER(ConvGeom), p, p, p, p, i32, p, p, i64, p, p]
+        L.pipe_lower_conv_input.argtypes = [C.POINTER(ConvGeom), p, p, i64, p]
         L.pipe_diag_select_kernel.argtypes = [i32]
         L.pipe_diag_mma_i8_rate.argtypes = [i32, i64, i32, C.POINTER(C.c_double), p]
         L.pipe_diag_bounded_wait.argtypes = [i64, p]
@@ -338,6 +340,13 @@ def pipe_expanded_conv2d_q8(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor,
     _check(lib().pipe_expanded_conv2d_q8(C.byref(desc), C.byref(geom), _dp(blob), _dp(xq_nhwc), _dp(sx), _dp(bias),
                                          int(relu), _dp(out_scale), _dp(yq), yq.stride(0), _dp(partials),
                                          _stream_ptr(stream)), "pipe_expanded_conv2d_q8")
+
+
+def pipe_lower_conv_input(geom: ConvGeom, xq_nhwc: torch.Tensor, rows: torch.Tensor, stream=None) -> None:
+    """xq_nhwc: cuda int8 [N, H, W, C] contiguous; rows: cuda int8 [N*Ho*Wo, >= kh*kw*C] (last dim contiguous)."""
+    assert xq_nhwc.is_contiguous() and xq_nhwc.dtype == torch.int8 and rows.dtype == torch.int8 and rows.stride(1) == 1
+    _check(lib().pipe_lower_conv_input(C.byref(geom), _dp(xq_nhwc), _dp(rows), rows.stride(0), _stream_ptr(stream)),
+           "pipe_lower_conv_input")
 
 
 def pipe_ensemble_conv2d(desc: LayerDesc, geom: ConvGeom, blob: torch.Tensor, xq_m, sx_m, y_m, bias: torch.Tensor | None = None,

@@ -361,3 +361,69 @@ extern "C" pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t
   count_launch(2);
   return launch_status();
 }
+
+// ------------------------------------------------------------------------------------------------
+// Explicit lowering of a quantized NHWC tensor to the rows of the convolution's GEMM, for the geometries the implicit
+// convolution does not take (channel counts that are not multiples of 128: a network's first layer, narrow layers).
+namespace pipe {
+
+struct LowerArgs {
+  const int8_t* x;
+  int8_t* rows;
+  int64_t ld_rows, total;   // total = T * kh * kw * ceil(C / 16) pieces of up to 16 channels
+  int N, H, W, C, kh, kw, ph, pw, sh, sw, Ho, Wo, cpieces;
+  int vec;                  // 16-byte loads and stores are possible (C % 16 == 0, aligned pointers and pitch)
+};
+
+__global__ void __launch_bounds__(256) lower_conv_input_kernel(const __grid_constant__ LowerArgs a) {
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < a.total; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int piece = static_cast<int>(i % a.cpieces);
+    int64_t r = i / a.cpieces;
+    const int tap = static_cast<int>(r % (a.kh * a.kw));
+    const int64_t t = r / (a.kh * a.kw);
+    const int wo = static_cast<int>(t % a.Wo);
+    const int ho = static_cast<int>((t / a.Wo) % a.Ho);
+    const int n = static_cast<int>(t / (static_cast<int64_t>(a.Wo) * a.Ho));
+    const int h = a.sh * ho + tap / a.kw - a.ph, w = a.sw * wo + tap % a.kw - a.pw;
+    const bool in = h >= 0 && h < a.H && w >= 0 && w < a.W;
+    const int c0 = piece * 16, nc = min(16, a.C - c0);
+    int8_t* dst = a.rows + t * a.ld_rows + static_cast<int64_t>(tap) * a.C + c0;
+    const int8_t* src = a.x + ((static_cast<int64_t>(n) * a.H + h) * a.W + w) * a.C + c0;
+    if (a.vec) {
+      *reinterpret_cast<uint4*>(dst) = in ? __ldg(reinterpret_cast<const uint4*>(src)) : make_uint4(0, 0, 0, 0);
+    } else {
+      for (int c = 0; c < nc; ++c) dst[c] = in ? __ldg(src + c) : static_cast<int8_t>(0);
+    }
+  }
+}
+
+}  // namespace pipe
+
+extern "C" pipe_status pipe_lower_conv_input(const pipe_conv_geom* geom, const int8_t* d_xq, int8_t* d_rows, int64_t ld_rows,
+                                             void* stream) {
+  if (!geom || !d_xq || !d_rows) return PIPE_ERR_INVALID_ARG;
+  if (geom->batch < 1 || geom->height < 1 || geom->width < 1 || geom->channels < 1 || geom->kernel_h < 1 || geom->kernel_w < 1 ||
+      geom->stride_h < 0 || geom->stride_w < 0 || geom->pad_h < 0 || geom->pad_w < 0)
+    return PIPE_ERR_INVALID_ARG;
+  const int sh = geom->stride_h > 0 ? geom->stride_h : 1, sw = geom->stride_w > 0 ? geom->stride_w : 1;
+  if (geom->pad_h >= geom->kernel_h || geom->pad_w >= geom->kernel_w) return PIPE_ERR_SHAPE;
+  if (geom->height + 2 * geom->pad_h < geom->kernel_h || geom->width + 2 * geom->pad_w < geom->kernel_w) return PIPE_ERR_SHAPE;
+  const int64_t I = static_cast<int64_t>(geom->kernel_h) * geom->kernel_w * geom->channels;
+  if (I > INT32_MAX || ld_rows < I) return PIPE_ERR_INVALID_ARG;
+  LowerArgs a;
+  a.x = d_xq; a.rows = d_rows; a.ld_rows = ld_rows;
+  a.N = geom->batch; a.H = geom->height; a.W = geom->width; a.C = geom->channels;
+  a.kh = geom->kernel_h; a.kw = geom->kernel_w; a.ph = geom->pad_h; a.pw = geom->pad_w; a.sh = sh; a.sw = sw;
+  a.Ho = (a.H + 2 * a.ph - a.kh) / sh + 1;
+  a.Wo = (a.W + 2 * a.pw - a.kw) / sw + 1;
+  a.cpieces = ceil_div(a.C, 16);
+  a.total = static_cast<int64_t>(a.N) * a.Ho * a.Wo * a.kh * a.kw * a.cpieces;
+  a.vec = (a.C % 16 == 0 && ld_rows % 16 == 0 && !(reinterpret_cast<uintptr_t>(d_xq) & 15) && !(reinterpret_cast<uintptr_t>(d_rows) & 15)) ? 1 : 0;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t want = ceil_div<int64_t>(a.total, 256);
+  const int grid = static_cast<int>(want < static_cast<int64_t>(sms) * 16 ? want : static_cast<int64_t>(sms) * 16);
+  lower_conv_input_kernel<<<grid > 0 ? grid : 1, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  count_launch(1);
+  return launch_status();
+}

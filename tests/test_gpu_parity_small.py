@@ -497,3 +497,45 @@ def test_ensemble_convolution_inner_layer_matches_oracle(oracle):
     assert B.pipe_poll_status() == B.PIPE_OK
     for m in range(M):
         np.testing.assert_array_equal(yq[m].cpu().numpy(), want[m])
+
+
+LOWER_CASES = [
+    # N, H, W, C, kh, kw, pad, stride, pitch_extra
+    (2, 20, 18, 3, 7, 7, 3, 2, 13),      # a first layer: 7 x 7 on three channels, stride 2 (I = 147, pitch 160)
+    (1, 9, 11, 24, 3, 3, 1, 1, 0),       # channels not a multiple of 16
+    (2, 8, 8, 64, 3, 3, 1, 1, 0),        # 16-byte pieces
+    (1, 10, 6, 96, 1, 1, 0, 2, 32),
+]
+
+
+@pytest.mark.parametrize("N,Hh,Ww,Cc,kh,kw,pad,stride,extra", LOWER_CASES)
+def test_explicit_lowering_and_first_layer_convolution(oracle, N, Hh, Ww, Cc, kh, kw, pad, stride, extra):
+    """pipe_lower_conv_input == the lowering written out on the host, and pipe_expanded_linear on its rows == the
+    oracle: the route for convolutions whose channel count the implicit form does not take."""
+    rng = np.random.default_rng(N + Hh + Cc)
+    x4 = rng.standard_normal((N, Hh, Ww, Cc)).astype(np.float32)
+    xq4, sx = H.gpu_quantize(x4.reshape(-1, Cc))
+    xq_o, sx_o = oracle.quantize_act(x4.reshape(-1, Cc))
+    want_rows, Ho, Wo = _lower_im2col(xq_o.reshape(N, Hh, Ww, Cc), kh, kw, pad, pad, stride)
+    I = kh * kw * Cc
+    T = N * Ho * Wo
+    buf = torch.full((T, I + extra), 77, dtype=torch.int8, device="cuda")
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, pad, pad
+    geom.stride_h = geom.stride_w = stride
+    B.pipe_lower_conv_input(geom, xq4.view(N, Hh, Ww, Cc), buf)
+    torch.cuda.synchronize()
+    got = buf.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :I], want_rows)
+    assert (got[:, I:] == 77).all(), "bytes beyond the row were written"
+    O, bits, K, g, n_keep = 64, (8 if I % 2 else 4), 3, 8, 3   # (a row of 4-bit codes is a whole number of bytes)
+    W = _w(rng, O, I)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep), W)
+    f = oracle.forward(e, want_rows, sx_o)
+    y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
+    B.pipe_expanded_linear(layer.desc, layer.blob, buf[:, :I], sx, y)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), f.y.view(np.uint32))
