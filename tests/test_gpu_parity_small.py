@@ -539,3 +539,46 @@ def test_explicit_lowering_and_first_layer_convolution(oracle, N, Hh, Ww, Cc, kh
     torch.cuda.synchronize()
     assert B.pipe_poll_status() == B.PIPE_OK
     np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), f.y.view(np.uint32))
+
+
+def test_two_layer_convolutional_ensemble_chain(oracle):
+    """Sec. 3.2 / Fig. 2 on a small ConvNet: two predictors, each a chain of two convolutions on its own tensors; the
+    inner layer hands Q(ReLU(y_m)) to the same predictor's next layer, the last layer's outputs are summed.  Equal, bit
+    for bit, to the same composition of the oracle's pinned functions on explicitly lowered rows."""
+    rng = np.random.default_rng(5)
+    N, Hh, Ww, C0, C1, O, bits, K, g, M = 2, 12, 12, 128, 128, 40, 4, 4, 8, 2
+    W1, W2 = _w(rng, C1, 9 * C0), _w(rng, O, 9 * C1)
+    b1, b2 = rng.standard_normal(C1).astype(np.float32), rng.standard_normal(O).astype(np.float32)
+    e1, e2 = oracle.expand(W1, bits, K, g, 6), oracle.expand(W2, bits, K, g, 2)
+    l1 = H.gpu_expand(H.desc_of(C1, 9 * C0, bits, K, g, 6, M), W1)
+    l2 = H.gpu_expand(H.desc_of(O, 9 * C1, bits, K, g, 2, M), W2)
+    split = oracle.balanced_split(K, M)
+    begin = np.concatenate([[0], np.cumsum(split)]).astype(int)
+    x4 = np.maximum(rng.standard_normal((N, Hh, Ww, C0)), 0).astype(np.float32)
+    xq4, sx = H.gpu_quantize(x4.reshape(-1, C0))
+    xq_o, sx_o = oracle.quantize_act(x4.reshape(-1, C0))
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, C0
+    geom.kernel_h = geom.kernel_w = 3
+    geom.pad_h = geom.pad_w = 1
+    geom.stride_h = geom.stride_w = 1
+    T = N * Hh * Ww
+    steps = [0.04, 0.09]
+    # layer 1: both predictors read the network's input; predictor m keeps its own int8 tensor
+    mid = [torch.full((T, C1), 99, dtype=torch.int8, device="cuda") for _ in range(M)]
+    so = [torch.tensor([s], dtype=torch.float32, device="cuda") for s in steps]
+    B.pipe_ensemble_conv2d_q8(l1.desc, geom, l1.blob, [xq4.view(N, Hh, Ww, C0)] * M, [sx] * M, so, mid, torch.from_numpy(b1).cuda(), True)
+    # layer 2: predictor m's tensor with its step; the outputs are summed
+    y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
+    geom.channels = C1
+    B.pipe_ensemble_conv2d(l2.desc, geom, l2.blob, [t.view(N, Hh, Ww, C1) for t in mid], so, [y], torch.from_numpy(b2).cuda(), True)
+    torch.cuda.synchronize()
+    assert B.pipe_poll_status() == B.PIPE_OK
+    rows0, _, _ = _lower_im2col(xq_o.reshape(N, Hh, Ww, C0), 3, 3, 1, 1, 1)
+    rows1 = []
+    for m in range(M):
+        q = oracle.forward_requantized(e1, rows0, sx_o, steps[m], int(begin[m]), int(begin[m + 1]), bias=b1 if m == 0 else None, relu=True)
+        np.testing.assert_array_equal(mid[m].cpu().numpy(), q)
+        rows1.append(_lower_im2col(q.reshape(N, Hh, Ww, C1), 3, 3, 1, 1, 1)[0])
+    want, _ = oracle.ensemble(e2, np.stack(rows1), steps, split, bias=b2, sum_branches=True)
+    np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), want.view(np.uint32))
