@@ -738,10 +738,37 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
 // ---------------------------------------------------------------------------------------------
 }  // namespace tc
 
+// A tensor map depends on the address, the shape and the box only, and a decoding loop presents the same few
+// activation buffers call after call: the last encodings of a host thread are kept (encoding one costs the host about
+// as much as the rest of a small-token forward call).
 bool make_tensor_map_2d_u8(CUtensorMap* map, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
                            uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
-  return tcc::make_map_2d(map, base, inner_bytes, rows, pitch_bytes, box_inner, box_rows,
-                         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
+  struct Entry {
+    const void* base = nullptr;
+    uint64_t inner = 0, rows = 0, pitch = 0;
+    uint32_t box_inner = 0, box_rows = 0;
+    bool swz = false, valid = false;
+    CUtensorMap map;
+  };
+  constexpr int kEntries = 8;
+  thread_local Entry cache[kEntries];
+  thread_local int next = 0;
+  for (int i = 0; i < kEntries; ++i) {
+    const Entry& e = cache[i];
+    if (e.valid && e.base == base && e.inner == inner_bytes && e.rows == rows && e.pitch == pitch_bytes && e.box_inner == box_inner &&
+        e.box_rows == box_rows && e.swz == swizzle128) {
+      *map = e.map;
+      return true;
+    }
+  }
+  if (!tcc::make_map_2d(map, base, inner_bytes, rows, pitch_bytes, box_inner, box_rows,
+                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE))
+    return false;
+  Entry& e = cache[next];
+  next = (next + 1) % kEntries;
+  e.base = base, e.inner = inner_bytes, e.rows = rows, e.pitch = pitch_bytes, e.box_inner = box_inner, e.box_rows = box_rows;
+  e.swz = swizzle128, e.valid = true, e.map = *map;
+  return true;
 }
 
 namespace tc {
