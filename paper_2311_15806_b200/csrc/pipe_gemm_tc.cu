@@ -633,7 +633,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_forward_kernel(const __grid_co
           const int half = static_cast<int>(hb);
           int n, h0, w0;
           patch_origin(p, 2 * p.tpt * tt + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-          tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[0], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
+          tma_load_4d(g.stage0 + rp.slot * p.stage_bytes + half * (kABytes / 2), &p.tmap_a[m], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh,
                       n, g.a_full0 + 8u * rp.slot);
         }
       }
@@ -829,7 +829,7 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   }
   if (a.g % 8 != 0 || BN == 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
-  if (a.conv_on && (a.cC % kKStep != 0 || a.num_branches != 1)) return PIPE_ERR_UNSUPPORTED;
+  if (a.conv_on && a.cC % kKStep != 0) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
     if (reinterpret_cast<uintptr_t>(a.branch[m].xq) & 15) return PIPE_ERR_UNSUPPORTED;
   }
@@ -887,7 +887,8 @@ static pipe_status launch_tc(const ForwardArgs& a, cudaStream_t stream) {
   const int dyn_smem = p.depth * p.stage_bytes + 1024;
 
   if (a.conv_on) {
-    if (!make_map_nhwc(&p.tmap_a[0], a.branch[0].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
+    for (int m = 0; m < a.num_branches; ++m)
+      if (!make_map_nhwc(&p.tmap_a[m], a.branch[m].xq, a.cN, a.cH, a.cW, a.cC, a.csh, a.csw)) return PIPE_ERR_CUDA;
   } else
   for (int m = 0; m < a.num_branches; ++m) {
     if (!make_map_2d(&p.tmap_a[m], a.branch[m].xq, static_cast<uint64_t>(a.I), static_cast<uint64_t>(a.T),

@@ -420,6 +420,8 @@ ENSEMBLE_CONV_CASES = [
     (2, 16, 16, 256, 80, 1, 1, 2, 4, 16, 2, 2, 2, False),   # strided 1x1, ternary
     (1, 15, 17, 128, 64, 3, 3, 4, 4, 8, 4, 2, 2, True),     # summed: one launch per predictor, in order
     (2, 12, 12, 128, 48, 3, 3, 8, 2, 8, 3, 2, 1, True),
+    (1, 15, 11, 256, 48, 1, 3, 2, 4, 8, 2, 3, 1, False),    # ternary with groups of 8: the one-SM kernel's turn
+    (3, 15, 22, 128, 72, 5, 3, 2, 4, 8, 4, 2, 2, True),
 ]
 
 
