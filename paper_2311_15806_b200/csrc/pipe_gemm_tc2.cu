@@ -1091,6 +1091,14 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   }
   // (a single token tile: the second CTA of a pair then stages zeros and stores nothing, but still unpacks its half of
   // every block, which is what such a launch spends its time on)
+  if (p.ntok_tiles == 1 && kernel_choice() == 0) {
+    // ... unless the whole layer is a handful of blocks: then nothing is there to share and the one-SM kernel's shorter
+    // set-up wins (a forced choice of this kernel still takes the launch)
+    int64_t rows = 0;
+    for (int m = 0; m < a.num_branches; ++m)
+      for (int k = a.branch[m].k_begin; k < a.branch[m].k_end; ++k) rows += a.order[k].rows;
+    if (rows <= 4 * PIPE_BLOCK_ROWS) return PIPE_ERR_UNSUPPORTED;
+  }
   p.ntt = ceil_div(p.ntok_tiles, 2);
   // the tile count is known on the device only (block counts of the tables); a table never has more blocks than groups
   if (static_cast<int64_t>(a.G) * p.ntt * a.num_branches > INT32_MAX) return PIPE_ERR_UNSUPPORTED;
