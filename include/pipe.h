@@ -17,6 +17,15 @@
  *     stayed in bounds.  Nothing throws, aborts, traps or prints.
  *   - there is no CPU fallback: without a CUDA device every compute call returns
  *     PIPE_ERR_CUDA.
+ *   - the forward kernels are launched with programmatic stream serialization: their prologue
+ *     may overlap the tail of the preceding launch on `stream`, and the weight-streaming kernel
+ *     (at most 16 tokens) starts copying the blob's packed codes during that overlap.  The
+ *     library orders this correctly against its own calls (a forward call that directly follows
+ *     pipe_expand_weights* on the same stream waits for it in full).  A caller that writes
+ *     d_blob by other means must let that work complete -- an event, a synchronize, or any other
+ *     library call in between -- before queueing a forward call on the same stream.  Inputs
+ *     other than d_blob (activations, scales, bias, outputs) are only touched after the
+ *     preceding launch has completed, whoever queued it.
  */
 #ifndef PIPE_H_
 #define PIPE_H_

@@ -31,6 +31,10 @@ constexpr int kPlanSMs = 148;   // SMs of the B200 the decode plan is laid out f
 int* device_status_word();
 void count_launch(int n = 1);
 int kernel_choice();
+// Streams whose last library call was an expansion (which writes the blob a forward call on the same stream may be about
+// to read): an expansion marks its stream, every other call on a stream takes the mark away and learns whether it was there.
+void mark_expansion(cudaStream_t stream);
+bool take_expansion_mark(cudaStream_t stream);
 
 inline pipe_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PIPE_OK : PIPE_ERR_CUDA; }
 
@@ -178,6 +182,8 @@ struct ForwardArgs {
   int cHo, cWo, csh, csw;   // output height / width and the strides
   // fused inner-layer epilogue (q8_out != 0): yq = clamp(rne(act(y) / out_scale)) as int8, row pitch ldyq; y is not written
   int decode_split;   // CTAs that share a decode unit's reduction axis (from the layout; 0 = no decode tables)
+  int blob_settled;   // the library's last call on this stream was no expansion: a kernel launched with programmatic stream
+                      // serialization may read the expanded layer before it waits for the launch before it
   int q8_out, relu;   // relu: the activation kind (see apply_activation; the name is from the first version)
   int64_t ldyq;
 };

@@ -747,6 +747,7 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
       count_launch(1);
     }
   }
+  mark_expansion(s);   // a forward call that follows on this stream must not read the blob ahead of its dependency wait
   return launch_status();
 }
 

@@ -52,6 +52,7 @@ struct Params {
   int nstages;            // stages per pass
   int nkmax;              // most orders any branch has
   int own_max;            // most slabs any CTA owns
+  int prefetch;           // the expanded layer is not being written by the launch before: weights may be fetched ahead of the dependency wait
   int ctas_per_branch;    // every branch has its own CTAs, so no CTA's range crosses a branch boundary
 };
 
@@ -185,9 +186,12 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   const int cnt = base + (cib < rem ? 1 : 0);
 
   // A launch of this kernel that follows in the stream may be brought onto the SMs as they become free: its CTAs
-  // then exist, with their barriers set up, when this launch's last CTA ends, instead of being launched only then
-  // (a chain of small-token layers otherwise pays a launch gap per layer).  They wait below, before their first
-  // access to global memory, until this launch is complete.
+  // then exist when this launch's last CTA ends, instead of being launched only then (a chain of small-token layers
+  // otherwise pays a launch gap and a cold start per layer).  Until the launch before it is complete such a CTA
+  // touches nothing that launch may have written: with p.prefetch (the host knows that the expanded layer is not
+  // being written: its last call on this stream was no expansion) it builds its tables and fills its whole ring
+  // with WEIGHTS first, which belong to the layer alone, and waits only then, before the first access to
+  // activations, steps, bias or outputs; without it, it waits before its first access to global memory.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -202,7 +206,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   // passes: pieces of at most pass_slabs slabs of the CTA's range (which lies in one branch)
   const int npass = min((cnt + p.pass_slabs - 1) / p.pass_slabs, kMaxPasses);
   for (int e = threadIdx.x; e < p.pass_slabs * NP * NT * 4 * 32; e += kThreads) sums[e] = 0;
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!p.prefetch) asm volatile("griddepcontrol.wait;" ::: "memory");
   // ---- which orders keep each own slab, and where its 8 rows start
   for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
     const int li = e / p.nkmax, ko = e % p.nkmax;
@@ -290,25 +294,36 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
       __syncwarp();
       if (*abort_flag) break;
       // jobs of a stage: per reduction block, the activation tile and then one run of rows per order
+      // (what: 0 all of them, 1 the weights only, 2 the activation tiles only)
       const int njobs = KBPS * (1 + nk);
-      for (int j0 = 0; j0 < KBPS * (1 + p.nkmax); j0 += kJobLanes) {   // same trip count in every lane; lanes without a job idle
-        const int j = j0 + job0;
-        if (valid && j < njobs) {
-          const int kbs = j / (1 + nk), idx = j - kbs * (1 + nk);
-          const int kb = ks * KBPS + kbs;
-          if (kb < p.kblocks) {
-            if (idx == 0) {
-              // activations: token rows beyond T and reduction bytes beyond I come back as zeros
-              tma_load_2d(sbase + kbs * kXTile, &p.tmap_x[P.branch], kb * 128, 0, bar);
-            } else if (P.seg_rows[idx - 1] > 0) {
-              const int ko = idx - 1;
-              const OrderView& ov = p.f.order[br.k_begin + ko];
-              const uint8_t* src = ov.kcodes + (static_cast<size_t>(kb) * ov.rows + P.seg_row0[ko]) * p.pk;
-              bulk_load(sbase + P.seg_off[ko] + kbs * P.seg_rows[ko] * p.pk, src, static_cast<uint32_t>(P.seg_rows[ko] * p.pk), bar);
+      auto issue_jobs = [&](int what) {
+        for (int j0 = 0; j0 < KBPS * (1 + p.nkmax); j0 += kJobLanes) {   // same trip count in every lane; lanes without a job idle
+          const int j = j0 + job0;
+          if (valid && j < njobs) {
+            const int kbs = j / (1 + nk), idx = j - kbs * (1 + nk);
+            const int kb = ks * KBPS + kbs;
+            if (kb < p.kblocks) {
+              if (idx == 0) {
+                // activations: token rows beyond T and reduction bytes beyond I come back as zeros
+                if (what != 1) tma_load_2d(sbase + kbs * kXTile, &p.tmap_x[P.branch], kb * 128, 0, bar);
+              } else if (what != 2 && P.seg_rows[idx - 1] > 0) {
+                const int ko = idx - 1;
+                const OrderView& ov = p.f.order[br.k_begin + ko];
+                const uint8_t* src = ov.kcodes + (static_cast<size_t>(kb) * ov.rows + P.seg_row0[ko]) * p.pk;
+                bulk_load(sbase + P.seg_off[ko] + kbs * P.seg_rows[ko] * p.pk, src, static_cast<uint32_t>(P.seg_rows[ko] * p.pk), bar);
+              }
             }
           }
+          __syncwarp();
         }
-        __syncwarp();
+      };
+      if (p.prefetch && it0 < static_cast<uint32_t>(depth)) {
+        // the first use of the ring: its weights go ahead of the wait for the launch before, its activation tiles after
+        issue_jobs(1);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        issue_jobs(2);
+      } else {
+        issue_jobs(0);
       }
     }
     __syncwarp();
@@ -322,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
     }
   } else {
     // ================================================================== consumer warps
+    if (p.prefetch) asm volatile("griddepcontrol.wait;" ::: "memory");   // (the steps and the bias are the caller's data)
     // scale products s_k * lambda_x and bias of every own slab (needed at the end of a pass only;
     // the loads overlap the first copies)
     for (int e = threadIdx.x; e < cnt * p.nkmax * 8; e += 32 * kConsWarps) {
@@ -610,6 +626,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   if (max_cluster > kMaxOrd) return PIPE_ERR_UNSUPPORTED;
   Params p;
   p.f = a;
+  p.prefetch = a.blob_settled ? 1 : 0;
   const int nt = a.T <= 8 ? 1 : 2;
   const int np = max_cluster <= 2 ? 1 : (max_cluster <= 4 ? 2 : 4);
   const int spw = (np * nt <= 2) ? 5 : (np * nt == 4 ? 2 : 1);

@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "pipe_common.cuh"
 #include "pipe_diag.h"
@@ -15,6 +16,33 @@ static std::atomic<int> g_kernel_choice{0};
 
 void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
 int kernel_choice() { return g_kernel_choice.load(); }
+
+namespace {
+std::mutex g_mark_mutex;
+constexpr int kMaxMarked = 64;
+cudaStream_t g_marked[kMaxMarked];
+int g_num_marked = 0;
+bool g_mark_overflow = false;   // more streams than the table holds: every call is then treated as following an expansion
+}  // namespace
+
+void mark_expansion(cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_mark_mutex);
+  for (int i = 0; i < g_num_marked; ++i)
+    if (g_marked[i] == stream) return;
+  if (g_num_marked < kMaxMarked) g_marked[g_num_marked++] = stream;
+  else g_mark_overflow = true;
+}
+
+bool take_expansion_mark(cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_mark_mutex);
+  if (g_mark_overflow) return true;
+  for (int i = 0; i < g_num_marked; ++i)
+    if (g_marked[i] == stream) {
+      g_marked[i] = g_marked[--g_num_marked];
+      return true;
+    }
+  return false;
+}
 
 int* device_status_word() {
   // The symbol is per device; its address is looked up once for whichever device is current and kept.

@@ -316,6 +316,7 @@ extern "C" pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I,
       (reinterpret_cast<uintptr_t>(d_sx) & 3))
     return PIPE_ERR_ALIGNMENT;
   if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
+  take_expansion_mark(static_cast<cudaStream_t>(stream));   // (this call's kernels now stand between an expansion and what follows)
   return quantize_act_impl(d_x, T, I, ldx, d_static_scale, d_xq, ldxq, d_sx, static_cast<uint32_t*>(d_ws),
                            static_cast<cudaStream_t>(stream));
 }
@@ -336,6 +337,7 @@ extern "C" pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t
     return PIPE_ERR_ALIGNMENT;
   if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  take_expansion_mark(s);
   int* status = device_status_word();
   if (!status) return PIPE_ERR_CUDA;
   if (T == 0) {
@@ -423,6 +425,7 @@ extern "C" pipe_status pipe_lower_conv_input(const pipe_conv_geom* geom, const i
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int64_t want = ceil_div<int64_t>(a.total, 256);
   const int grid = static_cast<int>(want < static_cast<int64_t>(sms) * 16 ? want : static_cast<int64_t>(sms) * 16);
+  take_expansion_mark(static_cast<cudaStream_t>(stream));
   lower_conv_input_kernel<<<grid > 0 ? grid : 1, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
   count_launch(1);
   return launch_status();
