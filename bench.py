@@ -113,12 +113,12 @@ def workload_spec(name: str):
 # program (summaries under profiles/, named in the comment).  A workload without a capture of the present
 # kernel has no entry and reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "cfg2": 33277696 + 54557440,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
-    "cfg3a": 9437440 + 46843136,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
-    "cfg4a_t4096": 91016704 + 313291008,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
-    "cfg5": 431076352 + 1026774528,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
-    "cfg4a_t1": 56557056 + 22784,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
-    "cfg4a_t16": 56685056 + 248064,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
+    "cfg2": 33161984 + 52870912,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
+    "cfg3a": 9438464 + 46983680,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
+    "cfg4a_t4096": 90846208 + 312983808,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
+    "cfg5": 431581952 + 1026934272,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
+    "cfg4a_t1": 56559872 + 62464,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
+    "cfg4a_t16": 56687616 + 119040,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
 }
 
 

@@ -192,7 +192,9 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   // being written: its last call on this stream was no expansion) it builds its tables and fills its whole ring
   // with WEIGHTS first, which belong to the layer alone, and waits only then, before the first access to
   // activations, steps, bias or outputs; without it, it waits before its first access to global memory.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Its own dependents start at once in the first case (the layer before was complete, or past this same point, when
+  // this CTA started, so no expansion queued earlier is still running beside them) and after the wait in the second.
+  if (p.prefetch) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < depth; ++s) {
@@ -206,7 +208,10 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
   // passes: pieces of at most pass_slabs slabs of the CTA's range (which lies in one branch)
   const int npass = min((cnt + p.pass_slabs - 1) / p.pass_slabs, kMaxPasses);
   for (int e = threadIdx.x; e < p.pass_slabs * NP * NT * 4 * 32; e += kThreads) sums[e] = 0;
-  if (!p.prefetch) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!p.prefetch) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   // ---- which orders keep each own slab, and where its 8 rows start
   for (int e = threadIdx.x; e < cnt * p.nkmax; e += kThreads) {
     const int li = e / p.nkmax, ko = e % p.nkmax;

@@ -804,11 +804,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   g.abort_flag = &abort_flag_s;
   g.ntot = ntot_s;
 
-  // A launch of this kernel that follows in the stream may be brought onto the SMs as they become free (its CTAs then
-  // exist when this launch's last pair ends); it waits here, before its first access to global memory, until the
-  // launch before it is complete.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A launch that follows in the stream may be brought onto the SMs as they become free (its CTAs then exist when this
+  // launch's last pair ends).  This kernel waits here, before its first access to global memory, until the launch
+  // before it is complete, and lets its own dependents start only after that: a dependent that reads weights ahead
+  // of ITS wait (the weight-streaming kernel) then never runs beside an expansion queued before this launch.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x >= 32 && threadIdx.x < 32 + 2 * PIPE_MAX_ORDERS) {
     // (inputs of this launch: written before it started)
     const int i = threadIdx.x - 32, m = i % PIPE_MAX_ORDERS;
