@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 DEFAULT_WORKLOAD = "cfg5"
 TABLE_WORKLOADS = (["cfg1", "cfg2", "cfg3a", "cfg3b"] + [f"cfg4{ab}_t{T}" for ab in "ab" for T in (1, 16, 128, 1024, 4096)]
                    + ["cfg5"])
+# rows measured once more on a layer that keeps its codes as int8 in the tensor-core operand layout as well
+# (pipe_layer_desc.int8_copy: twice the packed bytes of 4-bit codes in HBM, no widening in shared memory)
+INT8_COPY_WORKLOADS = ["cfg3a", "cfg3b", "cfg4a_t128", "cfg4a_t1024", "cfg4a_t4096", "cfg4b_t4096"]
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -324,6 +327,9 @@ def forward_row(run, spec, fwd_ms, fwd_best_ms, how, clocks, peaks, int8, sms: i
            "ops_per_launch": ops, "bytes_per_launch": nbytes, "effective_tops": tops, "gbs": gbs,
            "arithmetic_intensity": ai, "bound": bound,
            "frac_int8_probe_burst": tops / int8["probe_burst"],
+           # (the timing loop runs for a few tenths of a second: long enough for a dense kernel to meet the power cap
+           # that the 1.5 s probe loop settles under, so that figure is given beside the burst one)
+           "frac_int8_probe_sustained": (tops / int8["probe_sustained"]) if int8.get("probe_sustained") else None,
            "frac_int8_int_mm": (tops / int8["int_mm_8192"]) if int8.get("int_mm_8192") else None,
            "frac_int8_2x_bf16_burst": tops / (2.0 * peaks["bf16_tflops"]),
            "frac_int8_nominal_4500": tops / 4500.0,
@@ -518,14 +524,14 @@ def run_ours(args):
     table = []
     host_us = None
     if world == 1 and not args.no_table:
-        for name in TABLE_WORKLOADS:
-            if name == spec.name:
+        for name, int8_copy in [(n, False) for n in TABLE_WORKLOADS] + [(n, True) for n in INT8_COPY_WORKLOADS]:
+            if name == spec.name and not int8_copy:
                 table.append(head_row)
                 continue
             del run
             torch.cuda.empty_cache()
             s2 = workload_spec(name)
-            run = LayerRunner(s2)
+            run = LayerRunner(s2, int8_copy=int8_copy)
             run.load()
             run.expand()
             q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -543,7 +549,11 @@ def run_ours(args):
                 continue
             row = forward_row(run, s2, ms, best, how2, ck, peaks, int8, sms)
             row["quantize_ms"] = q0.elapsed_time(q1)
-            if name == "cfg4a_t1":
+            if int8_copy:
+                row["workload"] = name + "+int8_copy"
+                row["weights"] = "int8 copy in the operand layout beside the packed codes"
+                row["traffic"] = None
+            if name == "cfg4a_t1" and not int8_copy:
                 host_us = host_time_per_forward_call(run, B, torch)
                 row["host_us_per_call"] = host_us
             st = B.pipe_poll_status()

@@ -77,6 +77,12 @@ typedef struct pipe_layer_desc {
                             keep_elems entries of the current residual with the largest magnitude are quantized (ties
                             to the lower index), the others get the code 0 and keep their residual.  Needs
                             keep_groups = G: an unstructured R^k keeps every row */
+  int32_t int8_copy;     /* 0 or 1.  1: the blob also holds every order's codes widened to int8 in the operand layout of
+                            the tensor-core kernel (wcodes_off below; needs g % 8 == 0).  The kernels for more than 16
+                            tokens then copy weight tiles straight into place instead of widening packed codes in
+                            shared memory on every use -- the choice for layers evaluated on many tokens at a time, at
+                            the price of I_pad more bytes per kept row in HBM.  Results are the same bits either way; the
+                            small-token kernels keep streaming the packed codes */
 } pipe_layer_desc;
 
 #define PIPE_ACT_IDENTITY 0
@@ -111,6 +117,11 @@ typedef struct pipe_layer_desc {
  *                 reduction order: int4 -> code 4h+j of the word's 8 codes sits in nibble 2j+h;
  *                 ternary -> code 4h+j of the word's 16 codes sits in bits 8j+2h..8j+2h+1;
  *                 int8 -> unchanged.
+ *   wcodes_off[k] (int8_copy only, else 0) the codes as int8, block-major like kcodes_off: [I_pad/128][rows[k]][128]
+ *                 bytes, with the 16-byte pieces of a row permuted the way the tensor core's 128-byte swizzle expects
+ *                 them in shared memory: piece c (codes 16c .. 16c+15 of the block) of compacted row r is stored as
+ *                 piece c ^ (r & 7) of that row.  A run of kept rows of one block is then one contiguous run of bytes
+ *                 that lands in an operand tile by a plain bulk copy (kept-row runs start at multiples of g, hence of 8).
  * Channel-block tables, one per cluster of orders that a forward call can evaluate on one input: entry m < M
  * for predictor m (Sec. 3.2), entry M for all K orders (pipe_expanded_linear, pipe_expanded_conv2d).
  *   blk_off[m]    int32 [2 + blk_cap[m]]: n, then b_0 = 0 < b_1 < ... < b_n = G.  Block i is the channel groups
@@ -152,6 +163,7 @@ typedef struct pipe_layer_layout {
   int32_t branch_orders[PIPE_MAX_ORDERS]; /* the resolved [K_1..K_M] */
   uint64_t codes_off[PIPE_MAX_ORDERS];
   uint64_t kcodes_off[PIPE_MAX_ORDERS];
+  uint64_t wcodes_off[PIPE_MAX_ORDERS];  /* int8 operand-layout copy (see above); 0 without int8_copy */
   uint64_t scales_off[PIPE_MAX_ORDERS];
   uint64_t kept_off[PIPE_MAX_ORDERS];
   uint64_t cum_off[PIPE_MAX_ORDERS];

@@ -46,7 +46,7 @@ class LayerDesc(C.Structure):
     _fields_ = [("out_features", C.c_int32), ("in_features", C.c_int32), ("weight_bits", C.c_int32),
                 ("num_orders", C.c_int32), ("group_size", C.c_int32), ("keep_groups", C.c_int32),
                 ("num_branches", C.c_int32), ("branch_orders", C.c_int32 * MAX_ORDERS),
-                ("score_mode", C.c_int32), ("keep_elems", C.c_int32)]
+                ("score_mode", C.c_int32), ("keep_elems", C.c_int32), ("int8_copy", C.c_int32)]
 
 
 class ConvGeom(C.Structure):
@@ -60,6 +60,7 @@ class LayerLayout(C.Structure):
                 ("kernel_row_bytes", C.c_int32), ("rows", C.c_int32 * MAX_ORDERS),
                 ("kept_groups", C.c_int32 * MAX_ORDERS), ("branch_orders", C.c_int32 * MAX_ORDERS),
                 ("codes_off", C.c_uint64 * MAX_ORDERS), ("kcodes_off", C.c_uint64 * MAX_ORDERS),
+                ("wcodes_off", C.c_uint64 * MAX_ORDERS),
                 ("scales_off", C.c_uint64 * MAX_ORDERS), ("kept_off", C.c_uint64 * MAX_ORDERS),
                 ("cum_off", C.c_uint64 * MAX_ORDERS), ("blk_off", C.c_uint64 * (MAX_ORDERS + 1)),
                 ("blk_cap", C.c_int32 * (MAX_ORDERS + 1)), ("rec_off", C.c_uint64 * (MAX_ORDERS + 1)),
@@ -240,11 +241,12 @@ ACT_IDENTITY, ACT_RELU, ACT_SILU, ACT_GELU, ACT_SIGMOID = 0, 1, 2, 3, 4
 
 
 def make_desc(O: int, I: int, bits: int, K: int, g: int, keep_groups: int, M: int = 1,
-              branch_orders=None, score_mode: int = 0, keep_elems: int = 0) -> LayerDesc:
+              branch_orders=None, score_mode: int = 0, keep_elems: int = 0, int8_copy: bool = False) -> LayerDesc:
     d = LayerDesc()
     d.out_features, d.in_features, d.weight_bits, d.num_orders = O, I, bits, K
     d.group_size, d.keep_groups, d.num_branches = g, keep_groups, M
     d.score_mode, d.keep_elems = score_mode, keep_elems
+    d.int8_copy = 1 if int8_copy else 0
     if branch_orders is not None:
         for m, v in enumerate(branch_orders):
             d.branch_orders[m] = int(v)
@@ -464,6 +466,14 @@ class ExpandedLayer:
     def kcodes(self, k: int) -> torch.Tensor:
         n = self.layout.rows[k] * self.layout.kernel_row_bytes
         return self.section(self.layout.kcodes_off[k], n).view(self.layout.rows[k], self.layout.kernel_row_bytes)
+
+    def wcodes(self, k: int) -> torch.Tensor | None:
+        """The int8 copy of order k as stored: [I_pad / 128, rows, 128] bytes (None without int8_copy)."""
+        if not self.layout.wcodes_off[k]:
+            return None
+        ipad = (self.desc.in_features + 127) // 128 * 128
+        n = self.layout.rows[k] * ipad
+        return self.section(self.layout.wcodes_off[k], n).view(ipad // 128, self.layout.rows[k], 128)
 
     def scales(self, k: int) -> torch.Tensor:
         return self.section(self.layout.scales_off[k], self.layout.rows[k] * 4).view(torch.float32)

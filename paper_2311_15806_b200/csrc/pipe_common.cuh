@@ -130,6 +130,7 @@ __device__ __forceinline__ float apply_activation(float v, int kind) {
 struct OrderView {
   const uint8_t* codes;   // canonical packed codes
   const uint8_t* kcodes;  // kernel-layout codes
+  const uint8_t* wcodes;  // int8 copy in the tensor-core operand layout, or nullptr
   const float* scales;
   const int32_t* cum;     // [G+1]
   int rows;
@@ -141,6 +142,7 @@ inline OrderView order_view(const LayerInfo& L, const void* blob, int k) {
   OrderView v;
   v.codes = b + L.lay.codes_off[k];
   v.kcodes = b + L.lay.kcodes_off[k];
+  v.wcodes = L.lay.wcodes_off[k] ? b + L.lay.wcodes_off[k] : nullptr;
   v.scales = reinterpret_cast<const float*>(b + L.lay.scales_off[k]);
   v.cum = reinterpret_cast<const int32_t*>(b + L.lay.cum_off[k]);
   v.rows = L.lay.rows[k];

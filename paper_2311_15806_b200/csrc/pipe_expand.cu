@@ -279,6 +279,7 @@ struct QuantizeRowsArgs {
   const int32_t* kept;   // [rows/g] ascending kept groups
   uint8_t* codes;        // canonical [rows, canon_row_bytes]
   uint8_t* kcodes;       // streaming layout [ceil(I/128), rows, 128*BITS/8]
+  uint8_t* wcodes;       // int8 copy in the tensor-core operand layout [ceil(I/128), rows, 128] or nullptr (see pipe.h)
   int rows;              // compacted rows of this order
   float* scales;         // [rows]
   int I, g, qmax;
@@ -356,6 +357,7 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
         const int e0 = base + w * 128 + lane * 4;
         float x[4] = {v[w].x, v[w].y, v[w].z, v[w].w};
         uint32_t cc = 0, ck = 0;
+        uint32_t f4[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           float c = 0.f;
@@ -366,7 +368,8 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
             x[j] = __fmaf_rn(-s, c, x[j]);         // exact new residual, rounded once
           }
           m = max(m, abs_key(x[j]));
-          const uint32_t f = static_cast<uint32_t>(static_cast<int>(c)) & fmask;
+          f4[j] = static_cast<uint32_t>(static_cast<int>(c));
+          const uint32_t f = f4[j] & fmask;
           cc |= f << (BITS * (4 * h + j));          // canonical: field e at bit e * b of the stream
           ck |= f << (8 * j + BITS * h);            // streaming layout: see include/pipe.h
         }
@@ -375,6 +378,13 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
         for (int d = 1; d < LPW; d <<= 1) {
           cc |= __shfl_xor_sync(0xffffffffu, cc, d);
           ck |= __shfl_xor_sync(0xffffffffu, ck, d);
+        }
+        if (p.wcodes && e0 < I_pad) {
+          // the lane's four codes are four bytes of piece (e0 & 127) / 16 of the row's block, which is stored as piece
+          // ((e0 & 127) / 16) ^ (n & 7)
+          const uint32_t wv = __byte_perm(__byte_perm(f4[0], f4[1], 0x0040), __byte_perm(f4[2], f4[3], 0x0040), 0x5410);
+          uint8_t* wdst = p.wcodes + (static_cast<int64_t>(e0 >> 7) * p.rows + n) * 128 + (((((e0 & 127) >> 4) ^ (n & 7)) << 4) | (e0 & 15));
+          *reinterpret_cast<uint32_t*>(wdst) = wv;
         }
         if (h == 0 && e0 < I_pad) {
           uint8_t* kdst = p.kcodes + (static_cast<int64_t>(e0 >> 7) * p.rows + n) * kStepBytes + (e0 & 127) * BITS / 8;
@@ -423,6 +433,15 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
     }
     uint32_t canon[4], kern[4];
     pack16<BITS>(q, canon, kern);
+    if (p.wcodes) {
+      uint32_t wv[4];
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        wv[w] = (static_cast<uint32_t>(q[4 * w]) & 0xffu) | ((static_cast<uint32_t>(q[4 * w + 1]) & 0xffu) << 8) |
+                ((static_cast<uint32_t>(q[4 * w + 2]) & 0xffu) << 16) | (static_cast<uint32_t>(q[4 * w + 3]) << 24);
+      uint8_t* wdst = p.wcodes + (static_cast<int64_t>(i0 >> 7) * p.rows + n) * 128 + ((((i0 & 127) >> 4) ^ (n & 7)) << 4);
+      *reinterpret_cast<uint4*>(wdst) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    }
     const int byte0 = i0 * BITS / 8;
     // streaming layout: reduction-block major, [i0 / 128][row][128 codes]; padded, always whole words
     uint8_t* kdst = p.kcodes + (static_cast<int64_t>(i0 >> 7) * p.rows + n) * kStepBytes + (i0 & 127) * BITS / 8;
@@ -664,6 +683,7 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     q.kept = kept;
     q.codes = blob + L.lay.codes_off[k];
     q.kcodes = blob + L.lay.kcodes_off[k];
+    q.wcodes = L.lay.wcodes_off[k] ? blob + L.lay.wcodes_off[k] : nullptr;
     q.scales = reinterpret_cast<float*>(blob + L.lay.scales_off[k]);
     q.I = L.I; q.g = L.g; q.qmax = L.qmax;
     q.canon_row_bytes = L.lay.canon_row_bytes;

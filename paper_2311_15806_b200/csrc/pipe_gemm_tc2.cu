@@ -62,6 +62,7 @@ struct Params {
   int depth;              // stages in the ring
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
   int shift;              // 8 - b
+  int direct;             // the weights come from the layer's int8 copy in the operand layout (bits reads 8, shift 0)
   int conv_pw, conv_pp, conv_np, conv_chunks;   // patches per image row / per image / in total; 128-channel chunks per tap
   const uint8_t* kbase;   // lowest address of the streaming-layout sections (16-byte aligned)
   uint32_t koff[PIPE_MAX_ORDERS];  // (kcodes of order k - kbase) / 16
@@ -309,7 +310,10 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
     const bool real = kbs < p.kblocks && mine > 0;     // false: the empty position behind an odd block count
     const uint32_t bt_off = slot * kStageBytes + kStageBOff + sub * kBtBytes;
     uint8_t* bt = g.stage_gen + bt_off;
-    if constexpr (BITS == 8) {
+    bool through_registers = false;
+    if constexpr (BITS == 8) through_registers = !p.direct;
+    if (through_registers) {
+      if constexpr (BITS == 8) {
 #pragma unroll
       for (int pass = 0; pass < ITEMS / PASS; ++pass) {
         uint4 w[PASS];
@@ -342,7 +346,9 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
           }
         }
       }
+      }
     } else {
+      // (int8 rows in the operand layout -- the layer's int8 copy -- are complete when their copies have landed)
       // everything the copies need is prepared before the wait for the slot: what follows the wait is on the
       // critical path of the ring (the barrier of the packed rows belongs to this warp alone, so its byte count can
       // be posted while the slot is still being read)
@@ -371,6 +377,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
         // of this kernel are most sensitive to).  The widened rows of the first half lie in the part of the slot
         // that holds no packed bytes; those of the second half cover the packed rows of both, all of which are in
         // registers (or used up) once every lane has loaded its share of the second half.
+        if constexpr (BITS != 8) {
         const uint4* pk_in = reinterpret_cast<const uint4*>(bt + kPackedOff) + lane;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -401,6 +408,7 @@ __device__ __forceinline__ void unpack_role(const Params& p, const Rings& g, int
               *reinterpret_cast<uint4*>(row + (((c0 + h) ^ sw) << 4)) = v;
             }
           }
+        }
         }
         }
       }
@@ -875,36 +883,54 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     const int sub = lane / per_block, half = lane % per_block;
     if (lane < kSub * per_block) {
       RingPos rp{0, 0};
-      int tile = g.pair, ks = 0;
+      // Everything a copy needs is worked out before the wait for its stage (what follows that wait is on the critical
+      // path of the ring): the tile's place once per tile, the filter tap of a reduction block by stepping, not by
+      // dividing.
+      int tile = g.pair - g.npairs, ks = p.ksteps;
+      int m = 0, ttile = 0;
+      int pn = 0, ph0 = 0, pw0 = 0;     // convolution: image and origin of this lane's patch of the tile
+      int chunk = 0, th = 0, tw = 0;    // convolution: 128-channel chunk and filter tap (row, column) of block kb
       for (uint32_t it = 0; it < total_steps; ++it, rp.advance(1, depth), ++ks) {
         if (ks == p.ksteps) {
           ks = 0;
           tile += g.npairs;
+          int cb, tt;
+          locate_tile(p, g.tile_base, tile, m, cb, tt);
+          ttile = 2 * tt + g.rank;   // this CTA's 128 token rows of the pair's tile
+          if (p.f.conv_on) {
+            patch_origin(p, 2 * ttile + half, pn, ph0, pw0);   // a patch index beyond the last one reads zeros (n >= N)
+            const int tap = sub / p.conv_chunks;
+            chunk = sub - tap * p.conv_chunks;
+            th = tap / p.f.ckw;
+            tw = tap - th * p.f.ckw;
+          }
         }
-        int m, cb, tt;
-        locate_tile(p, g.tile_base, tile, m, cb, tt);
-        const int ttile = 2 * tt + g.rank;   // this CTA's 128 token rows of the pair's tile
         const int nsub = min(kSub, p.kblocks - ks * kSub);   // the last stage of a tile may hold one block only
         const int kb = ks * kSub + sub;
+        const uint32_t bar = g.full_lead0 + 8u * rp.slot;
+        const uint32_t dst = g.stage0 + rp.slot * kStageBytes + sub * kABytes + (p.f.conv_on ? half * (kABytes / 2) : 0);
+        // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
+        const int c0 = p.f.conv_on ? chunk * kKStep : kb * kKStep;
+        const int c1 = p.f.conv_on ? p.f.csw * pw0 + tw - p.f.cpw : ttile * kTileM;
+        const int c2 = p.f.csh * ph0 + th - p.f.cph;
+        if (p.f.conv_on) {   // block kb + kSub, for the next stage
+          chunk += kSub;
+          while (chunk >= p.conv_chunks) {
+            chunk -= p.conv_chunks;
+            if (++tw == p.f.ckw) {
+              tw = 0;
+              ++th;
+            }
+          }
+        }
         // (the byte count of the stage barrier must NOT be posted ahead of this wait: the producer runs up to a ring
         // ahead of the MMAs, so the barrier's phase of the slot's use before may still be collecting its arrivals,
         // and an early arrival would be counted into that phase)
         if (!mbar_wait(g.done0 + 8u * rp.slot, rp.phase ^ 1, g.abort_flag, p.f.status)) break;
         if (g.rank == 0 && lane == 0) mbar_expect_tx(g.full0 + 8u * rp.slot, 2 * nsub * kABytes);
         if (sub >= nsub) continue;
-        const uint32_t bar = g.full_lead0 + 8u * rp.slot;
-        const uint32_t dst = g.stage0 + rp.slot * kStageBytes + sub * kABytes;
-        if (!p.f.conv_on) {
-          // rows beyond T read zeros
-          tma_pair_load_2d(dst, &p.tmap_a[m], kb * kKStep, ttile * kTileM, bar);
-        } else {
-          // reduction block kb = (filter tap, 128-channel chunk); the tap shifts the patch window
-          const int tap = kb / p.conv_chunks, chunk = kb - tap * p.conv_chunks;
-          const int dh = tap / p.f.ckw - p.f.cph, dw = tap % p.f.ckw - p.f.cpw;
-          int n, h0, w0;
-          patch_origin(p, 2 * ttile + half, n, h0, w0);   // a patch index beyond the last one reads zeros (n >= N)
-          tma_pair_load_4d(dst + half * (kABytes / 2), &p.tmap_a[m], chunk * kKStep, p.f.csw * w0 + dw, p.f.csh * h0 + dh, n, bar);
-        }
+        if (!p.f.conv_on) tma_pair_load_2d(dst, &p.tmap_a[m], c0, c1, bar);   // rows beyond T read zeros
+        else tma_pair_load_4d(dst, &p.tmap_a[m], c0, c1, c2, pn, bar);
       }
     }
     __syncwarp();
@@ -1071,7 +1097,14 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   for (int m = 0; m < a.num_branches; ++m)
     if (!a.branch[m].blk || !a.branch[m].rec) return PIPE_ERR_UNSUPPORTED;
   if (a.g % 8 != 0) return PIPE_ERR_UNSUPPORTED;
-  if (a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
+  int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
+  for (int m = 0; m < a.num_branches; ++m) {
+    k_lo = min(k_lo, a.branch[m].k_begin);
+    k_hi = max(k_hi, a.branch[m].k_end);
+  }
+  bool direct = true;   // every order of the call has its int8 copy
+  for (int k = k_lo; k < k_hi; ++k) direct = direct && a.order[k].wcodes != nullptr;
+  if (!direct && a.bits == 2 && a.g % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // an unpack item is 16 rows of 2-bit codes and must lie in one order
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.conv_on && a.cC % kKStep != 0) return PIPE_ERR_UNSUPPORTED;
   for (int m = 0; m < a.num_branches; ++m) {
@@ -1080,6 +1113,9 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T > (1ll << 30)) return PIPE_ERR_UNSUPPORTED;
 
   p.f = a;
+  p.direct = direct ? 1 : 0;
+  const int row_bytes = direct ? round_up(a.I, kKStep) : a.kernel_row_bytes;   // bytes of a row over all reduction blocks
+  if (direct) p.f.bits = 8;   // the kernel then treats the layer as one of int8 codes
   p.nkmax = max_cluster;
   p.ntok_tiles = static_cast<int>(ceil_div<int64_t>(a.T, kTileM));
   p.conv_pw = p.conv_pp = p.conv_np = p.conv_chunks = 1;
@@ -1109,26 +1145,22 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
     // bytes one branch sweeps in either order: its activations, or the packed rows of its orders
     const int64_t x_bytes = a.conv_on ? static_cast<int64_t>(a.cN) * a.cH * a.cW * a.cC : a.T * static_cast<int64_t>(a.I);
     int64_t w_bytes = 0;
-    for (int k = a.branch[0].k_begin; k < a.branch[0].k_end; ++k) w_bytes += static_cast<int64_t>(a.order[k].rows) * a.kernel_row_bytes;
+    for (int k = a.branch[0].k_begin; k < a.branch[0].k_end; ++k) w_bytes += static_cast<int64_t>(a.order[k].rows) * row_bytes;
     // (sweeping the activations once per channel block is the better order while they stay in L2 beside the outputs
     // streaming through it -- the pairs working together then share one weight block -- so the other order is taken
     // only for activations of tens of megabytes)
     p.blocks_fastest = (x_bytes > w_bytes && x_bytes > (48ll << 20)) ? 1 : 0;
   }
-  p.pk = kKStep * a.bits / 8;
-  p.shift = 8 - a.bits;
+  p.pk = kKStep * p.f.bits / 8;
+  p.shift = 8 - p.f.bits;
 
-  int k_lo = PIPE_MAX_ORDERS, k_hi = 0;
-  for (int m = 0; m < a.num_branches; ++m) {
-    k_lo = min(k_lo, a.branch[m].k_begin);
-    k_hi = max(k_hi, a.branch[m].k_end);
-  }
-  const uint8_t* kbase = a.order[k_lo].kcodes;
-  for (int k = k_lo; k < k_hi; ++k) kbase = a.order[k].kcodes < kbase ? a.order[k].kcodes : kbase;
+  auto section = [&](int k) { return direct ? a.order[k].wcodes : a.order[k].kcodes; };
+  const uint8_t* kbase = section(k_lo);
+  for (int k = k_lo; k < k_hi; ++k) kbase = section(k) < kbase ? section(k) : kbase;
   p.kbase = kbase;
   for (int k = k_lo; k < k_hi; ++k) {
-    const uint64_t d = static_cast<uint64_t>(a.order[k].kcodes - kbase);
-    const uint64_t end = (d + static_cast<uint64_t>(a.order[k].rows) * a.kernel_row_bytes) >> 4;
+    const uint64_t d = static_cast<uint64_t>(section(k) - kbase);
+    const uint64_t end = (d + static_cast<uint64_t>(a.order[k].rows) * row_bytes) >> 4;
     if ((d & 15) || end >= 0xffffffffull) return PIPE_ERR_UNSUPPORTED;
     p.koff[k] = static_cast<uint32_t>(d >> 4);
   }

@@ -66,9 +66,11 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     return PIPE_ERR_INVALID_ARG;
   if (d->score_mode != PIPE_SCORE_MAXABS && d->score_mode != PIPE_SCORE_L2) return PIPE_ERR_INVALID_ARG;
   if (d->keep_elems < 0 || d->keep_elems > d->in_features) return PIPE_ERR_INVALID_ARG;
+  if (d->int8_copy != 0 && d->int8_copy != 1) return PIPE_ERR_INVALID_ARG;
   if (d->num_orders < 1 || d->num_orders > PIPE_MAX_ORDERS) return PIPE_ERR_INVALID_ARG;
   if (d->group_size < 1) return PIPE_ERR_INVALID_ARG;
   if (d->out_features % d->group_size != 0) return PIPE_ERR_SHAPE;
+  if (d->int8_copy && d->group_size % 8 != 0) return PIPE_ERR_SHAPE;   // kept-row runs must keep the 8-row swizzle atoms whole
   const int container = d->weight_bits == 2 ? 2 : (d->weight_bits <= 4 ? 4 : 8);   // storage format of the codes
   const int per_byte = 8 / container;
   if (d->in_features % per_byte != 0) return PIPE_ERR_SHAPE;
@@ -137,6 +139,11 @@ pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
     off = align_up64(off + static_cast<uint64_t>(L.G + 1) * 4, 1024);
     y.kcodes_off[k] = off;
     off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * y.kernel_row_bytes, 1024);
+    y.wcodes_off[k] = 0;
+    if (d->int8_copy) {
+      y.wcodes_off[k] = off;
+      off = align_up64(off + static_cast<uint64_t>(y.rows[k]) * round_up(L.I, kKernelKAlign), 1024);
+    }
   }
   // channel-block tables: predictors 0..M-1, then the cluster of all K orders
   for (int m = 0; m <= L.M; ++m) {

@@ -15,12 +15,13 @@ from . import synth
 
 class LayerRunner:
     def __init__(self, spec: synth.LayerSpec, device="cuda", distinct_inputs: bool = True, second_layer: bool = False,
-                 implicit_conv: bool = True):
+                 implicit_conv: bool = True, int8_copy: bool = False):
         self.spec = spec
         self.device = torch.device(device)
         G = spec.O // spec.g
         self.n_keep = B.pipe_keep_groups_from_gamma(G, spec.gamma)
-        self.desc = B.make_desc(spec.O, spec.I, spec.bits, spec.K, spec.g, self.n_keep, spec.M)
+        # int8_copy: the blob also keeps the codes as int8 in the tensor-core operand layout (pipe_layer_desc.int8_copy)
+        self.desc = B.make_desc(spec.O, spec.I, spec.bits, spec.K, spec.g, self.n_keep, spec.M, int8_copy=int8_copy)
         self.layout = B.pipe_layout(self.desc)
         self.second_layer = second_layer
         # a convolution workload runs as implicit GEMM on the NHWC tensor when the library takes its shape
@@ -163,7 +164,10 @@ class LayerRunner:
     def forward_bytes(self) -> int:
         """Algorithmic bytes of one forward call: streamed codes + scales + xq + fp32 outputs."""
         lay, s = self.layout, self.spec
-        codes = sum(lay.rows[k] * lay.kernel_row_bytes for k in range(s.K))
+        row_bytes = lay.kernel_row_bytes
+        if self.desc.int8_copy and self.T > 16:      # the kernels for more than 16 tokens read the int8 copy instead
+            row_bytes = (s.I + 127) // 128 * 128
+        codes = sum(lay.rows[k] * row_bytes for k in range(s.K))
         scales = 4 * self.total_rows + 4 * (lay.num_groups + 1) * s.K
         return codes + scales + sum(x.numel() for x in self.xq) + 4 * self.M * self.T * s.O
 
@@ -175,6 +179,8 @@ class LayerRunner:
         for k in range(s.K):
             b += 4 * lay.rows[k] * s.I * (2 if k + 1 < s.K else 1)
             b += lay.rows[k] * (lay.canon_row_bytes + lay.kernel_row_bytes)
+            if self.desc.int8_copy:
+                b += lay.rows[k] * ((s.I + 127) // 128 * 128)
         return b
 
     def quantize_bytes(self) -> int:

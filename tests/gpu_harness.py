@@ -16,8 +16,13 @@ def ensure_built():
     B.lib()
 
 
-def desc_of(O, I, bits, K, g, n_keep, M=1, branch_orders=None):
-    return B.make_desc(O, I, bits, K, g, n_keep, M, branch_orders)
+INT8_COPY_DEFAULT = False   # tests/test_gpu_int8_copy.py runs other modules' cases with this switched on
+
+
+def desc_of(O, I, bits, K, g, n_keep, M=1, branch_orders=None, int8_copy=None):
+    if int8_copy is None:
+        int8_copy = INT8_COPY_DEFAULT and g % 8 == 0
+    return B.make_desc(O, I, bits, K, g, n_keep, M, branch_orders, int8_copy=int8_copy)
 
 
 def gpu_expand(desc, W: np.ndarray) -> B.ExpandedLayer:
@@ -68,7 +73,28 @@ def assert_expansion_matches(layer: B.ExpandedLayer, e, oracle, check_kernel_lay
             np.testing.assert_array_equal(layer.kcodes(k).cpu().numpy(),
                                           kernel_layout_from_codes(e.order_codes(k), 2 if e.bits == 2 else (4 if e.bits <= 4 else 8)),
                                           err_msg=f"streaming layout, order {k}")
+        w = layer.wcodes(k)
+        if layer.desc.int8_copy:
+            np.testing.assert_array_equal(w.cpu().numpy().view(np.int8), int8_copy_from_codes(e.order_codes(k)),
+                                          err_msg=f"int8 copy, order {k}")
+        else:
+            assert w is None
     assert_block_tables_match(layer, e)
+
+
+def int8_copy_from_codes(codes: np.ndarray) -> np.ndarray:
+    """The int8 operand-layout copy (include/pipe.h) from int8 codes [rows, I]: [I_pad / 128, rows, 128], the 16-byte
+    piece c of compacted row r stored as piece c ^ (r & 7)."""
+    rows, I = codes.shape
+    Ipad = (I + 127) // 128 * 128
+    c = np.zeros((rows, Ipad), np.int8)
+    c[:, :I] = codes
+    pieces = c.reshape(rows, Ipad // 128, 8, 16)
+    out = np.zeros_like(pieces)
+    for a in range(8):          # rows with r & 7 == a
+        for p in range(8):
+            out[a::8, :, p ^ a, :] = pieces[a::8, :, p, :]
+    return np.ascontiguousarray(out.transpose(1, 0, 2, 3)).reshape(Ipad // 128, rows, 128)
 
 
 def expected_decode_table(kept_lists, G: int, g: int, row_limit: int, channel_limit: int = 512):

@@ -80,6 +80,37 @@ def test_layout_sections_are_disjoint_and_aligned(lib):
     assert lay2.expand_ws_bytes >= 16 * 200 * 4
 
 
+def test_layout_with_an_int8_copy(lib):
+    plain = B.pipe_layout(B.make_desc(256, 2300, 4, 3, 8, 8, 1))
+    assert all(plain.wcodes_off[k] == 0 for k in range(16))
+    d = B.make_desc(256, 2300, 4, 3, 8, 8, 1, int8_copy=True)
+    lay = B.pipe_layout(d)
+    ipad = 2304
+    spans = []
+    for k in range(3):
+        assert lay.wcodes_off[k] % 1024 == 0 and lay.wcodes_off[k] > 0
+        spans += [(lay.codes_off[k], lay.rows[k] * lay.canon_row_bytes), (lay.scales_off[k], lay.rows[k] * 4),
+                  (lay.kept_off[k], lay.kept_groups[k] * 4), (lay.cum_off[k], 33 * 4),
+                  (lay.kcodes_off[k], lay.rows[k] * lay.kernel_row_bytes), (lay.wcodes_off[k], lay.rows[k] * ipad)]
+    spans += [(lay.blk_off[m], 4 * (lay.blk_cap[m] + 2)) for m in range(2)]
+    spans += [(lay.rec_off[m], B.BLOCK_RECORD_BYTES * lay.rec_cap[m]) for m in range(2)]
+    spans.sort()
+    for (o0, n0), (o1, _) in zip(spans, spans[1:]):
+        assert o0 + n0 <= o1
+    assert spans[-1][0] + spans[-1][1] <= lay.blob_bytes
+    assert lay.blob_bytes >= plain.blob_bytes + sum(lay.rows[k] for k in range(3)) * ipad
+    # the copy keeps 8-row atoms whole, so the group size must be a multiple of 8; the flag is 0 or 1
+    bad = B.make_desc(256, 2304, 4, 3, 4, 8, 1, int8_copy=True)
+    with pytest.raises(B.PipeError) as ex:
+        B.pipe_layout(bad)
+    assert ex.value.status == B.PIPE_ERR_SHAPE
+    bad = B.make_desc(256, 2304, 4, 3, 8, 8, 1)
+    bad.int8_copy = 2
+    with pytest.raises(B.PipeError) as ex:
+        B.pipe_layout(bad)
+    assert ex.value.status == B.PIPE_ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("kwargs,status", [
     (dict(O=0), B.PIPE_ERR_INVALID_ARG), (dict(bits=5), B.PIPE_ERR_INVALID_ARG), (dict(K=17), B.PIPE_ERR_INVALID_ARG),
     (dict(g=7), B.PIPE_ERR_SHAPE), (dict(keep=0), B.PIPE_ERR_INVALID_ARG), (dict(keep=9), B.PIPE_ERR_INVALID_ARG),

@@ -211,12 +211,12 @@ FORWARD_CASES = [
 
 @pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", FORWARD_CASES)
-def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
+def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M, int8_copy=False):
     rng = np.random.default_rng(O + 3 * I + 5 * T)
     W = _w(rng, O, I, heavy=(bits == 2))
     bias = rng.standard_normal(O).astype(np.float32)
     e = oracle.expand(W, bits, K, g, n_keep)
-    d = H.desc_of(O, I, bits, K, g, n_keep, M)
+    d = H.desc_of(O, I, bits, K, g, n_keep, M, int8_copy=int8_copy)
     layer = H.gpu_expand(d, W)
     H.assert_expansion_matches(layer, e, oracle, check_kernel_layout=False)
     split = [layer.layout.branch_orders[m] for m in range(M)]
@@ -257,6 +257,14 @@ def test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
     y_o, _ = oracle.ensemble(e, np.stack([qo[0][0]] * M), [qo[0][1]] * M, split, bias=bias, sum_branches=True)
     np.testing.assert_array_equal(ys[0].view(np.uint32), y_o.view(np.uint32))
     assert (np.abs(ys[0] - f.y64) <= H.REL_TOL * f.yabs + 1e-30).all()
+
+
+@pytest.mark.parametrize("kernel", [B.KERNEL_AUTO, B.KERNEL_TCGEN05_PAIR, B.KERNEL_TCGEN05, B.KERNEL_STREAM])
+@pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", [c for c in FORWARD_CASES if c[5] % 8 == 0])
+def test_forward_with_int8_copy_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
+    """A layer that also keeps its codes as int8 in the tensor-core operand layout: the copy is what the definition
+    says, the kernels that use it (the SM-pair kernel) and those that do not give the oracle's bits."""
+    test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M, int8_copy=True)
 
 
 def test_forward_zero_tokens_and_strided_io(oracle):

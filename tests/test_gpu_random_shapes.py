@@ -32,3 +32,9 @@ def _cases(n, seed):
 def test_random_shapes_match_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M):
     TP.test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M)
     assert B.pipe_poll_status() == B.PIPE_OK
+
+
+@pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", _cases(24, 20231116))
+def test_random_shapes_with_int8_copy_match_oracle(oracle, O, I, T, bits, K, g, n_keep, M):
+    TP.test_forward_matches_oracle(oracle, B.KERNEL_TCGEN05_PAIR, O, I, T, bits, K, g, n_keep, M, int8_copy=True)
+    assert B.pipe_poll_status() == B.PIPE_OK
