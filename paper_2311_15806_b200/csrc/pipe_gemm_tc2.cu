@@ -940,9 +940,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     if (lane == 0 && g.rank == 0 && *g.abort_flag) drain_ring(g.full0, total_steps, p.depth, 20000000ll);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (first CTA of the pair)
-    if (lane == 0 && g.rank == 0) {
+    // The whole warp runs the loop and its waits; one lane issues.  Everything the loop computes is then the same in
+    // all lanes, which lets the compiler keep the descriptors in the warp's uniform registers, where the MMA
+    // instruction takes them from: a loop run by one lane of a diverged warp moves every descriptor there
+    // instruction by instruction, and this thread's instruction count is what paces a layer with a short reduction
+    // axis.
+    if (g.rank == 0) {
       RingPos rp{0, 0};
+      // (the address field of a descriptor is its low 14 bits, in 16-byte units: offsets inside the ring never carry
+      // out of it, so only the low word changes from MMA to MMA)
       const uint64_t adesc0 = smem_desc_sw128(g.stage0), bdesc0 = smem_desc_sw128(g.stage0 + kStageBOff);
+      const uint32_t a_lo = static_cast<uint32_t>(adesc0), a_hi = static_cast<uint32_t>(adesc0 >> 32);
+      const uint32_t b_lo = static_cast<uint32_t>(bdesc0), b_hi = static_cast<uint32_t>(bdesc0 >> 32);
       uint32_t tcount = 0;
       bool ok = true;
       // The stacked rows of a tile (the only tile metadata this role needs) come from the unpack warps, which decode
@@ -955,22 +964,29 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
         uint32_t idesc = 0;
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
         for (int ks = 0; ks < p.ksteps; ++ks, rp.advance(1, depth)) {
-          if (!mbar_wait<true>(g.full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
+          // (a plain wait: these threads read none of the stage's bytes themselves -- the tensor cores of the two SMs
+          // do, for which the writers' proxy fences and the copies' own completion have made them visible)
+          if (!mbar_wait(g.full0 + 8u * rp.slot, rp.phase, g.abort_flag, p.f.status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           // (written by an unpack warp of this CTA before its arrival on the barrier just waited for)
           if (ks == 0) idesc = idesc_i8(2 * kTileM, pair_mma_rows(g.ntot[tcount % kTileRing], p.f.bits));
-          const uint64_t so = static_cast<uint64_t>(rp.slot * (kStageBytes >> 4));
+          const uint32_t so = rp.slot * (kStageBytes >> 4);
           const int nsub = min(kSub, p.kblocks - ks * kSub);
-          for (int sub = 0; sub < nsub; ++sub) {
-            const uint64_t adesc = adesc0 + so + static_cast<uint64_t>(sub * (kABytes >> 4));
-            const uint64_t bdesc = bdesc0 + so + static_cast<uint64_t>(sub * (kBtBytes >> 4));
+          if (lane == 0) {
+            for (int sub = 0; sub < nsub; ++sub) {
+              const uint32_t al = a_lo + so + static_cast<uint32_t>(sub * (kABytes >> 4));
+              const uint32_t bl = b_lo + so + static_cast<uint32_t>(sub * (kBtBytes >> 4));
 #pragma unroll
-            for (int k = 0; k < kKStep / 32; ++k)
-              mma_i8_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 2), idesc, (ks | sub | k) != 0);
+              for (int k = 0; k < kKStep / 32; ++k)
+                mma_i8_pair(d_tmem, (static_cast<uint64_t>(a_hi) << 32) | (al + 2u * k), (static_cast<uint64_t>(b_hi) << 32) | (bl + 2u * k), idesc,
+                            (ks | sub | k) != 0);
+            }
+            mma_commit_pair(g.done0 + 8u * rp.slot);   // frees the stage for the producers of both CTAs
           }
-          mma_commit_pair(g.done0 + 8u * rp.slot);   // frees the stage for the producers of both CTAs
+          __syncwarp();
         }
-        if (ok) mma_commit_pair(g.tfull0 + 8u * buf);
+        if (ok && lane == 0) mma_commit_pair(g.tfull0 + 8u * buf);
+        __syncwarp();
       }
     }
   } else if (warp < 2 + kUnpackWarps) {
