@@ -98,6 +98,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_lead(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// One lane of a converged warp (the form the compiler recognises as "one thread of a uniform warp").
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -940,7 +946,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     if (lane == 0 && g.rank == 0 && *g.abort_flag) drain_ring(g.full0, total_steps, p.depth, 20000000ll);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (first CTA of the pair)
-    // The whole warp runs the loop and its waits; one lane issues.  Everything the loop computes is then the same in
+    // The whole warp runs the loop and its waits; one elected lane issues.  Everything the loop computes is then the same in
     // all lanes, which lets the compiler keep the descriptors in the warp's uniform registers, where the MMA
     // instruction takes them from: a loop run by one lane of a diverged warp moves every descriptor there
     // instruction by instruction, and this thread's instruction count is what paces a layer with a short reduction
@@ -972,7 +978,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
           if (ks == 0) idesc = idesc_i8(2 * kTileM, pair_mma_rows(g.ntot[tcount % kTileRing], p.f.bits));
           const uint32_t so = rp.slot * (kStageBytes >> 4);
           const int nsub = min(kSub, p.kblocks - ks * kSub);
-          if (lane == 0) {
+          if (elect_one()) {
             for (int sub = 0; sub < nsub; ++sub) {
               const uint32_t al = a_lo + so + static_cast<uint32_t>(sub * (kABytes >> 4));
               const uint32_t bl = b_lo + so + static_cast<uint32_t>(sub * (kBtBytes >> 4));
@@ -985,7 +991,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
           }
           __syncwarp();
         }
-        if (ok && lane == 0) mma_commit_pair(g.tfull0 + 8u * buf);
+        if (ok && elect_one()) mma_commit_pair(g.tfull0 + 8u * buf);
         __syncwarp();
       }
     }

@@ -1,6 +1,6 @@
 """Run the forward call of one benchmark configuration a few times (for profilers and quick looks).
 
-    python -m paper_2311_15806_b200.run_case cfg2 [--launches 3] [--kernel K]
+    python -m paper_2311_15806_b200.run_case cfg2 [--launches 3] [--kernel K] [--int8-copy]
 
 Loads the seeded synthetic layer, expands the weights, quantizes the activations and launches the expanded GEMM
 `--launches` times; prints the CUDA-event time of the last launch.  Nothing is checked here: parity lives in tests/.
@@ -22,11 +22,13 @@ def main() -> None:
     ap.add_argument("workload")
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--kernel", type=int, default=0, help="force a GEMM kernel (pipe_diag_select_kernel)")
+    ap.add_argument("--int8-copy", action="store_true",
+                    help="the layer also keeps its codes as int8 in the tensor-core operand layout (pipe_layer_desc.int8_copy)")
     args = ap.parse_args()
     pipe_build.build()
     B.lib()
     spec = synth.paper_workloads()[args.workload]
-    run = LayerRunner(spec)
+    run = LayerRunner(spec, int8_copy=args.int8_copy)
     run.load()
     run.expand()
     run.quantize()
