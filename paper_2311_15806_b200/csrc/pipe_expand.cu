@@ -57,23 +57,19 @@ __global__ void group_score_kernel(const float* __restrict__ a, int G, int g, fl
 // result does not depend on any reduction order.
 template <typename S>
 __global__ void group_rank_kernel(const S* __restrict__ score, int G, int n_keep, int32_t* __restrict__ keep) {
-  __shared__ S tile[1024];
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  const S sj = j < G ? score[j] : S(0);
+  // one warp per group: its lanes share the G comparisons (a count, so the order of the additions does not matter)
+  const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (j >= G) return;
+  const S sj = score[j];
   int rank = 0;
-  for (int base = 0; base < G; base += 1024) {
-    const int n = min(1024, G - base);
-    __syncthreads();
-    for (int t = threadIdx.x; t < n; t += blockDim.x) tile[t] = score[base + t];
-    __syncthreads();
-    if (j < G) {
-      for (int t = 0; t < n; ++t) {
-        const S si = tile[t];
-        rank += (si > sj) || (si == sj && base + t < j);
-      }
-    }
+  for (int t = lane; t < G; t += 32) {
+    const S si = score[t];
+    rank += (si > sj) || (si == sj && t < j);
   }
-  if (j < G) keep[j] = rank < n_keep ? 1 : 0;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, d);
+  if (lane == 0) keep[j] = rank < n_keep ? 1 : 0;
 }
 
 // Second score of the structured mask (PIPE_SCORE_L2): the squared Euclidean norm of the group's residual rows in
@@ -185,27 +181,57 @@ __global__ void __launch_bounds__(1024) group_compact_kernel(const int32_t* __re
 // Group selection of one order in ONE block, for layers of up to kFusedGroups groups: scores, ranks and
 // the compacted list stay in shared memory (three tiny launches less per sparse order).  Same rule and
 // same exact comparisons as the three kernels above.
-constexpr int kFusedGroups = 512;   // one group per thread: the ranking is G comparisons per thread
+constexpr int kFusedGroups = 512;   // one group per thread; a power of two (the sorting network's size)
 __global__ void __launch_bounds__(kFusedGroups) group_select_kernel(const float* __restrict__ a, int G, int g, int n_keep,
                                                             int32_t* __restrict__ cum, int32_t* __restrict__ kept) {
-  __shared__ float score[kFusedGroups];
+  // Rank = position in the order (score descending, index ascending), found by sorting the keys
+  // (score bits, ~index) in descending order: scores are non-negative floats, whose order is the order of their bit
+  // patterns, so the keys are distinct integers and the sorted order is unique (a bitonic network of 45 rounds over
+  // the 512 slots; slots beyond G hold the smallest key and end up last).
+  __shared__ unsigned long long key[kFusedGroups];
   __shared__ int32_t flag[kFusedGroups];
   __shared__ int32_t chunk_sum[kFusedGroups];
-  for (int j = threadIdx.x; j < G; j += blockDim.x) {
-    float m = 0.f;
-    for (int u = 0; u < g; ++u) m = fmaxf(m, a[static_cast<int64_t>(j) * g + u]);
-    score[j] = m;
+  const int tid = threadIdx.x;
+  {
+    unsigned long long kv = 0ull;
+    if (tid < G) {
+      // the group's row maxima: independent loads (four at a time where the rows allow vector loads)
+      const float* rows = a + static_cast<int64_t>(tid) * g;
+      float m0 = 0.f, m1 = 0.f, m2 = 0.f, m3 = 0.f;
+      int u = 0;
+      if ((g & 3) == 0 && (reinterpret_cast<uintptr_t>(rows) & 15) == 0) {
+#pragma unroll 4
+        for (; u < g; u += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(rows + u);
+          m0 = fmaxf(m0, v.x);
+          m1 = fmaxf(m1, v.y);
+          m2 = fmaxf(m2, v.z);
+          m3 = fmaxf(m3, v.w);
+        }
+      }
+#pragma unroll 4
+      for (; u < g; ++u) m0 = fmaxf(m0, rows[u]);
+      const float m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      kv = (static_cast<unsigned long long>(__float_as_uint(m)) << 32) | (0xffffffffu - static_cast<uint32_t>(tid));
+    }
+    key[tid] = kv;
   }
   __syncthreads();
-  for (int j = threadIdx.x; j < G; j += blockDim.x) {
-    const float sj = score[j];
-    int rank = 0;
-    for (int t = 0; t < G; ++t) {
-      const float si = score[t];
-      rank += (si > sj) || (si == sj && t < j);
+  for (int k = 2; k <= kFusedGroups; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      const int other = tid ^ j;
+      if (other > tid) {
+        const unsigned long long x = key[tid], y = key[other];
+        const bool descending = (tid & k) == 0;
+        if (descending ? x < y : x > y) {
+          key[tid] = y;
+          key[other] = x;
+        }
+      }
+      __syncthreads();
     }
-    flag[j] = rank < n_keep ? 1 : 0;
   }
+  if (tid < G) flag[0xffffffffu - static_cast<uint32_t>(key[tid])] = tid < n_keep ? 1 : 0;
   __syncthreads();
   const int per = (G + blockDim.x - 1) / blockDim.x;
   const int b = threadIdx.x * per, e = min(G, b + per);
@@ -467,44 +493,91 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
 // when the next group would take its stacked rows beyond PIPE_BLOCK_ROWS or its channels beyond PIPE_BLOCK_CHANNELS.
 // One thread block per cluster: all threads gather the rows every group stacks (kept orders of the cluster only),
 // thread 0 then cuts the blocks.
+constexpr int kTableSets = 2 * (PIPE_MAX_ORDERS + 1);   // channel-block tables, then decode-unit tables
 struct BlockTableArgs {
-  const int32_t* cum[PIPE_MAX_ORDERS + 1][8];   // prefix counts of the cluster's orders
-  int nk[PIPE_MAX_ORDERS + 1];
-  int32_t* out[PIPE_MAX_ORDERS + 1];
-  int cap[PIPE_MAX_ORDERS + 1];
-  int limit[PIPE_MAX_ORDERS + 1];   // rows a block of the cluster may stack
+  const int32_t* cum[kTableSets][8];   // prefix counts of the cluster's orders
+  int nk[kTableSets];
+  int32_t* out[kTableSets];
+  int cap[kTableSets];
+  int limit[kTableSets];   // rows a block of the cluster may stack
   int G, g;
 };
 
 constexpr int kTableChunk = 2048;
+constexpr int kTableThreads = 256;
 
-__global__ void block_table_kernel(const __grid_constant__ BlockTableArgs a) {
-  __shared__ int rows_s[kTableChunk];
+// One thread block per table.  The groups are taken in chunks: all threads gather the rows every group of the chunk
+// stacks (kept orders of the cluster only) and form their running sums; the first warp then cuts the blocks.  The
+// greedy rule "close the block when the next group would take it beyond the limit" needs, for a block that starts at
+// group b, the first group whose running sum from b exceeds the limit (or that would be the block's max_groups + 1-th):
+// the sums are non-decreasing, so the lanes test 32 candidates at a time and the first hit is the cut.
+__global__ void __launch_bounds__(kTableThreads) block_table_kernel(const __grid_constant__ BlockTableArgs a) {
+  __shared__ int pre_s[kTableChunk];            // inclusive running sum of the chunk's rows
+  __shared__ int part_s[kTableThreads];
   const int m = blockIdx.x;
   int32_t* out = a.out[m];
   if (!out) return;
-  int cur_rows = 0, cur_groups = 0, n = 0;
+  int cur_rows = 0, cur_groups = 0, n = 0;      // (warp 0: the same in every lane)
   const int max_groups = PIPE_BLOCK_CHANNELS / a.g > 0 ? PIPE_BLOCK_CHANNELS / a.g : 1;
+  const int lane = threadIdx.x & 31;
+  constexpr int kPer = kTableChunk / kTableThreads;
   for (int base = 0; base < a.G; base += kTableChunk) {
     const int cnt = min(kTableChunk, a.G - base);
-    for (int j = threadIdx.x; j < cnt; j += blockDim.x) {
-      int r = 0;
-      for (int q = 0; q < a.nk[m]; ++q) r += (a.cum[m][q][base + j + 1] - a.cum[m][q][base + j]) * a.g;
-      rows_s[j] = r;
+    // rows of this thread's kPer consecutive groups, then a scan of the threads' totals
+    int r[kPer];
+    int tot = 0;
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) {
+      const int j = threadIdx.x * kPer + u;
+      int v = 0;
+      if (j < cnt)
+        for (int q = 0; q < a.nk[m]; ++q) v += (a.cum[m][q][base + j + 1] - a.cum[m][q][base + j]) * a.g;
+      tot += v;
+      r[u] = tot;
+    }
+    part_s[threadIdx.x] = tot;
+    __syncthreads();
+    for (int d = 1; d < kTableThreads; d <<= 1) {
+      const int v = threadIdx.x >= d ? part_s[threadIdx.x - d] : 0;
+      __syncthreads();
+      part_s[threadIdx.x] += v;
+      __syncthreads();
+    }
+    const int before = threadIdx.x == 0 ? 0 : part_s[threadIdx.x - 1];
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) {
+      const int j = threadIdx.x * kPer + u;
+      if (j < cnt) pre_s[j] = before + r[u];
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      if (base == 0) out[1] = 0;
-      for (int j = 0; j < cnt; ++j) {
-        const int r = rows_s[j];
-        if (cur_groups > 0 && (cur_rows + r > a.limit[m] || cur_groups + 1 > max_groups)) {
-          if (n < a.cap[m]) out[2 + n] = base + j;   // (the capacity bound holds by construction; never write past it)
-          ++n;
-          cur_rows = 0;
-          cur_groups = 0;
+    if (threadIdx.x < 32) {
+      if (base == 0 && lane == 0) out[1] = 0;
+      int pos = 0, s0 = 0;   // next group of the chunk to place; running sum before it
+      while (pos < cnt) {
+        for (int off = 0;; off += 32) {
+          const int c = pos + off + lane;
+          const bool valid = c < cnt;
+          const int rsum = valid ? pre_s[c] - s0 : 0;   // rows of the groups pos .. c
+          const int ng = cur_groups + off + lane;       // groups of the block before c
+          const bool cut = valid && ng > 0 && (cur_rows + rsum > a.limit[m] || ng + 1 > max_groups);
+          const unsigned hit = __ballot_sync(0xffffffffu, cut);
+          if (hit) {
+            const int f = off + __ffs(hit) - 1;         // group pos + f opens the next block
+            if (lane == 0 && n < a.cap[m]) out[2 + n] = base + pos + f;   // (the capacity bound holds by construction; never write past it)
+            ++n;
+            cur_rows = 0;
+            cur_groups = 0;
+            pos += f;
+            s0 = pos > 0 ? pre_s[pos - 1] : 0;
+            break;
+          }
+          if (pos + off + 32 >= cnt) {                  // the rest of the chunk joins the block under construction
+            cur_rows += pre_s[cnt - 1] - s0;
+            cur_groups += cnt - pos;
+            pos = cnt;
+            break;
+          }
         }
-        cur_rows += r;
-        ++cur_groups;
       }
     }
     __syncthreads();
@@ -662,11 +735,11 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
         // (a sparse order is never the first, so the current residual is in the workspace)
         row_sumsq_kernel<<<ceil_div(L.O, 8), 256, 0, s>>>(resid, I4, L.O, L.I, rowsq);
         group_score_l2_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(rowsq, L.G, L.g, score64);
-        group_rank_kernel<double><<<ceil_div(L.G, 256), 256, 0, s>>>(score64, L.G, L.n_keep, keep);
+        group_rank_kernel<double><<<ceil_div(L.G, 8), 256, 0, s>>>(score64, L.G, L.n_keep, keep);
         count_launch(3);
       } else if (!dense) {
         group_score_kernel<<<ceil_div(L.G, 256), 256, 0, s>>>(a, L.G, L.g, score);
-        group_rank_kernel<float><<<ceil_div(L.G, 256), 256, 0, s>>>(score, L.G, L.n_keep, keep);
+        group_rank_kernel<float><<<ceil_div(L.G, 8), 256, 0, s>>>(score, L.G, L.n_keep, keep);
         count_launch(2);
       }
       group_compact_kernel<<<1, 1024, 0, s>>>(dense ? nullptr : keep, L.G, cum, kept);
@@ -704,27 +777,41 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
     count_launch(1);
   }
   {
+    // channel-block tables (entries 0 .. M) and decode-unit tables (entries M + 1 .. 2 M + 1: the same cut with the
+    // layout's row limits) in one launch, one thread block per table
     BlockTableArgs t;
     std::memset(&t, 0, sizeof(t));
     t.G = L.G;
     t.g = L.g;
-    bool any = false;
+    bool any = false, any_blk = false;
     for (int m = 0; m <= L.M; ++m) {
-      if (L.lay.blk_off[m] == 0) continue;
       const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
-      t.nk[m] = k1 - k0;
-      for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
-      t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.blk_off[m]);
-      t.cap[m] = L.lay.blk_cap[m];
-      // even blocks: the fewest blocks that could hold the cluster's rows, their mean size plus one group of slack
-      int64_t R = 0;
-      for (int k = k0; k < k1; ++k) R += L.lay.rows[k];
-      t.limit[m] = block_row_limit(R, L.O, k1 - k0, L.g);
-      any = true;
+      if (L.lay.blk_off[m] != 0) {
+        t.nk[m] = k1 - k0;
+        for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
+        t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.blk_off[m]);
+        t.cap[m] = L.lay.blk_cap[m];
+        // even blocks: the fewest blocks that could hold the cluster's rows, their mean size plus one group of slack
+        int64_t R = 0;
+        for (int k = k0; k < k1; ++k) R += L.lay.rows[k];
+        t.limit[m] = block_row_limit(R, L.O, k1 - k0, L.g);
+        any = any_blk = true;
+      }
+      if (L.lay.dec_off[m] != 0) {
+        const int e = L.M + 1 + m;
+        t.nk[e] = k1 - k0;
+        for (int q = 0; q < k1 - k0; ++q) t.cum[e][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
+        t.out[e] = reinterpret_cast<int32_t*>(blob + L.lay.dec_off[m]);
+        t.cap[e] = L.G;
+        t.limit[e] = L.lay.dec_limit[m];
+        any = true;
+      }
     }
     if (any) {
-      block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
+      block_table_kernel<<<2 * (L.M + 1), kTableThreads, 0, s>>>(t);
       count_launch(1);
+    }
+    if (any_blk) {
       // the records of the blocks just cut
       BlockRecordArgs r;
       std::memset(&r, 0, sizeof(r));
@@ -748,23 +835,6 @@ extern "C" pipe_status pipe_expand_weights(const pipe_layer_desc* desc, const fl
         block_record_kernel<<<dim3(max_cap, L.M + 1), 256, 0, s>>>(r);
         count_launch(1);
       }
-    }
-    // the decode-unit tables: the same cut with the layout's row limits
-    any = false;
-    for (int m = 0; m <= L.M; ++m) {
-      t.out[m] = nullptr;
-      if (L.lay.dec_off[m] == 0) continue;
-      const int k0 = (m < L.M) ? L.branch_begin[m] : 0, k1 = (m < L.M) ? L.branch_begin[m + 1] : L.K;
-      t.nk[m] = k1 - k0;
-      for (int q = 0; q < k1 - k0; ++q) t.cum[m][q] = reinterpret_cast<const int32_t*>(blob + L.lay.cum_off[k0 + q]);
-      t.out[m] = reinterpret_cast<int32_t*>(blob + L.lay.dec_off[m]);
-      t.cap[m] = L.G;
-      t.limit[m] = L.lay.dec_limit[m];
-      any = true;
-    }
-    if (any) {
-      block_table_kernel<<<L.M + 1, 256, 0, s>>>(t);
-      count_launch(1);
     }
   }
   mark_expansion(s);   // a forward call that follows on this stream must not read the blob ahead of its dependency wait
