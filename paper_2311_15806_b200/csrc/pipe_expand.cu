@@ -369,7 +369,6 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
     // to their places in both layouts and the lanes OR their parts together.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int h = lane & (LPW - 1);
-    const uint32_t fmask = (1u << BITS) - 1u;
     for (int base = warp * 512; base < I_pad; base += nwarps * 512) {
       float4 v[4];
 #pragma unroll
@@ -382,24 +381,42 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
       for (int w = 0; w < 4; ++w) {
         const int e0 = base + w * 128 + lane * 4;
         float x[4] = {v[w].x, v[w].y, v[w].z, v[w].w};
-        uint32_t cc = 0, ck = 0;
         uint32_t f4[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           float c = 0.f;
-          const uint32_t key = abs_key(x[j]);
-          if (s != 0.f && (!masked || key > mthr || (key == mthr && e0 + j <= mcut))) {
+          bool take = s != 0.f;
+          if (masked) {
+            const uint32_t key = abs_key(x[j]);
+            take = take && (key > mthr || (key == mthr && e0 + j <= mcut));
+          }
+          if (take) {
             c = rintf(__fdiv_rn(x[j], s));         // round half to even
             c = fminf(fmaxf(c, -fq), fq);
             x[j] = __fmaf_rn(-s, c, x[j]);         // exact new residual, rounded once
           }
           m = max(m, abs_key(x[j]));
           f4[j] = static_cast<uint32_t>(static_cast<int>(c));
-          const uint32_t f = f4[j] & fmask;
-          cc |= f << (BITS * (4 * h + j));          // canonical: field e at bit e * b of the stream
-          ck |= f << (8 * j + BITS * h);            // streaming layout: see include/pipe.h
         }
         if (dst && e0 < I) *reinterpret_cast<float4*>(dst + e0) = make_float4(x[0], x[1], x[2], x[3]);
+        // The four codes as the four bytes of a word, then both packed layouts from that word with masks and shifts
+        // on all four fields at once.  Canonical: field e at bit e * b of the stream (this lane's four fields are
+        // e = 4 h + j); streaming layout: field 4 h + j at bit 8 j + b h (see include/pipe.h).
+        const uint32_t wv = __byte_perm(__byte_perm(f4[0], f4[1], 0x0040), __byte_perm(f4[2], f4[3], 0x0040), 0x5410);
+        uint32_t cc, ck;
+        if (BITS == 8) {
+          cc = ck = wv;
+        } else if (BITS == 4) {
+          const uint32_t t = wv & 0x0F0F0F0Fu;
+          const uint32_t u = (t | (t >> 4)) & 0x00FF00FFu;
+          cc = ((u | (u >> 8)) & 0xFFFFu) << (16 * h);
+          ck = t << (4 * h);
+        } else {
+          const uint32_t t = wv & 0x03030303u;
+          const uint32_t u = (t | (t >> 6)) & 0x000F000Fu;
+          cc = ((u | (u >> 12)) & 0xFFu) << (8 * h);
+          ck = t << (2 * h);
+        }
 #pragma unroll
         for (int d = 1; d < LPW; d <<= 1) {
           cc |= __shfl_xor_sync(0xffffffffu, cc, d);
@@ -408,7 +425,6 @@ __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const Quanti
         if (p.wcodes && e0 < I_pad) {
           // the lane's four codes are four bytes of piece (e0 & 127) / 16 of the row's block, which is stored as piece
           // ((e0 & 127) / 16) ^ (n & 7)
-          const uint32_t wv = __byte_perm(__byte_perm(f4[0], f4[1], 0x0040), __byte_perm(f4[2], f4[3], 0x0040), 0x5410);
           uint8_t* wdst = p.wcodes + (static_cast<int64_t>(e0 >> 7) * p.rows + n) * 128 + (((((e0 & 127) >> 4) ^ (n & 7)) << 4) | (e0 & 15));
           *reinterpret_cast<uint32_t*>(wdst) = wv;
         }
