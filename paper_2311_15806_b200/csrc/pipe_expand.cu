@@ -316,7 +316,7 @@ struct QuantizeRowsArgs {
 
 // One block per compacted row: Eq. 1 on the residual, then the residual update of Eq. 3.
 template <int BITS>
-__global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const QuantizeRowsArgs p) {
+__global__ void __launch_bounds__(kRowThreads, 5) quantize_rows_kernel(const QuantizeRowsArgs p) {
   const int n = blockIdx.x;
   const int o = p.kept[n / p.g] * p.g + n % p.g;
   const float* src = p.src + static_cast<int64_t>(o) * p.ld_src;
