@@ -35,6 +35,7 @@ int kernel_choice();
 // to read): an expansion marks its stream, every other call on a stream takes the mark away and learns whether it was there.
 void mark_expansion(cudaStream_t stream);
 bool take_expansion_mark(cudaStream_t stream);
+bool expansion_marked(cudaStream_t stream);   // the same question without clearing the mark
 
 inline pipe_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PIPE_OK : PIPE_ERR_CUDA; }
 

@@ -8,6 +8,9 @@ static const int32_t* block_table(const LayerInfo& L, const void* d_blob, int m)
   return L.lay.blk_off[m] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.blk_off[m]) : nullptr;
 }
 
+static pipe_status dispatch_forward(const ForwardArgs& a, const LayerInfo& L, int M, int64_t T, const int32_t* const* zp,
+                                    cudaStream_t stream);
+
 static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, const int8_t* const* xq,
                                const float* const* sx, float* const* y, const int* k_begin, const int* k_end,
                                int64_t T, int64_t ldxq, int64_t ldy, const float* d_bias, int sum_branches,
@@ -57,7 +60,7 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     b.dec = L.lay.dec_off[set] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.dec_off[set]) : nullptr;
   }
   a.decode_split = (M == 1 && k_end[0] - k_begin[0] == L.K) ? L.lay.decode_split_all : L.lay.decode_split;
-  a.blob_settled = take_expansion_mark(stream) ? 0 : 1;
+  a.blob_settled = expansion_marked(stream) ? 0 : 1;   // (the mark is cleared once this call has queued a kernel)
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = T; a.ldxq = ldxq; a.ldy = ldy;
   a.bias = d_bias;
@@ -74,6 +77,13 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
   a.relu = relu;
   a.ldyq = ldyq;
 
+  const pipe_status st = dispatch_forward(a, L, M, T, zp, stream);
+  if (st == PIPE_OK && T > 0) take_expansion_mark(stream);   // this call's kernels now stand behind the expansion
+  return st;
+}
+
+static pipe_status dispatch_forward(const ForwardArgs& a, const LayerInfo& L, int M, int64_t T, const int32_t* const* zp,
+                                    cudaStream_t stream) {
   const int choice = kernel_choice();
   if (zp) {   // asymmetric codes: the CUDA-core kernel folds the zero point in (the others decline)
     if (static_cast<int64_t>(255) * L.qmax * L.I >= (static_cast<int64_t>(1) << 31)) return PIPE_ERR_ACC_OVERFLOW;
@@ -228,7 +238,7 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
     b.out_scale = q8 ? out_scale[m] : nullptr;
   }
   a.decode_split = 0;
-  a.blob_settled = take_expansion_mark(static_cast<cudaStream_t>(stream)) ? 0 : 1;
+  a.blob_settled = expansion_marked(static_cast<cudaStream_t>(stream)) ? 0 : 1;
   a.q8_out = q8 ? 1 : 0;
   a.relu = relu;
   a.ldyq = ldyq;
@@ -248,10 +258,14 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
   a.ckh = geom->kernel_h; a.ckw = geom->kernel_w; a.cph = geom->pad_h; a.cpw = geom->pad_w;
   a.cHo = Ho; a.cWo = Wo; a.csh = sh; a.csw = sw;
   const int choice = kernel_choice();
-  if (choice == 4) return forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
-  if (choice == 2) return forward_tcgen05(a, static_cast<cudaStream_t>(stream));
-  pipe_status cst = forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
-  if (cst == PIPE_ERR_UNSUPPORTED) cst = forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  pipe_status cst;
+  if (choice == 4) cst = forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
+  else if (choice == 2) cst = forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  else {
+    cst = forward_tcgen05_pair(a, static_cast<cudaStream_t>(stream));
+    if (cst == PIPE_ERR_UNSUPPORTED) cst = forward_tcgen05(a, static_cast<cudaStream_t>(stream));
+  }
+  if (cst == PIPE_OK && a.T > 0) take_expansion_mark(static_cast<cudaStream_t>(stream));
   return cst;
 }
 

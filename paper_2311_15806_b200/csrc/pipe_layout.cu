@@ -44,6 +44,14 @@ bool take_expansion_mark(cudaStream_t stream) {
   return false;
 }
 
+bool expansion_marked(cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_mark_mutex);
+  if (g_mark_overflow) return true;
+  for (int i = 0; i < g_num_marked; ++i)
+    if (g_marked[i] == stream) return true;
+  return false;
+}
+
 int* device_status_word() {
   // The symbol is per device; its address is looked up once for whichever device is current and kept.
   constexpr int kMaxDevices = 64;

@@ -316,9 +316,11 @@ extern "C" pipe_status pipe_quantize_act(const float* d_x, int64_t T, int32_t I,
       (reinterpret_cast<uintptr_t>(d_sx) & 3))
     return PIPE_ERR_ALIGNMENT;
   if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
-  take_expansion_mark(static_cast<cudaStream_t>(stream));   // (this call's kernels now stand between an expansion and what follows)
-  return quantize_act_impl(d_x, T, I, ldx, d_static_scale, d_xq, ldxq, d_sx, static_cast<uint32_t*>(d_ws),
-                           static_cast<cudaStream_t>(stream));
+  const pipe_status st = quantize_act_impl(d_x, T, I, ldx, d_static_scale, d_xq, ldxq, d_sx, static_cast<uint32_t*>(d_ws),
+                                           static_cast<cudaStream_t>(stream));
+  // (this call's kernels now stand between an expansion and what follows)
+  if (st == PIPE_OK) take_expansion_mark(static_cast<cudaStream_t>(stream));
+  return st;
 }
 
 extern "C" pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t I, int64_t ldx, int32_t act_bits,
@@ -337,9 +339,9 @@ extern "C" pipe_status pipe_quantize_act_ex(const float* d_x, int64_t T, int32_t
     return PIPE_ERR_ALIGNMENT;
   if (ws_bytes < 256) return PIPE_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  take_expansion_mark(s);
   int* status = device_status_word();
   if (!status) return PIPE_ERR_CUDA;
+  take_expansion_mark(s);   // (kernels follow: they stand between an expansion and what comes next on the stream)
   if (T == 0) {
     act_empty_ex_kernel<<<1, 32, 0, s>>>(d_static_scale, d_sx, d_zp);
     count_launch(1);

@@ -35,8 +35,20 @@ def test_forward_directly_behind_an_expansion_sees_its_blob(oracle, O, I, T, bit
     Wd = [torch.from_numpy(w).cuda() for w in Ws]
     ys = [torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda") for _ in Ws]
     torch.cuda.synchronize()
+    zp = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(M)]
+    scratch_y = [torch.empty((T, O), dtype=torch.float32, device="cuda") for _ in range(M)]
     for r in range(len(Ws)):
         B.pipe_expand_weights(d, Wd[r], blob, ws)
+        if r % 2 == 1:
+            # a forward call that is refused after it has looked at its arguments (a zero point with a back end forced
+            # that takes none) queues nothing, so it must not count as "something stands behind the expansion now"
+            B.pipe_diag_select_kernel(B.KERNEL_STREAM)
+            try:
+                with pytest.raises(B.PipeError) as ex:
+                    B.pipe_ensemble_forward_zp(d, blob, [xq] * M, [sx] * M, zp, scratch_y, None, False, None)
+                assert ex.value.status == B.PIPE_ERR_UNSUPPORTED
+            finally:
+                B.pipe_diag_select_kernel(B.KERNEL_AUTO)
         if M == 1:
             B.pipe_expanded_linear(d, blob, xq, sx, ys[r], None, None)
         else:
