@@ -367,7 +367,10 @@ pipe_status pipe_expanded_linear(const pipe_layer_desc* desc, const void* d_blob
  * only after the last layer.  One layer of all M predictors as ONE grouped launch.
  * h_xq_m, h_sx_m, h_y_m: HOST arrays of M device pointers (int8 [T,I] pitch ldxq; 1 float;
  * float [T,O] pitch ldy); inputs may alias (shared input, the first layer of a network).
- * sum_branches != 0: only h_y_m[0] is written, with ((y_1 + y_2) + ...) + y_M.
+ * sum_branches != 0: only h_y_m[0] is written, with ((y_1 + y_2) + ...) + y_M, every y_m being predictor m's own
+ * chain from zero (the bias closing y_1).  Predictors that share input and step (the same pointers) run as one launch
+ * for more than 16 tokens when the layer has the channel-block table of all K orders (K <= 8): the sums are formed in
+ * registers; with distinct inputs it is one launch per predictor, in order, each adding into h_y_m[0].
  * d_partials as in pipe_expanded_linear.
  */
 pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,
@@ -457,7 +460,8 @@ pipe_status pipe_expanded_conv2d_q8(const pipe_layer_desc* desc, const pipe_conv
  * pipe_expanded_conv2d (geometry, layouts, alignment) and pipe_ensemble_forward (bias with predictor 0 only;
  * sum_branches != 0: the predictors' outputs are added in ascending m into h_y_m[0], each by the thread that wrote it;
  * otherwise predictor m writes h_y_m[m]; d_partials covers all K orders, each from its own predictor's input).
- * h_* are host arrays of num_branches device pointers.  One grouped launch unless sum_branches is set.
+ * h_* are host arrays of num_branches device pointers.  One grouped launch; with sum_branches one launch if the
+ * predictors share input and step (see pipe_ensemble_forward), one per predictor otherwise.
  */
 pipe_status pipe_ensemble_conv2d(const pipe_layer_desc* desc, const pipe_conv_geom* geom, const void* d_blob,
                                  const int8_t* const* h_xq_m, const float* const* h_sx_m, const float* d_bias,

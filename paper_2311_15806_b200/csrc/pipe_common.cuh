@@ -188,6 +188,10 @@ struct ForwardArgs {
   int blob_settled;   // the library's last call on this stream was no expansion: a kernel launched with programmatic stream
                       // serialization may read the expanded layer before it waits for the launch before it
   int q8_out, relu;   // relu: the activation kind (see apply_activation; the name is from the first version)
+  // the channel-block table and block records of the cluster of ALL orders, for a summed ensemble whose predictors
+  // share one input (nullptr: the layer has none, or the call is no such ensemble)
+  const int32_t* sum_blk;
+  const uint8_t* sum_rec;
   int64_t ldyq;
 };
 

@@ -60,6 +60,12 @@ static pipe_status run_forward(const LayerInfo& L, const void* d_blob, int M, co
     b.dec = L.lay.dec_off[set] ? reinterpret_cast<const int32_t*>(static_cast<const uint8_t*>(d_blob) + L.lay.dec_off[set]) : nullptr;
   }
   a.decode_split = (M == 1 && k_end[0] - k_begin[0] == L.K) ? L.lay.decode_split_all : L.lay.decode_split;
+  a.sum_blk = nullptr;
+  a.sum_rec = nullptr;
+  if (sum_branches && M > 1 && L.lay.rec_off[L.M]) {
+    a.sum_blk = block_table(L, d_blob, L.M);
+    a.sum_rec = static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[L.M];
+  }
   a.blob_settled = expansion_marked(stream) ? 0 : 1;   // (the mark is cleared once this call has queued a kernel)
   a.O = L.O; a.I = L.I; a.bits = L.bits; a.g = L.g; a.G = L.G;
   a.T = T; a.ldxq = ldxq; a.ldy = ldy;
@@ -238,6 +244,12 @@ static pipe_status run_conv(const pipe_layer_desc* desc, const pipe_conv_geom* g
     b.out_scale = q8 ? out_scale[m] : nullptr;
   }
   a.decode_split = 0;
+  a.sum_blk = nullptr;
+  a.sum_rec = nullptr;
+  if (sum_branches && M > 1 && !all_orders && L.lay.rec_off[L.M]) {
+    a.sum_blk = block_table(L, d_blob, L.M);
+    a.sum_rec = static_cast<const uint8_t*>(d_blob) + L.lay.rec_off[L.M];
+  }
   a.blob_settled = expansion_marked(static_cast<cudaStream_t>(stream)) ? 0 : 1;
   a.q8_out = q8 ? 1 : 0;
   a.relu = relu;

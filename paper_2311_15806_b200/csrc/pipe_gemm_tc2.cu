@@ -63,6 +63,8 @@ struct Params {
   int pk;                 // packed bytes of one row of one reduction block (128*b/8)
   int shift;              // 8 - b
   int direct;             // the weights come from the layer's int8 copy in the operand layout (bits reads 8, shift 0)
+  uint32_t split_mask;    // summed ensemble on one shared input, run as ONE cluster of all orders: bit k is set where
+                          // order k (k > 0) opens the next predictor, whose chain the epilogue starts from zero
   int conv_pw, conv_pp, conv_np, conv_chunks;   // patches per image row / per image / in total; 128-channel chunks per tap
   const uint8_t* kbase;   // lowest address of the streaming-layout sections (16-byte aligned)
   uint32_t koff[PIPE_MAX_ORDERS];  // (kcodes of order k - kbase) / 16
@@ -461,7 +463,11 @@ struct EpiCtx {
 // Q8: the fused inner-layer epilogue (activation function and the next layer's input quantizer, see the one-SM
 // kernel) replaces the fp32 store; a lane then stores the 16 codes of its own row itself and the staging block holds
 // the bias of the tile's channels.
-template <int NKMAX, bool PARTIALS, bool Q8>
+// SUMMED: the tile stacks the orders of ALL predictors of an ensemble whose predictors share one input and whose
+// outputs are summed after the layer (Sec. 3.2): every predictor's chain starts from zero, the bias closes the first
+// one, and the chains are added in ascending predictor order in this thread -- the same additions, in the same
+// order, as one launch per predictor summing into y, without the read-modify-write of y.
+template <int NKMAX, bool PARTIALS, bool Q8, bool SUMMED>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
   constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
   const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
@@ -580,7 +586,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
       qalign = (bits & 15) == 0 ? 16 : ((bits & 3) == 0 ? 4 : 1);
       for (int c = lane; c < c1 - c0; c += 32) x.stg[c] = (br.add_bias && p.f.bias) ? __ldg(p.f.bias + c0 + c) : 0.f;
     }
-    const bool add_bias = br.add_bias && p.f.bias;
+    const bool add_bias = !SUMMED && br.add_bias && p.f.bias;   // (a summed ensemble adds it inside the chain)
     const float* bias_q = add_bias ? p.f.bias + c0 + 4 * sj : nullptr;
     const int ngrp = (nch + 1) >> 1;
     __syncwarp();
@@ -634,8 +640,31 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
           float y[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) y[e] = 0.f;
+          float ysum[8];          // SUMMED: the predictors closed so far
+          bool first_chain = true;
+          // closes the running predictor's chain: the bias ends the first one, the others are added to the sum
+          auto close_chain = [&]() {
+            if (first_chain) {
+              if (p.f.bias) {
+                const float* bp = p.f.bias + c0 + 8 * chunk;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) y[e] = __fadd_rn(y[e], __ldg(bp + e));
+              }
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ysum[e] = y[e];
+              first_chain = false;
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ysum[e] = __fadd_rn(ysum[e], y[e]);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = 0.f;
+          };
 #pragma unroll
           for (int ko = 0; ko < NKMAX; ++ko) {
+            if constexpr (SUMMED) {
+              if (ko > 0 && ((p.split_mask >> ko) & 1u)) close_chain();
+            }
             if (cols[u][ko] < 0) continue;
             float cs[8];
             const uint32_t ca = cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
@@ -661,6 +690,11 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 #pragma unroll
               for (int e = 0; e < 8; ++e) prow[e] = acc[u][ko][e];
             }
+          }
+          if constexpr (SUMMED) {
+            close_chain();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = ysum[e];
           }
           if constexpr (Q8) {
             // bias last, sigma, then Q of the next layer (Sec. 3.2): eight codes of this lane's own row
@@ -783,7 +817,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   __syncwarp();
 }
 
-template <bool Q8>
+template <bool Q8, bool SUMMED>
 __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
@@ -1025,13 +1059,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.nparts = kEpiWarps / 4;
     e.stg = epi_stage[ew];
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
-      if (p.nkmax <= 2) epilogue_role<2, true, Q8>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, true, Q8>(p, e);
-      else epilogue_role<8, true, Q8>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, true, Q8, SUMMED>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true, Q8, SUMMED>(p, e);
+      else epilogue_role<8, true, Q8, SUMMED>(p, e);
     } else {
-      if (p.nkmax <= 2) epilogue_role<2, false, Q8>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, false, Q8>(p, e);
-      else epilogue_role<8, false, Q8>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, false, Q8, SUMMED>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false, Q8, SUMMED>(p, e);
+      else epilogue_role<8, false, Q8, SUMMED>(p, e);
     }
   }
 
@@ -1072,18 +1106,22 @@ static const DeviceSetup& device_setup() {
     int smem_max = 0, sms = 0;
     if (cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
-    cudaFuncAttributes f0, f1;
-    if (cudaFuncGetAttributes(&f0, tc2_forward_kernel<false>) != cudaSuccess) return;
-    if (cudaFuncGetAttributes(&f1, tc2_forward_kernel<true>) != cudaSuccess) return;
-    const int fixed = static_cast<int>(f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes);
+    cudaFuncAttributes f0, f1, f2;
+    if (cudaFuncGetAttributes(&f0, tc2_forward_kernel<false, false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f1, tc2_forward_kernel<true, false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f2, tc2_forward_kernel<false, true>) != cudaSuccess) return;
+    size_t fixed_b = f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes;
+    fixed_b = fixed_b > f2.sharedSizeBytes ? fixed_b : f2.sharedSizeBytes;
+    const int fixed = static_cast<int>(fixed_b);
     d.depth = (smem_max - fixed - 1024) / kStageBytes;   // static shared memory, alignment slack
     if (d.depth > kMaxRing) d.depth = kMaxRing;
     d.status = PIPE_ERR_UNSUPPORTED;
     if (d.depth * kSub != kUnpackWarps) return;   // every unpack warp owns one block slot of the ring
     d.dyn_smem = d.depth * kStageBytes + 1024;
     d.status = PIPE_ERR_CUDA;
-    if (cudaFuncSetAttribute(tc2_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
-    if (cudaFuncSetAttribute(tc2_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1097,7 +1135,7 @@ static const DeviceSetup& device_setup() {
     cfg.numAttrs = 1;
     int n = 0;
     d.status = PIPE_ERR_UNSUPPORTED;
-    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel<false>, &cfg) != cudaSuccess || n < 1) return;
+    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel<false, false>, &cfg) != cudaSuccess || n < 1) return;
     d.max_pairs = n < sms / 2 ? n : sms / 2;
     d.status = PIPE_OK;
   });
@@ -1106,7 +1144,7 @@ static const DeviceSetup& device_setup() {
 
 }  // namespace tc2
 
-static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
+static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream, uint32_t split_mask = 0) {
   using namespace tc2;
   const DeviceSetup& ds = device_setup();
   if (ds.status != PIPE_OK) return ds.status;
@@ -1136,6 +1174,7 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
 
   p.f = a;
   p.direct = direct ? 1 : 0;
+  p.split_mask = split_mask;
   const int row_bytes = direct ? round_up(a.I, kKStep) : a.kernel_row_bytes;   // bytes of a row over all reduction blocks
   if (direct) p.f.bits = 8;   // the kernel then treats the layer as one of int8 codes
   p.nkmax = max_cluster;
@@ -1223,7 +1262,9 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream) {
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = a.q8_out ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true>, p) : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false>, p);
+  const cudaError_t e = a.q8_out    ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true, false>, p)
+                        : split_mask ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, true>, p)
+                                     : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, false>, p);
   if (e != cudaSuccess) return PIPE_ERR_CUDA;
   count_launch(1);
   return launch_status();
@@ -1233,6 +1274,29 @@ pipe_status forward_tcgen05_pair(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T == 0) return PIPE_OK;
   const bool sum_mode = a.num_branches > 1 && a.branch[1].accumulate;
   if (!sum_mode) return launch_tc2(a, stream);
+  // Predictors that share one input (the first layer of an ensemble, Sec. 3.2): ONE launch on the cluster of all
+  // orders -- the activations are staged once, the MMAs run at the width of the whole cluster, and the epilogue
+  // closes each predictor's chain and adds them in ascending order in registers.
+  if (a.sum_blk && a.sum_rec && !a.q8_out) {
+    bool shared = true;
+    for (int m = 1; m < a.num_branches; ++m)
+      shared = shared && a.branch[m].xq == a.branch[0].xq && a.branch[m].sx == a.branch[0].sx &&
+               a.branch[m].k_begin == a.branch[m - 1].k_end && a.branch[m].y == a.branch[0].y;
+    const int k0 = a.branch[0].k_begin, k1 = a.branch[a.num_branches - 1].k_end;
+    if (shared && k1 - k0 <= tc2::kMaxClusterOrders) {
+      ForwardArgs one = a;
+      one.num_branches = 1;
+      one.branch[0] = a.branch[0];
+      one.branch[0].k_end = k1;
+      one.branch[0].blk = a.sum_blk;
+      one.branch[0].rec = a.sum_rec;
+      one.branch[0].accumulate = 0;
+      uint32_t split = 0;
+      for (int m = 1; m < a.num_branches; ++m) split |= 1u << (a.branch[m].k_begin - k0);
+      const pipe_status st = launch_tc2(one, stream, split);
+      if (st != PIPE_ERR_UNSUPPORTED) return st;
+    }
+  }
   // Summed ensemble: one launch per branch, in order, so that y = ((y_1 + y_2) + ...) is formed
   // by the same thread in a fixed order.
   for (int m = 0; m < a.num_branches; ++m) {

@@ -267,6 +267,41 @@ def test_forward_with_int8_copy_matches_oracle(oracle, kernel, O, I, T, bits, K,
     test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M, int8_copy=True)
 
 
+def test_summed_ensemble_on_a_shared_input_is_one_launch(oracle):
+    """Predictors that share their input and are summed after the layer (Sec. 3.2) run as ONE launch of the SM-pair
+    kernel on the cluster of all orders; with distinct inputs it is one launch per predictor.  Both give the oracle's
+    bits (each predictor's chain from zero, the bias closing the first, the chains added in ascending order)."""
+    O, I, T, bits, K, g, n_keep, M = 512, 640, 300, 4, 6, 8, 24, 3
+    rng = np.random.default_rng(77)
+    W = _w(rng, O, I)
+    bias = rng.standard_normal(O).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep, M), W)
+    split = [layer.layout.branch_orders[m] for m in range(M)]
+    xs = [(rng.standard_normal((T, I)) * (1 + m)).astype(np.float32) for m in range(M)]
+    q = [H.gpu_quantize(x) for x in xs]
+    qo = [oracle.quantize_act(x) for x in xs]
+    bd = torch.from_numpy(bias).cuda()
+    for shared in (True, False):
+        xq = [q[0][0]] * M if shared else [a for a, _ in q]
+        sx = [q[0][1]] * M if shared else [b for _, b in q]
+        y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
+        B.pipe_diag_select_kernel(B.KERNEL_TCGEN05_PAIR)
+        try:
+            before = B.pipe_launch_count()
+            B.pipe_ensemble_forward(layer.desc, layer.blob, xq, sx, [y], bd, True, None)
+            launches = B.pipe_launch_count() - before
+            torch.cuda.synchronize()
+        finally:
+            B.pipe_diag_select_kernel(B.KERNEL_AUTO)
+        assert B.pipe_poll_status() == B.PIPE_OK
+        assert launches == (1 if shared else M)
+        xo = np.stack([qo[0][0]] * M) if shared else np.stack([a for a, _ in qo])
+        so = [qo[0][1]] * M if shared else [b for _, b in qo]
+        y_o, _ = oracle.ensemble(e, xo, so, split, bias=bias, sum_branches=True)
+        np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), y_o.view(np.uint32))
+
+
 def test_forward_zero_tokens_and_strided_io(oracle):
     rng = np.random.default_rng(77)
     O, I, T = 64, 96, 10
