@@ -369,8 +369,8 @@ pipe_status pipe_expanded_linear(const pipe_layer_desc* desc, const void* d_blob
  * float [T,O] pitch ldy); inputs may alias (shared input, the first layer of a network).
  * sum_branches != 0: only h_y_m[0] is written, with ((y_1 + y_2) + ...) + y_M, every y_m being predictor m's own
  * chain from zero (the bias closing y_1).  Predictors that share input and step (the same pointers) run as one launch
- * for more than 16 tokens when the layer has the channel-block table of all K orders (K <= 8): the sums are formed in
- * registers; with distinct inputs it is one launch per predictor, in order, each adding into h_y_m[0].
+ * when K <= 8 (for more than 16 tokens the layer must also have the channel-block table of all K orders): the sums are
+ * formed in registers; with distinct inputs it is one launch per predictor, in order, each adding into h_y_m[0].
  * d_partials as in pipe_expanded_linear.
  */
 pipe_status pipe_ensemble_forward(const pipe_layer_desc* desc, const void* d_blob, const int8_t* const* h_xq_m,

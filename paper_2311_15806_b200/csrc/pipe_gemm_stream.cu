@@ -53,6 +53,8 @@ struct Params {
   int nkmax;              // most orders any branch has
   int own_max;            // most slabs any CTA owns
   int prefetch;           // the expanded layer is not being written by the launch before: weights may be fetched ahead of the dependency wait
+  uint32_t split_mask;    // summed ensemble on one shared input, run as ONE cluster of all orders: bit k marks the order (k > 0)
+                          // that opens the next predictor, whose chain the epilogue starts from zero
   int ctas_per_branch;    // every branch has its own CTAs, so no CTA's range crosses a branch boundary
 };
 
@@ -152,7 +154,7 @@ __device__ __forceinline__ int rows_before(const int32_t* cum, int c, int O, int
   return lo * g + (hi > lo ? c - j * g : 0);
 }
 
-template <int BITS, int NT, int NP>
+template <int BITS, int NT, int NP, bool SUMMED>
 __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __grid_constant__ Params p) {
   constexpr int SPW = (NP * NT <= 2) ? 5 : (NP * NT == 4 ? 2 : 1);   // slabs per consumer warp and pass
   constexpr int CHK = 128 / BITS;               // codes per 16-byte chunk
@@ -508,6 +510,28 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
         float y[NT][2];
 #pragma unroll
         for (int t = 0; t < NT; ++t) y[t][0] = y[t][1] = 0.f;
+        // Summed ensemble on a shared input (split_mask != 0): every predictor's chain starts from zero, the bias closes
+        // the first one, the chains are added in ascending predictor order -- the additions one launch per predictor
+        // summing into y would make, in the same order.
+        float ysum[NT][2];
+        bool first_chain = true;
+        int next_order = 1;   // orders below this one have had their predictor boundaries handled
+        const float bv = biastab[li * 8 + gid];
+        auto close_chain = [&]() {
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              if (first_chain) ysum[t][e] = (p.f.bias && br.add_bias) ? __fadd_rn(y[t][e], bv) : y[t][e];
+              else ysum[t][e] = __fadd_rn(ysum[t][e], y[t][e]);
+              y[t][e] = 0.f;
+            }
+          first_chain = false;
+        };
+        auto close_up_to = [&](int ko) {   // the boundaries at orders next_order .. ko
+          for (; next_order <= ko; ++next_order)
+            if ((p.split_mask >> next_order) & 1u) close_chain();
+        };
 #pragma unroll
         for (int q = 0; q < NP; ++q) {
           if (2 * q >= nch) continue;
@@ -525,6 +549,7 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
             const int ci = 2 * q + half;
             if (ci >= nch) continue;
             const int ko = kos[ci];
+            if constexpr (SUMMED) close_up_to(ko);
             const float cs = cstab[(li * p.nkmax + ko) * 8 + gid];
             const int row = slabmeta[li * p.nkmax + ko] + gid, roff = p.f.order[br.k_begin + ko].row_off;
 #pragma unroll
@@ -538,8 +563,13 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
               }
           }
         }
-        const bool bias = p.f.bias && br.add_bias;
-        const float bv = biastab[li * 8 + gid];
+        if constexpr (SUMMED) {
+          close_up_to(nk - 1);
+          close_chain();
+#pragma unroll
+          for (int t = 0; t < NT; ++t) y[t][0] = ysum[t][0], y[t][1] = ysum[t][1];
+        }
+        const bool bias = p.f.bias && br.add_bias && !SUMMED;   // (a summed ensemble has added it inside the chain)
 #pragma unroll
         for (int t = 0; t < NT; ++t)
 #pragma unroll
@@ -582,7 +612,7 @@ struct DeviceCache {
   std::mutex mu;
   bool ready = false;
   int smem_max = 0, sms = 0, n = 0;
-  KernelInfo k[24];
+  KernelInfo k[40];
 };
 
 static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* smem_max, int* sms, int* fixed) {
@@ -601,7 +631,7 @@ static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* sm
   for (int i = 0; i < c.n; ++i)
     if (c.k[i].fn == reinterpret_cast<const void*>(kern)) ki = &c.k[i];
   if (!ki) {
-    if (c.n >= 24) return false;
+    if (c.n >= 40) return false;
     cudaFuncAttributes fattr;
     if (cudaFuncGetAttributes(&fattr, kern) != cudaSuccess) return false;
     ki = &c.k[c.n++];
@@ -620,7 +650,7 @@ static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* sm
 
 }  // namespace st
 
-static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
+static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream, uint32_t split_mask = 0) {
   using namespace st;
   if (a.T > 16 || a.g % 8 != 0 || a.O % 8 != 0) return PIPE_ERR_UNSUPPORTED;
   if (a.ldxq % 16 != 0) return PIPE_ERR_UNSUPPORTED;   // tensor-map row pitch
@@ -632,6 +662,7 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   Params p;
   p.f = a;
   p.prefetch = a.blob_settled ? 1 : 0;
+  p.split_mask = split_mask;
   const int nt = a.T <= 8 ? 1 : 2;
   const int np = max_cluster <= 2 ? 1 : (max_cluster <= 4 ? 2 : 4);
   const int spw = (np * nt <= 2) ? 5 : (np * nt == 4 ? 2 : 1);
@@ -646,10 +677,14 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream) {
   p.pass_slabs = kGroupWarps * spw;
   // (the kernel instantiation depends only on bits, tokens and orders, all known here)
   void (*kern)(const Params) = nullptr;
-#define PIPE_ST_PICK(B)                                                                     \
-  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1> : (np == 2 ? stream_forward_kernel<B, 1, 2> : stream_forward_kernel<B, 1, 4>); \
-  else kern = np == 1 ? stream_forward_kernel<B, 2, 1> : (np == 2 ? stream_forward_kernel<B, 2, 2> : stream_forward_kernel<B, 2, 4>);
-  if (a.bits == 8) { PIPE_ST_PICK(8) } else if (a.bits == 4) { PIPE_ST_PICK(4) } else { PIPE_ST_PICK(2) }
+#define PIPE_ST_PICK(B, S)                                                                     \
+  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1, S> : (np == 2 ? stream_forward_kernel<B, 1, 2, S> : stream_forward_kernel<B, 1, 4, S>); \
+  else kern = np == 1 ? stream_forward_kernel<B, 2, 1, S> : (np == 2 ? stream_forward_kernel<B, 2, 2, S> : stream_forward_kernel<B, 2, 4, S>);
+  if (split_mask == 0) {
+    if (a.bits == 8) { PIPE_ST_PICK(8, false) } else if (a.bits == 4) { PIPE_ST_PICK(4, false) } else { PIPE_ST_PICK(2, false) }
+  } else {   // a summed ensemble on a shared input: the epilogue that closes the predictors' chains
+    if (a.bits == 8) { PIPE_ST_PICK(8, true) } else if (a.bits == 4) { PIPE_ST_PICK(4, true) } else { PIPE_ST_PICK(2, true) }
+  }
 #undef PIPE_ST_PICK
   int smem_max = 0, sms = 0, fixed = 0;
   if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
@@ -699,6 +734,25 @@ pipe_status forward_stream(const ForwardArgs& a, cudaStream_t stream) {
   if (a.T == 0) return PIPE_OK;
   const bool sum_mode = a.num_branches > 1 && a.branch[1].accumulate;
   if (!sum_mode) return launch_stream(a, stream);
+  // predictors that share input and step: one launch on the cluster of all orders, the chains added in registers
+  if (!a.q8_out) {
+    bool shared = true;
+    for (int m = 1; m < a.num_branches; ++m)
+      shared = shared && a.branch[m].xq == a.branch[0].xq && a.branch[m].sx == a.branch[0].sx &&
+               a.branch[m].k_begin == a.branch[m - 1].k_end && a.branch[m].y == a.branch[0].y;
+    const int k0 = a.branch[0].k_begin, k1 = a.branch[a.num_branches - 1].k_end;
+    if (shared && k0 == 0) {
+      ForwardArgs one = a;
+      one.num_branches = 1;
+      one.branch[0] = a.branch[0];
+      one.branch[0].k_end = k1;
+      one.branch[0].accumulate = 0;
+      uint32_t split = 0;
+      for (int m = 1; m < a.num_branches; ++m) split |= 1u << a.branch[m].k_begin;
+      const pipe_status st = launch_stream(one, stream, split);
+      if (st != PIPE_ERR_UNSUPPORTED) return st;
+    }
+  }
   for (int m = 0; m < a.num_branches; ++m) {
     ForwardArgs one = a;
     one.num_branches = 1;

@@ -267,11 +267,13 @@ def test_forward_with_int8_copy_matches_oracle(oracle, kernel, O, I, T, bits, K,
     test_forward_matches_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep, M, int8_copy=True)
 
 
-def test_summed_ensemble_on_a_shared_input_is_one_launch(oracle):
+@pytest.mark.parametrize("kernel,T", [(B.KERNEL_TCGEN05_PAIR, 300), (B.KERNEL_STREAM, 7), (B.KERNEL_STREAM, 16), (B.KERNEL_AUTO, 1)])
+def test_summed_ensemble_on_a_shared_input_is_one_launch(oracle, kernel, T):
     """Predictors that share their input and are summed after the layer (Sec. 3.2) run as ONE launch of the SM-pair
-    kernel on the cluster of all orders; with distinct inputs it is one launch per predictor.  Both give the oracle's
-    bits (each predictor's chain from zero, the bias closing the first, the chains added in ascending order)."""
-    O, I, T, bits, K, g, n_keep, M = 512, 640, 300, 4, 6, 8, 24, 3
+    kernel (of the weight-streaming kernel for up to 16 tokens) on the cluster of all orders; with distinct inputs it is
+    one launch per predictor.  Both give the oracle's bits (each predictor's chain from zero, the bias closing the
+    first, the chains added in ascending order)."""
+    O, I, bits, K, g, n_keep, M = 512, 640, 4, 6, 8, 24, 3
     rng = np.random.default_rng(77)
     W = _w(rng, O, I)
     bias = rng.standard_normal(O).astype(np.float32)
@@ -286,7 +288,7 @@ def test_summed_ensemble_on_a_shared_input_is_one_launch(oracle):
         xq = [q[0][0]] * M if shared else [a for a, _ in q]
         sx = [q[0][1]] * M if shared else [b for _, b in q]
         y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
-        B.pipe_diag_select_kernel(B.KERNEL_TCGEN05_PAIR)
+        B.pipe_diag_select_kernel(kernel)
         try:
             before = B.pipe_launch_count()
             B.pipe_ensemble_forward(layer.desc, layer.blob, xq, sx, [y], bd, True, None)
