@@ -28,8 +28,8 @@ def _built():
     H.ensure_built()
 
 
-def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_check=True):
-    run = LayerRunner(spec, second_layer=second_layer)
+def _check_layer(oracle, spec, token_counts=None, second_layer=False, cross_check=True, int8_copy=False):
+    run = LayerRunner(spec, second_layer=second_layer, int8_copy=int8_copy)
     W = run.host_weights()
     e = oracle.expand(W, spec.bits, spec.K, spec.g, run.n_keep)
     split = [int(v) for v in oracle.balanced_split(spec.K, spec.M)]
@@ -162,3 +162,11 @@ def test_cfg5_ternary(oracle):
 def test_cfg5_ternary_cross_check_on_a_token_slice(oracle):
     """The CUDA-core kernel needs seconds for the full 1.5e12 MACs; cross-check 1024 tokens."""
     _check_layer(oracle, WORK["cfg5"].with_tokens(1024), cross_check=True)
+
+
+def test_layers_with_an_int8_copy_at_full_size(oracle):
+    """The rows bench.py measures once more on layers that keep the int8 copy of their codes: same checks, same bits."""
+    _check_layer(oracle, WORK["cfg3a"], int8_copy=True)
+    _check_layer(oracle, WORK["cfg3b"], second_layer=True, int8_copy=True)
+    _check_layer(oracle, WORK["cfg4a_t1"], token_counts=[16, 128, 1024, 4096], int8_copy=True)
+    _check_layer(oracle, WORK["cfg4b_t1"], token_counts=[4096], second_layer=True, int8_copy=True)
