@@ -509,6 +509,45 @@ def test_ensemble_convolution_matches_oracle(oracle, N, Hh, Ww, Cc, O, kh, kw, b
     np.testing.assert_array_equal(got.view(np.uint32), want_y.view(np.uint32))
 
 
+@pytest.mark.parametrize("N,Hh,Ww,Cc,O,kh,kw,bits,K,g,n_keep,M,stride", [
+    (1, 15, 17, 128, 64, 3, 3, 4, 4, 8, 4, 2, 2), (2, 12, 12, 128, 48, 3, 3, 8, 3, 8, 3, 3, 1), (1, 16, 16, 256, 96, 1, 1, 2, 6, 16, 3, 3, 1)])
+def test_summed_ensemble_convolution_on_a_shared_input(oracle, N, Hh, Ww, Cc, O, kh, kw, bits, K, g, n_keep, M, stride):
+    """The predictors of a first convolution share the image and are summed after the layer: one launch on the cluster of
+    all orders (the chains closed and added in registers), the oracle's bits."""
+    rng = np.random.default_rng(N * 977 + Hh * 13 + Cc + M)
+    I = kh * kw * Cc
+    W = _w(rng, O, I, heavy=(bits == 2))
+    bias = rng.standard_normal(O).astype(np.float32)
+    e = oracle.expand(W, bits, K, g, n_keep)
+    layer = H.gpu_expand(H.desc_of(O, I, bits, K, g, n_keep, M), W)
+    split = oracle.balanced_split(K, M)
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    x4 = np.maximum(rng.standard_normal((N, Hh, Ww, Cc)), 0).astype(np.float32)
+    xq4, sx = H.gpu_quantize(x4.reshape(-1, Cc))
+    xq_o, s_o = oracle.quantize_act(x4.reshape(-1, Cc))
+    rows, Ho, Wo = _lower_im2col(xq_o.reshape(N, Hh, Ww, Cc), kh, kw, ph, pw, stride)
+    want_y, want_part = oracle.ensemble(e, np.stack([rows] * M), [s_o] * M, split, bias=bias, sum_branches=True)
+    geom = B.ConvGeom()
+    geom.batch, geom.height, geom.width, geom.channels = N, Hh, Ww, Cc
+    geom.kernel_h, geom.kernel_w, geom.pad_h, geom.pad_w = kh, kw, ph, pw
+    geom.stride_h = geom.stride_w = stride
+    T = N * Ho * Wo
+    y = torch.full((T, O), float("nan"), dtype=torch.float32, device="cuda")
+    part = torch.zeros((T, layer.layout.total_rows), dtype=torch.int32, device="cuda")
+    B.pipe_diag_select_kernel(B.KERNEL_TCGEN05_PAIR)   # (the automatic choice sends layers this small to the one-SM kernel)
+    try:
+        before = B.pipe_launch_count()
+        B.pipe_ensemble_conv2d(layer.desc, geom, layer.blob, [xq4.view(N, Hh, Ww, Cc)] * M, [sx] * M, [y], torch.from_numpy(bias).cuda(), True, part)
+        launches = B.pipe_launch_count() - before
+        torch.cuda.synchronize()
+    finally:
+        B.pipe_diag_select_kernel(B.KERNEL_AUTO)
+    assert B.pipe_poll_status() == B.PIPE_OK
+    assert launches == 1
+    np.testing.assert_array_equal(part.cpu().numpy(), want_part)
+    np.testing.assert_array_equal(y.cpu().numpy().view(np.uint32), want_y.view(np.uint32))
+
+
 def test_ensemble_convolution_inner_layer_matches_oracle(oracle):
     """pipe_ensemble_conv2d_q8: every predictor's int8 output equals forward -> ReLU -> quantize(static step) of the
     oracle on the lowered rows of that predictor's input."""
