@@ -11,7 +11,7 @@ from tests import test_gpu_parity_small as TP
 pytestmark = pytest.mark.gpu
 
 
-def _cases(n, seed):
+def _cases(n, seed, tokens=(17, 31, 64, 100, 128, 129, 255, 256, 257, 300, 511, 640, 1000)):
     rng = np.random.default_rng(seed)
     out = []
     for _ in range(n):
@@ -22,7 +22,7 @@ def _cases(n, seed):
         M = int(rng.integers(1, min(K, 4) + 1))
         n_keep = int(rng.integers(1, G + 1))
         I = int(rng.integers(1, 40)) * int(rng.choice([8, 16, 56, 128]))
-        T = int(rng.choice([17, 31, 64, 100, 128, 129, 255, 256, 257, 300, 511, 640, 1000]))
+        T = int(rng.choice(tokens))
         out.append((G * g, I, T, bits, K, g, n_keep, M))
     return out
 
@@ -37,4 +37,12 @@ def test_random_shapes_match_oracle(oracle, kernel, O, I, T, bits, K, g, n_keep,
 @pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", _cases(24, 20231116))
 def test_random_shapes_with_int8_copy_match_oracle(oracle, O, I, T, bits, K, g, n_keep, M):
     TP.test_forward_matches_oracle(oracle, B.KERNEL_TCGEN05_PAIR, O, I, T, bits, K, g, n_keep, M, int8_copy=True)
+    assert B.pipe_poll_status() == B.PIPE_OK
+
+
+@pytest.mark.parametrize("O,I,T,bits,K,g,n_keep,M", _cases(16, 20231117, tokens=(1, 2, 5, 8, 9, 16)))
+def test_random_shapes_on_few_tokens_match_oracle(oracle, O, I, T, bits, K, g, n_keep, M):
+    """Up to 16 tokens: the weight-streaming kernel (and whatever the automatic choice falls back to), the summed
+    ensemble on a shared input as one launch included."""
+    TP.test_forward_matches_oracle(oracle, B.KERNEL_AUTO, O, I, T, bits, K, g, n_keep, M)
     assert B.pipe_poll_status() == B.PIPE_OK
