@@ -67,8 +67,37 @@ int* device_status_word() {
 
 static uint64_t align_up64(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
+static pipe_status resolve_layer_uncached(const pipe_layer_desc* d, LayerInfo* out);
+
+// Every entry point resolves its descriptor; a serving loop passes the same few descriptors again and again, so
+// each host thread keeps the last ones it resolved (the result is a pure function of the descriptor's bytes).
 pipe_status resolve_layer(const pipe_layer_desc* d, LayerInfo* out) {
   if (!d || !out) return PIPE_ERR_INVALID_ARG;
+  constexpr int kKept = 4;
+  struct Entry {
+    pipe_layer_desc desc;
+    LayerInfo info;
+    bool valid;
+  };
+  thread_local Entry kept[kKept] = {};
+  thread_local int next = 0;
+  for (int i = 0; i < kKept; ++i)
+    if (kept[i].valid && std::memcmp(&kept[i].desc, d, sizeof(pipe_layer_desc)) == 0) {
+      *out = kept[i].info;
+      return PIPE_OK;
+    }
+  const pipe_status st = resolve_layer_uncached(d, out);
+  if (st == PIPE_OK) {
+    Entry& e = kept[next];
+    next = (next + 1) % kKept;
+    e.desc = *d;
+    e.info = *out;
+    e.valid = true;
+  }
+  return st;
+}
+
+static pipe_status resolve_layer_uncached(const pipe_layer_desc* d, LayerInfo* out) {
   if (d->out_features <= 0 || d->in_features <= 0) return PIPE_ERR_INVALID_ARG;
   if (!(d->weight_bits == 8 || d->weight_bits == 6 || d->weight_bits == 4 || d->weight_bits == 3 || d->weight_bits == 2))
     return PIPE_ERR_INVALID_ARG;
