@@ -127,7 +127,10 @@ typedef struct pipe_layer_desc {
  *   blk_off[m]    int32 [2 + blk_cap[m]]: n, then b_0 = 0 < b_1 < ... < b_n = G.  Block i is the channel groups
  *                 b_i .. b_{i+1} - 1.  With R the rows the cluster's orders keep in the whole layer and
  *                 n0 = max(ceil(R / PIPE_BLOCK_ROWS), ceil(O / PIPE_BLOCK_CHANNELS)) the fewest blocks that could
- *                 hold them, the limit of a block is L = min(PIPE_BLOCK_ROWS, roundup(ceil(R / n0), 16) + orders * g):
+ *                 hold them, the limit of a block is L = min(PIPE_BLOCK_ROWS, roundup(ceil(R / n0), 16) + orders * g)
+ *                 -- except for a cluster of few blocks: with h = orders * g / 2 and
+ *                 ne = max(ceil(R / (PIPE_BLOCK_ROWS - h)), ceil(O / PIPE_BLOCK_CHANNELS)), a cluster with
+ *                 ne <= PIPE_EVEN_BLOCKS has L = min(PIPE_BLOCK_ROWS, ceil(R / ne) + h), which gives blocks of one size --:
  *                 the groups are walked from 0 and a block is closed when the next group would take the rows it
  *                 stacks over the cluster's orders (kept groups only) beyond L or its channels beyond
  *                 PIPE_BLOCK_CHANNELS.  Blocks are the unit of work of the SM-pair tensor-core kernel, whose MMAs then
@@ -152,6 +155,7 @@ typedef struct pipe_layer_desc {
  */
 #define PIPE_BLOCK_ROWS 256
 #define PIPE_BLOCK_CHANNELS 512
+#define PIPE_EVEN_BLOCKS 8   /* clusters of at most this many blocks are cut into blocks of one size (see blk_off) */
 #define PIPE_BLOCK_RECORD_BYTES (32 * 4 + 8 * (PIPE_BLOCK_CHANNELS / 8) * 2 + PIPE_BLOCK_ROWS * 4)
 typedef struct pipe_layer_layout {
   int32_t num_groups;        /* G = O / g */

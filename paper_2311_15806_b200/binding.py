@@ -17,6 +17,7 @@ from . import build as _build
 MAX_ORDERS = 16
 BLOCK_ROWS = 256
 BLOCK_CHANNELS = 512
+EVEN_BLOCKS = 8   # PIPE_EVEN_BLOCKS
 BLOCK_RECORD_BYTES = 32 * 4 + 8 * (BLOCK_CHANNELS // 8) * 2 + BLOCK_ROWS * 4
 BLOB_ALIGN = 1024
 

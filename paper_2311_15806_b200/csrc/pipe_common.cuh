@@ -62,6 +62,21 @@ static_assert(kRecBytes == PIPE_BLOCK_RECORD_BYTES && kRecBytes % 16 == 0, "reco
 
 // Row limit of the blocks of a channel-block table (the definition in pipe.h): R rows kept by the cluster's nk orders.
 inline int block_row_limit(int64_t R, int O, int nk, int g) {
+  // A cluster of a few blocks (at most PIPE_EVEN_BLOCKS) is cut into blocks of ONE size: a block is closed when the
+  // next group would take it beyond the limit, so it ends up to one group (at most nk * g rows) short of it, half a
+  // group on average; n blocks of that average size hold the rows, and the limit is the mean block plus that half
+  // group.  (Filled to PIPE_BLOCK_ROWS instead, the last block of such a cluster is a small one that costs a tile
+  // like the others.)  A cluster of many blocks keeps the widest blocks: there the MMA's width is worth more.
+  {
+    const int64_t half = (static_cast<int64_t>(nk) * g) / 2;
+    const int64_t room = PIPE_BLOCK_ROWS - half > 0 ? PIPE_BLOCK_ROWS - half : 1;
+    const int64_t ner = ceil_div<int64_t>(R, room), nec = ceil_div<int64_t>(O, PIPE_BLOCK_CHANNELS);
+    const int64_t ne = ner > nec ? ner : nec;
+    if (ne >= 1 && ne <= PIPE_EVEN_BLOCKS) {
+      const int64_t even = ceil_div<int64_t>(R, ne) + half;
+      return static_cast<int>(even < PIPE_BLOCK_ROWS ? even : PIPE_BLOCK_ROWS);
+    }
+  }
   const int64_t n0r = ceil_div<int64_t>(R, PIPE_BLOCK_ROWS), n0c = ceil_div<int64_t>(O, PIPE_BLOCK_CHANNELS);
   const int64_t n0 = n0r > n0c ? n0r : n0c;
   const int64_t even = round_up<int64_t>(ceil_div<int64_t>(R, n0 > 0 ? n0 : 1), 16) + static_cast<int64_t>(nk) * g;

@@ -123,8 +123,13 @@ def expected_block_table(kept_lists, G: int, g: int, row_max: int = 256, channel
     for kept in kept_lists:
         rows[np.asarray(kept)] += g
     R = int(rows.sum())
-    n0 = max(-(-R // row_max), -(-(G * g) // channel_limit))
-    row_limit = min(row_max, (-(-(-(-R // n0)) // 16)) * 16 + len(kept_lists) * g)
+    half = len(kept_lists) * g // 2
+    ne = max(-(-R // max(row_max - half, 1)), -(-(G * g) // channel_limit))
+    if 1 <= ne <= B.EVEN_BLOCKS:
+        row_limit = min(row_max, -(-R // ne) + half)
+    else:
+        n0 = max(-(-R // row_max), -(-(G * g) // channel_limit))
+        row_limit = min(row_max, (-(-(-(-R // n0)) // 16)) * 16 + len(kept_lists) * g)
     bounds = [0]
     cur_rows, cur_groups = 0, 0
     for j in range(G):
