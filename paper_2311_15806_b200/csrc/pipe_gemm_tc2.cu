@@ -447,6 +447,7 @@ struct EpiCtx {
   uint32_t tempty_lead0;   // the accumulator-released barriers of the pair's first CTA (cluster address)
   int part, nparts;  // share of the 16-channel groups this warp drains (two warps per lane quarter)
   float* stg;        // 32 rows x 16 floats, swizzled
+  uint32_t zero_s;   // shared address of eight zero floats
 };
 
 // Epilogue role (8 warps, one TMEM lane quarter each; a lane owns one token row of a token tile).
@@ -467,9 +468,13 @@ struct EpiCtx {
 // outputs are summed after the layer (Sec. 3.2): every predictor's chain starts from zero, the bias closes the first
 // one, and the chains are added in ascending predictor order in this thread -- the same additions, in the same
 // order, as one launch per predictor summing into y, without the read-modify-write of y.
-template <int NKMAX, bool PARTIALS, bool Q8, bool SUMMED>
+template <int NKMAX, bool PARTIALS, bool Q8, bool SUMMED, bool SHORT_K>
 __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) {
   constexpr int CH = (NKMAX <= 2) ? 2 : 1;   // chunks per batch of accumulator loads
+  // STRAIGHT: the chain of a chunk without branches (see below).  It trades some arithmetic on pruned (chunk, order)
+  // pairs for a loop body the compiler can interleave freely, which pays where the drain paces the layer -- a short
+  // reduction axis (cfg3a 49.3 -> 46.1 us) -- and costs a percent where it does not, so the host picks it by the axis.
+  constexpr bool STRAIGHT = SHORT_K && !PARTIALS && NKMAX <= 2;
   const int q = x.warp & 3;                  // TMEM lane quarter this warp may read
   const int lane = x.lane;
   uint32_t tcount = 0;
@@ -630,8 +635,10 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
 #pragma unroll
         for (int u = 0; u < CH; ++u)
 #pragma unroll
-          for (int ko = 0; ko < NKMAX; ++ko)
-            if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
+          for (int ko = 0; ko < NKMAX; ++ko) {
+            if constexpr (STRAIGHT) tmem_ld8(tbase + (cols[u][ko] >= 0 ? cols[u][ko] : 0), acc[u][ko]);
+            else if (cols[u][ko] >= 0) tmem_ld8(tbase + cols[u][ko], acc[u][ko]);
+          }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
         for (int u = 0; u < CH; ++u) {
@@ -665,9 +672,13 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
             if constexpr (SUMMED) {
               if (ko > 0 && ((p.split_mask >> ko) & 1u)) close_chain();
             }
-            if (cols[u][ko] < 0) continue;
+            if constexpr (!STRAIGHT) {
+              if (cols[u][ko] < 0) continue;
+            }
             float cs[8];
-            const uint32_t ca = cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
+            // (STRAIGHT: an order that pruned the chunk's group takes part with the scale 0 and whatever integers column 0
+            // holds -- finite, times zero, added to a y that is never -0: the same bits, and no branch in the chain)
+            const uint32_t ca = (STRAIGHT && cols[u][ko] < 0) ? x.zero_s : cscale_s + static_cast<uint32_t>(cols[u][ko] * 4);
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[0]), "=f"(cs[1]), "=f"(cs[2]), "=f"(cs[3]) : "r"(ca));
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(cs[4]), "=f"(cs[5]), "=f"(cs[6]), "=f"(cs[7]) : "r"(ca + 16));
             if constexpr (PARTIALS) {
@@ -817,7 +828,7 @@ __device__ __forceinline__ void epilogue_role(const Params& p, const EpiCtx& x) 
   __syncwarp();
 }
 
-template <bool Q8, bool SUMMED>
+template <bool Q8, bool SUMMED, bool SHORT_K>
 __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t bars[2 * kMaxRing + 4];  // full[3] done[3] tmem_full[2] tmem_empty[2]
@@ -830,6 +841,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   __shared__ __align__(16) uint8_t tile_recs[kRecBufs][kRecBytes];   // block records of the tiles in the epilogue's hands
   __shared__ __align__(16) float cfold_s[kRecBufs][kMaxN];            // s_k * lambda_x of the stacked rows of those tiles
   __shared__ uint64_t pre_bars[kRecBufs];
+  __shared__ __align__(16) float zero8_s[8];
   __shared__ float sx_s[2 * PIPE_MAX_ORDERS];                        // lambda_x of every branch, then the fused epilogue's output steps
   __shared__ __align__(1024) float epi_stage[kEpiWarps][32 * 16];   // per epilogue warp: 32 token rows x 16 channels (the
                                                                     // source of tensor stores with the 64-byte swizzle)
@@ -870,6 +882,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
   }
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    for (int i = 0; i < 8; ++i) zero8_s[i] = 0.f;
     int acc = 0;
     for (int m = 0; m < p.f.num_branches; ++m) {
       tile_base_s[m] = acc;
@@ -1058,14 +1071,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc2_forward_kernel(const __grid_c
     e.part = ew >> 2;
     e.nparts = kEpiWarps / 4;
     e.stg = epi_stage[ew];
+    e.zero_s = smem_u32(zero8_s);
     if (p.f.partials) {   // verification output: every integer accumulator is also written out
-      if (p.nkmax <= 2) epilogue_role<2, true, Q8, SUMMED>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, true, Q8, SUMMED>(p, e);
-      else epilogue_role<8, true, Q8, SUMMED>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, true, Q8, SUMMED, SHORT_K>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, true, Q8, SUMMED, SHORT_K>(p, e);
+      else epilogue_role<8, true, Q8, SUMMED, SHORT_K>(p, e);
     } else {
-      if (p.nkmax <= 2) epilogue_role<2, false, Q8, SUMMED>(p, e);
-      else if (p.nkmax <= 4) epilogue_role<4, false, Q8, SUMMED>(p, e);
-      else epilogue_role<8, false, Q8, SUMMED>(p, e);
+      if (p.nkmax <= 2) epilogue_role<2, false, Q8, SUMMED, SHORT_K>(p, e);
+      else if (p.nkmax <= 4) epilogue_role<4, false, Q8, SUMMED, SHORT_K>(p, e);
+      else epilogue_role<8, false, Q8, SUMMED, SHORT_K>(p, e);
     }
   }
 
@@ -1107,9 +1121,9 @@ static const DeviceSetup& device_setup() {
     if (cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
     cudaFuncAttributes f0, f1, f2;
-    if (cudaFuncGetAttributes(&f0, tc2_forward_kernel<false, false>) != cudaSuccess) return;
-    if (cudaFuncGetAttributes(&f1, tc2_forward_kernel<true, false>) != cudaSuccess) return;
-    if (cudaFuncGetAttributes(&f2, tc2_forward_kernel<false, true>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f0, tc2_forward_kernel<false, false, false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f1, tc2_forward_kernel<true, false, false>) != cudaSuccess) return;
+    if (cudaFuncGetAttributes(&f2, tc2_forward_kernel<false, true, false>) != cudaSuccess) return;
     size_t fixed_b = f0.sharedSizeBytes > f1.sharedSizeBytes ? f0.sharedSizeBytes : f1.sharedSizeBytes;
     fixed_b = fixed_b > f2.sharedSizeBytes ? fixed_b : f2.sharedSizeBytes;
     const int fixed = static_cast<int>(fixed_b);
@@ -1119,9 +1133,11 @@ static const DeviceSetup& device_setup() {
     if (d.depth * kSub != kUnpackWarps) return;   // every unpack warp owns one block slot of the ring
     d.dyn_smem = d.depth * kStageBytes + 1024;
     d.status = PIPE_ERR_CUDA;
-    if (cudaFuncSetAttribute(tc2_forward_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
-    if (cudaFuncSetAttribute(tc2_forward_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
-    if (cudaFuncSetAttribute(tc2_forward_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
+    if (cudaFuncSetAttribute(tc2_forward_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, d.dyn_smem) != cudaSuccess) return;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1135,7 +1151,7 @@ static const DeviceSetup& device_setup() {
     cfg.numAttrs = 1;
     int n = 0;
     d.status = PIPE_ERR_UNSUPPORTED;
-    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel<false, false>, &cfg) != cudaSuccess || n < 1) return;
+    if (cudaOccupancyMaxActiveClusters(&n, tc2_forward_kernel<false, false, false>, &cfg) != cudaSuccess || n < 1) return;
     d.max_pairs = n < sms / 2 ? n : sms / 2;
     d.status = PIPE_OK;
   });
@@ -1262,9 +1278,13 @@ static pipe_status launch_tc2(const ForwardArgs& a, cudaStream_t stream, uint32_
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = a.q8_out    ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true, false>, p)
-                        : split_mask ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, true>, p)
-                                     : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, false>, p);
+  // (a reduction axis of at most 8 blocks: the drain paces the layer, see STRAIGHT in the epilogue)
+  const bool short_k = p.kblocks <= 8;
+  const cudaError_t e = a.q8_out    ? (short_k ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true, false, true>, p)
+                                               : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<true, false, false>, p))
+                        : split_mask ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, true, false>, p)
+                        : short_k    ? cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, false, true>, p)
+                                     : cudaLaunchKernelEx(&cfg, tc2_forward_kernel<false, false, false>, p);
   if (e != cudaSuccess) return PIPE_ERR_CUDA;
   count_launch(1);
   return launch_status();
