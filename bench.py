@@ -116,14 +116,14 @@ def workload_spec(name: str):
 # program (summaries under profiles/, named in the comment).  A workload without a capture of the present
 # kernel has no entry and reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "cfg2": 28680192 + 51124480,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
-    "cfg3a": 9438464 + 47748096,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
-    "cfg4a_t4096": 90854144 + 313195520,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
-    "cfg5": 495110144 + 1027253760,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
+    "cfg2": 29294336 + 51489280,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
+    "cfg3a": 9440512 + 47313152,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
+    "cfg4a_t4096": 90993408 + 312856320,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
+    "cfg5": 490662400 + 1028348928,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
     "cfg4a_t1": 56559872 + 62464,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
     "cfg4a_t16": 56687616 + 119040,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
-    "cfg4a_t4096+int8_copy": 148761088 + 316460288,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
-    "cfg3b+int8_copy": 31192832 + 1270528,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
+    "cfg4a_t4096+int8_copy": 148933632 + 316924928,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
+    "cfg3b+int8_copy": 31190784 + 717824,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
 }
 
 
