@@ -154,7 +154,11 @@ __device__ __forceinline__ int rows_before(const int32_t* cum, int c, int O, int
   return lo * g + (hi > lo ? c - j * g : 0);
 }
 
-template <int BITS, int NT, int NP, bool SUMMED>
+// FULL: nearly every slab slot of every consumer warp holds a slab (the host knows: one pass, more than SPW - 1 slabs per
+// warp): the loop over a warp's slabs then runs without its per-slab branches -- an absent chunk takes part with zero
+// weights -- so that the slabs' load-and-MMA chains are one block the compiler may interleave (cfg4a T = 1: 17.6 -> 16.8 us;
+// a launch with two slabs per warp would do 2.5 times its work that way, hence the choice per launch).
+template <int BITS, int NT, int NP, bool SUMMED, bool FULL>
 __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __grid_constant__ Params p) {
   constexpr int SPW = (NP * NT <= 2) ? 5 : (NP * NT == 4 ? 2 : 1);   // slabs per consumer warp and pass
   constexpr int CHK = 128 / BITS;               // codes per 16-byte chunk
@@ -451,10 +455,20 @@ __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __gri
           for (int s = 0; s < SPW; ++s) {
 #pragma unroll
             for (int q = 0; q < NP; ++q) {
-              if (2 * q >= nchunks[s]) continue;
               uint4 wa = make_uint4(0, 0, 0, 0), wb = make_uint4(0, 0, 0, 0);
-              if (live) wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
-              if (live && 2 * q + 1 < nchunks[s]) wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
+              if constexpr (FULL) {
+                // (an absent chunk, or a block beyond the reduction axis, reads some valid address of the stage and is
+                // replaced by zero weights)
+                wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
+                wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
+                const bool ha = live && 2 * q < nchunks[s], hb = live && 2 * q + 1 < nchunks[s];
+                wa = ha ? wa : make_uint4(0, 0, 0, 0);
+                wb = hb ? wb : make_uint4(0, 0, 0, 0);
+              } else {
+                if (2 * q >= nchunks[s]) continue;
+                if (live) wa = lds128(sgen, woff[s][2 * q] + kbs * wstr[s][2 * q] + wbyte);
+                if (live && 2 * q + 1 < nchunks[s]) wb = lds128(sgen, woff[s][2 * q + 1] + kbs * wstr[s][2 * q + 1] + wbyte);
+              }
 #pragma unroll
               for (int mm = 0; mm < 2 * XCH; ++mm) {
                 uint32_t a0, a1, b0, b1;
@@ -678,14 +692,18 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream, uint
   // (the kernel instantiation depends only on bits, tokens and orders, all known here)
   void (*kern)(const Params) = nullptr;
 #define PIPE_ST_PICK(B, S)                                                                     \
-  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1, S> : (np == 2 ? stream_forward_kernel<B, 1, 2, S> : stream_forward_kernel<B, 1, 4, S>); \
-  else kern = np == 1 ? stream_forward_kernel<B, 2, 1, S> : (np == 2 ? stream_forward_kernel<B, 2, 2, S> : stream_forward_kernel<B, 2, 4, S>);
+  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1, S, false> : (np == 2 ? stream_forward_kernel<B, 1, 2, S, false> : stream_forward_kernel<B, 1, 4, S, false>); \
+  else kern = np == 1 ? stream_forward_kernel<B, 2, 1, S, false> : (np == 2 ? stream_forward_kernel<B, 2, 2, S, false> : stream_forward_kernel<B, 2, 4, S, false>);
   if (split_mask == 0) {
     if (a.bits == 8) { PIPE_ST_PICK(8, false) } else if (a.bits == 4) { PIPE_ST_PICK(4, false) } else { PIPE_ST_PICK(2, false) }
   } else {   // a summed ensemble on a shared input: the epilogue that closes the predictors' chains
     if (a.bits == 8) { PIPE_ST_PICK(8, true) } else if (a.bits == 4) { PIPE_ST_PICK(4, true) } else { PIPE_ST_PICK(2, true) }
   }
 #undef PIPE_ST_PICK
+  void (*kern_full)(const Params) = nullptr;   // the same kernel without per-slab branches (up to 8 tokens, one order pair)
+  if (split_mask == 0 && nt == 1 && np == 1)
+    kern_full = a.bits == 8 ? stream_forward_kernel<8, 1, 1, false, true>
+                            : (a.bits == 4 ? stream_forward_kernel<4, 1, 1, false, true> : stream_forward_kernel<2, 1, 1, false, true>);
   int smem_max = 0, sms = 0, fixed = 0;
   if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
   p.ctas_per_branch = sms / a.num_branches;
@@ -693,6 +711,11 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream, uint
   if (p.ctas_per_branch > p.slabs_per_branch) p.ctas_per_branch = p.slabs_per_branch;
   const int grid = p.ctas_per_branch * a.num_branches;
   p.own_max = ceil_div(p.slabs_per_branch, p.ctas_per_branch);
+  // one pass whose slab slots are (nearly) all taken: the kernel without per-slab branches
+  if (kern_full && p.own_max <= p.pass_slabs && p.own_max > (spw - 1) * kGroupWarps) {
+    kern = kern_full;
+    if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
+  }
   // passes a CTA may need: its range cut into pieces of pass_slabs
   if (ceil_div(p.own_max, p.pass_slabs) > kMaxPasses) return PIPE_ERR_UNSUPPORTED;
   // a stage holds one reduction block (two for 2-bit codes) of every order for the slabs of a pass, all kept

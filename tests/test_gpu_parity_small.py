@@ -206,6 +206,9 @@ FORWARD_CASES = [
     (320, 1024, 7, 2, 8, 8, 10, 1),
     (200, 1152, 16, 2, 3, 8, 11, 1),
     (24832, 128, 5, 4, 2, 8, 1552, 1),
+    # 18 slabs per CTA on 148 SMs: nearly every slab slot of a consumer warp is taken (the kernel without per-slab branches)
+    (21312, 128, 3, 4, 2, 8, 1000, 1),
+    (21312, 256, 8, 2, 2, 16, 700, 1),
 ]
 
 
