@@ -116,14 +116,14 @@ def workload_spec(name: str):
 # program (summaries under profiles/, named in the comment).  A workload without a capture of the present
 # kernel has no entry and reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "cfg2": 29294336 + 51489280,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
-    "cfg3a": 9440512 + 47313152,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
-    "cfg4a_t4096": 90993408 + 312856320,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
-    "cfg5": 490662400 + 1028348928,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
-    "cfg4a_t1": 56559872 + 62464,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
-    "cfg4a_t16": 56687616 + 119040,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
-    "cfg4a_t4096+int8_copy": 148933632 + 316924928,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
-    "cfg3b+int8_copy": 31190784 + 717824,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
+    "cfg2": 29206784 + 50998016,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
+    "cfg3a": 9449728 + 47143680,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
+    "cfg4a_t4096": 91097856 + 313175552,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
+    "cfg5": 509625088 + 1027933440,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
+    "cfg4a_t1": 56559872 + 30464,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
+    "cfg4a_t16": 56688640 + 161280,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
+    "cfg4a_t4096+int8_copy": 150005504 + 316969216,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
+    "cfg3b+int8_copy": 31191040 + 1042688,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
 }
 
 
