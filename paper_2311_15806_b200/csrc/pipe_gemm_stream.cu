@@ -154,13 +154,14 @@ __device__ __forceinline__ int rows_before(const int32_t* cum, int c, int O, int
   return lo * g + (hi > lo ? c - j * g : 0);
 }
 
-// FULL: nearly every slab slot of every consumer warp holds a slab (the host knows: one pass, more than SPW - 1 slabs per
-// warp): the loop over a warp's slabs then runs without its per-slab branches -- an absent chunk takes part with zero
-// weights -- so that the slabs' load-and-MMA chains are one block the compiler may interleave (cfg4a T = 1: 17.6 -> 16.8 us;
-// a launch with two slabs per warp would do 2.5 times its work that way, hence the choice per launch).
-template <int BITS, int NT, int NP, bool SUMMED, bool FULL>
+// FULL != 0: a consumer warp has FULL slab slots per pass and (nearly) every one of them holds a slab (the host knows:
+// one pass, FULL = ceil(slabs of a CTA / warps of a group)): the loop over a warp's slabs then runs without its per-slab
+// branches -- an absent chunk takes part with zero weights -- so that the slabs' load-and-MMA chains are one block the
+// compiler may interleave (cfg4a T = 1, five slabs per warp: 17.6 -> 16.8 us; cfg4b T = 1, two: 21.2 -> 19.4 us; with the
+// slots of the general kernel, five, a launch with two slabs per warp would do 2.5 times its work that way).
+template <int BITS, int NT, int NP, bool SUMMED, int FULL>
 __global__ void __launch_bounds__(kThreads, 1) stream_forward_kernel(const __grid_constant__ Params p) {
-  constexpr int SPW = (NP * NT <= 2) ? 5 : (NP * NT == 4 ? 2 : 1);   // slabs per consumer warp and pass
+  constexpr int SPW = FULL ? FULL : ((NP * NT <= 2) ? 5 : (NP * NT == 4 ? 2 : 1));   // slabs per consumer warp and pass
   constexpr int CHK = 128 / BITS;               // codes per 16-byte chunk
   constexpr int KBPS = (BITS == 2) ? 2 : 1;     // reduction blocks per stage
   constexpr int MS = KBPS * 128 / (4 * CHK);    // macro steps (4 chunks per row of 8 lanes x 4) per stage
@@ -626,7 +627,7 @@ struct DeviceCache {
   std::mutex mu;
   bool ready = false;
   int smem_max = 0, sms = 0, n = 0;
-  KernelInfo k[40];
+  KernelInfo k[64];
 };
 
 static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* smem_max, int* sms, int* fixed) {
@@ -645,7 +646,7 @@ static bool kernel_info(void (*kern)(const Params), int dyn_wanted_or_0, int* sm
   for (int i = 0; i < c.n; ++i)
     if (c.k[i].fn == reinterpret_cast<const void*>(kern)) ki = &c.k[i];
   if (!ki) {
-    if (c.n >= 40) return false;
+    if (c.n >= 64) return false;
     cudaFuncAttributes fattr;
     if (cudaFuncGetAttributes(&fattr, kern) != cudaSuccess) return false;
     ki = &c.k[c.n++];
@@ -692,18 +693,32 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream, uint
   // (the kernel instantiation depends only on bits, tokens and orders, all known here)
   void (*kern)(const Params) = nullptr;
 #define PIPE_ST_PICK(B, S)                                                                     \
-  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1, S, false> : (np == 2 ? stream_forward_kernel<B, 1, 2, S, false> : stream_forward_kernel<B, 1, 4, S, false>); \
-  else kern = np == 1 ? stream_forward_kernel<B, 2, 1, S, false> : (np == 2 ? stream_forward_kernel<B, 2, 2, S, false> : stream_forward_kernel<B, 2, 4, S, false>);
+  if (nt == 1) kern = np == 1 ? stream_forward_kernel<B, 1, 1, S, 0> : (np == 2 ? stream_forward_kernel<B, 1, 2, S, 0> : stream_forward_kernel<B, 1, 4, S, 0>); \
+  else kern = np == 1 ? stream_forward_kernel<B, 2, 1, S, 0> : (np == 2 ? stream_forward_kernel<B, 2, 2, S, 0> : stream_forward_kernel<B, 2, 4, S, 0>);
   if (split_mask == 0) {
     if (a.bits == 8) { PIPE_ST_PICK(8, false) } else if (a.bits == 4) { PIPE_ST_PICK(4, false) } else { PIPE_ST_PICK(2, false) }
   } else {   // a summed ensemble on a shared input: the epilogue that closes the predictors' chains
     if (a.bits == 8) { PIPE_ST_PICK(8, true) } else if (a.bits == 4) { PIPE_ST_PICK(4, true) } else { PIPE_ST_PICK(2, true) }
   }
 #undef PIPE_ST_PICK
-  void (*kern_full)(const Params) = nullptr;   // the same kernel without per-slab branches (up to 8 tokens, one order pair)
-  if (split_mask == 0 && nt == 1 && np == 1)
-    kern_full = a.bits == 8 ? stream_forward_kernel<8, 1, 1, false, true>
-                            : (a.bits == 4 ? stream_forward_kernel<4, 1, 1, false, true> : stream_forward_kernel<2, 1, 1, false, true>);
+  // the same kernel without per-slab branches, by slab slots per warp (one order pair; up to 8 tokens: 2 to 5 slots,
+  // 9 to 16 tokens: 2 or 3 -- more would spill)
+  auto full_kernel = [&](int slots) -> void (*)(const Params) {
+    if (split_mask != 0 || np != 1) return nullptr;
+#define PIPE_ST_FULL(B)                                                                                       \
+  if (nt == 1) {                                                                                              \
+    if (slots == 2) return stream_forward_kernel<B, 1, 1, false, 2>;                                          \
+    if (slots == 3) return stream_forward_kernel<B, 1, 1, false, 3>;                                          \
+    if (slots == 4) return stream_forward_kernel<B, 1, 1, false, 4>;                                          \
+    if (slots == 5) return stream_forward_kernel<B, 1, 1, false, 5>;                                          \
+  } else {                                                                                                    \
+    if (slots == 2) return stream_forward_kernel<B, 2, 1, false, 2>;                                          \
+    if (slots == 3) return stream_forward_kernel<B, 2, 1, false, 3>;                                          \
+  }
+    if (a.bits == 8) { PIPE_ST_FULL(8) } else if (a.bits == 4) { PIPE_ST_FULL(4) } else { PIPE_ST_FULL(2) }
+#undef PIPE_ST_FULL
+    return nullptr;
+  };
   int smem_max = 0, sms = 0, fixed = 0;
   if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
   p.ctas_per_branch = sms / a.num_branches;
@@ -711,10 +726,15 @@ static pipe_status launch_stream(const ForwardArgs& a, cudaStream_t stream, uint
   if (p.ctas_per_branch > p.slabs_per_branch) p.ctas_per_branch = p.slabs_per_branch;
   const int grid = p.ctas_per_branch * a.num_branches;
   p.own_max = ceil_div(p.slabs_per_branch, p.ctas_per_branch);
-  // one pass whose slab slots are (nearly) all taken: the kernel without per-slab branches
-  if (kern_full && p.own_max <= p.pass_slabs && p.own_max > (spw - 1) * kGroupWarps) {
-    kern = kern_full;
-    if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
+  // one pass whose slab slots are (nearly) all taken: the kernel without per-slab branches, with just the slots it needs
+  {
+    const int slots = ceil_div(p.own_max, kGroupWarps);
+    void (*kern_full)(const Params) = (p.own_max > kGroupWarps) ? full_kernel(slots) : nullptr;
+    if (kern_full) {
+      kern = kern_full;
+      p.pass_slabs = kGroupWarps * slots;
+      if (!kernel_info(kern, 0, &smem_max, &sms, &fixed)) return PIPE_ERR_CUDA;
+    }
   }
   // passes a CTA may need: its range cut into pieces of pass_slabs
   if (ceil_div(p.own_max, p.pass_slabs) > kMaxPasses) return PIPE_ERR_UNSUPPORTED;

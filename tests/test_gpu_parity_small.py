@@ -209,6 +209,11 @@ FORWARD_CASES = [
     # 18 slabs per CTA on 148 SMs: nearly every slab slot of a consumer warp is taken (the kernel without per-slab branches)
     (21312, 128, 3, 4, 2, 8, 1000, 1),
     (21312, 256, 8, 2, 2, 16, 700, 1),
+    # ... and with 6, 10 and 14 slabs per CTA (two, three, four slab slots per warp), up to 8 and up to 16 tokens
+    (7104, 128, 12, 4, 2, 8, 400, 1),
+    (7104, 256, 2, 8, 2, 8, 300, 1),
+    (11840, 128, 16, 4, 2, 8, 700, 1),
+    (16576, 128, 1, 2, 2, 16, 500, 1),
 ]
 
 
