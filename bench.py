@@ -116,14 +116,14 @@ def workload_spec(name: str):
 # program (summaries under profiles/, named in the comment).  A workload without a capture of the present
 # kernel has no entry and reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "cfg2": 29206784 + 50998016,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
-    "cfg3a": 9449728 + 47143680,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
-    "cfg4a_t4096": 91097856 + 313175552,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
-    "cfg5": 509625088 + 1027933440,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
-    "cfg4a_t1": 56559872 + 30464,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
-    "cfg4a_t16": 56688640 + 161280,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
-    "cfg4a_t4096+int8_copy": 150005504 + 316969216,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
-    "cfg3b+int8_copy": 31191040 + 1042688,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
+    "cfg2": 29317632 + 51065600,           # profiles/ncu_tc2_forward_kernel_cfg2.txt
+    "cfg3a": 9438976 + 49971456,           # profiles/ncu_tc2_forward_kernel_cfg3a.txt
+    "cfg4a_t4096": 91033600 + 313256192,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096.txt
+    "cfg5": 478397440 + 1029014784,        # profiles/ncu_tc2_forward_kernel_cfg5.txt
+    "cfg4a_t1": 56559616 + 98304,          # profiles/ncu_stream_forward_kernel_cfg4a_t1.txt
+    "cfg4a_t16": 56688128 + 303872,         # profiles/ncu_stream_forward_kernel_cfg4a_t16.txt
+    "cfg4a_t4096+int8_copy": 149131520 + 316639744,   # profiles/ncu_tc2_forward_kernel_cfg4a_t4096_int8_copy.txt
+    "cfg3b+int8_copy": 31190784 + 930048,           # profiles/ncu_tc2_forward_kernel_cfg3b_int8_copy.txt
 }
 
 
